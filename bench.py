@@ -1,0 +1,305 @@
+#!/usr/bin/env python
+"""Benchmark of the 0/1 Adam optimizer-step path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload bert_large]
+    python bench.py --impl reference ...        # the CPU oracle on the host cores
+
+A step is one iteration of Algorithm 1 for all W workers under the workload's
+own T_u / T_v policies (fused sync kernel on sync steps, local-step kernel
+otherwise, variance update where due), over one batch of synthetic gradients
+that is already resident in device memory.  Prints ONE JSON line (rank 0).
+"""
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "optimizer step throughput (params*workers/s)"
+UNIT = "params*workers/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+# ---- byte model: what the method must move, per launch -------------------------
+def sync_step_bytes(n, W, chunk):
+    """Fused sync step: per parameter and worker read g, m, u, delta (16 B), write
+    delta, x, m, u (16 B) and 1 sign bit, plus one scale per chunk; per parameter
+    read delta_bar, v, x_sync (12 B), write delta_bar, x_sync (8 B) and 1 sign bit."""
+    n_chunks = -(-n // chunk)
+    return n * W * (32 + 1 / 8) + n_chunks * W * 4 + n * (20 + 1 / 8) + n_chunks * 4
+
+
+def local_step_bytes(n, W):
+    """Local step: per parameter and worker read g, m, x, u and write m, x, u (28 B); v read once."""
+    return n * W * 28 + n * 4
+
+
+def variance_bytes(n, W):
+    return n * W * 4 + n * 8
+
+
+def measured_hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ---- clocks during the timed region ----------------------------------------------
+class ClockSampler:
+    def __init__(self, index):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._dev = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self._dev, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self._nv = None
+
+    def _run(self):
+        nv = self._nv
+        names = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "hw_thermal_slowdown": 0x40,
+                 "sw_thermal_slowdown": 0x20, "hw_power_brake": 0x80}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self._dev, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self._dev)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._dev)
+                self.reasons.update(k for k, bit in names.items() if mask & bit)
+            except Exception:
+                pass
+            self._stop.wait(0.1)
+
+    def __enter__(self):
+        if self._nv:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+
+    def summary(self):
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ---- the CPU oracle, timed as it stands (baseline and --impl reference) ---------------
+def time_oracle(wl, sample_elems, steps, seed=1):
+    """Runs the oracle (oracle/, single thread) on the first `sample_elems`
+    parameters of the workload for the given step indices; returns
+    (params*workers/s, description)."""
+    import numpy as np
+    from oracle import zoa_oracle as zo
+
+    d = min(sample_elems, wl.n)
+    rng = np.random.default_rng(seed)
+    o = zo.Oracle(d, wl.W, wl.chunk, wl.beta1, wl.beta2, wl.eps, dtype=np.float32)
+    o.set_params((rng.standard_normal(d) * wl.x0_std).astype(np.float32))
+    g = rng.standard_normal((wl.W, d)).astype(np.float32)
+    o.step(g, np.float32(wl.lr), 0, True, True)          # untimed: touch every page once
+    t0 = time.perf_counter()
+    for k, t in enumerate(steps):
+        o.step(g, np.float32(wl.lr), k + 1, wl.in_T_u(t), wl.in_T_v(t))
+    dt = time.perf_counter() - t0
+    n_sync = sum(wl.in_T_u(t) for t in steps)
+    desc = (f"first {d} parameters x {wl.W} workers of {wl.name}, {len(steps)} steps of its schedule "
+            f"(t={steps[0]}..{steps[-1]}: {n_sync} sync, {len(steps) - n_sync} local), oracle/zoa_oracle.c float build")
+    return d * wl.W * len(steps) / dt, desc, dt
+
+
+def run_reference(args, wl):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    steps = list(range(60, 60 + max(1, min(args.steps, 10))))
+    for _ in range(min(args.warmup, 1)):
+        time_oracle(wl, 1 << 18, steps[:2])
+    value, desc, dt = time_oracle(wl, args.cpu_sample, steps)
+    per_step_ms = dt / len(steps) * 1e3 * (wl.n / min(args.cpu_sample, wl.n))
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step_ms,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic", "config": {"workload": wl.name, "n_params": wl.n, "W": wl.W, "chunk": wl.chunk},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0,
+            "note": "ms_per_step is the sampled time scaled to the full parameter count"}
+    print(json.dumps(line))
+
+
+# ---- the CUDA path -------------------------------------------------------------------
+def run_ours(args, wl):
+    import torch
+    import torch.distributed as dist
+    from paper_2202_06009_b200 import Zoa, synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # Every rank owns a contiguous chunk range of an N-times larger flat vector: the
+    # method is chunk-local, so there is no exchange between ranks (weak scaling).
+    seed = synth.DEFAULT_SEED + rank
+    opt = Zoa(wl.n, wl.W, wl.beta1, wl.beta2, wl.eps, wl.chunk)
+    opt.set_params(synth.initial_params(wl, "cuda", seed))
+    opt.set_policies(wl.var_steps, wl.sync_boundaries, wl.sync_intervals)
+    stream = synth.GradientStream(wl, "cuda", seed)
+    from paper_2202_06009_b200 import binding as B
+
+    K, Wu = args.steps, max(args.warmup, 3)
+    for t in range(Wu):                                   # warm-up: the first steps of the schedule
+        opt.step_auto(stream.fill(t), wl.lr_at(t), t)
+    # also warm the local-step kernel, then rewind the step counter (timing does not depend on values)
+    opt.step(stream.bufs, wl.lr, Wu)
+    B.zoa_set_scalars(opt.h, 0.0, 0, -1)
+    barrier()
+
+    launches0 = opt.stats()["n_launches"]
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    kinds = []
+    with ClockSampler(local_rank) as clocks:
+        barrier()
+        wall0 = time.perf_counter()
+        for t in range(K):
+            bufs = stream.fill(t)                         # untimed: the batch is resident before the step starts
+            ev[t][0].record()
+            opt.step_auto(bufs, wl.lr_at(t), t)
+            ev[t][1].record()
+            kinds.append(("sync" if wl.in_T_u(t) else "local") + ("+var" if wl.in_T_v(t) else ""))
+        barrier()
+        wall = time.perf_counter() - wall0
+    opt.check_device()
+    ms = [a.elapsed_time(b) for a, b in ev]
+    total_ms = sum(ms)
+    if world > 1:
+        tt = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = float(tt.item())
+    launches = opt.stats()["n_launches"] - launches0
+
+    by_kind = {}
+    for k, m in zip(kinds, ms):
+        by_kind.setdefault(k, []).append(m)
+    peak, peak_kind = measured_hbm_peak()
+    bytes_of = {"sync": sync_step_bytes(wl.n, wl.W, wl.chunk), "local": local_step_bytes(wl.n, wl.W)}
+    bytes_of["sync+var"] = bytes_of["sync"] + variance_bytes(wl.n, wl.W)
+    bytes_of["local+var"] = bytes_of["local"] + wl.n * 4
+    step_types = {k: {"count": len(v), "ms": statistics.mean(v), "algorithmic_GB": bytes_of[k] / 1e9,
+                      "GBps": bytes_of[k] / 1e6 / statistics.mean(v)} for k, v in by_kind.items()}
+    total_bytes = sum(bytes_of[k] for k in kinds)
+    dominant = "sync" if "sync" in by_kind else ("sync+var" if "sync+var" in by_kind else kinds[0])
+    achieved = bytes_of[dominant] / 1e6 / statistics.mean(by_kind[dominant])
+    roofline = {"bound": "hbm", "kernel": "step_sync_kernel" if dominant.startswith("sync") else "local_step_kernel",
+                "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "peak_kind": f"of {peak_kind}", "frac_of_8TBps_nominal": achieved / 8000.0,
+                "traffic": None, "launch_ms": statistics.mean(by_kind[dominant]),
+                "algorithmic_bytes_per_launch": bytes_of[dominant]}
+
+    # ---- end to end: host gradients in, worker 0's model out, through zoa_step_host ----
+    e2e = None
+    if rank == 0 or world > 1:
+        ke = max(1, min(args.e2e_steps, K))
+        host_g = torch.empty(wl.n, dtype=torch.float32).pin_memory()
+        host_g.copy_(stream.bufs[0])
+        host_x = torch.empty(wl.n, dtype=torch.float32).pin_memory()
+        B.zoa_set_scalars(opt.h, 0.0, 0, -1)
+        opt.step_host([host_g] * wl.W, wl.lr, 0, host_x)  # allocates the staging area; untimed
+        B.zoa_set_scalars(opt.h, 0.0, 0, -1)
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for t in range(ke):
+            opt.step_host([host_g] * wl.W, wl.lr_at(t), t, host_x)
+        b.record()
+        barrier()
+        e_ms = a.elapsed_time(b)
+        if world > 1:
+            tt = torch.tensor([e_ms], device="cuda", dtype=torch.float64)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            e_ms = float(tt.item())
+        e2e = {"value": wl.n * wl.W * ke * world / (e_ms / 1e3), "unit": UNIT,
+               "h2d_bytes_per_step": wl.n * wl.W * 4, "d2h_bytes_per_step": wl.n * 4, "steps": ke,
+               "ms_per_step": e_ms / ke,
+               "how": "zoa_step_host: W copies from pinned host memory (one pinned buffer serves every "
+                      "worker), the step, worker 0's model copied back"}
+    opt.close()
+
+    if rank == 0:
+        cpu = None
+        if world == 1 and not args.no_cpu_baseline:
+            value, desc, _ = time_oracle(wl, args.cpu_sample, list(range(60, 70)))
+            cpu = {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc}
+        line = {"metric": METRIC, "value": wl.n * wl.W * K * world / (total_ms / 1e3), "unit": UNIT,
+                "n_gpus": world, "steps": K, "warmup": Wu, "ms_per_step": total_ms / K,
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+                "data": "synthetic",
+                "config": {"workload": wl.name, "n_params": wl.n, "W": wl.W, "chunk": wl.chunk,
+                           "schedule": f"t=0..{K - 1} of the workload's T_u/T_v policies",
+                           "l2": "inputs larger than L2 (gradients and state are read once per step)",
+                           "parallelism": f"{world} x independent chunk ranges, no collective"},
+                "hbm_GBps": total_bytes / 1e6 / total_ms, "hbm_frac_of_measured_peak": total_bytes / 1e6 / total_ms / peak,
+                "step_types": step_types, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e,
+                "gpu_launches": launches, "clocks": clocks.summary(), "wall_s_timed_region": wall}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="bert_large")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--cpu-sample", type=int, default=1 << 22, help="parameters in the oracle's timed sample")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    if args.impl == "reference":
+        # the oracle needs no CUDA library; import only the workload tables
+        import importlib.util
+        spec = importlib.util.spec_from_file_location("_synth", os.path.join(ROOT, "paper_2202_06009_b200", "synth.py"))
+        synth = importlib.util.module_from_spec(spec)
+        sys.modules["_synth"] = synth
+        spec.loader.exec_module(synth)
+        wl = synth.WORKLOADS[args.workload]()
+        if args.steps is None:
+            args.steps = wl.steps
+        return run_reference(args, wl)
+
+    from paper_2202_06009_b200 import synth
+    wl = synth.WORKLOADS[args.workload]()
+    if args.steps is None:
+        args.steps = wl.steps
+    run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,165 @@
+/*
+ * zoa - the per-parameter optimizer step of 0/1 Adam (arXiv 2202.06009) for W
+ * data-parallel workers held as separate state buffers on one NVIDIA B200.
+ *
+ * Plain C ABI.  Pointers are marked (device) or (host).  The library owns all
+ * optimizer state; gradients are borrowed, read-only, and must stay valid until
+ * the stream has finished the call's work.  Every call that takes a stream
+ * enqueues its work on that stream and returns after host-side validation
+ * only; nothing synchronises unless stated.  A handle is not thread-safe.
+ *
+ * Arithmetic contract (what "the same result" means for every entry point):
+ * all state is IEEE binary32; each elementwise operation is one
+ * round-to-nearest binary32 operation (no fused multiply-add, subnormals
+ * kept); the three reductions of the method - the l1 norm of a chunk, the mean
+ * over workers of the compressed buffers, the mean over workers of the
+ * gradients - accumulate in binary64 and are rounded to binary32 once.
+ *
+ * State layout in device memory (n = n_params, row stride n_pad = n rounded up
+ * to 128 elements, padding always zero):
+ *   x, m, u, delta_w   float [W][n_pad]     per-worker model, momentum, buffer, error
+ *   v, delta_s, x_sync float [n_pad]        variance, server error, model at the last sync
+ *   words_w            uint32 [W][n_pad/32] sign bits each worker sent
+ *   scales_w           float  [W][n_chunks] one magnitude per chunk and worker
+ *   words_s, scales_s  uint32 [n_pad/32], float [n_chunks]   what the server sent back
+ * Coordinate j is bit (j mod 32), least significant first, of word j / 32;
+ * unused bits are zero.  Chunk c covers coordinates [c*chunk, min((c+1)*chunk, n)).
+ */
+#ifndef ZOA_H
+#define ZOA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct zoa_handle_s *zoa_handle;
+
+typedef enum {
+    ZOA_OK = 0,
+    ZOA_ERR_ARG = 1,    /* a bad argument; nothing was changed */
+    ZOA_ERR_ALLOC = 2,  /* device or host memory could not be had */
+    ZOA_ERR_CUDA = 3,   /* a CUDA call or an earlier kernel failed; see zoa_last_error */
+    ZOA_ERR_STATE = 4,  /* calls out of order: t not increasing, reduce with nothing accumulated */
+    ZOA_ERR_DEVICE = 5  /* a kernel gave up on a bounded wait; state is undefined */
+} zoa_status;
+
+typedef enum {
+    ZOA_BUF_X = 0, ZOA_BUF_M = 1, ZOA_BUF_U = 2, ZOA_BUF_DELTA_W = 3,
+    ZOA_BUF_V = 4, ZOA_BUF_DELTA_S = 5, ZOA_BUF_X_SYNC = 6,
+    ZOA_BUF_WORDS_W = 7, ZOA_BUF_SCALES_W = 8, ZOA_BUF_WORDS_S = 9, ZOA_BUF_SCALES_S = 10
+} zoa_buffer;
+
+typedef struct {
+    int64_t n_steps;        /* optimizer steps taken (Algorithm 1 iterations) */
+    int64_t n_syncs;        /* 1-bit AllReduce rounds */
+    int64_t n_var_updates;  /* variance updates (steps in T_v) */
+    int64_t n_launches;     /* kernels this handle has launched */
+    int64_t bits_per_worker;/* bits a worker would have sent so far: n_syncs * (n + 32 n_chunks) */
+    int64_t t_last;         /* last step index seen, -1 before the first */
+    int64_t t_sync;         /* t' of Algorithm 1 */
+    double gamma_sum;       /* learning rates accumulated into u since the last sync */
+} zoa_stats;
+
+/* Algorithm 1, "Require" line: creates the state for a d = n_params
+ * dimensional model on W workers with m_0 = v_0 = u_0 = 0, both compression
+ * errors 0 (Algorithm 3), x_0 = 0 until zoa_set_params, t' = 0, on the current
+ * CUDA device.  chunk is the number of consecutive coordinates that share one
+ * magnitude in the compressor of Eq. 3 (chunk >= n_params gives Eq. 3 as printed).
+ * Requires n_params >= 1, 1 <= W <= 64, 0 <= beta < 1, eps > 0, chunk a
+ * multiple of 32 in [32, 16384].  Allocates device memory (cudaMalloc). */
+zoa_status zoa_create(zoa_handle *out, size_t n_params, int W, float beta1, float beta2,
+                      float eps, int chunk);
+
+/* Frees everything the handle owns.  Synchronises the device first. */
+zoa_status zoa_destroy(zoa_handle h);
+
+/* x_0 of Algorithm 1: copies x0 (device, n_params floats) into every worker's
+ * model and into x_sync.  All workers start from the same model, as the
+ * analysis of the method assumes. */
+zoa_status zoa_set_params(zoa_handle h, const float *x0, void *stream);
+
+/* T_v of Algorithm 1 as an explicit list of step indices (host, any order).
+ * Default: empty (the variance is never updated). */
+zoa_status zoa_set_var_steps(zoa_handle h, const int64_t *steps, size_t count);
+
+/* T_v by the rule of Section 6 ("Policy for T_v and T_u"): the j-th update is
+ * at k_j with k_0 = 0 and k_{j+1} - k_j = 2^floor(j / kappa), for k_j < freeze_at. */
+zoa_status zoa_set_var_policy_doubling(zoa_handle h, int kappa, int64_t freeze_at);
+
+/* T_u of Algorithm 1 as a piecewise-constant interval: piece r starts at step
+ * boundaries[r] (host, strictly increasing, boundaries[0] = 0) and has a sync
+ * at every step t with (t - boundaries[r]) % intervals[r] == 0.  Default: one
+ * piece with interval 1 (sync at every step). */
+zoa_status zoa_set_sync_policy(zoa_handle h, const int64_t *boundaries, const int32_t *intervals,
+                               size_t count);
+
+/* Membership tests, 1 or 0 (negative on a bad handle). */
+int zoa_sync_due(zoa_handle h, int64_t t);
+int zoa_var_due(zoa_handle h, int64_t t);
+
+/* Algorithm 1 lines 3-5 for every worker, and lines 14-15 when t is in T_v
+ * (the new variance takes effect from the next step on, so that a following
+ * zoa_onebit_reduce still uses v_t as line 9 does).
+ * grads: (host) array of W (device) pointers, n_params floats each, worker i's
+ * gradient at step t; 16-byte aligned pointers take the vector path.
+ * lr is gamma_t; t must be larger than at the previous step. */
+zoa_status zoa_step(zoa_handle h, const float *const *grads, float lr, int64_t t, void *stream);
+
+/* Algorithm 1 lines 7-11 with Algorithm 3 inside: compresses u + delta per
+ * worker (Eq. 3 per chunk), averages, compresses again on the "server" with its
+ * own error, then m = u_bar / sum(gamma), x = x_sync - u_bar / sqrt(v_t + eps),
+ * u = 0 on every worker.  ZOA_ERR_STATE if nothing was accumulated since the
+ * last sync (the divisor of line 8 would be zero). */
+zoa_status zoa_onebit_reduce(zoa_handle h, void *stream);
+
+/* zoa_step followed by zoa_onebit_reduce, same results bit for bit, in one
+ * pass over memory that never writes the half-step values. */
+zoa_status zoa_step_sync(zoa_handle h, const float *const *grads, float lr, int64_t t,
+                         void *stream);
+
+/* One iteration of Algorithm 1 under the handle's own policies: zoa_step_sync
+ * if t is in T_u, else zoa_step. */
+zoa_status zoa_step_auto(zoa_handle h, const float *const *grads, float lr, int64_t t,
+                         void *stream);
+
+/* The same iteration with gradients in (host) memory: host_grads is an array
+ * of W (host) pointers of n_params floats (pinned memory copies fastest).
+ * Copies them to a device staging area the handle allocates on first use,
+ * runs zoa_step_auto, and, if host_x_out is not NULL, copies worker 0's model
+ * back (n_params floats).  All on `stream`; does not synchronise. */
+zoa_status zoa_step_host(zoa_handle h, const float *const *host_grads, float lr, int64_t t,
+                         float *host_x_out, void *stream);
+
+/* Borrowed (device) pointer to one row of a state buffer and its length in
+ * elements (n_pad, n_pad/32 or n_chunks).  worker is ignored for shared buffers. */
+zoa_status zoa_get_buffer(zoa_handle h, zoa_buffer which, int worker, void **dev_ptr,
+                          size_t *n_elems);
+
+/* Synchronous copies between a state row and (host) memory, in elements of the
+ * buffer's type from element `offset`; for checkpoints and tests. */
+zoa_status zoa_copy_out(zoa_handle h, zoa_buffer which, int worker, size_t offset, size_t count,
+                        void *host_dst);
+zoa_status zoa_copy_in(zoa_handle h, zoa_buffer which, int worker, size_t offset, size_t count,
+                       const void *host_src);
+
+/* Host scalars of Algorithm 1 (sum of gammas since the last sync, t', last t),
+ * to restore a checkpoint together with zoa_copy_in. */
+zoa_status zoa_set_scalars(zoa_handle h, double gamma_sum, int64_t t_sync, int64_t t_last);
+
+zoa_status zoa_get_stats(zoa_handle h, zoa_stats *out);
+
+/* Waits for the device and reports ZOA_ERR_DEVICE / ZOA_ERR_CUDA if any kernel
+ * of this handle failed since the last check. */
+zoa_status zoa_check_device(zoa_handle h);
+
+/* Text of the last error on this handle (or of the last failed zoa_create if h
+ * is NULL).  Never NULL. */
+const char *zoa_last_error(zoa_handle h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ZOA_H */

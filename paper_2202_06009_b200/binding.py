@@ -1,0 +1,160 @@
+"""ctypes binding of libzoa.so: the C ABI of include/zoa.h under the same names.
+
+Argument marshalling only; every step of the method runs in the CUDA kernels.
+The shared library must have been built (paper_2202_06009_b200/build.py); there
+is no fallback of any kind.
+"""
+import ctypes as C
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libzoa.so")
+
+OK, ERR_ARG, ERR_ALLOC, ERR_CUDA, ERR_STATE, ERR_DEVICE = range(6)
+(BUF_X, BUF_M, BUF_U, BUF_DELTA_W, BUF_V, BUF_DELTA_S, BUF_X_SYNC,
+ BUF_WORDS_W, BUF_SCALES_W, BUF_WORDS_S, BUF_SCALES_S) = range(11)
+WORD_BUFFERS = (BUF_WORDS_W, BUF_WORDS_S)
+
+
+class ZoaError(RuntimeError):
+    def __init__(self, status, message):
+        super().__init__(f"zoa status {status}: {message}")
+        self.status = status
+
+
+class Stats(C.Structure):
+    _fields_ = [("n_steps", C.c_int64), ("n_syncs", C.c_int64), ("n_var_updates", C.c_int64),
+                ("n_launches", C.c_int64), ("bits_per_worker", C.c_int64), ("t_last", C.c_int64),
+                ("t_sync", C.c_int64), ("gamma_sum", C.c_double)]
+
+
+def _load():
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2202_06009_b200.build` "
+                          "(or __graft_entry__.build()); this package has no CPU path")
+    lib = C.CDLL(LIB_PATH)
+    H, p = C.c_void_p, C.c_void_p
+    sigs = {
+        "zoa_create": ([C.POINTER(H), C.c_size_t, C.c_int, C.c_float, C.c_float, C.c_float, C.c_int], C.c_int),
+        "zoa_destroy": ([H], C.c_int),
+        "zoa_set_params": ([H, p, p], C.c_int),
+        "zoa_set_var_steps": ([H, C.POINTER(C.c_int64), C.c_size_t], C.c_int),
+        "zoa_set_var_policy_doubling": ([H, C.c_int, C.c_int64], C.c_int),
+        "zoa_set_sync_policy": ([H, C.POINTER(C.c_int64), C.POINTER(C.c_int32), C.c_size_t], C.c_int),
+        "zoa_sync_due": ([H, C.c_int64], C.c_int),
+        "zoa_var_due": ([H, C.c_int64], C.c_int),
+        "zoa_step": ([H, C.POINTER(p), C.c_float, C.c_int64, p], C.c_int),
+        "zoa_onebit_reduce": ([H, p], C.c_int),
+        "zoa_step_sync": ([H, C.POINTER(p), C.c_float, C.c_int64, p], C.c_int),
+        "zoa_step_auto": ([H, C.POINTER(p), C.c_float, C.c_int64, p], C.c_int),
+        "zoa_step_host": ([H, C.POINTER(p), C.c_float, C.c_int64, p, p], C.c_int),
+        "zoa_get_buffer": ([H, C.c_int, C.c_int, C.POINTER(p), C.POINTER(C.c_size_t)], C.c_int),
+        "zoa_copy_out": ([H, C.c_int, C.c_int, C.c_size_t, C.c_size_t, p], C.c_int),
+        "zoa_copy_in": ([H, C.c_int, C.c_int, C.c_size_t, C.c_size_t, p], C.c_int),
+        "zoa_set_scalars": ([H, C.c_double, C.c_int64, C.c_int64], C.c_int),
+        "zoa_get_stats": ([H, C.POINTER(Stats)], C.c_int),
+        "zoa_check_device": ([H], C.c_int),
+        "zoa_last_error": ([H], C.c_char_p),
+    }
+    for name, (argtypes, restype) in sigs.items():
+        fn = getattr(lib, name)
+        fn.argtypes, fn.restype = argtypes, restype
+    return lib, tuple(sigs)
+
+
+lib, EXPORTS = _load()
+
+
+def _check(handle, status):
+    if status != OK:
+        raise ZoaError(status, lib.zoa_last_error(handle).decode())
+
+
+def _ptr_array(ptrs):
+    return (C.c_void_p * len(ptrs))(*ptrs)
+
+
+# -- the C calls under their own names (handle = ctypes.c_void_p) ---------------
+def zoa_create(n_params, W, beta1, beta2, eps, chunk):
+    h = C.c_void_p()
+    _check(None, lib.zoa_create(C.byref(h), n_params, W, beta1, beta2, eps, chunk))
+    return h
+
+
+def zoa_destroy(h):
+    _check(None, lib.zoa_destroy(h))
+
+
+def zoa_set_params(h, x0_ptr, stream=0):
+    _check(h, lib.zoa_set_params(h, x0_ptr, stream))
+
+
+def zoa_set_var_steps(h, steps):
+    arr = (C.c_int64 * len(steps))(*steps)
+    _check(h, lib.zoa_set_var_steps(h, arr, len(steps)))
+
+
+def zoa_set_var_policy_doubling(h, kappa, freeze_at):
+    _check(h, lib.zoa_set_var_policy_doubling(h, kappa, freeze_at))
+
+
+def zoa_set_sync_policy(h, boundaries, intervals):
+    b = (C.c_int64 * len(boundaries))(*boundaries)
+    k = (C.c_int32 * len(intervals))(*intervals)
+    _check(h, lib.zoa_set_sync_policy(h, b, k, len(boundaries)))
+
+
+def zoa_sync_due(h, t):
+    return lib.zoa_sync_due(h, t)
+
+
+def zoa_var_due(h, t):
+    return lib.zoa_var_due(h, t)
+
+
+def zoa_step(h, grad_ptrs, lr, t, stream=0):
+    _check(h, lib.zoa_step(h, _ptr_array(grad_ptrs), lr, t, stream))
+
+
+def zoa_onebit_reduce(h, stream=0):
+    _check(h, lib.zoa_onebit_reduce(h, stream))
+
+
+def zoa_step_sync(h, grad_ptrs, lr, t, stream=0):
+    _check(h, lib.zoa_step_sync(h, _ptr_array(grad_ptrs), lr, t, stream))
+
+
+def zoa_step_auto(h, grad_ptrs, lr, t, stream=0):
+    _check(h, lib.zoa_step_auto(h, _ptr_array(grad_ptrs), lr, t, stream))
+
+
+def zoa_step_host(h, host_grad_ptrs, lr, t, host_x_out_ptr=None, stream=0):
+    _check(h, lib.zoa_step_host(h, _ptr_array(host_grad_ptrs), lr, t, host_x_out_ptr, stream))
+
+
+def zoa_get_buffer(h, which, worker=0):
+    ptr, n = C.c_void_p(), C.c_size_t()
+    _check(h, lib.zoa_get_buffer(h, which, worker, C.byref(ptr), C.byref(n)))
+    return ptr.value, n.value
+
+
+def zoa_copy_out(h, which, worker, offset, count, host_ptr):
+    _check(h, lib.zoa_copy_out(h, which, worker, offset, count, host_ptr))
+
+
+def zoa_copy_in(h, which, worker, offset, count, host_ptr):
+    _check(h, lib.zoa_copy_in(h, which, worker, offset, count, host_ptr))
+
+
+def zoa_set_scalars(h, gamma_sum, t_sync, t_last):
+    _check(h, lib.zoa_set_scalars(h, gamma_sum, t_sync, t_last))
+
+
+def zoa_get_stats(h):
+    s = Stats()
+    _check(h, lib.zoa_get_stats(h, C.byref(s)))
+    return {name: getattr(s, name) for name, _ in Stats._fields_}
+
+
+def zoa_check_device(h):
+    _check(h, lib.zoa_check_device(h))

@@ -1,0 +1,428 @@
+// The C ABI of include/zoa.h: handle, validation, policies, host scalars of
+// Algorithm 1 (sum of gammas, t', pending variance) and kernel dispatch.
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/zoa.h"
+#include "zoa_internal.h"
+
+using namespace zoa;
+
+struct zoa_handle_s {
+    int device = 0, sm_count = 148;
+    long long n = 0, n_pad = 0, n_chunks = 0, words_stride = 0;
+    int W = 0, chunk = 0;
+    Consts c{};
+    float *x = nullptr, *m = nullptr, *u = nullptr, *dw = nullptr;
+    float *v_cur = nullptr, *v_nxt = nullptr, *ds = nullptr, *xs = nullptr;
+    uint32_t *words_w = nullptr, *words_s = nullptr;
+    float *scales_w = nullptr, *scales_s = nullptr;
+    float *staging = nullptr;      // [W][n_pad], device copy of host gradients (zoa_step_host)
+    bool v_pending = false;        // v_nxt holds v_{t+1}; it becomes v at the next step
+    std::vector<int64_t> var_steps;                    // T_v, sorted
+    std::vector<int64_t> sync_bounds{0};               // T_u pieces
+    std::vector<int32_t> sync_intervals{1};
+    double gamma_sum = 0.0;
+    int64_t t_sync = 0, t_last = -1;
+    int64_t n_steps = 0, n_syncs = 0, n_var_updates = 0, n_launches = 0;
+    std::string err;
+};
+
+static std::string g_create_error;
+
+static zoa_status fail(zoa_handle h, zoa_status s, const std::string &msg)
+{
+    if (h) h->err = msg; else g_create_error = msg;
+    return s;
+}
+static zoa_status fail_cuda(zoa_handle h, cudaError_t e, const char *what)
+{
+    return fail(h, e == cudaErrorMemoryAllocation ? ZOA_ERR_ALLOC : ZOA_ERR_CUDA,
+                std::string(what) + ": " + cudaGetErrorString(e));
+}
+#define ZOA_CUDA(h, call)                                        \
+    do {                                                         \
+        cudaError_t e_ = (call);                                 \
+        if (e_ != cudaSuccess) return fail_cuda(h, e_, #call);   \
+    } while (0)
+
+static StateView view(zoa_handle h)
+{
+    StateView st{};
+    st.x = h->x; st.m = h->m; st.u = h->u; st.dw = h->dw;
+    st.v = h->v_cur; st.v_next = h->v_nxt; st.ds = h->ds; st.xs = h->xs;
+    st.words_w = h->words_w; st.scales_w = h->scales_w; st.words_s = h->words_s; st.scales_s = h->scales_s;
+    st.n = h->n; st.n_pad = h->n_pad; st.n_chunks = h->n_chunks; st.words_stride = h->words_stride;
+    st.W = h->W; st.chunk = h->chunk;
+    return st;
+}
+
+static void free_all(zoa_handle h)
+{
+    void *ptrs[] = {h->x, h->m, h->u, h->dw, h->v_cur, h->v_nxt, h->ds, h->xs,
+                    h->words_w, h->words_s, h->scales_w, h->scales_s, h->staging};
+    for (void *p : ptrs)
+        if (p) cudaFree(p);
+}
+
+template <typename T>
+static cudaError_t alloc_zero(T **p, size_t count)
+{
+    cudaError_t e = cudaMalloc(reinterpret_cast<void **>(p), count * sizeof(T));
+    if (e != cudaSuccess) { *p = nullptr; return e; }
+    return cudaMemset(*p, 0, count * sizeof(T));
+}
+
+extern "C" zoa_status zoa_create(zoa_handle *out, size_t n_params, int W, float beta1, float beta2,
+                                 float eps, int chunk)
+{
+    if (!out) return fail(nullptr, ZOA_ERR_ARG, "zoa_create: out is NULL");
+    *out = nullptr;
+    if (n_params < 1 || n_params > (size_t)1 << 40) return fail(nullptr, ZOA_ERR_ARG, "zoa_create: n_params out of range");
+    if (W < 1 || W > kMaxWorkers) return fail(nullptr, ZOA_ERR_ARG, "zoa_create: W must be in [1, 64]");
+    if (!(beta1 >= 0.f && beta1 < 1.f) || !(beta2 >= 0.f && beta2 < 1.f))
+        return fail(nullptr, ZOA_ERR_ARG, "zoa_create: beta1 and beta2 must be in [0, 1)");
+    if (!(eps > 0.f) || !std::isfinite(eps)) return fail(nullptr, ZOA_ERR_ARG, "zoa_create: eps must be positive");
+    if (chunk < 32 || chunk > kMaxChunk || chunk % 32 != 0)
+        return fail(nullptr, ZOA_ERR_ARG, "zoa_create: chunk must be a multiple of 32 in [32, 16384]");
+
+    zoa_handle h = new (std::nothrow) zoa_handle_s;
+    if (!h) return fail(nullptr, ZOA_ERR_ALLOC, "zoa_create: out of host memory");
+    cudaError_t e = cudaGetDevice(&h->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device);
+    if (e == cudaSuccess) e = configure_kernels();
+    if (e != cudaSuccess) { delete h; return fail_cuda(nullptr, e, "zoa_create: device set-up"); }
+
+    h->n = (long long)n_params;
+    h->n_pad = (h->n + kRowAlign - 1) / kRowAlign * kRowAlign;
+    h->W = W;
+    h->chunk = chunk;
+    h->n_chunks = (h->n + chunk - 1) / chunk;
+    h->words_stride = h->n_pad / 32;
+    h->c.b1 = beta1; h->c.ob1 = 1.0f - beta1;
+    h->c.b2 = beta2; h->c.ob2 = 1.0f - beta2;
+    h->c.eps = eps;
+
+    const size_t rows = (size_t)W * (size_t)h->n_pad, row = (size_t)h->n_pad;
+    if ((e = alloc_zero(&h->x, rows)) == cudaSuccess && (e = alloc_zero(&h->m, rows)) == cudaSuccess &&
+        (e = alloc_zero(&h->u, rows)) == cudaSuccess && (e = alloc_zero(&h->dw, rows)) == cudaSuccess &&
+        (e = alloc_zero(&h->v_cur, row)) == cudaSuccess && (e = alloc_zero(&h->v_nxt, row)) == cudaSuccess &&
+        (e = alloc_zero(&h->ds, row)) == cudaSuccess && (e = alloc_zero(&h->xs, row)) == cudaSuccess &&
+        (e = alloc_zero(&h->words_w, (size_t)W * h->words_stride)) == cudaSuccess &&
+        (e = alloc_zero(&h->words_s, (size_t)h->words_stride)) == cudaSuccess &&
+        (e = alloc_zero(&h->scales_w, (size_t)W * h->n_chunks)) == cudaSuccess &&
+        (e = alloc_zero(&h->scales_s, (size_t)h->n_chunks)) == cudaSuccess)
+        e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) {
+        free_all(h);
+        delete h;
+        cudaGetLastError();
+        return fail_cuda(nullptr, e, "zoa_create: allocating state");
+    }
+    *out = h;
+    return ZOA_OK;
+}
+
+extern "C" zoa_status zoa_destroy(zoa_handle h)
+{
+    if (!h) return ZOA_ERR_ARG;
+    cudaSetDevice(h->device);
+    cudaDeviceSynchronize();
+    free_all(h);
+    delete h;
+    return ZOA_OK;
+}
+
+extern "C" zoa_status zoa_set_params(zoa_handle h, const float *x0, void *stream)
+{
+    if (!h) return ZOA_ERR_ARG;
+    if (!x0) return fail(h, ZOA_ERR_ARG, "zoa_set_params: x0 is NULL");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t bytes = (size_t)h->n * sizeof(float);
+    for (int i = 0; i < h->W; ++i)
+        ZOA_CUDA(h, cudaMemcpyAsync(h->x + (size_t)i * h->n_pad, x0, bytes, cudaMemcpyDeviceToDevice, s));
+    ZOA_CUDA(h, cudaMemcpyAsync(h->xs, x0, bytes, cudaMemcpyDeviceToDevice, s));
+    return ZOA_OK;
+}
+
+extern "C" zoa_status zoa_set_var_steps(zoa_handle h, const int64_t *steps, size_t count)
+{
+    if (!h) return ZOA_ERR_ARG;
+    if (count && !steps) return fail(h, ZOA_ERR_ARG, "zoa_set_var_steps: steps is NULL");
+    for (size_t k = 0; k < count; ++k)
+        if (steps[k] < 0) return fail(h, ZOA_ERR_ARG, "zoa_set_var_steps: negative step index");
+    h->var_steps.assign(steps, steps + count);
+    std::sort(h->var_steps.begin(), h->var_steps.end());
+    h->var_steps.erase(std::unique(h->var_steps.begin(), h->var_steps.end()), h->var_steps.end());
+    return ZOA_OK;
+}
+
+extern "C" zoa_status zoa_set_var_policy_doubling(zoa_handle h, int kappa, int64_t freeze_at)
+{
+    if (!h) return ZOA_ERR_ARG;
+    if (kappa < 1 || freeze_at < 0) return fail(h, ZOA_ERR_ARG, "zoa_set_var_policy_doubling: kappa >= 1, freeze_at >= 0");
+    h->var_steps.clear();
+    int64_t k = 0;
+    for (int64_t j = 0; k < freeze_at; ++j) {
+        h->var_steps.push_back(k);
+        const int64_t e = j / kappa;
+        if (e >= 62) break;
+        k += (int64_t)1 << e;  // k_{j+1} - k_j = 2^floor(j / kappa)
+    }
+    return ZOA_OK;
+}
+
+extern "C" zoa_status zoa_set_sync_policy(zoa_handle h, const int64_t *boundaries, const int32_t *intervals,
+                                          size_t count)
+{
+    if (!h) return ZOA_ERR_ARG;
+    if (count < 1 || !boundaries || !intervals) return fail(h, ZOA_ERR_ARG, "zoa_set_sync_policy: need at least one piece");
+    if (boundaries[0] != 0) return fail(h, ZOA_ERR_ARG, "zoa_set_sync_policy: boundaries[0] must be 0");
+    for (size_t r = 0; r < count; ++r) {
+        if (intervals[r] < 1) return fail(h, ZOA_ERR_ARG, "zoa_set_sync_policy: intervals must be >= 1");
+        if (r && boundaries[r] <= boundaries[r - 1]) return fail(h, ZOA_ERR_ARG, "zoa_set_sync_policy: boundaries must increase");
+    }
+    h->sync_bounds.assign(boundaries, boundaries + count);
+    h->sync_intervals.assign(intervals, intervals + count);
+    return ZOA_OK;
+}
+
+extern "C" int zoa_sync_due(zoa_handle h, int64_t t)
+{
+    if (!h || t < 0) return -1;
+    size_t r = std::upper_bound(h->sync_bounds.begin(), h->sync_bounds.end(), t) - h->sync_bounds.begin() - 1;
+    return (t - h->sync_bounds[r]) % h->sync_intervals[r] == 0 ? 1 : 0;
+}
+
+extern "C" int zoa_var_due(zoa_handle h, int64_t t)
+{
+    if (!h || t < 0) return -1;
+    return std::binary_search(h->var_steps.begin(), h->var_steps.end(), t) ? 1 : 0;
+}
+
+// Checks shared by the step entry points; fills the pointer pack.
+static zoa_status check_step_args(zoa_handle h, const float *const *grads, float lr, int64_t t, GradPtrs *gp,
+                                  bool *aligned, const char *who)
+{
+    if (!h) return ZOA_ERR_ARG;
+    if (!grads) return fail(h, ZOA_ERR_ARG, std::string(who) + ": grads is NULL");
+    if (!std::isfinite(lr)) return fail(h, ZOA_ERR_ARG, std::string(who) + ": lr is not finite");
+    if (t < 0) return fail(h, ZOA_ERR_ARG, std::string(who) + ": t is negative");
+    if (t <= h->t_last) return fail(h, ZOA_ERR_STATE, std::string(who) + ": t must increase from step to step");
+    *aligned = true;
+    for (int i = 0; i < h->W; ++i) {
+        if (!grads[i]) return fail(h, ZOA_ERR_ARG, std::string(who) + ": a gradient pointer is NULL");
+        gp->p[i] = grads[i];
+        if (reinterpret_cast<uintptr_t>(grads[i]) & 15u) *aligned = false;
+    }
+    for (int i = h->W; i < kMaxWorkers; ++i) gp->p[i] = nullptr;
+    return ZOA_OK;
+}
+
+static void commit_variance(zoa_handle h)
+{
+    if (h->v_pending) {
+        std::swap(h->v_cur, h->v_nxt);
+        h->v_pending = false;
+    }
+}
+
+extern "C" zoa_status zoa_step(zoa_handle h, const float *const *grads, float lr, int64_t t, void *stream)
+{
+    GradPtrs gp;
+    bool aligned;
+    zoa_status rc = check_step_args(h, grads, lr, t, &gp, &aligned, "zoa_step");
+    if (rc != ZOA_OK) return rc;
+    commit_variance(h);
+    const bool do_var = zoa_var_due(h, t) == 1;
+    ZOA_CUDA(h, launch_local_step(view(h), gp, h->c, lr, do_var, aligned, h->sm_count, static_cast<cudaStream_t>(stream)));
+    h->n_launches += 1;
+    h->gamma_sum += (double)lr;
+    if (do_var) { h->v_pending = true; h->n_var_updates += 1; }
+    h->t_last = t;
+    h->n_steps += 1;
+    return ZOA_OK;
+}
+
+extern "C" zoa_status zoa_onebit_reduce(zoa_handle h, void *stream)
+{
+    if (!h) return ZOA_ERR_ARG;
+    const float gamma_sum = (float)h->gamma_sum;
+    if (!(h->gamma_sum > 0.0) || !(gamma_sum > 0.f) || !std::isfinite(gamma_sum))
+        return fail(h, ZOA_ERR_STATE, "zoa_onebit_reduce: nothing accumulated since the last sync (sum of learning rates is not positive)");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const StateView st = view(h);
+    ZOA_CUDA(h, launch_compress(st, s));
+    ZOA_CUDA(h, launch_reduce(st, h->c, gamma_sum, s));
+    h->n_launches += 2;
+    h->gamma_sum = 0.0;
+    h->t_sync = h->t_last;
+    h->n_syncs += 1;
+    return ZOA_OK;
+}
+
+extern "C" zoa_status zoa_step_sync(zoa_handle h, const float *const *grads, float lr, int64_t t, void *stream)
+{
+    GradPtrs gp;
+    bool aligned;
+    zoa_status rc = check_step_args(h, grads, lr, t, &gp, &aligned, "zoa_step_sync");
+    if (rc != ZOA_OK) return rc;
+    const double total = h->gamma_sum + (double)lr;
+    const float gamma_sum = (float)total;
+    if (!(total > 0.0) || !(gamma_sum > 0.f) || !std::isfinite(gamma_sum))
+        return fail(h, ZOA_ERR_STATE, "zoa_step_sync: sum of learning rates since the last sync is not positive");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    commit_variance(h);
+    const bool do_var = zoa_var_due(h, t) == 1;
+    const StateView st = view(h);
+    ZOA_CUDA(h, launch_step_sync(st, gp, h->c, lr, gamma_sum, aligned, s));
+    h->n_launches += 1;
+    if (do_var) {
+        ZOA_CUDA(h, launch_variance(st, gp, h->c, aligned, h->sm_count, s));
+        h->n_launches += 1;
+        h->v_pending = true;
+        h->n_var_updates += 1;
+    }
+    h->gamma_sum = 0.0;
+    h->t_last = t;
+    h->t_sync = t;
+    h->n_steps += 1;
+    h->n_syncs += 1;
+    return ZOA_OK;
+}
+
+extern "C" zoa_status zoa_step_auto(zoa_handle h, const float *const *grads, float lr, int64_t t, void *stream)
+{
+    if (!h) return ZOA_ERR_ARG;
+    return zoa_sync_due(h, t) == 1 ? zoa_step_sync(h, grads, lr, t, stream) : zoa_step(h, grads, lr, t, stream);
+}
+
+extern "C" zoa_status zoa_step_host(zoa_handle h, const float *const *host_grads, float lr, int64_t t,
+                                    float *host_x_out, void *stream)
+{
+    if (!h) return ZOA_ERR_ARG;
+    if (!host_grads) return fail(h, ZOA_ERR_ARG, "zoa_step_host: host_grads is NULL");
+    for (int i = 0; i < h->W; ++i)
+        if (!host_grads[i]) return fail(h, ZOA_ERR_ARG, "zoa_step_host: a gradient pointer is NULL");
+    if (!std::isfinite(lr) || t < 0) return fail(h, ZOA_ERR_ARG, "zoa_step_host: bad lr or t");
+    if (t <= h->t_last) return fail(h, ZOA_ERR_STATE, "zoa_step_host: t must increase from step to step");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (!h->staging) {
+        cudaError_t e = cudaMalloc(reinterpret_cast<void **>(&h->staging), (size_t)h->W * h->n_pad * sizeof(float));
+        if (e != cudaSuccess) { h->staging = nullptr; cudaGetLastError(); return fail_cuda(h, e, "zoa_step_host: staging area"); }
+    }
+    const float *dev[kMaxWorkers];
+    for (int i = 0; i < h->W; ++i) {
+        float *dst = h->staging + (size_t)i * h->n_pad;
+        ZOA_CUDA(h, cudaMemcpyAsync(dst, host_grads[i], (size_t)h->n * sizeof(float), cudaMemcpyHostToDevice, s));
+        dev[i] = dst;
+    }
+    zoa_status rc = zoa_step_auto(h, dev, lr, t, stream);
+    if (rc != ZOA_OK) return rc;
+    if (host_x_out)
+        ZOA_CUDA(h, cudaMemcpyAsync(host_x_out, h->x, (size_t)h->n * sizeof(float), cudaMemcpyDeviceToHost, s));
+    return ZOA_OK;
+}
+
+// Row base, element size and row length of a state buffer.
+static zoa_status locate(zoa_handle h, zoa_buffer which, int worker, char **base, size_t *elem, size_t *len)
+{
+    const bool per_worker = which == ZOA_BUF_X || which == ZOA_BUF_M || which == ZOA_BUF_U ||
+                            which == ZOA_BUF_DELTA_W || which == ZOA_BUF_WORDS_W || which == ZOA_BUF_SCALES_W;
+    if (per_worker && (worker < 0 || worker >= h->W)) return fail(h, ZOA_ERR_ARG, "worker index out of range");
+    const size_t i = per_worker ? (size_t)worker : 0;
+    *elem = 4;
+    switch (which) {
+    case ZOA_BUF_X: *base = (char *)(h->x + i * h->n_pad); *len = h->n_pad; break;
+    case ZOA_BUF_M: *base = (char *)(h->m + i * h->n_pad); *len = h->n_pad; break;
+    case ZOA_BUF_U: *base = (char *)(h->u + i * h->n_pad); *len = h->n_pad; break;
+    case ZOA_BUF_DELTA_W: *base = (char *)(h->dw + i * h->n_pad); *len = h->n_pad; break;
+    case ZOA_BUF_V: *base = (char *)(h->v_pending ? h->v_nxt : h->v_cur); *len = h->n_pad; break;
+    case ZOA_BUF_DELTA_S: *base = (char *)h->ds; *len = h->n_pad; break;
+    case ZOA_BUF_X_SYNC: *base = (char *)h->xs; *len = h->n_pad; break;
+    case ZOA_BUF_WORDS_W: *base = (char *)(h->words_w + i * h->words_stride); *len = h->words_stride; break;
+    case ZOA_BUF_SCALES_W: *base = (char *)(h->scales_w + i * h->n_chunks); *len = h->n_chunks; break;
+    case ZOA_BUF_WORDS_S: *base = (char *)h->words_s; *len = h->words_stride; break;
+    case ZOA_BUF_SCALES_S: *base = (char *)h->scales_s; *len = h->n_chunks; break;
+    default: return fail(h, ZOA_ERR_ARG, "unknown buffer");
+    }
+    return ZOA_OK;
+}
+
+extern "C" zoa_status zoa_get_buffer(zoa_handle h, zoa_buffer which, int worker, void **dev_ptr, size_t *n_elems)
+{
+    if (!h) return ZOA_ERR_ARG;
+    if (!dev_ptr) return fail(h, ZOA_ERR_ARG, "zoa_get_buffer: dev_ptr is NULL");
+    char *base; size_t elem, len;
+    zoa_status rc = locate(h, which, worker, &base, &elem, &len);
+    if (rc != ZOA_OK) return rc;
+    *dev_ptr = base;
+    if (n_elems) *n_elems = len;
+    return ZOA_OK;
+}
+
+extern "C" zoa_status zoa_copy_out(zoa_handle h, zoa_buffer which, int worker, size_t offset, size_t count, void *host_dst)
+{
+    if (!h) return ZOA_ERR_ARG;
+    char *base; size_t elem, len;
+    zoa_status rc = locate(h, which, worker, &base, &elem, &len);
+    if (rc != ZOA_OK) return rc;
+    if (!host_dst || offset > len || count > len - offset) return fail(h, ZOA_ERR_ARG, "zoa_copy_out: range outside the row");
+    ZOA_CUDA(h, cudaDeviceSynchronize());
+    ZOA_CUDA(h, cudaMemcpy(host_dst, base + offset * elem, count * elem, cudaMemcpyDeviceToHost));
+    return ZOA_OK;
+}
+
+extern "C" zoa_status zoa_copy_in(zoa_handle h, zoa_buffer which, int worker, size_t offset, size_t count, const void *host_src)
+{
+    if (!h) return ZOA_ERR_ARG;
+    char *base; size_t elem, len;
+    zoa_status rc = locate(h, which, worker, &base, &elem, &len);
+    if (rc != ZOA_OK) return rc;
+    if (!host_src || offset > len || count > len - offset) return fail(h, ZOA_ERR_ARG, "zoa_copy_in: range outside the row");
+    ZOA_CUDA(h, cudaDeviceSynchronize());
+    ZOA_CUDA(h, cudaMemcpy(base + offset * elem, host_src, count * elem, cudaMemcpyHostToDevice));
+    return ZOA_OK;
+}
+
+extern "C" zoa_status zoa_set_scalars(zoa_handle h, double gamma_sum, int64_t t_sync, int64_t t_last)
+{
+    if (!h) return ZOA_ERR_ARG;
+    if (!std::isfinite(gamma_sum) || gamma_sum < 0.0 || t_last < -1) return fail(h, ZOA_ERR_ARG, "zoa_set_scalars: bad value");
+    h->gamma_sum = gamma_sum;
+    h->t_sync = t_sync;
+    h->t_last = t_last;
+    return ZOA_OK;
+}
+
+extern "C" zoa_status zoa_get_stats(zoa_handle h, zoa_stats *out)
+{
+    if (!h || !out) return ZOA_ERR_ARG;
+    out->n_steps = h->n_steps;
+    out->n_syncs = h->n_syncs;
+    out->n_var_updates = h->n_var_updates;
+    out->n_launches = h->n_launches;
+    out->bits_per_worker = h->n_syncs * (h->n + 32 * h->n_chunks);
+    out->t_last = h->t_last;
+    out->t_sync = h->t_sync;
+    out->gamma_sum = h->gamma_sum;
+    return ZOA_OK;
+}
+
+extern "C" zoa_status zoa_check_device(zoa_handle h)
+{
+    if (!h) return ZOA_ERR_ARG;
+    ZOA_CUDA(h, cudaDeviceSynchronize());
+    ZOA_CUDA(h, cudaGetLastError());
+    return ZOA_OK;
+}
+
+extern "C" const char *zoa_last_error(zoa_handle h)
+{
+    return h ? h->err.c_str() : g_create_error.c_str();
+}

@@ -1,0 +1,142 @@
+// Device-side building blocks shared by the zoa kernels: the binary32
+// "one rounding per operation" arithmetic, 128-bit accesses, the block-wide
+// binary64 sum and the sign-bit packing.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace zoa {
+
+constexpr int kMaxWorkers = 64;
+constexpr int kMaxChunk = 16384;
+constexpr int kRowAlign = 128;  // elements; state rows are padded to this
+
+// W gradient pointers travel as one kernel argument.
+struct GradPtrs {
+    const float *p[kMaxWorkers];
+};
+
+// beta1, 1 - beta1, beta2, 1 - beta2, eps, all already rounded to binary32 on the host.
+struct Consts {
+    float b1, ob1, b2, ob2, eps;
+};
+
+// Borrowed view of a handle's device state (see include/zoa.h for the layout).
+struct StateView {
+    float *x, *m, *u, *dw;  // [W][n_pad]
+    const float *v;         // [n_pad] v_t
+    float *v_next;          // [n_pad] v_{t+1}, written on T_v steps
+    float *ds, *xs;         // [n_pad] server error, model at the last sync
+    uint32_t *words_w;      // [W][words_stride]
+    float *scales_w;        // [W][n_chunks]
+    uint32_t *words_s;      // [words_stride]
+    float *scales_s;        // [n_chunks]
+    long long n, n_pad, n_chunks, words_stride;
+    int W, chunk;
+};
+
+// ---- binary32 arithmetic, one IEEE rounding per operation, never contracted ----
+__device__ __forceinline__ float f_add(float a, float b) { return __fadd_rn(a, b); }
+__device__ __forceinline__ float f_sub(float a, float b) { return __fsub_rn(a, b); }
+__device__ __forceinline__ float f_mul(float a, float b) { return __fmul_rn(a, b); }
+__device__ __forceinline__ float f_div(float a, float b) { return __fdiv_rn(a, b); }
+__device__ __forceinline__ float f_sqrt(float a) { return __fsqrt_rn(a); }
+
+// Algorithm 1 line 3: m_{t+1/2} = beta1 m_t + (1 - beta1) g_t.
+__device__ __forceinline__ float momentum(const Consts &c, float m, float g)
+{
+    return f_add(f_mul(c.b1, m), f_mul(c.ob1, g));
+}
+// Denominator of lines 4 and 9: sqrt(v_t + eps).
+__device__ __forceinline__ float denom(const Consts &c, float v) { return f_sqrt(f_add(v, c.eps)); }
+// Algorithm 1 line 15: v_{t+1} = beta2 v_t + (1 - beta2) g_bar^2.
+__device__ __forceinline__ float variance(const Consts &c, float v, float g_bar)
+{
+    return f_add(f_mul(c.b2, v), f_mul(c.ob2, f_mul(g_bar, g_bar)));
+}
+// Mean over W workers of a binary64 sum, rounded once (Algorithm 4).
+__device__ __forceinline__ float mean_round(double sum, int W)
+{
+    return __double2float_rn(__ddiv_rn(sum, (double)W));
+}
+// Eq. 3 magnitude of a chunk: l1 / len, rounded once.
+__device__ __forceinline__ float chunk_scale(double l1, int len)
+{
+    return __double2float_rn(__ddiv_rn(l1, (double)len));
+}
+// Server input of Algorithm 3: mean of the compressed buffers plus the server error.
+__device__ __forceinline__ float server_input(double sum_hat, int W, float delta_bar)
+{
+    return __double2float_rn(__dadd_rn(__ddiv_rn(sum_hat, (double)W), (double)delta_bar));
+}
+
+// ---- 128-bit accesses ----
+__device__ __forceinline__ float4 ld4(const float *p) { return *reinterpret_cast<const float4 *>(p); }
+__device__ __forceinline__ void st4(float *p, float4 v) { *reinterpret_cast<float4 *>(p) = v; }
+// Streaming variants: data touched once per step should not displace the rest of L2.
+__device__ __forceinline__ float4 ld4_stream(const float *p)
+{
+    return __ldcs(reinterpret_cast<const float4 *>(p));
+}
+__device__ __forceinline__ void st4_stream(float *p, float4 v) { __stcs(reinterpret_cast<float4 *>(p), v); }
+
+// Four consecutive gradient values starting at j (j % 4 == 0); the user's buffer
+// has exactly n elements and may be unaligned, so the ragged end and the
+// unaligned case go through guarded scalar loads (zero beyond n).
+__device__ __forceinline__ float4 ld_grad4(const float *g, long long j, long long n, bool aligned)
+{
+    if (aligned && j + 4 <= n) return ld4_stream(g + j);
+    float4 r;
+    r.x = j + 0 < n ? g[j + 0] : 0.f;
+    r.y = j + 1 < n ? g[j + 1] : 0.f;
+    r.z = j + 2 < n ? g[j + 2] : 0.f;
+    r.w = j + 3 < n ? g[j + 3] : 0.f;
+    return r;
+}
+
+// ---- block-wide binary64 sum; every thread gets the result ----
+// `scratch` holds 33 doubles.  Fixed tree, so a launch is reproducible.
+__device__ __forceinline__ double block_sum(double v, double *scratch)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = (blockDim.x + 31) >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    __syncthreads();  // scratch may still be read from the previous sum
+    if (lane == 0) scratch[warp] = v;
+    __syncthreads();
+    if (warp == 0) {
+        double t = lane < n_warps ? scratch[lane] : 0.0;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+        if (lane == 0) scratch[32] = t;
+    }
+    __syncthreads();
+    return scratch[32];
+}
+
+// ---- sign-bit packing for the "lane l holds coordinates 4l..4l+3" layout ----
+// Spreads the 8 bits of `byte` to bit positions 0, 4, 8, ..., 28.
+__device__ __forceinline__ uint32_t spread8(uint32_t x)
+{
+    x = (x | (x << 12)) & 0x000F000Fu;
+    x = (x | (x << 6)) & 0x03030303u;
+    x = (x | (x << 3)) & 0x11111111u;
+    return x;
+}
+// A warp covers 128 consecutive coordinates = 4 words.  b[k] says whether the
+// lane's k-th coordinate is non-negative (and valid).  Returns, in lanes 0..3,
+// word `lane` of the tile (undefined in the other lanes).  All 32 lanes call it.
+__device__ __forceinline__ uint32_t pack_tile(const bool b[4])
+{
+    const int w = threadIdx.x & 3;
+    uint32_t word = 0;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const uint32_t ballot = __ballot_sync(0xffffffffu, b[k]);
+        word |= spread8((ballot >> (8 * w)) & 0xFFu) << k;
+    }
+    return word;
+}
+
+}  // namespace zoa

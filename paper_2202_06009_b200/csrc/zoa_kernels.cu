@@ -1,0 +1,398 @@
+// The zoa kernels, chunk-per-block form: correct for every shape the API
+// accepts (any chunk that is a multiple of 32, a ragged last chunk, unaligned
+// gradient pointers).
+//
+//   local_step_kernel   Algorithm 1 lines 3-5 (+ lines 14-15 on T_v steps)
+//   variance_kernel     Algorithm 1 lines 14-15 alone
+//   compress_kernel     Algorithm 3 worker side (Eq. 3 per chunk, error feedback)
+//   reduce_kernel       Algorithm 3 server side + Algorithm 1 lines 8-10
+//   step_sync_kernel    all of the above for a sync step, one pass over memory
+#include "zoa_internal.h"
+
+namespace zoa {
+
+// ---------------------------------------------------------------------------
+// Local step: elementwise, one thread per 4 coordinates, loop over workers so
+// that v is read once and the gradient mean for the variance comes for free.
+// ---------------------------------------------------------------------------
+template <bool DO_VAR>
+__global__ void __launch_bounds__(256)
+local_step_kernel(StateView st, GradPtrs g, Consts c, float gamma, int g_aligned)
+{
+    const long long n4 = (st.n + 3) >> 2;
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x; q < n4; q += stride) {
+        const long long j = q << 2;
+        const float4 v4 = ld4(st.v + j);
+        const float d[4] = {denom(c, v4.x), denom(c, v4.y), denom(c, v4.z), denom(c, v4.w)};
+        double G[4] = {0.0, 0.0, 0.0, 0.0};
+        for (int i = 0; i < st.W; ++i) {
+            const long long row = (long long)i * st.n_pad + j;
+            const float4 g4 = ld_grad4(g.p[i], j, st.n, g_aligned);
+            const float4 m4 = ld4(st.m + row), x4 = ld4(st.x + row), u4 = ld4(st.u + row);
+            const float gg[4] = {g4.x, g4.y, g4.z, g4.w};
+            const float mm[4] = {m4.x, m4.y, m4.z, m4.w};
+            const float xx[4] = {x4.x, x4.y, x4.z, x4.w};
+            const float uu[4] = {u4.x, u4.y, u4.z, u4.w};
+            float mo[4], xo[4], uo[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                mo[k] = momentum(c, mm[k], gg[k]);              // line 3
+                const float s = f_mul(gamma, mo[k]);
+                xo[k] = f_sub(xx[k], f_div(s, d[k]));           // line 4
+                uo[k] = f_add(uu[k], s);                        // line 5
+                if (DO_VAR) G[k] += (double)gg[k];
+            }
+            st4(st.m + row, make_float4(mo[0], mo[1], mo[2], mo[3]));
+            st4(st.x + row, make_float4(xo[0], xo[1], xo[2], xo[3]));
+            st4(st.u + row, make_float4(uo[0], uo[1], uo[2], uo[3]));
+        }
+        if (DO_VAR) {
+            const float vv[4] = {v4.x, v4.y, v4.z, v4.w};
+            float vo[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) vo[k] = variance(c, vv[k], mean_round(G[k], st.W));  // lines 14-15
+            st4(st.v_next + j, make_float4(vo[0], vo[1], vo[2], vo[3]));
+        }
+    }
+}
+
+__global__ void __launch_bounds__(256)
+variance_kernel(StateView st, GradPtrs g, Consts c, int g_aligned)
+{
+    const long long n4 = (st.n + 3) >> 2;
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x; q < n4; q += stride) {
+        const long long j = q << 2;
+        double G[4] = {0.0, 0.0, 0.0, 0.0};
+        for (int i = 0; i < st.W; ++i) {
+            const float4 g4 = ld_grad4(g.p[i], j, st.n, g_aligned);
+            G[0] += (double)g4.x; G[1] += (double)g4.y; G[2] += (double)g4.z; G[3] += (double)g4.w;
+        }
+        const float4 v4 = ld4(st.v + j);
+        st4(st.v_next + j, make_float4(variance(c, v4.x, mean_round(G[0], st.W)),
+                                       variance(c, v4.y, mean_round(G[1], st.W)),
+                                       variance(c, v4.z, mean_round(G[2], st.W)),
+                                       variance(c, v4.w, mean_round(G[3], st.W))));
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Chunk-per-block helpers.  A warp owns tiles of 128 consecutive coordinates of
+// the chunk (4 words), lane l the coordinates 4l..4l+3 of the tile; a thread
+// touches the same coordinates in every pass, so shared memory needs no
+// barrier beyond those of the block sums.
+// ---------------------------------------------------------------------------
+struct ChunkGeom {
+    long long c0;  // first coordinate of the chunk
+    int len;       // its true length (the last chunk may be short)
+};
+__device__ __forceinline__ ChunkGeom chunk_geom(const StateView &st, long long c)
+{
+    ChunkGeom g;
+    g.c0 = c * st.chunk;
+    const long long rest = st.n - g.c0;
+    g.len = rest < st.chunk ? (int)rest : st.chunk;
+    return g;
+}
+
+// Second half of Eq. 3 for one tile: sign bits, compressed values, error
+// (written back in place of the input), packed word.  z[k] is the value being
+// compressed; on return z[k] holds z - z_hat (0 where invalid) and hat[k] the
+// compressed value (0 where invalid).  Lanes 0..3 hold the tile's words.
+__device__ __forceinline__ uint32_t compress_tile(float z[4], float hat[4], float scale, int idx, int len)
+{
+    bool b[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const bool valid = idx + k < len;
+        b[k] = valid && (z[k] >= 0.0f);  // +0 and -0 count as non-negative, NaN as negative
+        hat[k] = valid ? (b[k] ? scale : -scale) : 0.0f;
+        z[k] = valid ? f_sub(z[k], hat[k]) : 0.0f;
+    }
+    return pack_tile(b);
+}
+
+// Worker side of Algorithm 3 for (chunk blockIdx.x, worker blockIdx.y).
+__global__ void compress_kernel(StateView st)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    double *scratch = reinterpret_cast<double *>(smem_raw);        // 33 doubles
+    float *z_s = reinterpret_cast<float *>(smem_raw + 34 * sizeof(double));
+    const ChunkGeom cg = chunk_geom(st, blockIdx.x);
+    const int i = blockIdx.y;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    const long long row = (long long)i * st.n_pad + cg.c0;
+
+    double l1 = 0.0;
+    for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
+        const int idx = base + 4 * lane;
+        if (idx < cg.len) {
+            const float4 u4 = ld4(st.u + row + idx), e4 = ld4(st.dw + row + idx);
+            const float4 z4 = make_float4(f_add(u4.x, e4.x), f_add(u4.y, e4.y), f_add(u4.z, e4.z), f_add(u4.w, e4.w));
+            st4(z_s + idx, z4);
+            l1 += fabs((double)z4.x) + fabs((double)z4.y) + fabs((double)z4.z) + fabs((double)z4.w);
+        }
+    }
+    const float scale = chunk_scale(block_sum(l1, scratch), cg.len);
+    for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
+        const int idx = base + 4 * lane;
+        float z[4] = {0.f, 0.f, 0.f, 0.f}, hat[4];
+        if (idx < cg.len) {
+            const float4 z4 = ld4(z_s + idx);
+            z[0] = z4.x; z[1] = z4.y; z[2] = z4.z; z[3] = z4.w;
+        }
+        const uint32_t word = compress_tile(z, hat, scale, idx, cg.len);
+        if (idx < cg.len) st4(st.dw + row + idx, make_float4(z[0], z[1], z[2], z[3]));
+        if (lane < 4 && base + 32 * lane < cg.len)
+            st.words_w[(long long)i * st.words_stride + ((cg.c0 + base) >> 5) + lane] = word;
+    }
+    if (threadIdx.x == 0) st.scales_w[(long long)i * st.n_chunks + blockIdx.x] = scale;
+}
+
+// Server side of Algorithm 3 and lines 8-10 of Algorithm 1 for one tile whose
+// server input a[k] is known: compress it, keep the server error, rebuild m and x,
+// clear u, on every worker.  `scale` is the chunk's server magnitude.
+__device__ __forceinline__ void server_tile(const StateView &st, const Consts &c, const ChunkGeom &cg,
+                                            int base, int lane, float a[4], float scale, float gamma_sum)
+{
+    const int idx = base + 4 * lane;
+    float hat[4];
+    const uint32_t word = compress_tile(a, hat, scale, idx, cg.len);  // a[] now holds the new server error
+    if (lane < 4 && base + 32 * lane < cg.len) st.words_s[((cg.c0 + base) >> 5) + lane] = word;
+    if (idx >= cg.len) return;
+    const long long j = cg.c0 + idx;
+    st4(st.ds + j, make_float4(a[0], a[1], a[2], a[3]));
+    const float4 v4 = ld4(st.v + j), xs4 = ld4(st.xs + j);
+    const float vv[4] = {v4.x, v4.y, v4.z, v4.w}, xs[4] = {xs4.x, xs4.y, xs4.z, xs4.w};
+    float mo[4], xo[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const bool valid = idx + k < cg.len;
+        mo[k] = valid ? f_div(hat[k], gamma_sum) : 0.0f;                        // line 8
+        xo[k] = valid ? f_sub(xs[k], f_div(hat[k], denom(c, vv[k]))) : 0.0f;    // line 9
+    }
+    const float4 m4 = make_float4(mo[0], mo[1], mo[2], mo[3]);
+    const float4 x4 = make_float4(xo[0], xo[1], xo[2], xo[3]);
+    const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+    st4(st.xs + j, x4);
+    for (int i = 0; i < st.W; ++i) {
+        const long long row = (long long)i * st.n_pad + j;
+        st4(st.m + row, m4);
+        st4(st.x + row, x4);
+        st4(st.u + row, zero);                                                   // line 10
+    }
+}
+
+// Server side for chunk blockIdx.x, reading what compress_kernel sent.
+__global__ void reduce_kernel(StateView st, Consts c, float gamma_sum)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    double *scratch = reinterpret_cast<double *>(smem_raw);
+    float *scales = reinterpret_cast<float *>(smem_raw + 34 * sizeof(double));  // kMaxWorkers floats
+    float *a_s = scales + kMaxWorkers;
+    const ChunkGeom cg = chunk_geom(st, blockIdx.x);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+
+    for (int i = threadIdx.x; i < st.W; i += blockDim.x) scales[i] = st.scales_w[(long long)i * st.n_chunks + blockIdx.x];
+    __syncthreads();
+
+    double l1 = 0.0;
+    for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
+        const int idx = base + 4 * lane;
+        if (idx < cg.len) {
+            double A[4] = {0.0, 0.0, 0.0, 0.0};
+            const long long word_idx = (cg.c0 + idx) >> 5;
+            const int shift = idx & 31;
+            for (int i = 0; i < st.W; ++i) {  // worker order
+                const uint32_t nib = st.words_w[(long long)i * st.words_stride + word_idx] >> shift;
+                const double s = (double)scales[i];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) A[k] += ((nib >> k) & 1u) ? s : -s;
+            }
+            const float4 e4 = ld4(st.ds + cg.c0 + idx);
+            const float ee[4] = {e4.x, e4.y, e4.z, e4.w};
+            float a[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                a[k] = idx + k < cg.len ? server_input(A[k], st.W, ee[k]) : 0.0f;
+                l1 += fabs((double)a[k]);
+            }
+            st4(a_s + idx, make_float4(a[0], a[1], a[2], a[3]));
+        }
+    }
+    const float scale = chunk_scale(block_sum(l1, scratch), cg.len);
+    for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
+        const int idx = base + 4 * lane;
+        float a[4] = {0.f, 0.f, 0.f, 0.f};
+        if (idx < cg.len) {
+            const float4 a4 = ld4(a_s + idx);
+            a[0] = a4.x; a[1] = a4.y; a[2] = a4.z; a[3] = a4.w;
+        }
+        server_tile(st, c, cg, base, lane, a, scale, gamma_sum);
+    }
+    if (threadIdx.x == 0) st.scales_s[blockIdx.x] = scale;
+}
+
+// A whole sync step for chunk blockIdx.x: lines 3-5 in registers, worker
+// compression, server, lines 8-10.  The half-step m, x, u never reach memory;
+// x is not even read (line 9 rebuilds it from x_sync).
+__global__ void step_sync_kernel(StateView st, GradPtrs g, Consts c, float gamma, float gamma_sum,
+                                 int g_aligned, long long chunk_offset)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    double *scratch = reinterpret_cast<double *>(smem_raw);                      // 34 doubles
+    double *A_s = scratch + 34;                                                  // [chunk]
+    float *z_s = reinterpret_cast<float *>(A_s + st.chunk);                      // [chunk]
+    const long long chunk_id = chunk_offset + blockIdx.x;
+    const ChunkGeom cg = chunk_geom(st, chunk_id);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+
+    for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
+        const int idx = base + 4 * lane;
+        if (idx < cg.len) { A_s[idx] = 0.0; A_s[idx + 1] = 0.0; A_s[idx + 2] = 0.0; A_s[idx + 3] = 0.0; }
+    }
+    for (int i = 0; i < st.W; ++i) {
+        const long long row = (long long)i * st.n_pad + cg.c0;
+        const float *gi = g.p[i];
+        double l1 = 0.0;
+        for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
+            const int idx = base + 4 * lane;
+            if (idx < cg.len) {
+                const float4 g4 = ld_grad4(gi, cg.c0 + idx, st.n, g_aligned);
+                const float4 m4 = ld4_stream(st.m + row + idx), u4 = ld4_stream(st.u + row + idx);
+                const float4 e4 = ld4_stream(st.dw + row + idx);
+                const float gg[4] = {g4.x, g4.y, g4.z, g4.w}, mm[4] = {m4.x, m4.y, m4.z, m4.w};
+                const float uu[4] = {u4.x, u4.y, u4.z, u4.w}, ee[4] = {e4.x, e4.y, e4.z, e4.w};
+                float z[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const float s = f_mul(gamma, momentum(c, mm[k], gg[k]));     // lines 3, 5
+                    z[k] = f_add(f_add(uu[k], s), ee[k]);                        // u_{t+1/2} + delta
+                    l1 += fabs((double)z[k]);
+                }
+                st4(z_s + idx, make_float4(z[0], z[1], z[2], z[3]));
+            }
+        }
+        const float scale = chunk_scale(block_sum(l1, scratch), cg.len);
+        for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
+            const int idx = base + 4 * lane;
+            float z[4] = {0.f, 0.f, 0.f, 0.f}, hat[4];
+            if (idx < cg.len) {
+                const float4 z4 = ld4(z_s + idx);
+                z[0] = z4.x; z[1] = z4.y; z[2] = z4.z; z[3] = z4.w;
+            }
+            const uint32_t word = compress_tile(z, hat, scale, idx, cg.len);
+            if (idx < cg.len) {
+                st4_stream(st.dw + row + idx, make_float4(z[0], z[1], z[2], z[3]));
+#pragma unroll
+                for (int k = 0; k < 4; ++k) A_s[idx + k] += (double)hat[k];      // worker order
+            }
+            if (lane < 4 && base + 32 * lane < cg.len)
+                st.words_w[(long long)i * st.words_stride + ((cg.c0 + base) >> 5) + lane] = word;
+        }
+        if (threadIdx.x == 0) st.scales_w[(long long)i * st.n_chunks + chunk_id] = scale;
+    }
+    double l1 = 0.0;
+    for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
+        const int idx = base + 4 * lane;
+        if (idx < cg.len) {
+            const float4 e4 = ld4(st.ds + cg.c0 + idx);
+            const float ee[4] = {e4.x, e4.y, e4.z, e4.w};
+            float a[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                a[k] = idx + k < cg.len ? server_input(A_s[idx + k], st.W, ee[k]) : 0.0f;
+                l1 += fabs((double)a[k]);
+            }
+            st4(z_s + idx, make_float4(a[0], a[1], a[2], a[3]));
+        }
+    }
+    const float scale = chunk_scale(block_sum(l1, scratch), cg.len);
+    for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
+        const int idx = base + 4 * lane;
+        float a[4] = {0.f, 0.f, 0.f, 0.f};
+        if (idx < cg.len) {
+            const float4 a4 = ld4(z_s + idx);
+            a[0] = a4.x; a[1] = a4.y; a[2] = a4.z; a[3] = a4.w;
+        }
+        server_tile(st, c, cg, base, lane, a, scale, gamma_sum);
+    }
+    if (threadIdx.x == 0) st.scales_s[chunk_id] = scale;
+}
+
+// ---------------------------------------------------------------------------
+// Launchers
+// ---------------------------------------------------------------------------
+static int block_threads_for_chunk(int chunk)
+{
+    int t = chunk / 8;  // 8 coordinates per thread
+    if (t < 128) t = 128;
+    if (t > 1024) t = 1024;
+    int p = 128;
+    while (p < t) p <<= 1;
+    return p;
+}
+
+static int elementwise_grid(long long n4, int sm_count)
+{
+    long long blocks = (n4 + 255) / 256;
+    const long long cap = (long long)sm_count * 8;  // 8 resident blocks of 256 threads per SM
+    if (blocks > cap) blocks = cap;
+    return (int)(blocks < 1 ? 1 : blocks);
+}
+
+cudaError_t launch_local_step(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
+                              bool do_var, bool g_aligned, int sm_count, cudaStream_t s)
+{
+    const int grid = elementwise_grid((st.n + 3) / 4, sm_count);
+    if (do_var)
+        local_step_kernel<true><<<grid, 256, 0, s>>>(st, g, c, gamma, g_aligned);
+    else
+        local_step_kernel<false><<<grid, 256, 0, s>>>(st, g, c, gamma, g_aligned);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_variance(const StateView &st, const GradPtrs &g, const Consts &c, bool g_aligned,
+                            int sm_count, cudaStream_t s)
+{
+    variance_kernel<<<elementwise_grid((st.n + 3) / 4, sm_count), 256, 0, s>>>(st, g, c, g_aligned);
+    return cudaGetLastError();
+}
+
+size_t compress_smem(int chunk) { return 34 * sizeof(double) + (size_t)chunk * sizeof(float); }
+size_t reduce_smem(int chunk) { return 34 * sizeof(double) + (kMaxWorkers + (size_t)chunk) * sizeof(float); }
+size_t step_sync_smem(int chunk) { return 34 * sizeof(double) + (size_t)chunk * (sizeof(double) + sizeof(float)); }
+
+cudaError_t configure_kernels()
+{
+    cudaError_t e;
+    e = cudaFuncSetAttribute(compress_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)compress_smem(kMaxChunk));
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(reduce_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)reduce_smem(kMaxChunk));
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(step_sync_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)step_sync_smem(kMaxChunk));
+}
+
+cudaError_t launch_compress(const StateView &st, cudaStream_t s)
+{
+    const dim3 grid((unsigned)st.n_chunks, (unsigned)st.W);
+    compress_kernel<<<grid, block_threads_for_chunk(st.chunk), compress_smem(st.chunk), s>>>(st);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_reduce(const StateView &st, const Consts &c, float gamma_sum, cudaStream_t s)
+{
+    reduce_kernel<<<(unsigned)st.n_chunks, block_threads_for_chunk(st.chunk), reduce_smem(st.chunk), s>>>(st, c, gamma_sum);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_step_sync(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
+                             float gamma_sum, bool g_aligned, cudaStream_t s)
+{
+    step_sync_kernel<<<(unsigned)st.n_chunks, block_threads_for_chunk(st.chunk), step_sync_smem(st.chunk), s>>>(
+        st, g, c, gamma, gamma_sum, g_aligned, 0);
+    return cudaGetLastError();
+}
+
+}  // namespace zoa

@@ -1,0 +1,111 @@
+"""Handle wrapper: owns a zoa handle, marshals torch tensors to raw pointers.
+
+No arithmetic happens here.  torch supplies device memory for the gradients
+and the CUDA stream; the optimizer state lives inside the library.
+"""
+import numpy as np
+import torch
+
+from . import binding as B
+
+_NAMES = {"x": B.BUF_X, "m": B.BUF_M, "u": B.BUF_U, "delta_w": B.BUF_DELTA_W, "v": B.BUF_V,
+          "delta_s": B.BUF_DELTA_S, "x_sync": B.BUF_X_SYNC, "words_w": B.BUF_WORDS_W,
+          "scales_w": B.BUF_SCALES_W, "words_s": B.BUF_WORDS_S, "scales_s": B.BUF_SCALES_S}
+PER_WORKER = ("x", "m", "u", "delta_w", "words_w", "scales_w")
+
+
+def _stream():
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _grad_ptrs(grads, n, W):
+    if isinstance(grads, torch.Tensor):
+        grads = list(grads)
+    if len(grads) != W:
+        raise ValueError(f"expected {W} gradient tensors, got {len(grads)}")
+    for g in grads:
+        if not (g.is_cuda and g.dtype == torch.float32 and g.is_contiguous() and g.numel() == n):
+            raise ValueError("each gradient must be a contiguous float32 CUDA tensor of n_params elements")
+    return [g.data_ptr() for g in grads]
+
+
+class Zoa:
+    def __init__(self, n_params, W, beta1=0.9, beta2=0.999, eps=1e-8, chunk=4096):
+        self.n, self.W, self.chunk = int(n_params), int(W), int(chunk)
+        self.n_chunks = (self.n + self.chunk - 1) // self.chunk
+        self.h = B.zoa_create(self.n, self.W, beta1, beta2, eps, self.chunk)
+
+    def close(self):
+        if self.h is not None:
+            B.zoa_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+    # -- set-up -------------------------------------------------------------
+    def set_params(self, x0):
+        x0 = x0.to(device="cuda", dtype=torch.float32).contiguous()
+        assert x0.numel() == self.n
+        B.zoa_set_params(self.h, x0.data_ptr(), _stream())
+        torch.cuda.current_stream().synchronize()   # x0 may be a temporary
+
+    def set_policies(self, var_steps, sync_boundaries, sync_intervals):
+        B.zoa_set_var_steps(self.h, list(var_steps))
+        B.zoa_set_sync_policy(self.h, list(sync_boundaries), list(sync_intervals))
+
+    def sync_due(self, t):
+        return B.zoa_sync_due(self.h, t) == 1
+
+    def var_due(self, t):
+        return B.zoa_var_due(self.h, t) == 1
+
+    # -- Algorithm 1 --------------------------------------------------------
+    def step(self, grads, lr, t):
+        B.zoa_step(self.h, _grad_ptrs(grads, self.n, self.W), lr, t, _stream())
+
+    def onebit_reduce(self):
+        B.zoa_onebit_reduce(self.h, _stream())
+
+    def step_sync(self, grads, lr, t):
+        B.zoa_step_sync(self.h, _grad_ptrs(grads, self.n, self.W), lr, t, _stream())
+
+    def step_auto(self, grads, lr, t):
+        B.zoa_step_auto(self.h, _grad_ptrs(grads, self.n, self.W), lr, t, _stream())
+
+    def step_host(self, host_grads, lr, t, host_x_out=None):
+        ptrs = [g.data_ptr() for g in host_grads]
+        out = host_x_out.data_ptr() if host_x_out is not None else None
+        B.zoa_step_host(self.h, ptrs, lr, t, out, _stream())
+
+    # -- state access (synchronous copies) ----------------------------------------
+    def read(self, name, worker=0, offset=0, count=None):
+        which = _NAMES[name]
+        _, row_len = B.zoa_get_buffer(self.h, which, worker)
+        if count is None:
+            count = {True: (self.n + 31) // 32}.get(which in B.WORD_BUFFERS,
+                                                      self.n_chunks if name.startswith("scales") else self.n)
+            count -= offset
+        out = np.empty(count, np.uint32 if which in B.WORD_BUFFERS else np.float32)
+        B.zoa_copy_out(self.h, which, worker, offset, count, out.ctypes.data)
+        return out
+
+    def write(self, name, values, worker=0, offset=0):
+        which = _NAMES[name]
+        values = np.ascontiguousarray(values, np.uint32 if which in B.WORD_BUFFERS else np.float32)
+        B.zoa_copy_in(self.h, which, worker, offset, values.size, values.ctypes.data)
+
+    def stats(self):
+        return B.zoa_get_stats(self.h)
+
+    def check_device(self):
+        B.zoa_check_device(self.h)

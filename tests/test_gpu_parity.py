@@ -1,0 +1,274 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle on identical
+seeded float32 inputs: packed sign words bit-exact, every float32 state within
+1e-5 relative (1e-7 absolute near zero), after every step."""
+import numpy as np
+import pytest
+import torch
+
+from helpers import ATOL, RTOL, Pair, assert_close
+from paper_2202_06009_b200 import Zoa, ZoaError, binding as B, synth
+
+pytestmark = pytest.mark.gpu
+
+
+def _grads(rng, W, n, scale=1.0, outliers=True):
+    g = rng.standard_normal((W, n)).astype(np.float32) * np.float32(scale)
+    if outliers:
+        g[rng.random((W, n)) < 0.01] *= np.float32(100.0)
+    return g
+
+
+SIZES = [1, 31, 32, 33, 127, 128, 129, 2047, 2048, 2049, 3 * 2048 + 17]
+
+
+@pytest.mark.parametrize("mode", ["fused", "two_call"])
+@pytest.mark.parametrize("n", SIZES)
+def test_ragged_sizes(n, mode):
+    """Sizes around word, tile and chunk boundaries; six steps mixing local, sync and variance steps."""
+    rng = np.random.default_rng(n)
+    W, chunk = 3, 2048
+    p = Pair(n, W, chunk, var_steps=(0, 1, 3), sync=((0, 2), (1, 2)), x0=rng.standard_normal(n) * 0.02)
+    try:
+        for t in range(6):
+            p.step(_grads(rng, W, n), 1e-3 * (1 + t), t, mode)
+            p.compare(f"n={n} t={t}")
+        p.padding_is_zero()
+    finally:
+        p.close()
+
+
+@pytest.mark.parametrize("W,chunk,n", [(1, 32, 1000), (2, 64, 4096 + 5), (5, 96, 96 * 7 + 3), (4, 1024, 20000),
+                                       (8, 4096, 3 * 4096 + 1852), (16, 4096, 2 * 4096 + 77), (4, 8192, 8192 * 2 + 704),
+                                       (2, 16384, 16384 * 2 + 100), (64, 256, 1500), (3, 4000, 9000)])
+@pytest.mark.parametrize("mode", ["fused", "two_call"])
+def test_worker_and_chunk_shapes(W, chunk, n, mode):
+    rng = np.random.default_rng(W * 131 + chunk)
+    p = Pair(n, W, chunk, var_steps=(0, 2), sync=((0, 3), (1, 2)), x0=rng.standard_normal(n) * 0.02)
+    try:
+        for t in range(6):
+            p.step(_grads(rng, W, n), 1e-3, t, mode)
+            p.compare(f"W={W} chunk={chunk} t={t}")
+        p.padding_is_zero()
+    finally:
+        p.close()
+
+
+def test_fused_equals_two_call_bit_for_bit():
+    rng = np.random.default_rng(77)
+    n, W, chunk = 5 * 1024 + 333, 4, 1024
+    x0 = torch.from_numpy((rng.standard_normal(n) * 0.02).astype(np.float32))
+    a, b = Zoa(n, W, chunk=chunk), Zoa(n, W, chunk=chunk)
+    try:
+        for z in (a, b):
+            z.set_params(x0)
+            z.set_policies((0, 1, 4), (0, 3), (1, 2))
+        for t in range(8):
+            g = list(torch.from_numpy(_grads(rng, W, n)).cuda())
+            a.step_auto(g, 2e-3, t)
+            b.step(g, 2e-3, t)
+            if b.sync_due(t):
+                b.onebit_reduce()
+            torch.cuda.synchronize()
+            for name in ("x", "m", "u", "delta_w", "words_w", "scales_w"):
+                for i in range(W):
+                    assert np.array_equal(a.read(name, i), b.read(name, i)), (name, i, t)
+            for name in ("v", "delta_s", "x_sync", "words_s", "scales_s"):
+                assert np.array_equal(a.read(name), b.read(name)), (name, t)
+        assert a.stats()["n_syncs"] == b.stats()["n_syncs"] == 6
+    finally:
+        a.close(), b.close()
+
+
+@pytest.mark.parametrize("mode", ["fused", "two_call"])
+def test_special_values(mode):
+    """Signed zeros, subnormals, an all-zero chunk, a chunk of one sign, a lone outlier."""
+    W, chunk, n = 2, 64, 64 * 6
+    g = np.zeros((W, n), np.float32)
+    g[:, 0:64] = 0.0                                   # all-zero chunk: scale 0, every bit 1
+    g[0, 64:128] = np.float32(-0.0)
+    g[1, 64:128] = np.float32(1e-42)                   # subnormal gradients
+    g[:, 128:192] = np.float32(3.0)                    # constant sign
+    g[0, 192:256] = np.float32(1e-3); g[0, 200] = np.float32(1e6)   # one outlier dominates the l1 norm
+    g[1, 192:256] = np.float32(-1e-3)
+    rng = np.random.default_rng(4)
+    g[:, 256:] = rng.standard_normal((W, n - 256)).astype(np.float32) * np.float32(1e-20)  # tiny values
+    p = Pair(n, W, chunk, var_steps=(0,), x0=np.zeros(n))
+    try:
+        for t in range(3):
+            p.step(g, 1e-3, t, mode)
+            p.compare(f"t={t}")
+        words = p.gpu.read("words_w", 0)
+        assert words[0] == 0xFFFFFFFF and words[1] == 0xFFFFFFFF
+    finally:
+        p.close()
+
+
+def test_tiny_config_full_run():
+    """The small configuration in full: 2^20 parameters, W = 4, chunk 2048, 64 steps,
+    T_v = {0,1,2,4,8,16}, sync every step until 16 then every other step; every
+    state compared after every step."""
+    wl = synth.tiny()
+    stream = synth.GradientStream(wl, "cuda")
+    x0 = synth.initial_params(wl, "cuda")
+    p = Pair(wl.n, wl.W, wl.chunk, wl.beta1, wl.beta2, wl.eps, wl.var_steps,
+             (wl.sync_boundaries, wl.sync_intervals), x0=x0.cpu().numpy())
+    try:
+        n_sync = 0
+        for t in range(wl.steps):
+            bufs = stream.fill(t)
+            g = torch.stack(bufs).cpu().numpy()
+            sync, var = wl.in_T_u(t), wl.in_T_v(t)
+            assert p.gpu.sync_due(t) == sync and p.gpu.var_due(t) == var
+            p.gpu.step_auto(bufs, wl.lr_at(t), t)
+            torch.cuda.synchronize()
+            assert p.cpu.step(g, np.float32(wl.lr_at(t)), t, sync, var) == 0
+            n_sync += sync
+            p.compare(f"t={t}", wire=sync)
+        assert n_sync == 40 and p.gpu.stats()["n_syncs"] == 40 and p.gpu.stats()["n_var_updates"] == 6
+    finally:
+        p.close()
+
+
+@pytest.mark.parametrize("name,divisor", [("bert_base", 64), ("gpt2_1p5b", 1024)])
+def test_shaped_workloads_scaled_down(name, divisor):
+    """BERT- and GPT-2-shaped layouts shrunk per tensor (per-tensor lognormal scales,
+    Student-t noise for GPT-2), their own policies, first 24 steps."""
+    wl = synth.scaled(synth.WORKLOADS[name](), divisor, steps=24)
+    stream = synth.GradientStream(wl, "cuda")
+    x0 = synth.initial_params(wl, "cuda")
+    p = Pair(wl.n, wl.W, wl.chunk, wl.beta1, wl.beta2, wl.eps, wl.var_steps,
+             (wl.sync_boundaries, wl.sync_intervals), x0=x0.cpu().numpy())
+    try:
+        for t in range(wl.steps):
+            bufs = stream.fill(t)
+            g = torch.stack(bufs).cpu().numpy()
+            p.gpu.step_auto(bufs, wl.lr, t)
+            torch.cuda.synchronize()
+            p.cpu.step(g, np.float32(wl.lr), t, wl.in_T_u(t), wl.in_T_v(t))
+            if t % 4 == 3 or t < 3:
+                p.compare(f"{name} t={t}", wire=wl.in_T_u(t))
+    finally:
+        p.close()
+
+
+def test_unaligned_gradient_pointers():
+    rng = np.random.default_rng(5)
+    n, W, chunk = 3000, 2, 1024
+    p = Pair(n, W, chunk, var_steps=(0,), sync=((0,), (2,)), x0=rng.standard_normal(n) * 0.02)
+    try:
+        for t in range(4):
+            g = _grads(rng, W, n)
+            backing = torch.zeros(W, n + 8, device="cuda")
+            views = [backing[i, 1 + i:1 + i + n] for i in range(W)]     # 4- and 8-byte offsets
+            for i in range(W):
+                views[i].copy_(torch.from_numpy(g[i]))
+            assert any(v.data_ptr() % 16 for v in views)
+            p.gpu.step_auto(views, 1e-3, t)
+            torch.cuda.synchronize()
+            p.cpu.step(g, np.float32(1e-3), t, p.gpu.sync_due(t), p.gpu.var_due(t))
+            p.compare(f"t={t}", wire=False)
+    finally:
+        p.close()
+
+
+def test_checkpoint_round_trip():
+    """k steps, export, import into a fresh handle, k more steps == 2k steps."""
+    rng = np.random.default_rng(6)
+    n, W, chunk = 5000, 3, 512
+    gs = [_grads(rng, W, n) for _ in range(8)]
+    x0 = torch.from_numpy((rng.standard_normal(n) * 0.02).astype(np.float32))
+    pol = ((0, 1, 5), (0, 2), (1, 3))
+    a, b = Zoa(n, W, chunk=chunk), Zoa(n, W, chunk=chunk)
+    try:
+        a.set_params(x0), a.set_policies(*pol), b.set_policies(*pol)
+        for t in range(4):
+            a.step_auto(list(torch.from_numpy(gs[t]).cuda()), 1e-3, t)
+        st = a.stats()
+        for name in ("x", "m", "u", "delta_w"):
+            for i in range(W):
+                b.write(name, a.read(name, i), i)
+        for name in ("v", "delta_s", "x_sync"):
+            b.write(name, a.read(name))
+        B.zoa_set_scalars(b.h, st["gamma_sum"], st["t_sync"], st["t_last"])
+        for t in range(4, 8):
+            g = list(torch.from_numpy(gs[t]).cuda())
+            a.step_auto(g, 1e-3, t), b.step_auto(g, 1e-3, t)
+        torch.cuda.synchronize()
+        for name in ("x", "m", "u", "delta_w"):
+            for i in range(W):
+                assert np.array_equal(a.read(name, i), b.read(name, i)), name
+        for name in ("v", "delta_s", "x_sync"):
+            assert np.array_equal(a.read(name), b.read(name)), name
+    finally:
+        a.close(), b.close()
+
+
+def test_host_gradient_entry_point():
+    rng = np.random.default_rng(8)
+    n, W, chunk = 4096 + 100, 2, 1024
+    a, b = Zoa(n, W, chunk=chunk), Zoa(n, W, chunk=chunk)
+    try:
+        for t in range(3):
+            g = torch.from_numpy(_grads(rng, W, n)).pin_memory()
+            out = torch.empty(n).pin_memory()
+            a.step_host(list(g), 1e-3, t, out)
+            b.step_auto(list(g.cuda()), 1e-3, t)
+            torch.cuda.synchronize()
+            assert np.array_equal(out.numpy(), b.read("x", 0))
+            assert np.array_equal(a.read("m", 1), b.read("m", 1))
+    finally:
+        a.close(), b.close()
+
+
+def test_argument_and_state_errors():
+    with pytest.raises(ZoaError) as e:
+        Zoa(100, 0)
+    assert e.value.status == B.ERR_ARG
+    for kw in (dict(chunk=48), dict(chunk=16), dict(chunk=32768), dict(beta1=1.0), dict(eps=0.0)):
+        with pytest.raises(ZoaError):
+            Zoa(100, 2, **kw)
+    z = Zoa(100, 2, chunk=32)
+    try:
+        with pytest.raises(ZoaError) as e:
+            z.onebit_reduce()                       # nothing accumulated: line 8 would divide by zero
+        assert e.value.status == B.ERR_STATE
+        g = list(torch.zeros(2, 100, device="cuda"))
+        z.step(g, 1e-3, 5)
+        with pytest.raises(ZoaError) as e:
+            z.step(g, 1e-3, 5)                      # t must increase
+        assert e.value.status == B.ERR_STATE
+        with pytest.raises(ZoaError):
+            z.step(g, float("nan"), 6)
+        with pytest.raises(ZoaError) as e:
+            z.step_sync(g, -1.0, 7)                 # the sum of learning rates would not be positive
+        assert e.value.status == B.ERR_STATE
+        z.onebit_reduce()
+        with pytest.raises(ZoaError):
+            z.onebit_reduce()
+        with pytest.raises(ZoaError):
+            z.read("x", worker=2)
+        z.check_device()
+        s = z.stats()
+        assert s["n_steps"] == 1 and s["n_syncs"] == 1 and s["n_launches"] == 3
+        assert s["bits_per_worker"] == 100 + 32 * 4
+    finally:
+        z.close()
+
+
+def test_policies_match_the_workload_tables():
+    for make in synth.WORKLOADS.values():
+        wl = synth.scaled(make(), 1 << 14)
+        z = Zoa(wl.n, wl.W, chunk=wl.chunk)
+        try:
+            z.set_policies(wl.var_steps, wl.sync_boundaries, wl.sync_intervals)
+            for t in range(wl.steps):
+                assert z.sync_due(t) == wl.in_T_u(t) and z.var_due(t) == wl.in_T_v(t)
+        finally:
+            z.close()
+    z = Zoa(64, 1, chunk=32)
+    try:
+        B.zoa_set_var_policy_doubling(z.h, 2, 40)   # gaps 1,1,2,2,4,4,8,8,...
+        got = [t for t in range(60) if z.var_due(t)]
+        assert got == [0, 1, 2, 4, 6, 10, 14, 22, 30]
+    finally:
+        z.close()
