@@ -222,7 +222,7 @@ def run_ours(args, wl):
 
     # ---- end to end: host gradients in, worker 0's model out, through zoa_step_host ----
     e2e = None
-    if rank == 0 or world > 1:
+    if args.e2e_steps > 0:
         ke = max(1, min(args.e2e_steps, K))
         host_g = torch.empty(wl.n, dtype=torch.float32).pin_memory()
         host_g.copy_(stream.bufs[0])
@@ -280,6 +280,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-sample", type=int, default=1 << 22, help="parameters in the oracle's timed sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--scale", type=int, default=1, help="shrink every tensor by this factor (profiling captures)")
     args = ap.parse_args()
 
     if args.impl == "reference":
@@ -290,12 +291,16 @@ def main():
         sys.modules["_synth"] = synth
         spec.loader.exec_module(synth)
         wl = synth.WORKLOADS[args.workload]()
+        if args.scale > 1:
+            wl = synth.scaled(wl, args.scale)
         if args.steps is None:
             args.steps = wl.steps
         return run_reference(args, wl)
 
     from paper_2202_06009_b200 import synth
     wl = synth.WORKLOADS[args.workload]()
+    if args.scale > 1:
+        wl = synth.scaled(wl, args.scale)
     if args.steps is None:
         args.steps = wl.steps
     run_ours(args, wl)
