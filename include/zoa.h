@@ -85,7 +85,7 @@ zoa_status zoa_set_params(zoa_handle h, const float *x0, void *stream);
  * Default: empty (the variance is never updated). */
 zoa_status zoa_set_var_steps(zoa_handle h, const int64_t *steps, size_t count);
 
-/* T_v by the rule of Section 6 ("Policy for T_v and T_u"): the j-th update is
+/* T_v by the rule of the paragraph "Policy for T_v and T_u": the j-th update is
  * at k_j with k_0 = 0 and k_{j+1} - k_j = 2^floor(j / kappa), for k_j < freeze_at. */
 zoa_status zoa_set_var_policy_doubling(zoa_handle h, int kappa, int64_t freeze_at);
 
@@ -158,6 +158,41 @@ zoa_status zoa_check_device(zoa_handle h);
 /* Text of the last error on this handle (or of the last failed zoa_create if h
  * is NULL).  Never NULL. */
 const char *zoa_last_error(zoa_handle h);
+
+/* (The paper has no counterpart to this entry point; it exists for callers that
+ * must not allocate device memory.)
+ * The error-feedback 1-bit AllReduce of Algorithm 3 on buffers the caller owns,
+ * without a handle and without allocating anything: no cudaMalloc, cudaFree or
+ * allocating library call is made.  It is meant for code that runs where
+ * device allocation is forbidden or harmful - inside a region whose memory a
+ * framework's allocator has already handed out, in a latency-critical loop that
+ * cannot afford cudaMalloc's implicit synchronisation, in a process whose
+ * memory is pre-partitioned between tenants, or in a clean-up path that runs
+ * when the device is already full.
+ *   z        (host) array of W (device) pointers, n floats each: the buffers to reduce, read-only
+ *   delta_w  (host) array of W (device) pointers, n floats each: worker errors, updated in place
+ *   delta_s  (device) n floats: server error, updated in place
+ *   z_bar    (device) n floats: the result, +-magnitude of the server's chunk
+ * The packed sign words and magnitudes that travel between the two kernels of
+ * a call live in an array built into the library (1,048,576 32-bit slots, 4 MiB,
+ * held by every GPU that loads the library until the process exits).  The call
+ * needs W * (ceil(n/32) + ceil(n/chunk)) slots and returns ZOA_ERR_ARG, with a
+ * text in zoa_static_last_error(), if that is more.  All calls on a device share
+ * the array: calls whose GPU work may overlap (different streams without
+ * ordering) race on it and must be serialised by the caller.  The array keeps
+ * the last call's contents; a call reads only what it wrote itself, so nothing
+ * needs clearing.  The first call on each device looks up the array's device
+ * address and raises two kernels' shared-memory limit: make that first call
+ * before any stream capture starts.  Pointers that are all 16-byte aligned take
+ * the 128-bit path, others a scalar one.  Work is enqueued on `stream`; the
+ * call does not synchronise. */
+zoa_status zoa_onebit_allreduce_static(const float *const *z, float *const *delta_w, float *delta_s,
+                                       float *z_bar, size_t n, int W, int chunk, void *stream);
+
+/* Capacity of that built-in array in 32-bit slots, and the text of the last
+ * error zoa_onebit_allreduce_static returned on this thread (never NULL). */
+size_t zoa_static_scratch_slots(void);
+const char *zoa_static_last_error(void);
 
 #ifdef __cplusplus
 }

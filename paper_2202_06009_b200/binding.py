@@ -55,6 +55,9 @@ def _load():
         "zoa_get_stats": ([H, C.POINTER(Stats)], C.c_int),
         "zoa_check_device": ([H], C.c_int),
         "zoa_last_error": ([H], C.c_char_p),
+        "zoa_onebit_allreduce_static": ([C.POINTER(p), C.POINTER(p), p, p, C.c_size_t, C.c_int, C.c_int, p], C.c_int),
+        "zoa_static_scratch_slots": ([], C.c_size_t),
+        "zoa_static_last_error": ([], C.c_char_p),
     }
     for name, (argtypes, restype) in sigs.items():
         fn = getattr(lib, name)
@@ -158,3 +161,15 @@ def zoa_get_stats(h):
 
 def zoa_check_device(h):
     _check(h, lib.zoa_check_device(h))
+
+
+def zoa_onebit_allreduce_static(z_ptrs, delta_w_ptrs, delta_s_ptr, z_bar_ptr, n, W, chunk, stream=0):
+    """Algorithm 3 on caller-owned device buffers, allocating nothing (see include/zoa.h)."""
+    status = lib.zoa_onebit_allreduce_static(_ptr_array(z_ptrs), _ptr_array(delta_w_ptrs), delta_s_ptr,
+                                             z_bar_ptr, n, W, chunk, stream)
+    if status != OK:
+        raise ZoaError(status, lib.zoa_static_last_error().decode())
+
+
+def zoa_static_scratch_slots():
+    return lib.zoa_static_scratch_slots()
