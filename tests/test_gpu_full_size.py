@@ -1,0 +1,94 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py
+times.  The method is chunk-local (every reduction stays inside one chunk), so
+the oracle runs on a sample of chunks - the first, the ragged last, chunks that
+straddle tensor boundaries, random ones - gathered into one short vector, and is
+compared with the same chunks of the full-size GPU state."""
+import numpy as np
+import pytest
+import torch
+
+from helpers import assert_close
+from oracle import zoa_oracle as zo
+from paper_2202_06009_b200 import Zoa, synth
+
+pytestmark = pytest.mark.gpu
+
+
+def _sample_chunks(wl, count, seed):
+    n_chunks = -(-wl.n // wl.chunk)
+    picks = {0, 1, n_chunks - 2}
+    off = 0
+    for size in wl.tensors[:40]:                      # chunks that straddle a tensor boundary
+        off += size
+        picks.add(min(off // wl.chunk, n_chunks - 2))
+    rng = np.random.default_rng(seed)
+    while len(picks) < count - 1:
+        picks.add(int(rng.integers(0, n_chunks - 1)))
+    return sorted(picks)[:count - 1] + [n_chunks - 1]    # the ragged last chunk stays last
+
+
+def _run(wl, steps, check_at, n_sample=40):
+    torch.cuda.empty_cache()
+    free, _ = torch.cuda.mem_get_info()
+    need = (5 * wl.W + 6) * wl.n * 4
+    if free < need * 1.03:
+        pytest.skip(f"needs {need / 1e9:.0f} GB of device memory, {free / 1e9:.0f} GB free")
+    chunks = _sample_chunks(wl, n_sample, 7)
+    spans = [(c * wl.chunk, min((c + 1) * wl.chunk, wl.n)) for c in chunks]
+    idx = torch.cat([torch.arange(a, b, device="cuda") for a, b in spans])
+    d = idx.numel()
+    stream = synth.GradientStream(wl, "cuda")
+    x0 = synth.initial_params(wl, "cuda")
+    cpu = zo.Oracle(d, wl.W, wl.chunk, wl.beta1, wl.beta2, wl.eps, dtype=np.float32)
+    cpu.set_params(x0[idx].cpu().numpy())
+    gpu = Zoa(wl.n, wl.W, wl.beta1, wl.beta2, wl.eps, wl.chunk)
+    try:
+        gpu.set_params(x0)
+        del x0
+        gpu.set_policies(wl.var_steps, wl.sync_boundaries, wl.sync_intervals)
+
+        def gather(name, worker=0):
+            return np.concatenate([gpu.read(name, worker, a, b - a) for a, b in spans])
+
+        for t in range(steps):
+            bufs = stream.fill(t)
+            g = np.stack([b[idx].cpu().numpy() for b in bufs])
+            gpu.step_auto(bufs, wl.lr_at(t), t)
+            assert cpu.step(g, np.float32(wl.lr_at(t)), t, wl.in_T_u(t), wl.in_T_v(t)) == 0
+            if t in check_at:
+                torch.cuda.synchronize()
+                for i in range(wl.W):
+                    assert_close(gather("x", i), cpu.x[i], f"t={t} x[{i}]")
+                    assert_close(gather("m", i), cpu.m[i], f"t={t} m[{i}]")
+                    assert_close(gather("u", i), cpu.u[i], f"t={t} u[{i}]")
+                    assert_close(gather("delta_w", i), cpu.delta[i], f"t={t} delta_w[{i}]")
+                assert_close(gather("v"), cpu.v, f"t={t} v")
+                assert_close(gather("delta_s"), cpu.delta_bar, f"t={t} delta_s")
+                assert_close(gather("x_sync"), cpu.x_sync, f"t={t} x_sync")
+                if wl.in_T_u(t):
+                    # packed words, bit-exact: oracle word k of sampled chunk j <-> GPU word (start_j/32 + k)
+                    per = wl.chunk // 32
+                    for j, (a, b) in enumerate(spans):
+                        nw = -(-(b - a) // 32)
+                        for i in (0, wl.W - 1):
+                            assert np.array_equal(gpu.read("words_w", i, a // 32, nw),
+                                                  cpu.words_worker[i][j * per:j * per + nw]), (t, j, i)
+                        assert np.array_equal(gpu.read("words_s", 0, a // 32, nw),
+                                              cpu.words_server[j * per:j * per + nw]), (t, j)
+                    got = np.array([gpu.read("scales_s", 0, c, 1)[0] for c in chunks])
+                    assert_close(got, cpu.scales_server, f"t={t} scales_s")
+        gpu.check_device()
+    finally:
+        gpu.close()
+        del stream
+        torch.cuda.empty_cache()
+
+
+def test_bert_large_full_size_sampled_chunks():
+    """336,226,108 parameters, W = 16, chunk 4096, all 100 steps of the schedule."""
+    _run(synth.bert_large(), 100, {0, 1, 2, 5, 17, 33, 63, 64, 65, 66, 67, 99})
+
+
+def test_gpt2_full_size_sampled_chunks():
+    """1,557,611,200 parameters, W = 4, chunk 8192, Student-t noise; first 22 steps (sync, local and variance steps)."""
+    _run(synth.gpt2_xl(), 22, {0, 3, 15, 16, 17, 19, 20, 21}, n_sample=24)
