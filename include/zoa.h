@@ -155,6 +155,13 @@ zoa_status zoa_get_stats(zoa_handle h, zoa_stats *out);
  * of this handle failed since the last check. */
 zoa_status zoa_check_device(zoa_handle h);
 
+/* Tuning switches.  ZOA_OPT_PIPELINE (default 1): run the fused sync step as the
+ * persistent bulk-copy-ring kernel where the shape allows (chunk 2048, 4096 or
+ * 8192, 16-byte aligned gradients); 0 forces the chunk-per-block kernel.  The
+ * results are the same bit for bit. */
+enum { ZOA_OPT_PIPELINE = 1 };
+zoa_status zoa_set_option(zoa_handle h, int option, int value);
+
 /* Text of the last error on this handle (or of the last failed zoa_create if h
  * is NULL).  Never NULL. */
 const char *zoa_last_error(zoa_handle h);

@@ -55,6 +55,7 @@ def _load():
         "zoa_get_stats": ([H, C.POINTER(Stats)], C.c_int),
         "zoa_check_device": ([H], C.c_int),
         "zoa_last_error": ([H], C.c_char_p),
+        "zoa_set_option": ([H, C.c_int, C.c_int], C.c_int),
         "zoa_onebit_allreduce_static": ([C.POINTER(p), C.POINTER(p), p, p, C.c_size_t, C.c_int, C.c_int, p], C.c_int),
         "zoa_static_scratch_slots": ([], C.c_size_t),
         "zoa_static_last_error": ([], C.c_char_p),
@@ -157,6 +158,13 @@ def zoa_get_stats(h):
     s = Stats()
     _check(h, lib.zoa_get_stats(h, C.byref(s)))
     return {name: getattr(s, name) for name, _ in Stats._fields_}
+
+
+OPT_PIPELINE = 1
+
+
+def zoa_set_option(h, option, value):
+    _check(h, lib.zoa_set_option(h, option, value))
 
 
 def zoa_check_device(h):

@@ -23,6 +23,9 @@ struct zoa_handle_s {
     uint32_t *words_w = nullptr, *words_s = nullptr;
     float *scales_w = nullptr, *scales_s = nullptr;
     float *staging = nullptr;      // [W][n_pad], device copy of host gradients (zoa_step_host)
+    int *error_flag = nullptr;     // device int: a kernel gave up on a bounded wait
+    unsigned long long *sched = nullptr;   // device [2]: chunk counter of the persistent kernel, finished blocks
+    bool use_pipeline = true;      // bulk-copy ring form of the fused sync step where the shape allows
     bool v_pending = false;        // v_nxt holds v_{t+1}; it becomes v at the next step
     std::vector<int64_t> var_steps;                    // T_v, sorted
     std::vector<int64_t> sync_bounds{0};               // T_u pieces
@@ -65,7 +68,7 @@ static StateView view(zoa_handle h)
 static void free_all(zoa_handle h)
 {
     void *ptrs[] = {h->x, h->m, h->u, h->dw, h->v_cur, h->v_nxt, h->ds, h->xs,
-                    h->words_w, h->words_s, h->scales_w, h->scales_s, h->staging};
+                    h->words_w, h->words_s, h->scales_w, h->scales_s, h->staging, h->error_flag, h->sched};
     for (void *p : ptrs)
         if (p) cudaFree(p);
 }
@@ -116,7 +119,8 @@ extern "C" zoa_status zoa_create(zoa_handle *out, size_t n_params, int W, float 
         (e = alloc_zero(&h->words_w, (size_t)W * h->words_stride)) == cudaSuccess &&
         (e = alloc_zero(&h->words_s, (size_t)h->words_stride)) == cudaSuccess &&
         (e = alloc_zero(&h->scales_w, (size_t)W * h->n_chunks)) == cudaSuccess &&
-        (e = alloc_zero(&h->scales_s, (size_t)h->n_chunks)) == cudaSuccess)
+        (e = alloc_zero(&h->scales_s, (size_t)h->n_chunks)) == cudaSuccess &&
+        (e = alloc_zero(&h->error_flag, 1)) == cudaSuccess && (e = alloc_zero(&h->sched, 2)) == cudaSuccess)
         e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
         free_all(h);
@@ -280,11 +284,29 @@ extern "C" zoa_status zoa_step_sync(zoa_handle h, const float *const *grads, flo
     commit_variance(h);
     const bool do_var = zoa_var_due(h, t) == 1;
     const StateView st = view(h);
-    ZOA_CUDA(h, launch_step_sync(st, gp, h->c, lr, gamma_sum, aligned, s));
-    h->n_launches += 1;
-    if (do_var) {
-        ZOA_CUDA(h, launch_variance(st, gp, h->c, aligned, h->sm_count, s));
+    const int stages = h->use_pipeline ? pipeline_stages(st, aligned) : 0;
+    long long var_first = 0;     // coordinates from here on still need lines 14-15
+    if (stages > 0) {
+        // Full chunks through the bulk-copy ring; a ragged last chunk through the chunk-per-block kernel.
+        const long long n_full = h->n / h->chunk;
+        bool var_fused = false;
+        ZOA_CUDA(h, launch_step_sync_pipelined(st, gp, h->c, lr, gamma_sum, do_var, stages, h->sm_count,
+                                               h->error_flag, h->sched, &var_fused, s));
         h->n_launches += 1;
+        if (n_full < h->n_chunks) {
+            ZOA_CUDA(h, launch_step_sync(st, gp, h->c, lr, gamma_sum, aligned, n_full, h->n_chunks - n_full, s));
+            h->n_launches += 1;
+        }
+        var_first = var_fused ? n_full * h->chunk : 0;
+    } else {
+        ZOA_CUDA(h, launch_step_sync(st, gp, h->c, lr, gamma_sum, aligned, 0, h->n_chunks, s));
+        h->n_launches += 1;
+    }
+    if (do_var) {
+        if (var_first < h->n) {
+            ZOA_CUDA(h, launch_variance(st, gp, h->c, aligned, var_first, h->sm_count, s));
+            h->n_launches += 1;
+        }
         h->v_pending = true;
         h->n_var_updates += 1;
     }
@@ -419,6 +441,21 @@ extern "C" zoa_status zoa_check_device(zoa_handle h)
     if (!h) return ZOA_ERR_ARG;
     ZOA_CUDA(h, cudaDeviceSynchronize());
     ZOA_CUDA(h, cudaGetLastError());
+    int flag = 0;
+    ZOA_CUDA(h, cudaMemcpy(&flag, h->error_flag, sizeof(int), cudaMemcpyDeviceToHost));
+    if (flag) {
+        cudaMemset(h->error_flag, 0, sizeof(int));
+        cudaMemset(h->sched, 0, 2 * sizeof(unsigned long long));
+        return fail(h, ZOA_ERR_DEVICE, "a kernel gave up waiting for its asynchronous copies; the optimizer state is undefined");
+    }
+    return ZOA_OK;
+}
+
+extern "C" zoa_status zoa_set_option(zoa_handle h, int option, int value)
+{
+    if (!h) return ZOA_ERR_ARG;
+    if (option != ZOA_OPT_PIPELINE) return fail(h, ZOA_ERR_ARG, "zoa_set_option: unknown option");
+    h->use_pipeline = value != 0;
     return ZOA_OK;
 }
 

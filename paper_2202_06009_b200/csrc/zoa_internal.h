@@ -10,10 +10,16 @@ cudaError_t configure_kernels();
 cudaError_t launch_local_step(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
                               bool do_var, bool g_aligned, int sm_count, cudaStream_t s);
 cudaError_t launch_variance(const StateView &st, const GradPtrs &g, const Consts &c, bool g_aligned,
-                            int sm_count, cudaStream_t s);
+                            long long first, int sm_count, cudaStream_t s);
 cudaError_t launch_compress(const StateView &st, cudaStream_t s);
 cudaError_t launch_reduce(const StateView &st, const Consts &c, float gamma_sum, cudaStream_t s);
 cudaError_t launch_step_sync(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
-                             float gamma_sum, bool g_aligned, cudaStream_t s);
+                             float gamma_sum, bool g_aligned, long long first_chunk, long long count, cudaStream_t s);
+
+// Pipelined (bulk-copy ring) form of the fused sync step, zoa_pipeline.cu.
+int pipeline_stages(const StateView &st, bool g_aligned);
+cudaError_t launch_step_sync_pipelined(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
+                                       float gamma_sum, bool do_var, int stages, int sm_count, int *error_flag,
+                                       unsigned long long *sched, bool *var_fused, cudaStream_t s);
 
 }  // namespace zoa

@@ -58,11 +58,11 @@ local_step_kernel(StateView st, GradPtrs g, Consts c, float gamma, int g_aligned
 }
 
 __global__ void __launch_bounds__(256)
-variance_kernel(StateView st, GradPtrs g, Consts c, int g_aligned)
+variance_kernel(StateView st, GradPtrs g, Consts c, int g_aligned, long long first4)
 {
     const long long n4 = (st.n + 3) >> 2;
     const long long stride = (long long)gridDim.x * blockDim.x;
-    for (long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x; q < n4; q += stride) {
+    for (long long q = first4 + (long long)blockIdx.x * blockDim.x + threadIdx.x; q < n4; q += stride) {
         const long long j = q << 2;
         double G[4] = {0.0, 0.0, 0.0, 0.0};
         for (int i = 0; i < st.W; ++i) {
@@ -355,10 +355,12 @@ cudaError_t launch_local_step(const StateView &st, const GradPtrs &g, const Cons
     return cudaGetLastError();
 }
 
+// Lines 14-15 for the coordinates [first, n); first is a multiple of 4.
 cudaError_t launch_variance(const StateView &st, const GradPtrs &g, const Consts &c, bool g_aligned,
-                            int sm_count, cudaStream_t s)
+                            long long first, int sm_count, cudaStream_t s)
 {
-    variance_kernel<<<elementwise_grid((st.n + 3) / 4, sm_count), 256, 0, s>>>(st, g, c, g_aligned);
+    const long long first4 = first >> 2;
+    variance_kernel<<<elementwise_grid((st.n + 3) / 4 - first4, sm_count), 256, 0, s>>>(st, g, c, g_aligned, first4);
     return cudaGetLastError();
 }
 
@@ -389,11 +391,12 @@ cudaError_t launch_reduce(const StateView &st, const Consts &c, float gamma_sum,
     return cudaGetLastError();
 }
 
+// The chunks [first_chunk, first_chunk + count) of a sync step, one block each.
 cudaError_t launch_step_sync(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
-                             float gamma_sum, bool g_aligned, cudaStream_t s)
+                             float gamma_sum, bool g_aligned, long long first_chunk, long long count, cudaStream_t s)
 {
-    step_sync_kernel<<<(unsigned)st.n_chunks, block_threads_for_chunk(st.chunk), step_sync_smem(st.chunk), s>>>(
-        st, g, c, gamma, gamma_sum, g_aligned, 0);
+    step_sync_kernel<<<(unsigned)count, block_threads_for_chunk(st.chunk), step_sync_smem(st.chunk), s>>>(
+        st, g, c, gamma, gamma_sum, g_aligned, first_chunk);
     return cudaGetLastError();
 }
 

@@ -1,0 +1,499 @@
+// step_sync_pipelined_kernel: the fused sync step (Algorithm 1 lines 3-11 with
+// Algorithm 3 inside) as a persistent, warp-specialised kernel for sm_100a.
+//
+// One block per SM takes chunks from a global counter (SMs do not all get the same
+// share of DRAM bandwidth, so a fixed split would leave the fast ones idle at the
+// end).  A producer warp streams
+// the inputs of each (chunk, worker) - tiles of 2048 coordinates of g, m, u and
+// the worker error - through a ring of shared-memory stages with 1-D bulk
+// asynchronous copies (cp.async.bulk ... mbarrier::complete_tx), several stages
+// ahead of the 512 consumer threads, so DRAM reads stay in flight while the
+// consumers sit in the block-wide l1 sums.  After the W workers of a chunk come
+// tiles of (server error, v, x_sync) for the server part.  Consumers keep a
+// chunk's z in registers (thread t owns coordinates 4t..4t+3 of every tile), so
+// shared memory holds only the ring, the packed bits and the magnitudes.
+//
+// Every wait on an mbarrier is bounded: after about two seconds a thread gives
+// up, raises the block's abort flag and the handle's device error flag, the
+// block stops issuing copies, waits (bounded) for those in flight and leaves.
+#include "zoa_internal.h"
+
+namespace zoa {
+
+namespace {
+
+constexpr int kConsumers = 512;                 // consumer threads (16 warps)
+constexpr int kConsumerWarps = kConsumers / 32;
+constexpr int kThreads = kConsumers + 32;       // + one producer warp
+constexpr int kTile = 4 * kConsumers;           // coordinates per ring stage and array
+constexpr int kTileBytes = kTile * 4;
+constexpr int kStageBytes = 4 * kTileBytes;     // g, m, u, delta  |  delta_bar, v, x_sync, (unused)
+constexpr int kMaxStages = 6;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+
+struct PipeArgs {
+    StateView st;
+    GradPtrs g;
+    Consts c;
+    float gamma, gamma_sum;
+    long long n_full_chunks;
+    int stages;
+    int *error_flag;  // device int, set non-zero when a wait ran out
+    unsigned long long *sched;  // device: [0] next chunk to hand out, [1] blocks that have finished
+};
+
+// Shared-memory header (the ring follows, 1024-byte aligned).
+struct PipeShared {
+    unsigned long long full[kMaxStages];
+    unsigned long long empty[kMaxStages];
+    double sums[2][kConsumerWarps];
+    long long chunk_queue[kMaxStages + 2];   // chunk ids in the order the producer took them; -1 = no more
+    int abort;
+};
+
+__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_timer_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait.  Returns false if the block has been aborted or the limit ran out
+// (in which case it raises both flags).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *error_flag)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long start = global_timer_ns();
+    for (unsigned it = 1;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if ((it & 63u) == 0 && global_timer_ns() - start > kWaitLimitNs) {
+            *abort_flag = 1;
+            atomicExch(error_flag, 1);
+            return false;
+        }
+    }
+}
+// 1-D bulk asynchronous copy global -> this block's shared memory, completion counted on `bar`.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ void consumer_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory"); }
+// Barrier over the consumers that also tells every one of them whether any had `flag` set.
+__device__ __forceinline__ bool consumer_any(bool flag)
+{
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "bar.red.or.pred p, 1, %2, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(out)
+        : "r"((uint32_t)flag), "n"(kConsumers)
+        : "memory");
+    return out != 0;
+}
+
+// Sum over the 512 consumers in binary64; every consumer gets the same value.
+// One named barrier per call (the two partial-sum arrays alternate).
+__device__ __forceinline__ double consumer_sum(double v, PipeShared *sh, int &flip)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    if ((threadIdx.x & 31) == 0) sh->sums[flip][threadIdx.x >> 5] = v;
+    consumer_barrier();
+    double t = 0.0;
+#pragma unroll
+    for (int w = 0; w < kConsumerWarps; ++w) t += sh->sums[flip][w];
+    flip ^= 1;
+    return t;
+}
+
+// Packs the sign bits of a float4-per-lane tile: lane l holds coordinates 4l..4l+3,
+// eight lanes make one word.  Returns the word in every lane of the 8-lane group.
+__device__ __forceinline__ uint32_t pack_group(const bool b[4])
+{
+    const int lane = threadIdx.x & 31;
+    const uint32_t nib = (b[0] ? 1u : 0u) | (b[1] ? 2u : 0u) | (b[2] ? 4u : 0u) | (b[3] ? 8u : 0u);
+    return __reduce_or_sync(0xFFu << (lane & 24), nib << ((lane & 7) * 4));
+}
+
+#ifdef ZOA_PIPE_PROFILE
+__device__ unsigned long long g_pipe_prof[256][8];
+#define PROF_T0() const long long prof_t0_ = clock64()
+#define PROF_ADD(slot) do { if (tid == 0) prof[slot] += clock64() - prof_t0_; } while (0)
+#else
+#define PROF_T0() do {} while (0)
+#define PROF_ADD(slot) do {} while (0)
+#endif
+
+}  // namespace
+
+#ifdef ZOA_PIPE_PROFILE
+extern "C" int zoa_debug_read_pipe_profile(unsigned long long *out)
+{
+    return (int)cudaMemcpyFromSymbol(out, g_pipe_prof, sizeof(g_pipe_prof));
+}
+#endif
+
+template <int TILES, bool DO_VAR>
+__global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const __grid_constant__ PipeArgs a)
+{
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    PipeShared *sh = reinterpret_cast<PipeShared *>(smem_raw);
+    const StateView &st = a.st;
+    const int W = st.W;
+    const int words_per_chunk = st.chunk >> 5;
+    uint32_t *bits_s = reinterpret_cast<uint32_t *>(smem_raw + 1024);                 // [W][words_per_chunk]
+    float *scales_s = reinterpret_cast<float *>(bits_s + W * words_per_chunk);         // [kConsumerWarps][W]
+    unsigned char *ring = smem_raw + ((1024 + (size_t)W * words_per_chunk * 4 + (size_t)kConsumerWarps * W * 4 + 1023) & ~(size_t)1023);
+    const int R = a.stages;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    volatile int *abort_flag = &sh->abort;
+
+    if (tid == 0) {
+        for (int s = 0; s < R; ++s) {
+            mbar_init(smem_addr(&sh->full[s]), 1);
+            mbar_init(smem_addr(&sh->empty[s]), kConsumerWarps);
+        }
+        sh->abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+
+    if (warp == kConsumerWarps) {
+        // ------------------------------ producer ------------------------------
+        if (lane != 0) return;
+        int s = 0;
+        uint32_t phase = 0;
+        long long issued = 0;
+        bool ok = true;
+        for (long long k = 0; ok; ++k) {
+            const long long chunk = (long long)atomicAdd(&a.sched[0], 1ull);
+            const bool last = chunk >= a.n_full_chunks;
+            // The chunk id travels to the consumers through shared memory; the arrive on the
+            // first tile's barrier below publishes it.  The queue cannot wrap onto an unread
+            // entry: the producer is at most `stages` tiles, hence chunks, ahead.
+            if (!mbar_wait(smem_addr(&sh->empty[s]), phase ^ 1u, abort_flag, a.error_flag)) { ok = false; break; }
+            sh->chunk_queue[k % (kMaxStages + 2)] = last ? -1 : chunk;
+            if (last) {
+                mbar_arrive(smem_addr(&sh->full[s]));       // an empty "tile": wakes the consumers to read the -1
+                break;
+            }
+            const long long c0 = chunk * st.chunk;
+            for (int i = 0; ok && i <= W; ++i) {            // i == W: the server's tiles
+                for (int t = 0; t < TILES; ++t) {
+                    const uint32_t full = smem_addr(&sh->full[s]);
+                    if (!mbar_wait(smem_addr(&sh->empty[s]), phase ^ 1u, abort_flag, a.error_flag)) { ok = false; break; }
+                    const uint32_t dst = smem_addr(ring + (size_t)s * kStageBytes);
+                    const long long off = c0 + (long long)t * kTile;
+                    if (i < W) {
+                        const long long row = (long long)i * st.n_pad + off;
+                        mbar_arrive_expect_tx(full, 4 * kTileBytes);
+                        bulk_load(dst, a.g.p[i] + off, kTileBytes, full);
+                        bulk_load(dst + kTileBytes, st.m + row, kTileBytes, full);
+                        bulk_load(dst + 2 * kTileBytes, st.u + row, kTileBytes, full);
+                        bulk_load(dst + 3 * kTileBytes, st.dw + row, kTileBytes, full);
+                    } else {
+                        mbar_arrive_expect_tx(full, 3 * kTileBytes);
+                        bulk_load(dst, st.ds + off, kTileBytes, full);
+                        bulk_load(dst + kTileBytes, st.v + off, kTileBytes, full);
+                        bulk_load(dst + 2 * kTileBytes, st.xs + off, kTileBytes, full);
+                    }
+                    ++issued;
+                    if (++s == R) { s = 0; phase ^= 1u; }
+                }
+            }
+        }
+        if (!ok) {
+            // Aborted: let the copies still in flight land before the block's shared memory is released.
+            const long long outstanding = issued < R ? issued : R;
+            for (long long k = 1; k <= outstanding; ++k) {
+                const long long q = issued - k;                      // sequence number of an issued tile
+                const uint32_t bar = smem_addr(&sh->full[q % R]);
+                const uint32_t par = (uint32_t)((q / R) & 1);
+                const unsigned long long start = global_timer_ns();
+                while (!mbar_try_wait(bar, par) && global_timer_ns() - start < kWaitLimitNs) {}
+            }
+        }
+        // The last block to finish taking chunks rearms the counters for the next launch.
+        if (atomicAdd(&a.sched[1], 1ull) == gridDim.x - 1) {
+            a.sched[0] = 0;
+            a.sched[1] = 0;
+        }
+        return;
+    }
+
+    // -------------------------------- consumers --------------------------------
+#ifdef ZOA_PIPE_PROFILE
+    unsigned long long prof[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    const long long prof_start = clock64();
+#endif
+    int s = 0;
+    uint32_t phase = 0;
+    int flip = 0;
+    const int pos = 4 * tid;                         // this thread's coordinates inside every tile
+    const int word_in_tile = pos >> 5;               // = warp * 4 + (lane >> 3)
+    const bool group_leader = (lane & 7) == 0;
+    float *my_scales = scales_s + warp * W;
+
+    // Lines 8-10 of the previous chunk, carried in registers: its 3 W tile stores are
+    // spread over the worker iterations of the next chunk (one worker's m, x, u after
+    // each worker's compression) instead of leaving in one burst, so that the block's
+    // stores and its ring's loads stay evenly mixed.  m is +-m_pos by the server's bit.
+    float x_prev[TILES][4];
+    uint32_t bits_prev = 0;
+    float m_pos_prev = 0.0f;
+    long long c0_prev = -1;
+    auto store_prev_worker = [&](int i) {
+        const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int t = 0; t < TILES; ++t) {
+            const long long row = (long long)i * st.n_pad + c0_prev + t * kTile + pos;
+            const uint32_t nib = bits_prev >> (4 * t);
+            st4_stream(st.m + row, make_float4((nib & 1u) ? m_pos_prev : -m_pos_prev, (nib & 2u) ? m_pos_prev : -m_pos_prev,
+                                               (nib & 4u) ? m_pos_prev : -m_pos_prev, (nib & 8u) ? m_pos_prev : -m_pos_prev));
+            st4_stream(st.x + row, make_float4(x_prev[t][0], x_prev[t][1], x_prev[t][2], x_prev[t][3]));
+            st4_stream(st.u + row, zero);                                      // line 10
+        }
+    };
+
+    for (long long k = 0;; ++k) {
+        // The first tile's barrier also publishes the chunk id (or the end mark).  Leaving the
+        // loop must be unanimous (the block sums below count on all 512 consumers), so a
+        // wait that ran out is put to the vote.
+        const bool gave_up = !mbar_wait(smem_addr(&sh->full[s]), phase, abort_flag, a.error_flag);
+        if (consumer_any(gave_up)) break;
+        const long long chunk = sh->chunk_queue[k % (kMaxStages + 2)];
+        if (chunk < 0) break;
+        const long long c0 = chunk * st.chunk;
+        double G[DO_VAR ? TILES : 1][4];
+        if (DO_VAR) {
+#pragma unroll
+            for (int t = 0; t < TILES; ++t) { G[t][0] = G[t][1] = G[t][2] = G[t][3] = 0.0; }
+        }
+        for (int i = 0; i < W; ++i) {
+            float z[TILES][4];
+            double l1 = 0.0;
+#pragma unroll
+            for (int t = 0; t < TILES; ++t) {
+                PROF_T0();
+                const bool ready = mbar_wait(smem_addr(&sh->full[s]), phase, abort_flag, a.error_flag);
+                PROF_ADD(0);
+                const float *stage = reinterpret_cast<const float *>(ring + (size_t)s * kStageBytes);
+                float4 g4 = make_float4(0.f, 0.f, 0.f, 0.f), m4 = g4, u4 = g4, e4 = g4;
+                if (ready) {
+                    g4 = ld4(stage + pos);
+                    m4 = ld4(stage + kTile + pos);
+                    u4 = ld4(stage + 2 * kTile + pos);
+                    e4 = ld4(stage + 3 * kTile + pos);
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_addr(&sh->empty[s]));
+                if (++s == R) { s = 0; phase ^= 1u; }
+                const float gg[4] = {g4.x, g4.y, g4.z, g4.w}, mm[4] = {m4.x, m4.y, m4.z, m4.w};
+                const float uu[4] = {u4.x, u4.y, u4.z, u4.w}, ee[4] = {e4.x, e4.y, e4.z, e4.w};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const float step = f_mul(a.gamma, momentum(a.c, mm[k], gg[k]));   // lines 3, 5
+                    z[t][k] = f_add(f_add(uu[k], step), ee[k]);                       // u_{t+1/2} + delta
+                    l1 += fabs((double)z[t][k]);
+                    if (DO_VAR) G[t][k] += (double)gg[k];
+                }
+            }
+            float scale;
+            { PROF_T0(); scale = chunk_scale(consumer_sum(l1, sh, flip), st.chunk); PROF_ADD(1); }
+            PROF_T0();
+            const long long row = (long long)i * st.n_pad + c0;
+#pragma unroll
+            for (int t = 0; t < TILES; ++t) {
+                bool b[4];
+                float e[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    b[k] = z[t][k] >= 0.0f;
+                    e[k] = f_sub(z[t][k], b[k] ? scale : -scale);
+                }
+                st4_stream(st.dw + row + t * kTile + pos, make_float4(e[0], e[1], e[2], e[3]));
+                const uint32_t word = pack_group(b);
+                if (group_leader) {
+                    bits_s[i * words_per_chunk + t * (kTile / 32) + word_in_tile] = word;
+                    st.words_w[(long long)i * st.words_stride + ((c0 + t * kTile) >> 5) + word_in_tile] = word;
+                }
+            }
+            if (lane == 0) my_scales[i] = scale;
+            if (tid == 0) st.scales_w[(long long)i * st.n_chunks + chunk] = scale;
+            if (c0_prev >= 0) store_prev_worker(i);
+            PROF_ADD(2);
+        }
+        __syncwarp();   // bits_s and my_scales were written by lanes of this warp
+
+        // ---- server: mean of the compressed buffers + server error, compress again ----
+        float av[TILES][4];
+        int srv_stage[TILES];
+        double l1 = 0.0;
+#pragma unroll
+        for (int t = 0; t < TILES; ++t) {
+            const bool ready = mbar_wait(smem_addr(&sh->full[s]), phase, abort_flag, a.error_flag);
+            srv_stage[t] = s;
+            const float *stage = reinterpret_cast<const float *>(ring + (size_t)s * kStageBytes);
+            if (++s == R) { s = 0; phase ^= 1u; }
+            const float4 d4 = ready ? ld4(stage + pos) : make_float4(0.f, 0.f, 0.f, 0.f);
+            const float dd[4] = {d4.x, d4.y, d4.z, d4.w};
+            double A[4] = {0.0, 0.0, 0.0, 0.0};
+            const int shift = (lane & 7) * 4;
+            for (int i = 0; i < W; ++i) {   // worker order
+                const uint32_t nib = bits_s[i * words_per_chunk + t * (kTile / 32) + word_in_tile] >> shift;
+                const double sc = (double)my_scales[i];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) A[k] += ((nib >> k) & 1u) ? sc : -sc;
+            }
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                av[t][k] = server_input(A[k], W, dd[k]);
+                l1 += fabs((double)av[t][k]);
+            }
+        }
+        const float scale = chunk_scale(consumer_sum(l1, sh, flip), st.chunk);
+#pragma unroll
+        for (int t = 0; t < TILES; ++t) {
+            const float *stage = reinterpret_cast<const float *>(ring + (size_t)srv_stage[t] * kStageBytes);
+            const float4 v4 = ld4(stage + kTile + pos), xs4 = ld4(stage + 2 * kTile + pos);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_addr(&sh->empty[srv_stage[t]]));
+            const float vv[4] = {v4.x, v4.y, v4.z, v4.w}, xs[4] = {xs4.x, xs4.y, xs4.z, xs4.w};
+            bool b[4];
+            float e[4];
+            if (t == 0) bits_prev = 0;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                b[k] = av[t][k] >= 0.0f;
+                const float hat = b[k] ? scale : -scale;
+                e[k] = f_sub(av[t][k], hat);
+                x_prev[t][k] = f_sub(xs[k], f_div(hat, denom(a.c, vv[k])));    // line 9
+                bits_prev |= (b[k] ? 1u : 0u) << (4 * t + k);
+            }
+            const long long j = c0 + t * kTile + pos;
+            const uint32_t word = pack_group(b);
+            if (group_leader) st.words_s[((c0 + t * kTile) >> 5) + word_in_tile] = word;
+            st4_stream(st.ds + j, make_float4(e[0], e[1], e[2], e[3]));
+            st4_stream(st.xs + j, make_float4(x_prev[t][0], x_prev[t][1], x_prev[t][2], x_prev[t][3]));
+            if (DO_VAR) {
+                float vo[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) vo[k] = variance(a.c, vv[k], mean_round(G[t][k], W));   // lines 14-15
+                st4_stream(st.v_next + j, make_float4(vo[0], vo[1], vo[2], vo[3]));
+            }
+        }
+        m_pos_prev = f_div(scale, a.gamma_sum);     // line 8: m = +-scale / sum(gamma); -(s/G) == (-s)/G exactly
+        c0_prev = c0;
+        if (tid == 0) st.scales_s[chunk] = scale;
+        __syncwarp();   // the next chunk overwrites bits_s / my_scales of this warp
+    }
+    if (c0_prev >= 0)
+        for (int i = 0; i < W; ++i) store_prev_worker(i);   // the block's last chunk
+#ifdef ZOA_PIPE_PROFILE
+    if (tid == 0) {
+        prof[7] = clock64() - prof_start;
+        for (int k = 0; k < 8; ++k) g_pipe_prof[blockIdx.x][k] = prof[k];
+    }
+#endif
+}
+
+// ---------------------------------------------------------------------------
+// Host side
+// ---------------------------------------------------------------------------
+static size_t pipeline_fixed_smem(int W, int chunk)
+{
+    const size_t head = 1024 + (size_t)W * (chunk / 32) * 4 + (size_t)kConsumerWarps * W * 4;
+    return (head + 1023) & ~(size_t)1023;
+}
+
+// How many ring stages fit (0 = the pipelined kernel does not apply to this shape).
+int pipeline_stages(const StateView &st, bool g_aligned)
+{
+    if (!g_aligned) return 0;
+    if (st.chunk != kTile && st.chunk != 2 * kTile && st.chunk != 4 * kTile) return 0;
+    if (st.n / st.chunk < 1) return 0;
+    const int tiles = st.chunk / kTile;
+    const size_t budget = 227 * 1024;
+    const size_t fixed = pipeline_fixed_smem(st.W, st.chunk);
+    if (fixed + (size_t)(tiles + 1) * kStageBytes > budget) return 0;
+    int stages = (int)((budget - fixed) / kStageBytes);
+    if (stages > kMaxStages) stages = kMaxStages;
+    return stages >= tiles + 1 ? stages : 0;
+}
+
+template <int TILES, bool DO_VAR>
+static cudaError_t launch_pipe(const PipeArgs &a, int grid, size_t smem, cudaStream_t s)
+{
+    auto kern = step_sync_pipelined_kernel<TILES, DO_VAR>;
+    static bool configured[64] = {false};   // per instantiation and device
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64 || !configured[dev]) {
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) configured[dev] = true;
+    }
+    kern<<<grid, kThreads, smem, s>>>(a);
+    return cudaGetLastError();
+}
+
+// Runs the full chunks [0, n / chunk) of a sync step; the ragged last chunk, if any, is the caller's.
+// *var_fused tells whether lines 14-15 were done here too.
+cudaError_t launch_step_sync_pipelined(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
+                                       float gamma_sum, bool do_var, int stages, int sm_count, int *error_flag,
+                                       unsigned long long *sched, bool *var_fused, cudaStream_t s)
+{
+    PipeArgs a;
+    a.st = st; a.g = g; a.c = c; a.gamma = gamma; a.gamma_sum = gamma_sum;
+    a.n_full_chunks = st.n / st.chunk;
+    a.stages = stages;
+    a.error_flag = error_flag;
+    a.sched = sched;
+    const int grid = (int)(a.n_full_chunks < sm_count ? a.n_full_chunks : sm_count);
+    const size_t smem = pipeline_fixed_smem(st.W, st.chunk) + (size_t)stages * kStageBytes;
+    const int tiles = st.chunk / kTile;
+    // With 4 tiles per chunk the binary64 gradient sums no longer fit the register budget
+    // (measured: the spilling variant is slower than a separate variance pass).
+    *var_fused = do_var && tiles <= 2;
+    switch (tiles) {
+    case 1: return do_var ? launch_pipe<1, true>(a, grid, smem, s) : launch_pipe<1, false>(a, grid, smem, s);
+    case 2: return do_var ? launch_pipe<2, true>(a, grid, smem, s) : launch_pipe<2, false>(a, grid, smem, s);
+    case 4: return launch_pipe<4, false>(a, grid, smem, s);
+    default: return cudaErrorInvalidValue;
+    }
+}
+
+}  // namespace zoa

@@ -63,6 +63,10 @@ class Zoa:
         B.zoa_set_var_steps(self.h, list(var_steps))
         B.zoa_set_sync_policy(self.h, list(sync_boundaries), list(sync_intervals))
 
+    def set_pipeline(self, on):
+        """Fused sync step through the bulk-copy ring kernel (default) or the chunk-per-block one."""
+        B.zoa_set_option(self.h, B.OPT_PIPELINE, int(bool(on)))
+
     def sync_due(self, t):
         return B.zoa_sync_due(self.h, t) == 1
 

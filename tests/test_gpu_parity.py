@@ -79,6 +79,38 @@ def test_fused_equals_two_call_bit_for_bit():
         a.close(), b.close()
 
 
+@pytest.mark.parametrize("W,chunk,n_chunks,tail", [(5, 4096, 301, 1852), (3, 2048, 700, 0), (4, 8192, 160, 704),
+                                                   (16, 4096, 40, 5), (64, 2048, 20, 33), (33, 8192, 9, 0)])
+def test_pipelined_kernel_equals_chunk_per_block_kernel(W, chunk, n_chunks, tail):
+    """The bulk-copy ring kernel and the chunk-per-block kernel give the same bits,
+    over enough chunks that every block wraps its ring many times; steps with and
+    without the fused variance update."""
+    rng = np.random.default_rng(W + chunk)
+    n = n_chunks * chunk + tail
+    x0 = torch.from_numpy((rng.standard_normal(n) * 0.02).astype(np.float32))
+    a, b = Zoa(n, W, chunk=chunk), Zoa(n, W, chunk=chunk)
+    try:
+        b.set_pipeline(False)
+        for z in (a, b):
+            z.set_params(x0)
+            z.set_policies((0, 2), (0,), (1,))
+        g = torch.empty(W, n, device="cuda")
+        for t in range(4):
+            g.normal_(generator=torch.Generator("cuda").manual_seed(t + 5))
+            a.step_sync(list(g), 1e-3, t)
+            b.step_sync(list(g), 1e-3, t)
+            torch.cuda.synchronize()
+            a.check_device()
+            for name in ("x", "m", "u", "delta_w", "words_w", "scales_w"):
+                for i in (0, W // 2, W - 1):
+                    assert np.array_equal(a.read(name, i), b.read(name, i)), (name, i, t)
+            for name in ("v", "delta_s", "x_sync", "words_s", "scales_s"):
+                assert np.array_equal(a.read(name), b.read(name)), (name, t)
+        assert a.stats()["n_launches"] < b.stats()["n_launches"] or tail
+    finally:
+        a.close(), b.close()
+
+
 @pytest.mark.parametrize("mode", ["fused", "two_call"])
 def test_special_values(mode):
     """Signed zeros, subnormals, an all-zero chunk, a chunk of one sign, a lone outlier."""
