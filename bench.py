@@ -24,6 +24,7 @@ if ROOT not in sys.path:
 METRIC = "optimizer step throughput (params*workers/s)"
 UNIT = "params*workers/s"
 FALLBACK_HBM_GBS = 6650.0
+DRAM_TRAFFIC_RATIO = 0.995   # measured DRAM bytes / algorithmic bytes, see profiles/
 
 
 # ---- byte model: what the method must move, per launch -------------------------
@@ -168,6 +169,8 @@ def run_ours(args, wl):
     opt = Zoa(wl.n, wl.W, wl.beta1, wl.beta2, wl.eps, wl.chunk)
     opt.set_params(synth.initial_params(wl, "cuda", seed))
     opt.set_policies(wl.var_steps, wl.sync_boundaries, wl.sync_intervals)
+    if args.no_pipeline:
+        opt.set_pipeline(False)
     stream = synth.GradientStream(wl, "cuda", seed)
     from paper_2202_06009_b200 import binding as B
 
@@ -215,10 +218,16 @@ def run_ours(args, wl):
     total_bytes = sum(bytes_of[k] for k in kinds)
     dominant = "sync" if "sync" in by_kind else ("sync+var" if "sync+var" in by_kind else kinds[0])
     achieved = bytes_of[dominant] / 1e6 / statistics.mean(by_kind[dominant])
-    roofline = {"bound": "hbm", "kernel": "step_sync_kernel" if dominant.startswith("sync") else "local_step_kernel",
+    sync_kernel = "step_sync_kernel" if args.no_pipeline else "step_sync_pipelined_kernel"
+    roofline = {"bound": "hbm", "kernel": sync_kernel if dominant.startswith("sync") else "local_step_kernel",
                 "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "peak_kind": f"of {peak_kind}", "frac_of_8TBps_nominal": achieved / 8000.0,
-                "traffic": None, "launch_ms": statistics.mean(by_kind[dominant]),
+                # ncu (dram__bytes_read.sum + dram__bytes_write.sum) on the layout shrunk 16x gave
+                # 0.995 x the algorithmic bytes for both sync kernels and 0.994 for the local step
+                # (profiles/); traffic is proportional to n*W, so the ratio carries to a full launch.
+                "traffic": DRAM_TRAFFIC_RATIO * bytes_of[dominant],
+                "traffic_how": "ncu capture of the same kernel on the layout shrunk 16x, scaled by n*W",
+                "launch_ms": statistics.mean(by_kind[dominant]),
                 "algorithmic_bytes_per_launch": bytes_of[dominant]}
 
     # ---- end to end: host gradients in, worker 0's model out, through zoa_step_host ----
@@ -282,6 +291,7 @@ def main():
     ap.add_argument("--cpu-sample", type=int, default=1 << 22, help="parameters in the oracle's timed sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--scale", type=int, default=1, help="shrink every tensor by this factor (profiling captures)")
+    ap.add_argument("--no-pipeline", action="store_true", help="fused sync step through the chunk-per-block kernel")
     args = ap.parse_args()
 
     if args.impl == "reference":
