@@ -280,6 +280,73 @@ def run_ours(args, wl):
         dist.destroy_process_group()
 
 
+# ---- kernel sweep: worker compression and W-way decompress-average on flat vectors ---------
+def run_sweep(args):
+    """Times zoa_onebit_compress (Algorithm 3, worker side) and zoa_onebit_average (server
+    side + lines 8-10 of Algorithm 1) alone, for n = 2^20 .. 2^30 in powers of 4,
+    W in {2,4,8,16}, chunk in {1024,4096,16384}; inputs N(0,1) with 1 % of the elements
+    scaled by 100.  One JSON line per combination."""
+    import torch
+    from paper_2202_06009_b200 import Zoa, ZoaError, binding as B
+
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    peak, peak_kind = measured_hbm_peak()
+    exps = [20, 22] if args.sweep == "quick" else [20, 22, 24, 26, 28, 30]
+    gen = torch.Generator("cuda").manual_seed(5)
+    for e in exps:
+        n = 1 << e
+        for W in (2, 4, 8, 16):
+            for chunk in (1024, 4096, 16384):
+                n_chunks = n // chunk
+                row = {"sweep": True, "n": n, "W": W, "chunk": chunk}
+                state_bytes = (4 * W + 4) * n * 4 + (W + 1) * n // 8
+                free, _ = torch.cuda.mem_get_info()
+                if state_bytes > 0.97 * free:
+                    row["skipped"] = f"memory: the handle's state needs {state_bytes / 1e9:.0f} GB"
+                    print(json.dumps(row), flush=True)
+                    continue
+                try:
+                    opt = Zoa(n, W, chunk=chunk)
+                except ZoaError as err:
+                    row["skipped"] = f"memory: {err}"
+                    print(json.dumps(row), flush=True)
+                    continue
+                tmp = torch.empty(min(n, 1 << 26), device="cuda")
+                for i in range(W):                        # u := N(0,1), 1 % of the elements x100
+                    u = opt.device_view("u", i)
+                    for lo in range(0, n, tmp.numel()):
+                        part = u[lo:lo + tmp.numel()]
+                        part.normal_(generator=gen)
+                        t = tmp[:part.numel()].uniform_(generator=gen)
+                        part.mul_(torch.where(t < 0.01, 100.0, 1.0))
+                del tmp
+                bytes_c = n * W * (12 + 1 / 8) + 4 * n_chunks * W
+                bytes_a = n * W * (12 + 1 / 8) + 4 * n_chunks * W + n * (20 + 1 / 8) + 4 * n_chunks
+                times = {"compress": [], "average": []}
+                for rep in range(args.sweep_reps + 1):      # rep 0: errors start at zero; later reps: non-zero errors
+                    B.zoa_set_scalars(opt.h, 1e-3, 0, rep)
+                    e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+                    e0.record()
+                    opt.onebit_compress()
+                    e1.record()
+                    opt.onebit_average()
+                    e2.record()
+                    torch.cuda.synchronize()
+                    times["compress"].append(e0.elapsed_time(e1))
+                    times["average"].append(e1.elapsed_time(e2))
+                opt.check_device()
+                opt.close()
+                tc0, ta0 = times["compress"][0], times["average"][0]
+                tc, ta = statistics.median(times["compress"][1:]), statistics.median(times["average"][1:])
+                row.update({"compress_ms_zero_errors": tc0, "compress_ms": tc, "compress_GBps": bytes_c / 1e6 / tc,
+                            "average_ms_zero_errors": ta0, "average_ms": ta, "average_GBps": bytes_a / 1e6 / ta,
+                            "both_GBps": (bytes_c + bytes_a) / 1e6 / (tc + ta),
+                            "both_frac_of_peak": (bytes_c + bytes_a) / 1e6 / (tc + ta) / peak, "peak_kind": peak_kind,
+                            "l2_resident": state_bytes < 126e6})
+                print(json.dumps(row), flush=True)
+                torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -292,8 +359,13 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--scale", type=int, default=1, help="shrink every tensor by this factor (profiling captures)")
     ap.add_argument("--no-pipeline", action="store_true", help="fused sync step through the chunk-per-block kernel")
+    ap.add_argument("--sweep", nargs="?", const="full", default=None, choices=["full", "quick"],
+                    help="time the compress / decompress-average kernels over the size grid instead")
+    ap.add_argument("--sweep-reps", type=int, default=3)
     args = ap.parse_args()
 
+    if args.sweep:
+        return run_sweep(args)
     if args.impl == "reference":
         # the oracle needs no CUDA library; import only the workload tables
         import importlib.util

@@ -115,6 +115,14 @@ zoa_status zoa_step(zoa_handle h, const float *const *grads, float lr, int64_t t
  * last sync (the divisor of line 8 would be zero). */
 zoa_status zoa_onebit_reduce(zoa_handle h, void *stream);
 
+/* The two halves of zoa_onebit_reduce, for callers that want to time or
+ * interleave them: zoa_onebit_compress is the worker side of Algorithm 3 (packs
+ * u + delta of every worker into words_w / scales_w, keeps the errors);
+ * zoa_onebit_average is the server side and lines 8-11 of Algorithm 1 (reads
+ * words_w / scales_w).  compress then average == zoa_onebit_reduce. */
+zoa_status zoa_onebit_compress(zoa_handle h, void *stream);
+zoa_status zoa_onebit_average(zoa_handle h, void *stream);
+
 /* zoa_step followed by zoa_onebit_reduce, same results bit for bit, in one
  * pass over memory that never writes the half-step values. */
 zoa_status zoa_step_sync(zoa_handle h, const float *const *grads, float lr, int64_t t,

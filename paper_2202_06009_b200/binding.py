@@ -45,6 +45,8 @@ def _load():
         "zoa_var_due": ([H, C.c_int64], C.c_int),
         "zoa_step": ([H, C.POINTER(p), C.c_float, C.c_int64, p], C.c_int),
         "zoa_onebit_reduce": ([H, p], C.c_int),
+        "zoa_onebit_compress": ([H, p], C.c_int),
+        "zoa_onebit_average": ([H, p], C.c_int),
         "zoa_step_sync": ([H, C.POINTER(p), C.c_float, C.c_int64, p], C.c_int),
         "zoa_step_auto": ([H, C.POINTER(p), C.c_float, C.c_int64, p], C.c_int),
         "zoa_step_host": ([H, C.POINTER(p), C.c_float, C.c_int64, p, p], C.c_int),
@@ -122,6 +124,14 @@ def zoa_step(h, grad_ptrs, lr, t, stream=0):
 
 def zoa_onebit_reduce(h, stream=0):
     _check(h, lib.zoa_onebit_reduce(h, stream))
+
+
+def zoa_onebit_compress(h, stream=0):
+    _check(h, lib.zoa_onebit_compress(h, stream))
+
+
+def zoa_onebit_average(h, stream=0):
+    _check(h, lib.zoa_onebit_average(h, stream))
 
 
 def zoa_step_sync(h, grad_ptrs, lr, t, stream=0):

@@ -270,6 +270,28 @@ extern "C" zoa_status zoa_onebit_reduce(zoa_handle h, void *stream)
     return ZOA_OK;
 }
 
+extern "C" zoa_status zoa_onebit_compress(zoa_handle h, void *stream)
+{
+    if (!h) return ZOA_ERR_ARG;
+    ZOA_CUDA(h, launch_compress(view(h), static_cast<cudaStream_t>(stream)));
+    h->n_launches += 1;
+    return ZOA_OK;
+}
+
+extern "C" zoa_status zoa_onebit_average(zoa_handle h, void *stream)
+{
+    if (!h) return ZOA_ERR_ARG;
+    const float gamma_sum = (float)h->gamma_sum;
+    if (!(h->gamma_sum > 0.0) || !(gamma_sum > 0.f) || !std::isfinite(gamma_sum))
+        return fail(h, ZOA_ERR_STATE, "zoa_onebit_average: nothing accumulated since the last sync (sum of learning rates is not positive)");
+    ZOA_CUDA(h, launch_reduce(view(h), h->c, gamma_sum, static_cast<cudaStream_t>(stream)));
+    h->n_launches += 1;
+    h->gamma_sum = 0.0;
+    h->t_sync = h->t_last;
+    h->n_syncs += 1;
+    return ZOA_OK;
+}
+
 extern "C" zoa_status zoa_step_sync(zoa_handle h, const float *const *grads, float lr, int64_t t, void *stream)
 {
     GradPtrs gp;

@@ -80,6 +80,24 @@ class Zoa:
     def onebit_reduce(self):
         B.zoa_onebit_reduce(self.h, _stream())
 
+    def onebit_compress(self):
+        B.zoa_onebit_compress(self.h, _stream())
+
+    def onebit_average(self):
+        B.zoa_onebit_average(self.h, _stream())
+
+    def device_view(self, name, worker=0):
+        """The state row as a torch tensor that aliases the library's memory (no copy)."""
+        which = _NAMES[name]
+        ptr, n = B.zoa_get_buffer(self.h, which, worker)
+        words = which in B.WORD_BUFFERS
+
+        class _Raw:
+            __cuda_array_interface__ = {"shape": (n,), "typestr": "<u4" if words else "<f4",
+                                        "data": (ptr, False), "version": 2}
+        t = torch.as_tensor(_Raw(), device="cuda")
+        return t.view(torch.int32) if words else t
+
     def step_sync(self, grads, lr, t):
         B.zoa_step_sync(self.h, _grad_ptrs(grads, self.n, self.W), lr, t, _stream())
 

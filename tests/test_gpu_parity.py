@@ -184,6 +184,32 @@ def test_shaped_workloads_scaled_down(name, divisor):
         p.close()
 
 
+@pytest.mark.parametrize("W,chunk", [(2, 1024), (16, 1024), (4, 4096), (8, 16384), (16, 16384)])
+def test_sweep_recipe_compress_then_average(W, chunk):
+    """The kernel sweep's recipe (N(0,1) with 1 % of the elements x100), through the two
+    halves of zoa_onebit_reduce called separately, two rounds so that the second sees
+    non-zero errors."""
+    rng = np.random.default_rng(W * chunk)
+    n = (1 << 20) // 8 + 77
+    p = Pair(n, W, chunk, x0=np.zeros(n))
+    try:
+        for r in range(2):
+            z = rng.standard_normal((W, n)).astype(np.float32)
+            z[rng.random((W, n)) < 0.01] *= np.float32(100.0)
+            for i in range(W):
+                p.gpu.write("u", z[i], i)
+                p.cpu.u[i] = z[i]
+            B.zoa_set_scalars(p.gpu.h, 1e-3, 0, r)
+            p.cpu._st.gamma_sum = 1e-3
+            p.gpu.onebit_compress()
+            p.gpu.onebit_average()
+            torch.cuda.synchronize()
+            assert p.cpu.sync(r) == 0
+            p.compare(f"round {r}")
+    finally:
+        p.close()
+
+
 def test_unaligned_gradient_pointers():
     rng = np.random.default_rng(5)
     n, W, chunk = 3000, 2, 1024
