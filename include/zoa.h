@@ -166,8 +166,14 @@ zoa_status zoa_check_device(zoa_handle h);
 /* Tuning switches.  ZOA_OPT_PIPELINE (default 1): run the fused sync step as the
  * persistent bulk-copy-ring kernel where the shape allows (chunk 2048, 4096 or
  * 8192, 16-byte aligned gradients); 0 forces the chunk-per-block kernel.  The
- * results are the same bit for bit. */
-enum { ZOA_OPT_PIPELINE = 1 };
+ * results are the same bit for bit.
+ * ZOA_OPT_WAIT_LIMIT_MS (default 2000): how long a kernel thread waits for an
+ * asynchronous copy before it gives up; the kernel then ends early, the state is
+ * undefined and zoa_check_device reports ZOA_ERR_DEVICE.
+ * ZOA_OPT_TEST_STOP_AFTER_TILES (default 0 = off): for testing that error path
+ * only - the copy-issuing lane of every block stops after this many tiles, so
+ * the waits of the other threads run out after the limit. */
+enum { ZOA_OPT_PIPELINE = 1, ZOA_OPT_WAIT_LIMIT_MS = 2, ZOA_OPT_TEST_STOP_AFTER_TILES = 3 };
 zoa_status zoa_set_option(zoa_handle h, int option, int value);
 
 /* Text of the last error on this handle (or of the last failed zoa_create if h

@@ -170,7 +170,7 @@ def zoa_get_stats(h):
     return {name: getattr(s, name) for name, _ in Stats._fields_}
 
 
-OPT_PIPELINE = 1
+OPT_PIPELINE, OPT_WAIT_LIMIT_MS, OPT_TEST_STOP_AFTER_TILES = 1, 2, 3
 
 
 def zoa_set_option(h, option, value):

@@ -26,6 +26,8 @@ struct zoa_handle_s {
     int *error_flag = nullptr;     // device int: a kernel gave up on a bounded wait
     unsigned long long *sched = nullptr;   // device [2]: chunk counter of the persistent kernel, finished blocks
     bool use_pipeline = true;      // bulk-copy ring form of the fused sync step where the shape allows
+    int wait_limit_ms = 2000;      // bound on every device-side wait
+    long long test_stop_after_tiles = 0;   // error-path test hook, see zoa_set_option
     bool v_pending = false;        // v_nxt holds v_{t+1}; it becomes v at the next step
     std::vector<int64_t> var_steps;                    // T_v, sorted
     std::vector<int64_t> sync_bounds{0};               // T_u pieces
@@ -210,6 +212,8 @@ extern "C" int zoa_var_due(zoa_handle h, int64_t t)
 }
 
 // Checks shared by the step entry points; fills the pointer pack.
+static bool on_own_device(zoa_handle h);
+
 static zoa_status check_step_args(zoa_handle h, const float *const *grads, float lr, int64_t t, GradPtrs *gp,
                                   bool *aligned, const char *who)
 {
@@ -218,6 +222,7 @@ static zoa_status check_step_args(zoa_handle h, const float *const *grads, float
     if (!std::isfinite(lr)) return fail(h, ZOA_ERR_ARG, std::string(who) + ": lr is not finite");
     if (t < 0) return fail(h, ZOA_ERR_ARG, std::string(who) + ": t is negative");
     if (t <= h->t_last) return fail(h, ZOA_ERR_STATE, std::string(who) + ": t must increase from step to step");
+    if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, std::string(who) + ": the handle's device is not the current CUDA device");
     *aligned = true;
     for (int i = 0; i < h->W; ++i) {
         if (!grads[i]) return fail(h, ZOA_ERR_ARG, std::string(who) + ": a gradient pointer is NULL");
@@ -226,6 +231,12 @@ static zoa_status check_step_args(zoa_handle h, const float *const *grads, float
     }
     for (int i = h->W; i < kMaxWorkers; ++i) gp->p[i] = nullptr;
     return ZOA_OK;
+}
+
+static bool on_own_device(zoa_handle h)
+{
+    int dev = -1;
+    return cudaGetDevice(&dev) == cudaSuccess && dev == h->device;
 }
 
 static void commit_variance(zoa_handle h)
@@ -259,6 +270,7 @@ extern "C" zoa_status zoa_onebit_reduce(zoa_handle h, void *stream)
     const float gamma_sum = (float)h->gamma_sum;
     if (!(h->gamma_sum > 0.0) || !(gamma_sum > 0.f) || !std::isfinite(gamma_sum))
         return fail(h, ZOA_ERR_STATE, "zoa_onebit_reduce: nothing accumulated since the last sync (sum of learning rates is not positive)");
+    if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, "zoa_onebit_reduce: the handle's device is not the current CUDA device");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const StateView st = view(h);
     ZOA_CUDA(h, launch_compress(st, s));
@@ -313,7 +325,8 @@ extern "C" zoa_status zoa_step_sync(zoa_handle h, const float *const *grads, flo
         const long long n_full = h->n / h->chunk;
         bool var_fused = false;
         ZOA_CUDA(h, launch_step_sync_pipelined(st, gp, h->c, lr, gamma_sum, do_var, stages, h->sm_count,
-                                               h->error_flag, h->sched, &var_fused, s));
+                                               h->error_flag, h->sched, (unsigned long long)h->wait_limit_ms * 1000000ull,
+                                               h->test_stop_after_tiles, &var_fused, s));
         h->n_launches += 1;
         if (n_full < h->n_chunks) {
             ZOA_CUDA(h, launch_step_sync(st, gp, h->c, lr, gamma_sum, aligned, n_full, h->n_chunks - n_full, s));
@@ -476,9 +489,18 @@ extern "C" zoa_status zoa_check_device(zoa_handle h)
 extern "C" zoa_status zoa_set_option(zoa_handle h, int option, int value)
 {
     if (!h) return ZOA_ERR_ARG;
-    if (option != ZOA_OPT_PIPELINE) return fail(h, ZOA_ERR_ARG, "zoa_set_option: unknown option");
-    h->use_pipeline = value != 0;
-    return ZOA_OK;
+    switch (option) {
+    case ZOA_OPT_PIPELINE: h->use_pipeline = value != 0; return ZOA_OK;
+    case ZOA_OPT_WAIT_LIMIT_MS:
+        if (value < 1 || value > 60000) return fail(h, ZOA_ERR_ARG, "zoa_set_option: wait limit must be 1..60000 ms");
+        h->wait_limit_ms = value;
+        return ZOA_OK;
+    case ZOA_OPT_TEST_STOP_AFTER_TILES:
+        if (value < 0) return fail(h, ZOA_ERR_ARG, "zoa_set_option: negative tile count");
+        h->test_stop_after_tiles = value;
+        return ZOA_OK;
+    default: return fail(h, ZOA_ERR_ARG, "zoa_set_option: unknown option");
+    }
 }
 
 extern "C" const char *zoa_last_error(zoa_handle h)

@@ -20,6 +20,7 @@ cudaError_t launch_step_sync(const StateView &st, const GradPtrs &g, const Const
 int pipeline_stages(const StateView &st, bool g_aligned);
 cudaError_t launch_step_sync_pipelined(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
                                        float gamma_sum, bool do_var, int stages, int sm_count, int *error_flag,
-                                       unsigned long long *sched, bool *var_fused, cudaStream_t s);
+                                       unsigned long long *sched, unsigned long long wait_limit_ns,
+                                       long long test_stop_after_tiles, bool *var_fused, cudaStream_t s);
 
 }  // namespace zoa

@@ -13,7 +13,7 @@
 // chunk's z in registers (thread t owns coordinates 4t..4t+3 of every tile), so
 // shared memory holds only the ring, the packed bits and the magnitudes.
 //
-// Every wait on an mbarrier is bounded: after about two seconds a thread gives
+// Every wait on an mbarrier is bounded: after the handle's limit (2 s by default) a thread gives
 // up, raises the block's abort flag and the handle's device error flag, the
 // block stops issuing copies, waits (bounded) for those in flight and leaves.
 #include "zoa_internal.h"
@@ -29,7 +29,6 @@ constexpr int kTile = 4 * kConsumers;           // coordinates per ring stage an
 constexpr int kTileBytes = kTile * 4;
 constexpr int kStageBytes = 4 * kTileBytes;     // g, m, u, delta  |  delta_bar, v, x_sync, (unused)
 constexpr int kMaxStages = 6;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 struct PipeArgs {
     StateView st;
@@ -40,6 +39,8 @@ struct PipeArgs {
     int stages;
     int *error_flag;  // device int, set non-zero when a wait ran out
     unsigned long long *sched;  // device: [0] next chunk to hand out, [1] blocks that have finished
+    unsigned long long wait_limit_ns;  // how long a thread waits on an mbarrier before it gives up
+    long long test_stop_after_tiles;   // > 0: each producer stops after this many tiles (error-path test)
 };
 
 // Shared-memory header (the ring follows, 1024-byte aligned).
@@ -85,14 +86,15 @@ __device__ __forceinline__ unsigned long long global_timer_ns()
 }
 // Bounded wait.  Returns false if the block has been aborted or the limit ran out
 // (in which case it raises both flags).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *error_flag)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *error_flag,
+                                          unsigned long long limit_ns)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long start = global_timer_ns();
     for (unsigned it = 1;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if ((it & 63u) == 0 && global_timer_ns() - start > kWaitLimitNs) {
+        if ((it & 63u) == 0 && global_timer_ns() - start > limit_ns) {
             *abort_flag = 1;
             atomicExch(error_flag, 1);
             return false;
@@ -203,7 +205,7 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
             // The chunk id travels to the consumers through shared memory; the arrive on the
             // first tile's barrier below publishes it.  The queue cannot wrap onto an unread
             // entry: the producer is at most `stages` tiles, hence chunks, ahead.
-            if (!mbar_wait(smem_addr(&sh->empty[s]), phase ^ 1u, abort_flag, a.error_flag)) { ok = false; break; }
+            if (!mbar_wait(smem_addr(&sh->empty[s]), phase ^ 1u, abort_flag, a.error_flag, a.wait_limit_ns)) { ok = false; break; }
             sh->chunk_queue[k % (kMaxStages + 2)] = last ? -1 : chunk;
             if (last) {
                 mbar_arrive(smem_addr(&sh->full[s]));       // an empty "tile": wakes the consumers to read the -1
@@ -213,7 +215,7 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
             for (int i = 0; ok && i <= W; ++i) {            // i == W: the server's tiles
                 for (int t = 0; t < TILES; ++t) {
                     const uint32_t full = smem_addr(&sh->full[s]);
-                    if (!mbar_wait(smem_addr(&sh->empty[s]), phase ^ 1u, abort_flag, a.error_flag)) { ok = false; break; }
+                    if (!mbar_wait(smem_addr(&sh->empty[s]), phase ^ 1u, abort_flag, a.error_flag, a.wait_limit_ns)) { ok = false; break; }
                     const uint32_t dst = smem_addr(ring + (size_t)s * kStageBytes);
                     const long long off = c0 + (long long)t * kTile;
                     if (i < W) {
@@ -231,6 +233,7 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
                     }
                     ++issued;
                     if (++s == R) { s = 0; phase ^= 1u; }
+                    if (a.test_stop_after_tiles > 0 && issued >= a.test_stop_after_tiles) { ok = false; break; }
                 }
             }
         }
@@ -242,7 +245,7 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
                 const uint32_t bar = smem_addr(&sh->full[q % R]);
                 const uint32_t par = (uint32_t)((q / R) & 1);
                 const unsigned long long start = global_timer_ns();
-                while (!mbar_try_wait(bar, par) && global_timer_ns() - start < kWaitLimitNs) {}
+                while (!mbar_try_wait(bar, par) && global_timer_ns() - start < a.wait_limit_ns) {}
             }
         }
         // The last block to finish taking chunks rearms the counters for the next launch.
@@ -291,7 +294,7 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
         // The first tile's barrier also publishes the chunk id (or the end mark).  Leaving the
         // loop must be unanimous (the block sums below count on all 512 consumers), so a
         // wait that ran out is put to the vote.
-        const bool gave_up = !mbar_wait(smem_addr(&sh->full[s]), phase, abort_flag, a.error_flag);
+        const bool gave_up = !mbar_wait(smem_addr(&sh->full[s]), phase, abort_flag, a.error_flag, a.wait_limit_ns);
         if (consumer_any(gave_up)) break;
         const long long chunk = sh->chunk_queue[k % (kMaxStages + 2)];
         if (chunk < 0) break;
@@ -307,7 +310,7 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
 #pragma unroll
             for (int t = 0; t < TILES; ++t) {
                 PROF_T0();
-                const bool ready = mbar_wait(smem_addr(&sh->full[s]), phase, abort_flag, a.error_flag);
+                const bool ready = mbar_wait(smem_addr(&sh->full[s]), phase, abort_flag, a.error_flag, a.wait_limit_ns);
                 PROF_ADD(0);
                 const float *stage = reinterpret_cast<const float *>(ring + (size_t)s * kStageBytes);
                 float4 g4 = make_float4(0.f, 0.f, 0.f, 0.f), m4 = g4, u4 = g4, e4 = g4;
@@ -363,7 +366,7 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
         double l1 = 0.0;
 #pragma unroll
         for (int t = 0; t < TILES; ++t) {
-            const bool ready = mbar_wait(smem_addr(&sh->full[s]), phase, abort_flag, a.error_flag);
+            const bool ready = mbar_wait(smem_addr(&sh->full[s]), phase, abort_flag, a.error_flag, a.wait_limit_ns);
             srv_stage[t] = s;
             const float *stage = reinterpret_cast<const float *>(ring + (size_t)s * kStageBytes);
             if (++s == R) { s = 0; phase ^= 1u; }
@@ -474,7 +477,8 @@ static cudaError_t launch_pipe(const PipeArgs &a, int grid, size_t smem, cudaStr
 // *var_fused tells whether lines 14-15 were done here too.
 cudaError_t launch_step_sync_pipelined(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
                                        float gamma_sum, bool do_var, int stages, int sm_count, int *error_flag,
-                                       unsigned long long *sched, bool *var_fused, cudaStream_t s)
+                                       unsigned long long *sched, unsigned long long wait_limit_ns,
+                                       long long test_stop_after_tiles, bool *var_fused, cudaStream_t s)
 {
     PipeArgs a;
     a.st = st; a.g = g; a.c = c; a.gamma = gamma; a.gamma_sum = gamma_sum;
@@ -482,6 +486,8 @@ cudaError_t launch_step_sync_pipelined(const StateView &st, const GradPtrs &g, c
     a.stages = stages;
     a.error_flag = error_flag;
     a.sched = sched;
+    a.wait_limit_ns = wait_limit_ns;
+    a.test_stop_after_tiles = test_stop_after_tiles;
     const int grid = (int)(a.n_full_chunks < sm_count ? a.n_full_chunks : sm_count);
     const size_t smem = pipeline_fixed_smem(st.W, st.chunk) + (size_t)stages * kStageBytes;
     const int tiles = st.chunk / kTile;
