@@ -273,14 +273,15 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
     // spread over the worker iterations of the next chunk (one worker's m, x, u after
     // each worker's compression) instead of leaving in one burst, so that the block's
     // stores and its ring's loads stay evenly mixed.  m is +-m_pos by the server's bit.
-    float x_prev[TILES][4];
+    constexpr bool DEFER = !(TILES == 4 && DO_VAR);   // that variant has no registers to spare: it stores at once
+    float x_prev[DEFER ? TILES : 1][4];
     uint32_t bits_prev = 0;
     float m_pos_prev = 0.0f;
     long long c0_prev = -1;
     auto store_prev_worker = [&](int i) {
         const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int t = 0; t < TILES; ++t) {
+        for (int t = 0; t < (DEFER ? TILES : 0); ++t) {
             const long long row = (long long)i * st.n_pad + c0_prev + t * kTile + pos;
             const uint32_t nib = bits_prev >> (4 * t);
             st4_stream(st.m + row, make_float4((nib & 1u) ? m_pos_prev : -m_pos_prev, (nib & 2u) ? m_pos_prev : -m_pos_prev,
@@ -355,7 +356,7 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
             }
             if (lane == 0) my_scales[i] = scale;
             if (tid == 0) st.scales_w[(long long)i * st.n_chunks + chunk] = scale;
-            if (c0_prev >= 0) store_prev_worker(i);
+            if (DEFER && c0_prev >= 0) store_prev_worker(i);
             PROF_ADD(2);
         }
         __syncwarp();   // bits_s and my_scales were written by lanes of this warp
@@ -395,21 +396,36 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
             if (lane == 0) mbar_arrive(smem_addr(&sh->empty[srv_stage[t]]));
             const float vv[4] = {v4.x, v4.y, v4.z, v4.w}, xs[4] = {xs4.x, xs4.y, xs4.z, xs4.w};
             bool b[4];
-            float e[4];
+            float e[4], xo[4];
             if (t == 0) bits_prev = 0;
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
                 b[k] = av[t][k] >= 0.0f;
                 const float hat = b[k] ? scale : -scale;
                 e[k] = f_sub(av[t][k], hat);
-                x_prev[t][k] = f_sub(xs[k], f_div(hat, denom(a.c, vv[k])));    // line 9
-                bits_prev |= (b[k] ? 1u : 0u) << (4 * t + k);
+                xo[k] = f_sub(xs[k], f_div(hat, denom(a.c, vv[k])));           // line 9
+                if (DEFER) {
+                    x_prev[t][k] = xo[k];
+                    bits_prev |= (b[k] ? 1u : 0u) << (4 * t + k);
+                }
             }
             const long long j = c0 + t * kTile + pos;
             const uint32_t word = pack_group(b);
             if (group_leader) st.words_s[((c0 + t * kTile) >> 5) + word_in_tile] = word;
             st4_stream(st.ds + j, make_float4(e[0], e[1], e[2], e[3]));
-            st4_stream(st.xs + j, make_float4(x_prev[t][0], x_prev[t][1], x_prev[t][2], x_prev[t][3]));
+            st4_stream(st.xs + j, make_float4(xo[0], xo[1], xo[2], xo[3]));
+            if (!DEFER) {
+                const float mp = f_div(scale, a.gamma_sum);                    // line 8
+                const float4 m4 = make_float4(b[0] ? mp : -mp, b[1] ? mp : -mp, b[2] ? mp : -mp, b[3] ? mp : -mp);
+                const float4 x4 = make_float4(xo[0], xo[1], xo[2], xo[3]);
+                const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int i = 0; i < W; ++i) {
+                    const long long row = (long long)i * st.n_pad + j;
+                    st4_stream(st.m + row, m4);
+                    st4_stream(st.x + row, x4);
+                    st4_stream(st.u + row, zero);                              // line 10
+                }
+            }
             if (DO_VAR) {
                 float vo[4];
 #pragma unroll
@@ -417,8 +433,10 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
                 st4_stream(st.v_next + j, make_float4(vo[0], vo[1], vo[2], vo[3]));
             }
         }
-        m_pos_prev = f_div(scale, a.gamma_sum);     // line 8: m = +-scale / sum(gamma); -(s/G) == (-s)/G exactly
-        c0_prev = c0;
+        if (DEFER) {
+            m_pos_prev = f_div(scale, a.gamma_sum);     // line 8: m = +-scale / sum(gamma); -(s/G) == (-s)/G exactly
+            c0_prev = c0;
+        }
         if (tid == 0) st.scales_s[chunk] = scale;
         __syncwarp();   // the next chunk overwrites bits_s / my_scales of this warp
     }
@@ -491,13 +509,11 @@ cudaError_t launch_step_sync_pipelined(const StateView &st, const GradPtrs &g, c
     const int grid = (int)(a.n_full_chunks < sm_count ? a.n_full_chunks : sm_count);
     const size_t smem = pipeline_fixed_smem(st.W, st.chunk) + (size_t)stages * kStageBytes;
     const int tiles = st.chunk / kTile;
-    // With 4 tiles per chunk the binary64 gradient sums no longer fit the register budget
-    // (measured: the spilling variant is slower than a separate variance pass).
-    *var_fused = do_var && tiles <= 2;
+    *var_fused = do_var;
     switch (tiles) {
     case 1: return do_var ? launch_pipe<1, true>(a, grid, smem, s) : launch_pipe<1, false>(a, grid, smem, s);
     case 2: return do_var ? launch_pipe<2, true>(a, grid, smem, s) : launch_pipe<2, false>(a, grid, smem, s);
-    case 4: return launch_pipe<4, false>(a, grid, smem, s);
+    case 4: return do_var ? launch_pipe<4, true>(a, grid, smem, s) : launch_pipe<4, false>(a, grid, smem, s);
     default: return cudaErrorInvalidValue;
     }
 }
