@@ -9,6 +9,8 @@
  * What it follows, in the paper's order and notation:
  *   Algorithm 1 (proposed 0/1 Adam)            -> zo_alg1_half_step, zo_alg1_sync,
  *                                                 zo_alg1_variance, zo_alg1_step
+ *   Algorithm 2 (frozen-variance 1-bit framework,
+ *                1-bit Adam as a special case)  -> zo_alg2_step
  *   Algorithm 3 (error-feedback 1bit-AllReduce) -> zo_onebit_allreduce
  *   Algorithm 4 (AllReduce, plain mean)         -> zo_allreduce
  *   Eq. 3       (1-bit compressor C[a])         -> zo_compress
@@ -48,6 +50,12 @@
  *      of 32-bit word floor(j/32); unused bits of the last word are 0; one
  *      scale per chunk.
  *  R8  Line 9 uses v_t; line 15 assigns v_{t+1} afterwards.
+ *  R9  Algorithm 2 also prints m_t in its model update.  It is introduced as the
+ *      special case of Algorithm 1 without local steps, so it takes the same
+ *      convention as R1: the momentum just computed.  (With the identity
+ *      compressor both algorithms are then the same Adam; `literal_momentum`
+ *      selects the printed, one-step-delayed form here too.)  Its model update
+ *      reads v_t, so the variance of a T_v step is assigned after it.
  *
  * Pins (tests/test_oracle_pins.py, none of which re-types these formulas):
  *  zo_compress          hand-worked fixtures; z = zhat + err; l1 preserved;
@@ -64,6 +72,10 @@
  *                       x = x_{t'} - u / sqrt(v + eps) between syncs;
  *                       hand-worked power-of-two fixture of one sync step;
  *                       sign and scale symmetries.
+ *  zo_alg2_step        identity compressor equals the closed form of Adam and
+ *                       equals zo_alg1_step with T_u = all steps; T_v = the first
+ *                       T0 steps is Adam for T0 steps and then keeps v; hand-worked
+ *                       compressed step; the received gradients telescope.
  *  The paper prints no worked numbers, so the values of a long trajectory are
  *  fixed only by these pins together.
  */
@@ -244,4 +256,33 @@ int ZO(zo_alg1_step)(ZO(zo_state) *st, const real *g, real gamma, int64_t t,
     if (in_T_u) rc = ZO(zo_alg1_sync)(st, t);   /* else line 13: keep the half-step values */
     if (in_T_v) ZO(zo_alg1_variance)(st, g, g_bar_scratch); /* else line 18: v stays (R8) */
     return rc;
+}
+
+/* One iteration t of Algorithm 2 (lines 2-11).  On a T_v step the workers
+ * exchange full-precision gradients (Algorithm 4) and the variance moves; on
+ * any other step they exchange 1-bit compressed gradients (Algorithm 3).
+ * Momentum and model are the same on every worker; they are kept per worker
+ * like the rest of the state.  g_bar_scratch is [d]. */
+void ZO(zo_alg2_step)(ZO(zo_state) *st, const real *g, real gamma, int in_T_v, real *g_bar_scratch)
+{
+    const real one_minus_beta1 = (real)1 - st->beta1, one_minus_beta2 = (real)1 - st->beta2;
+    const real *g_bar = g_bar_scratch;
+    if (in_T_v) {
+        ZO(zo_allreduce)(g, st->n, st->d, g_bar_scratch);                  /* line 4 */
+    } else {
+        ZO(zo_onebit_allreduce)(st, g);                                    /* line 7 */
+        g_bar = st->u_bar;
+    }
+    for (int i = 0; i < st->n; ++i)
+        for (int64_t j = 0; j < st->d; ++j) {
+            size_t k = (size_t)i * st->d + j;
+            real m_prev = st->m[k];
+            real m_next = st->beta1 * m_prev + one_minus_beta1 * g_bar[j]; /* line 10 */
+            real m_used = st->literal_momentum ? m_prev : m_next;          /* R9 */
+            st->x[k] = st->x[k] - (gamma * m_used) / ZO(zo_sqrt)(st->v[j] + st->eps); /* line 11 */
+            st->m[k] = m_next;
+        }
+    if (in_T_v)
+        for (int64_t j = 0; j < st->d; ++j)
+            st->v[j] = st->beta2 * st->v[j] + one_minus_beta2 * (g_bar[j] * g_bar[j]); /* line 5 */
 }

@@ -163,6 +163,14 @@ class Oracle:
         return f(C.byref(self._st), _ptr(g, self._real), self._real(gamma), C.c_int64(t),
                  C.c_int(bool(in_T_u)), C.c_int(bool(in_T_v)), _ptr(self._g_bar, self._real))
 
+    # -- Algorithm 2 ---------------------------------------------------------
+    def alg2_step(self, g, gamma, in_T_v):
+        g = self._g(g)
+        f = _fn("zo_alg2_step", self._suffix)
+        f.restype = None
+        f(C.byref(self._st), _ptr(g, self._real), self._real(gamma), C.c_int(bool(in_T_v)),
+          _ptr(self._g_bar, self._real))
+
     # -- Algorithm 3 on an arbitrary buffer ------------------------------------
     def onebit_allreduce(self, z):
         """Runs Algorithm 3 on z [n][d] with this state's errors; returns z_bar."""

@@ -367,3 +367,71 @@ def test_alg1_variance_bounds():
         assert (np.array_equal(o.v, v_before)) != in_v
         assert np.all(o.v >= 0) and o.v.max() <= g_max
         np.testing.assert_allclose(x_before - o.x[0], 1e-3 * o.m[0] / np.sqrt(v_before + 1e-8), rtol=1e-9, atol=1e-15)
+
+
+# --------------------------------------------------------------------------
+# Algorithm 2 (frozen-variance 1-bit framework; 1-bit Adam as a special case)
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_alg2_hand_worked(golden_dir, dtype):
+    fx = _load(golden_dir, "alg2_worked.json")
+    o = zo.Oracle(d=4, n=2, chunk=fx["chunk"], beta1=fx["beta1"], beta2=fx["beta2"], eps=fx["eps"], dtype=dtype)
+    o.set_params(fx["x0"])
+    tol = dict(rtol=0, atol=5e-7 if dtype == np.float32 else 1e-15)
+    for s in fx["steps"]:
+        o.alg2_step(np.array(s["g"], dtype), s["gamma"], s["in_T_v"])
+        for i in range(2):
+            np.testing.assert_allclose(o.m[i], np.array(s["m"], dtype), **tol)
+            np.testing.assert_allclose(o.x[i], np.array(s["x"], dtype), **tol)
+        np.testing.assert_allclose(o.v, np.array(s["v"], dtype), **tol)
+        np.testing.assert_allclose(o.delta, np.array(s["delta"], dtype), **tol)
+        np.testing.assert_allclose(o.delta_bar, np.array(s["delta_bar"], dtype), **tol)
+
+
+def test_alg2_identity_compressor_is_adam_and_equals_alg1_without_local_steps():
+    rng = np.random.default_rng(31)
+    n, d, T = 3, 50, 20
+    beta1, beta2, eps = 0.9, 0.999, 1e-8
+    g = rng.standard_normal((T, n, d))
+    gammas = 1e-3 * (1 + 0.05 * np.arange(T))
+    x0 = rng.standard_normal(d) * 0.02
+    two = zo.Oracle(d, n, 16, beta1, beta2, eps, dtype=np.float64, compressor=zo.IDENTITY)
+    one = zo.Oracle(d, n, 16, beta1, beta2, eps, dtype=np.float64, compressor=zo.IDENTITY)
+    two.set_params(x0), one.set_params(x0)
+    for t in range(T):
+        two.alg2_step(g[t], gammas[t], True)
+        one.step(g[t], gammas[t], t, True, True)
+    x, m, v = _adam_closed_form(g.mean(axis=1), gammas, beta1, beta2, eps, x0)
+    np.testing.assert_allclose(two.x[0], x, rtol=1e-10, atol=1e-13)
+    np.testing.assert_allclose(two.m[0], m, rtol=1e-10, atol=1e-14)
+    np.testing.assert_allclose(two.v, v, rtol=1e-11)
+    np.testing.assert_allclose(two.x, one.x, rtol=1e-9, atol=1e-13)     # Algorithm 1 with a sync at every step
+    np.testing.assert_allclose(two.m, one.m, rtol=1e-9, atol=1e-13)
+
+
+def test_alg2_one_bit_adam_special_case():
+    """T_v = the first T0 steps: plain Adam for T0 steps, then the variance is
+    frozen, the workers agree, and the received gradients telescope: their sum
+    is the sum of the true means minus the errors still held back."""
+    rng = np.random.default_rng(32)
+    n, d, T0, T = 4, 300, 5, 14
+    o = zo.Oracle(d, n, 64, dtype=np.float64)
+    x0 = rng.standard_normal(d) * 0.02
+    o.set_params(x0)
+    g = rng.standard_normal((T, n, d))
+    for t in range(T0):
+        o.alg2_step(g[t], 1e-3, True)
+    x, m, v = _adam_closed_form(g[:T0].mean(axis=1), [1e-3] * T0, 0.9, 0.999, 1e-8, x0)
+    np.testing.assert_allclose(o.x[0], x, rtol=1e-10, atol=1e-13)
+    assert np.all(o.delta == 0) and np.all(o.delta_bar == 0)
+    v_frozen, m_before = o.v.copy(), o.m[0].copy()
+    received = np.zeros(d)
+    for t in range(T0, T):
+        m_prev = o.m[0].copy()
+        o.alg2_step(g[t], 1e-3, False)
+        assert np.array_equal(o.v, v_frozen)
+        received += (o.m[0] - 0.9 * m_prev) / (1 - 0.9)             # the g_bar this step used
+        for i in range(1, n):
+            assert np.array_equal(o.x[i], o.x[0]) and np.array_equal(o.m[i], o.m[0])
+    np.testing.assert_allclose(received, g[T0:].mean(axis=1).sum(axis=0) - (o.delta.mean(axis=0) + o.delta_bar),
+                               rtol=0, atol=1e-11)
