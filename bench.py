@@ -45,6 +45,19 @@ def variance_bytes(n, W):
     return n * W * 4 + n * 8
 
 
+def alg2_compressed_bytes(n, W, chunk):
+    """Algorithm 2, compressed step: per parameter and worker read g, delta, m, x (16 B), write
+    delta, m, x (12 B) and 1 sign bit + a scale per chunk; per parameter read delta_bar, v,
+    write delta_bar (12 B) and 1 sign bit."""
+    n_chunks = -(-n // chunk)
+    return n * W * (28 + 1 / 8) + n_chunks * W * 4 + n * (12 + 1 / 8) + n_chunks * 4
+
+
+def alg2_full_bytes(n, W):
+    """Algorithm 2, T_v step: per parameter and worker read g, m, x, write m, x (20 B); v in and out."""
+    return n * W * 20 + n * 8
+
+
 def measured_hbm_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -191,9 +204,13 @@ def run_ours(args, wl):
         for t in range(K):
             bufs = stream.fill(t)                         # untimed: the batch is resident before the step starts
             ev[t][0].record()
-            opt.step_auto(bufs, wl.lr_at(t), t)
+            if args.algorithm == "alg2":
+                opt.alg2_step(bufs, wl.lr_at(t), t)
+                kinds.append("alg2_full" if wl.in_T_v(t) else "alg2_compressed")
+            else:
+                opt.step_auto(bufs, wl.lr_at(t), t)
+                kinds.append(("sync" if wl.in_T_u(t) else "local") + ("+var" if wl.in_T_v(t) else ""))
             ev[t][1].record()
-            kinds.append(("sync" if wl.in_T_u(t) else "local") + ("+var" if wl.in_T_v(t) else ""))
         barrier()
         wall = time.perf_counter() - wall0
     opt.check_device()
@@ -213,13 +230,17 @@ def run_ours(args, wl):
     # the variance update needs nothing beyond writing v_{t+1}: g and v are read anyway
     bytes_of["sync+var"] = bytes_of["sync"] + wl.n * 4
     bytes_of["local+var"] = bytes_of["local"] + wl.n * 4
+    bytes_of["alg2_compressed"] = alg2_compressed_bytes(wl.n, wl.W, wl.chunk)
+    bytes_of["alg2_full"] = alg2_full_bytes(wl.n, wl.W)
     step_types = {k: {"count": len(v), "ms": statistics.mean(v), "algorithmic_GB": bytes_of[k] / 1e9,
                       "GBps": bytes_of[k] / 1e6 / statistics.mean(v)} for k, v in by_kind.items()}
     total_bytes = sum(bytes_of[k] for k in kinds)
-    dominant = "sync" if "sync" in by_kind else ("sync+var" if "sync+var" in by_kind else kinds[0])
+    dominant = next((k for k in ("sync", "sync+var", "alg2_compressed") if k in by_kind), kinds[0])
     achieved = bytes_of[dominant] / 1e6 / statistics.mean(by_kind[dominant])
     sync_kernel = "step_sync_kernel" if args.no_pipeline else "step_sync_pipelined_kernel"
-    roofline = {"bound": "hbm", "kernel": sync_kernel if dominant.startswith("sync") else "local_step_kernel",
+    kernel_of = {"sync": sync_kernel, "sync+var": sync_kernel, "alg2_compressed": "alg2_compressed_kernel",
+                 "alg2_full": "alg2_full_kernel"}
+    roofline = {"bound": "hbm", "kernel": kernel_of.get(dominant, "local_step_kernel"),
                 "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "peak_kind": f"of {peak_kind}", "frac_of_8TBps_nominal": achieved / 8000.0,
                 # ncu (dram__bytes_read.sum + dram__bytes_write.sum) on the layout shrunk 16x gave
@@ -232,7 +253,7 @@ def run_ours(args, wl):
 
     # ---- end to end: host gradients in, worker 0's model out, through zoa_step_host ----
     e2e = None
-    if args.e2e_steps > 0:
+    if args.e2e_steps > 0 and args.algorithm == "alg1":
         ke = max(1, min(args.e2e_steps, K))
         host_g = torch.empty(wl.n, dtype=torch.float32).pin_memory()
         host_g.copy_(stream.bufs[0])
@@ -269,6 +290,8 @@ def run_ours(args, wl):
                 "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
                 "data": "synthetic",
                 "config": {"workload": wl.name, "n_params": wl.n, "W": wl.W, "chunk": wl.chunk,
+                           "algorithm": "Algorithm 1 (0/1 Adam)" if args.algorithm == "alg1" else
+                                        "Algorithm 2 (gradients through the 1-bit AllReduce, full precision on T_v steps)",
                            "schedule": f"t=0..{K - 1} of the workload's T_u/T_v policies",
                            "l2": "inputs larger than L2 (gradients and state are read once per step)",
                            "parallelism": f"{world} x independent chunk ranges, no collective"},
@@ -359,6 +382,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--scale", type=int, default=1, help="shrink every tensor by this factor (profiling captures)")
     ap.add_argument("--no-pipeline", action="store_true", help="fused sync step through the chunk-per-block kernel")
+    ap.add_argument("--algorithm", default="alg1", choices=["alg1", "alg2"],
+                    help="alg1: 0/1 Adam (the headline); alg2: the paper's frozen-variance 1-bit framework")
     ap.add_argument("--sweep", nargs="?", const="full", default=None, choices=["full", "quick"],
                     help="time the compress / decompress-average kernels over the size grid instead")
     ap.add_argument("--sweep-reps", type=int, default=3)

@@ -128,6 +128,18 @@ zoa_status zoa_onebit_average(zoa_handle h, void *stream);
 zoa_status zoa_step_sync(zoa_handle h, const float *const *grads, float lr, int64_t t,
                          void *stream);
 
+/* One iteration of Algorithm 2 (the frozen-variance framework that exchanges
+ * gradients, not accumulated updates; 1-bit Adam when T_v is an initial run of
+ * steps).  If t is in T_v: g_bar = mean of the W gradients (Algorithm 4) and the
+ * variance moves (effective from the next step); otherwise g_bar is the output
+ * of the error-feedback 1-bit AllReduce of the gradients (Algorithm 3, same
+ * error buffers and wire buffers as zoa_onebit_reduce).  Then on every worker
+ * m = beta1 m + (1 - beta1) g_bar and x = x - lr m / sqrt(v_t + eps), m being the
+ * momentum just computed (the convention that makes this the no-local-step case
+ * of Algorithm 1).  u, x_sync and the sum of learning rates are not touched.
+ * Arguments and errors as zoa_step. */
+zoa_status zoa_alg2_step(zoa_handle h, const float *const *grads, float lr, int64_t t, void *stream);
+
 /* One iteration of Algorithm 1 under the handle's own policies: zoa_step_sync
  * if t is in T_u, else zoa_step. */
 zoa_status zoa_step_auto(zoa_handle h, const float *const *grads, float lr, int64_t t,

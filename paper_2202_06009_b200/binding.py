@@ -49,6 +49,7 @@ def _load():
         "zoa_onebit_average": ([H, p], C.c_int),
         "zoa_step_sync": ([H, C.POINTER(p), C.c_float, C.c_int64, p], C.c_int),
         "zoa_step_auto": ([H, C.POINTER(p), C.c_float, C.c_int64, p], C.c_int),
+        "zoa_alg2_step": ([H, C.POINTER(p), C.c_float, C.c_int64, p], C.c_int),
         "zoa_step_host": ([H, C.POINTER(p), C.c_float, C.c_int64, p, p], C.c_int),
         "zoa_get_buffer": ([H, C.c_int, C.c_int, C.POINTER(p), C.POINTER(C.c_size_t)], C.c_int),
         "zoa_copy_out": ([H, C.c_int, C.c_int, C.c_size_t, C.c_size_t, p], C.c_int),
@@ -140,6 +141,10 @@ def zoa_step_sync(h, grad_ptrs, lr, t, stream=0):
 
 def zoa_step_auto(h, grad_ptrs, lr, t, stream=0):
     _check(h, lib.zoa_step_auto(h, _ptr_array(grad_ptrs), lr, t, stream))
+
+
+def zoa_alg2_step(h, grad_ptrs, lr, t, stream=0):
+    _check(h, lib.zoa_alg2_step(h, _ptr_array(grad_ptrs), lr, t, stream))
 
 
 def zoa_step_host(h, host_grad_ptrs, lr, t, host_x_out_ptr=None, stream=0):

@@ -353,6 +353,22 @@ extern "C" zoa_status zoa_step_sync(zoa_handle h, const float *const *grads, flo
     return ZOA_OK;
 }
 
+extern "C" zoa_status zoa_alg2_step(zoa_handle h, const float *const *grads, float lr, int64_t t, void *stream)
+{
+    GradPtrs gp;
+    bool aligned;
+    zoa_status rc = check_step_args(h, grads, lr, t, &gp, &aligned, "zoa_alg2_step");
+    if (rc != ZOA_OK) return rc;
+    commit_variance(h);
+    const bool full = zoa_var_due(h, t) == 1;
+    ZOA_CUDA(h, launch_alg2(view(h), gp, h->c, lr, full, aligned, h->sm_count, static_cast<cudaStream_t>(stream)));
+    h->n_launches += 1;
+    if (full) { h->v_pending = true; h->n_var_updates += 1; } else h->n_syncs += 1;
+    h->t_last = t;
+    h->n_steps += 1;
+    return ZOA_OK;
+}
+
 extern "C" zoa_status zoa_step_auto(zoa_handle h, const float *const *grads, float lr, int64_t t, void *stream)
 {
     if (!h) return ZOA_ERR_ARG;

@@ -16,6 +16,9 @@ cudaError_t launch_reduce(const StateView &st, const Consts &c, float gamma_sum,
 cudaError_t launch_step_sync(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
                              float gamma_sum, bool g_aligned, long long first_chunk, long long count, cudaStream_t s);
 
+cudaError_t launch_alg2(const StateView &st, const GradPtrs &g, const Consts &c, float gamma, bool full_precision,
+                        bool g_aligned, int sm_count, cudaStream_t s);
+
 // Pipelined (bulk-copy ring) form of the fused sync step, zoa_pipeline.cu.
 int pipeline_stages(const StateView &st, bool g_aligned);
 cudaError_t launch_step_sync_pipelined(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,

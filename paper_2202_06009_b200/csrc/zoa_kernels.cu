@@ -322,6 +322,158 @@ __global__ void step_sync_kernel(StateView st, GradPtrs g, Consts c, float gamma
 }
 
 // ---------------------------------------------------------------------------
+// Algorithm 2: the frozen-variance framework that exchanges gradients instead of
+// accumulated updates (1-bit Adam when T_v is an initial run of steps).
+// ---------------------------------------------------------------------------
+
+// A T_v step of Algorithm 2 (lines 4-5, 10-11): full-precision mean of the
+// gradients, momentum and model update with v_t on every worker, then v_{t+1}.
+__global__ void __launch_bounds__(256)
+alg2_full_kernel(StateView st, GradPtrs g, Consts c, float gamma, int g_aligned)
+{
+    const long long n4 = (st.n + 3) >> 2;
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x; q < n4; q += stride) {
+        const long long j = q << 2;
+        double G[4] = {0.0, 0.0, 0.0, 0.0};
+        for (int i = 0; i < st.W; ++i) {
+            const float4 g4 = ld_grad4(g.p[i], j, st.n, g_aligned);
+            G[0] += (double)g4.x; G[1] += (double)g4.y; G[2] += (double)g4.z; G[3] += (double)g4.w;
+        }
+        const float4 v4 = ld4(st.v + j);
+        const float vv[4] = {v4.x, v4.y, v4.z, v4.w};
+        float gb[4], d[4], vo[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            gb[k] = mean_round(G[k], st.W);                     // line 4 (Algorithm 4)
+            d[k] = denom(c, vv[k]);
+            vo[k] = variance(c, vv[k], gb[k]);                  // line 5
+        }
+        st4(st.v_next + j, make_float4(vo[0], vo[1], vo[2], vo[3]));
+        for (int i = 0; i < st.W; ++i) {
+            const long long row = (long long)i * st.n_pad + j;
+            const float4 m4 = ld4(st.m + row), x4 = ld4(st.x + row);
+            const float mm[4] = {m4.x, m4.y, m4.z, m4.w}, xx[4] = {x4.x, x4.y, x4.z, x4.w};
+            float mo[4], xo[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                mo[k] = momentum(c, mm[k], gb[k]);                              // line 10
+                xo[k] = f_sub(xx[k], f_div(f_mul(gamma, mo[k]), d[k]));         // line 11
+            }
+            st4(st.m + row, make_float4(mo[0], mo[1], mo[2], mo[3]));
+            st4(st.x + row, make_float4(xo[0], xo[1], xo[2], xo[3]));
+        }
+    }
+}
+
+// Any other step of Algorithm 2 for chunk blockIdx.x (lines 7, 10-11): the
+// gradients go through the error-feedback 1-bit AllReduce (Algorithm 3), the
+// decompressed mean drives momentum and model on every worker.
+__global__ void __launch_bounds__(512, 2) alg2_compressed_kernel(StateView st, GradPtrs g, Consts c, float gamma, int g_aligned)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    double *scratch = reinterpret_cast<double *>(smem_raw);
+    double *A_s = scratch + 34;
+    float *z_s = reinterpret_cast<float *>(A_s + st.chunk);
+    const ChunkGeom cg = chunk_geom(st, blockIdx.x);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+
+    for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
+        const int idx = base + 4 * lane;
+        if (idx < cg.len) { A_s[idx] = 0.0; A_s[idx + 1] = 0.0; A_s[idx + 2] = 0.0; A_s[idx + 3] = 0.0; }
+    }
+    for (int i = 0; i < st.W; ++i) {
+        const long long row = (long long)i * st.n_pad + cg.c0;
+        double l1 = 0.0;
+        for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
+            const int idx = base + 4 * lane;
+            if (idx < cg.len) {
+                const float4 g4 = ld_grad4(g.p[i], cg.c0 + idx, st.n, g_aligned);
+                const float4 e4 = ld4_stream(st.dw + row + idx);
+                const float4 z4 = make_float4(f_add(g4.x, e4.x), f_add(g4.y, e4.y), f_add(g4.z, e4.z), f_add(g4.w, e4.w));
+                st4(z_s + idx, z4);
+                l1 += fabs((double)z4.x) + fabs((double)z4.y) + fabs((double)z4.z) + fabs((double)z4.w);
+            }
+        }
+        const float scale = chunk_scale(block_sum(l1, scratch), cg.len);
+        for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
+            const int idx = base + 4 * lane;
+            float z[4] = {0.f, 0.f, 0.f, 0.f}, hat[4];
+            if (idx < cg.len) {
+                const float4 z4 = ld4(z_s + idx);
+                z[0] = z4.x; z[1] = z4.y; z[2] = z4.z; z[3] = z4.w;
+            }
+            const uint32_t word = compress_tile(z, hat, scale, idx, cg.len);
+            if (idx < cg.len) {
+                st4_stream(st.dw + row + idx, make_float4(z[0], z[1], z[2], z[3]));
+#pragma unroll
+                for (int k = 0; k < 4; ++k) A_s[idx + k] += (double)hat[k];
+            }
+            if (lane < 4 && base + 32 * lane < cg.len)
+                st.words_w[(long long)i * st.words_stride + ((cg.c0 + base) >> 5) + lane] = word;
+        }
+        if (threadIdx.x == 0) st.scales_w[(long long)i * st.n_chunks + blockIdx.x] = scale;
+    }
+    double l1 = 0.0;
+    for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
+        const int idx = base + 4 * lane;
+        if (idx < cg.len) {
+            const float4 e4 = ld4(st.ds + cg.c0 + idx);
+            const float ee[4] = {e4.x, e4.y, e4.z, e4.w};
+            float a[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                a[k] = idx + k < cg.len ? server_input(A_s[idx + k], st.W, ee[k]) : 0.0f;
+                l1 += fabs((double)a[k]);
+            }
+            st4(z_s + idx, make_float4(a[0], a[1], a[2], a[3]));
+        }
+    }
+    const float scale = chunk_scale(block_sum(l1, scratch), cg.len);
+    for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
+        const int idx = base + 4 * lane;
+        float a[4] = {0.f, 0.f, 0.f, 0.f}, gb[4];
+        if (idx < cg.len) {
+            const float4 a4 = ld4(z_s + idx);
+            a[0] = a4.x; a[1] = a4.y; a[2] = a4.z; a[3] = a4.w;
+        }
+        const uint32_t word = compress_tile(a, gb, scale, idx, cg.len);   // gb = the mean gradient the workers receive
+        if (lane < 4 && base + 32 * lane < cg.len) st.words_s[((cg.c0 + base) >> 5) + lane] = word;
+        if (idx >= cg.len) continue;
+        const long long j = cg.c0 + idx;
+        st4(st.ds + j, make_float4(a[0], a[1], a[2], a[3]));
+        const float4 v4 = ld4(st.v + j);
+        const float d[4] = {denom(c, v4.x), denom(c, v4.y), denom(c, v4.z), denom(c, v4.w)};
+        // four workers at a time: all eight loads are issued before the first dependent store
+        for (int i0 = 0; i0 < st.W; i0 += 4) {
+            float4 m4[4], x4[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                if (i0 + q < st.W) {
+                    const long long row = (long long)(i0 + q) * st.n_pad + j;
+                    m4[q] = ld4_stream(st.m + row);
+                    x4[q] = ld4_stream(st.x + row);
+                }
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                if (i0 + q < st.W) {
+                    const long long row = (long long)(i0 + q) * st.n_pad + j;
+                    const float mm[4] = {m4[q].x, m4[q].y, m4[q].z, m4[q].w}, xx[4] = {x4[q].x, x4[q].y, x4[q].z, x4[q].w};
+                    float mo[4], xo[4];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        mo[k] = momentum(c, mm[k], gb[k]);                              // line 10
+                        xo[k] = f_sub(xx[k], f_div(f_mul(gamma, mo[k]), d[k]));         // line 11
+                    }
+                    st4_stream(st.m + row, make_float4(mo[0], mo[1], mo[2], mo[3]));
+                    st4_stream(st.x + row, make_float4(xo[0], xo[1], xo[2], xo[3]));
+                }
+        }
+    }
+    if (threadIdx.x == 0) st.scales_s[blockIdx.x] = scale;
+}
+
+// ---------------------------------------------------------------------------
 // Launchers
 // ---------------------------------------------------------------------------
 static int block_threads_for_chunk(int chunk)
@@ -378,7 +530,20 @@ cudaError_t configure_kernels()
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(reduce_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)reduce_smem(kMaxChunk));
     if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(alg2_compressed_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)step_sync_smem(kMaxChunk));
+    if (e != cudaSuccess) return e;
     return cudaFuncSetAttribute(step_sync_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)step_sync_smem(kMaxChunk));
+}
+
+cudaError_t launch_alg2(const StateView &st, const GradPtrs &g, const Consts &c, float gamma, bool full_precision,
+                        bool g_aligned, int sm_count, cudaStream_t s)
+{
+    if (full_precision)
+        alg2_full_kernel<<<elementwise_grid((st.n + 3) / 4, sm_count), 256, 0, s>>>(st, g, c, gamma, g_aligned);
+    else
+        alg2_compressed_kernel<<<(unsigned)st.n_chunks, block_threads_for_chunk(st.chunk), step_sync_smem(st.chunk), s>>>(
+            st, g, c, gamma, g_aligned);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_compress(const StateView &st, cudaStream_t s)

@@ -104,6 +104,9 @@ class Zoa:
     def step_auto(self, grads, lr, t):
         B.zoa_step_auto(self.h, _grad_ptrs(grads, self.n, self.W), lr, t, _stream())
 
+    def alg2_step(self, grads, lr, t):
+        B.zoa_alg2_step(self.h, _grad_ptrs(grads, self.n, self.W), lr, t, _stream())
+
     def step_host(self, host_grads, lr, t, host_x_out=None):
         ptrs = [g.data_ptr() for g in host_grads]
         out = host_x_out.data_ptr() if host_x_out is not None else None

@@ -359,3 +359,47 @@ def test_device_wait_runs_out_and_is_reported():
         z.check_device()                                  # flag cleared, chunk counter rearmed
     finally:
         z.close()
+
+
+# --------------------------------------------------------------------------
+# Algorithm 2 (gradients through the 1-bit AllReduce; 1-bit Adam special case)
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("W,chunk,n", [(3, 2048, 1), (3, 2048, 33), (3, 2048, 2049), (2, 64, 4096 + 5), (5, 96, 96 * 7 + 3),
+                                       (8, 4096, 3 * 4096 + 1852), (4, 8192, 8192 * 2 + 704), (2, 16384, 16384 * 2 + 100),
+                                       (64, 256, 1500), (16, 4096, 40 * 4096 + 77)])
+def test_alg2_parity(W, chunk, n):
+    """Ten steps of Algorithm 2: a full-precision stage (T_v = {0,1,2}) then compressed steps,
+    i.e. the 1-bit Adam special case; every state after every step."""
+    rng = np.random.default_rng(W + chunk + n)
+    p = Pair(n, W, chunk, var_steps=(0, 1, 2), x0=rng.standard_normal(n) * 0.02)
+    try:
+        for t in range(10):
+            g = _grads(rng, W, n)
+            p.gpu.alg2_step(list(torch.from_numpy(g).cuda()), 1e-3 * (1 + t % 3), t)
+            torch.cuda.synchronize()
+            p.cpu.alg2_step(g, np.float32(1e-3 * (1 + t % 3)), t in (0, 1, 2))
+            p.compare(f"t={t}", wire=t > 2)
+        p.padding_is_zero()
+        s = p.gpu.stats()
+        assert s["n_var_updates"] == 3 and s["n_syncs"] == 7 and s["n_steps"] == 10
+    finally:
+        p.close()
+
+
+def test_alg2_unaligned_and_interleaved_variance_steps():
+    rng = np.random.default_rng(55)
+    n, W, chunk = 5000, 3, 1024
+    p = Pair(n, W, chunk, var_steps=(0, 3, 4), x0=rng.standard_normal(n) * 0.02)
+    try:
+        for t in range(7):
+            g = _grads(rng, W, n)
+            backing = torch.zeros(W, n + 8, device="cuda")
+            views = [backing[i, 1:1 + n] for i in range(W)]
+            for i in range(W):
+                views[i].copy_(torch.from_numpy(g[i]))
+            p.gpu.alg2_step(views, 2e-3, t)
+            torch.cuda.synchronize()
+            p.cpu.alg2_step(g, np.float32(2e-3), t in (0, 3, 4))
+            p.compare(f"t={t}", wire=False)
+    finally:
+        p.close()
