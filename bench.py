@@ -238,6 +238,8 @@ def run_ours(args, wl):
     dominant = next((k for k in ("sync", "sync+var", "alg2_compressed") if k in by_kind), kinds[0])
     achieved = bytes_of[dominant] / 1e6 / statistics.mean(by_kind[dominant])
     sync_kernel = "step_sync_kernel" if args.no_pipeline else "step_sync_pipelined_kernel"
+    if wl.chunk > 16384:
+        sync_kernel = "local_step_kernel + lc_* (multi-pass large-chunk kernels)"
     kernel_of = {"sync": sync_kernel, "sync+var": sync_kernel, "alg2_compressed": "alg2_compressed_kernel",
                  "alg2_full": "alg2_full_kernel"}
     roofline = {"bound": "hbm", "kernel": kernel_of.get(dominant, "local_step_kernel"),
@@ -382,6 +384,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--scale", type=int, default=1, help="shrink every tensor by this factor (profiling captures)")
     ap.add_argument("--no-pipeline", action="store_true", help="fused sync step through the chunk-per-block kernel")
+    ap.add_argument("--chunk", type=int, default=0,
+                    help="override the workload's chunk (e.g. 1073741824 = one magnitude for the whole vector, Eq. 3 as printed)")
     ap.add_argument("--algorithm", default="alg1", choices=["alg1", "alg2"],
                     help="alg1: 0/1 Adam (the headline); alg2: the paper's frozen-variance 1-bit framework")
     ap.add_argument("--sweep", nargs="?", const="full", default=None, choices=["full", "quick"],
@@ -409,6 +413,8 @@ def main():
     wl = synth.WORKLOADS[args.workload]()
     if args.scale > 1:
         wl = synth.scaled(wl, args.scale)
+    if args.chunk:
+        wl.chunk = args.chunk
     if args.steps is None:
         args.steps = wl.steps
     run_ours(args, wl)

@@ -69,7 +69,10 @@ typedef struct {
  * CUDA device.  chunk is the number of consecutive coordinates that share one
  * magnitude in the compressor of Eq. 3 (chunk >= n_params gives Eq. 3 as printed).
  * Requires n_params >= 1, 1 <= W <= 64, 0 <= beta < 1, eps > 0, chunk a
- * multiple of 32 in [32, 16384].  Allocates device memory (cudaMalloc). */
+ * multiple of 32 in [32, 2^30].  Chunks up to 16384 are handled by one thread
+ * block each (the fast kernels); larger ones, up to the whole vector, by
+ * multi-pass kernels that take each l1 norm in two steps.  Allocates device
+ * memory (cudaMalloc). */
 zoa_status zoa_create(zoa_handle *out, size_t n_params, int W, float beta1, float beta2,
                       float eps, int chunk);
 
@@ -88,6 +91,25 @@ zoa_status zoa_set_var_steps(zoa_handle h, const int64_t *steps, size_t count);
 /* T_v by the rule of the paragraph "Policy for T_v and T_u": the j-th update is
  * at k_j with k_0 = 0 and k_{j+1} - k_j = 2^floor(j / kappa), for k_j < freeze_at. */
 zoa_status zoa_set_var_policy_doubling(zoa_handle h, int kappa, int64_t freeze_at);
+
+/* The two schedules of the paragraph "Policy for T_v and T_u" as plain host
+ * functions (no handle, no GPU).  Both return the number of entries the full
+ * answer has and write at most `capacity` of them (pass NULL, 0 to size).
+ * zoa_policy_var_steps: k_0 = 0, k_{j+1} - k_j = 2^floor(j / kappa) while
+ * k_j < freeze_at (the paper uses kappa = 16).
+ * zoa_policy_sync_pieces: the interval between syncs is 1 through the learning
+ * rate warm-up and then doubles every `double_every` steps (the steps in which
+ * the learning rate halves), never above max_interval (the paper: warm-up 12.5K
+ * steps, 32678, 16 for BERT); returned as pieces for zoa_set_sync_policy. */
+size_t zoa_policy_var_steps(int kappa, int64_t freeze_at, int64_t *out, size_t capacity);
+size_t zoa_policy_sync_pieces(int64_t warmup, int64_t double_every, int32_t max_interval,
+                              int64_t *boundaries, int32_t *intervals, size_t capacity);
+
+/* Installs zoa_policy_sync_pieces on the handle.  With freeze_variance != 0 it
+ * also drops every T_v step from the first step whose sync interval exceeds 1
+ * (the paper stops updating the variance there); call it after the T_v setter. */
+zoa_status zoa_set_sync_policy_doubling(zoa_handle h, int64_t warmup, int64_t double_every,
+                                        int32_t max_interval, int freeze_variance);
 
 /* T_u of Algorithm 1 as a piecewise-constant interval: piece r starts at step
  * boundaries[r] (host, strictly increasing, boundaries[0] = 0) and has a sync

@@ -41,6 +41,10 @@ def _load():
         "zoa_set_var_steps": ([H, C.POINTER(C.c_int64), C.c_size_t], C.c_int),
         "zoa_set_var_policy_doubling": ([H, C.c_int, C.c_int64], C.c_int),
         "zoa_set_sync_policy": ([H, C.POINTER(C.c_int64), C.POINTER(C.c_int32), C.c_size_t], C.c_int),
+        "zoa_policy_var_steps": ([C.c_int, C.c_int64, C.POINTER(C.c_int64), C.c_size_t], C.c_size_t),
+        "zoa_policy_sync_pieces": ([C.c_int64, C.c_int64, C.c_int32, C.POINTER(C.c_int64), C.POINTER(C.c_int32),
+                                    C.c_size_t], C.c_size_t),
+        "zoa_set_sync_policy_doubling": ([H, C.c_int64, C.c_int64, C.c_int32, C.c_int], C.c_int),
         "zoa_sync_due": ([H, C.c_int64], C.c_int),
         "zoa_var_due": ([H, C.c_int64], C.c_int),
         "zoa_step": ([H, C.POINTER(p), C.c_float, C.c_int64, p], C.c_int),
@@ -109,6 +113,24 @@ def zoa_set_sync_policy(h, boundaries, intervals):
     b = (C.c_int64 * len(boundaries))(*boundaries)
     k = (C.c_int32 * len(intervals))(*intervals)
     _check(h, lib.zoa_set_sync_policy(h, b, k, len(boundaries)))
+
+
+def zoa_policy_var_steps(kappa, freeze_at):
+    n = lib.zoa_policy_var_steps(kappa, freeze_at, None, 0)
+    out = (C.c_int64 * n)()
+    lib.zoa_policy_var_steps(kappa, freeze_at, out, n)
+    return list(out)
+
+
+def zoa_policy_sync_pieces(warmup, double_every, max_interval):
+    n = lib.zoa_policy_sync_pieces(warmup, double_every, max_interval, None, None, 0)
+    b, k = (C.c_int64 * n)(), (C.c_int32 * n)()
+    lib.zoa_policy_sync_pieces(warmup, double_every, max_interval, b, k, n)
+    return list(b), list(k)
+
+
+def zoa_set_sync_policy_doubling(h, warmup, double_every, max_interval, freeze_variance=True):
+    _check(h, lib.zoa_set_sync_policy_doubling(h, warmup, double_every, max_interval, int(bool(freeze_variance))))
 
 
 def zoa_sync_due(h, t):

@@ -25,6 +25,8 @@ struct zoa_handle_s {
     float *staging = nullptr;      // [W][n_pad], device copy of host gradients (zoa_step_host)
     int *error_flag = nullptr;     // device int: a kernel gave up on a bounded wait
     unsigned long long *sched = nullptr;   // device [2]: chunk counter of the persistent kernel, finished blocks
+    double *partials = nullptr;    // device [W + 1][n_chunks * segments]: per-segment l1 sums, chunk > 16384 only
+    bool large_chunk = false;
     bool use_pipeline = true;      // bulk-copy ring form of the fused sync step where the shape allows
     int wait_limit_ms = 2000;      // bound on every device-side wait
     long long test_stop_after_tiles = 0;   // error-path test hook, see zoa_set_option
@@ -70,7 +72,7 @@ static StateView view(zoa_handle h)
 static void free_all(zoa_handle h)
 {
     void *ptrs[] = {h->x, h->m, h->u, h->dw, h->v_cur, h->v_nxt, h->ds, h->xs,
-                    h->words_w, h->words_s, h->scales_w, h->scales_s, h->staging, h->error_flag, h->sched};
+                    h->words_w, h->words_s, h->scales_w, h->scales_s, h->staging, h->error_flag, h->sched, h->partials};
     for (void *p : ptrs)
         if (p) cudaFree(p);
 }
@@ -93,8 +95,8 @@ extern "C" zoa_status zoa_create(zoa_handle *out, size_t n_params, int W, float 
     if (!(beta1 >= 0.f && beta1 < 1.f) || !(beta2 >= 0.f && beta2 < 1.f))
         return fail(nullptr, ZOA_ERR_ARG, "zoa_create: beta1 and beta2 must be in [0, 1)");
     if (!(eps > 0.f) || !std::isfinite(eps)) return fail(nullptr, ZOA_ERR_ARG, "zoa_create: eps must be positive");
-    if (chunk < 32 || chunk > kMaxChunk || chunk % 32 != 0)
-        return fail(nullptr, ZOA_ERR_ARG, "zoa_create: chunk must be a multiple of 32 in [32, 16384]");
+    if (chunk < 32 || chunk > (1 << 30) || chunk % 32 != 0)
+        return fail(nullptr, ZOA_ERR_ARG, "zoa_create: chunk must be a multiple of 32 in [32, 2^30]");
 
     zoa_handle h = new (std::nothrow) zoa_handle_s;
     if (!h) return fail(nullptr, ZOA_ERR_ALLOC, "zoa_create: out of host memory");
@@ -122,8 +124,12 @@ extern "C" zoa_status zoa_create(zoa_handle *out, size_t n_params, int W, float 
         (e = alloc_zero(&h->words_s, (size_t)h->words_stride)) == cudaSuccess &&
         (e = alloc_zero(&h->scales_w, (size_t)W * h->n_chunks)) == cudaSuccess &&
         (e = alloc_zero(&h->scales_s, (size_t)h->n_chunks)) == cudaSuccess &&
-        (e = alloc_zero(&h->error_flag, 1)) == cudaSuccess && (e = alloc_zero(&h->sched, 2)) == cudaSuccess)
-        e = cudaDeviceSynchronize();
+        (e = alloc_zero(&h->error_flag, 1)) == cudaSuccess && (e = alloc_zero(&h->sched, 2)) == cudaSuccess) {
+        h->large_chunk = chunk > kMaxChunk;
+        if (h->large_chunk)
+            e = alloc_zero(&h->partials, (size_t)(W + 1) * (size_t)h->n_chunks * (size_t)large_chunk_segments(view(h)));
+        if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    }
     if (e != cudaSuccess) {
         free_all(h);
         delete h;
@@ -168,17 +174,71 @@ extern "C" zoa_status zoa_set_var_steps(zoa_handle h, const int64_t *steps, size
     return ZOA_OK;
 }
 
+// ---- the paper's schedules as plain host functions (no handle, no GPU) ----------------------
+
+// T_v: k_0 = 0, k_{j+1} - k_j = 2^floor(j / kappa), for k_j < freeze_at.
+extern "C" size_t zoa_policy_var_steps(int kappa, int64_t freeze_at, int64_t *out, size_t capacity)
+{
+    if (kappa < 1 || freeze_at < 0) return 0;
+    size_t count = 0;
+    int64_t k = 0;
+    for (int64_t j = 0; k < freeze_at; ++j) {
+        if (out && count < capacity) out[count] = k;
+        ++count;
+        const int64_t e = j / kappa;
+        if (e >= 62) break;
+        k += (int64_t)1 << e;
+    }
+    return count;
+}
+
+// T_u: the interval between syncs is 1 through the warm-up and then doubles every `double_every`
+// steps, as the learning rate halves: interval(t) = min(2^floor((t - warmup) / double_every), max_interval)
+// for t >= warmup.  Written as pieces (boundary, interval).
+extern "C" size_t zoa_policy_sync_pieces(int64_t warmup, int64_t double_every, int32_t max_interval,
+                                         int64_t *boundaries, int32_t *intervals, size_t capacity)
+{
+    if (warmup < 0 || double_every < 1 || max_interval < 1) return 0;
+    size_t count = 0;
+    auto push = [&](int64_t b, int32_t k) {
+        if (boundaries && intervals && count < capacity) { boundaries[count] = b; intervals[count] = k; }
+        ++count;
+    };
+    push(0, 1);
+    int32_t interval = 1;
+    for (int64_t r = 1; interval < max_interval; ++r) {
+        interval = interval > max_interval / 2 ? max_interval : interval * 2;
+        push(warmup + r * double_every, interval);
+    }
+    return count;
+}
+
 extern "C" zoa_status zoa_set_var_policy_doubling(zoa_handle h, int kappa, int64_t freeze_at)
 {
     if (!h) return ZOA_ERR_ARG;
     if (kappa < 1 || freeze_at < 0) return fail(h, ZOA_ERR_ARG, "zoa_set_var_policy_doubling: kappa >= 1, freeze_at >= 0");
-    h->var_steps.clear();
-    int64_t k = 0;
-    for (int64_t j = 0; k < freeze_at; ++j) {
-        h->var_steps.push_back(k);
-        const int64_t e = j / kappa;
-        if (e >= 62) break;
-        k += (int64_t)1 << e;  // k_{j+1} - k_j = 2^floor(j / kappa)
+    const size_t count = zoa_policy_var_steps(kappa, freeze_at, nullptr, 0);
+    h->var_steps.assign(count, 0);
+    zoa_policy_var_steps(kappa, freeze_at, h->var_steps.data(), count);
+    return ZOA_OK;
+}
+
+extern "C" zoa_status zoa_set_sync_policy_doubling(zoa_handle h, int64_t warmup, int64_t double_every,
+                                                   int32_t max_interval, int freeze_variance)
+{
+    if (!h) return ZOA_ERR_ARG;
+    const size_t count = zoa_policy_sync_pieces(warmup, double_every, max_interval, nullptr, nullptr, 0);
+    if (count == 0) return fail(h, ZOA_ERR_ARG, "zoa_set_sync_policy_doubling: warmup >= 0, double_every >= 1, max_interval >= 1");
+    h->sync_bounds.assign(count, 0);
+    h->sync_intervals.assign(count, 1);
+    zoa_policy_sync_pieces(warmup, double_every, max_interval, h->sync_bounds.data(), h->sync_intervals.data(), count);
+    if (freeze_variance) {
+        // no variance updates once the interval between syncs exceeds 1
+        int64_t first_sparse = -1;
+        for (size_t r = 0; r < count; ++r)
+            if (h->sync_intervals[r] > 1) { first_sparse = h->sync_bounds[r]; break; }
+        if (first_sparse >= 0)
+            h->var_steps.erase(std::lower_bound(h->var_steps.begin(), h->var_steps.end(), first_sparse), h->var_steps.end());
     }
     return ZOA_OK;
 }
@@ -247,6 +307,35 @@ static void commit_variance(zoa_handle h)
     }
 }
 
+// Worker side / server side of the 1-bit AllReduce of u, by the kernels that fit the chunk size.
+static cudaError_t run_compress(zoa_handle h, cudaStream_t s)
+{
+    int launches = 0;
+    cudaError_t e;
+    if (h->large_chunk) {
+        GradPtrs none{};
+        e = launch_large_compress(view(h), none, false, true, h->partials, &launches, s);
+    } else {
+        e = launch_compress(view(h), s);
+        launches = 1;
+    }
+    h->n_launches += launches;
+    return e;
+}
+static cudaError_t run_server(zoa_handle h, float gamma_sum, cudaStream_t s)
+{
+    int launches = 0;
+    cudaError_t e;
+    if (h->large_chunk) {
+        e = launch_large_server(view(h), h->c, 1, gamma_sum, h->partials, &launches, s);
+    } else {
+        e = launch_reduce(view(h), h->c, gamma_sum, s);
+        launches = 1;
+    }
+    h->n_launches += launches;
+    return e;
+}
+
 extern "C" zoa_status zoa_step(zoa_handle h, const float *const *grads, float lr, int64_t t, void *stream)
 {
     GradPtrs gp;
@@ -272,10 +361,8 @@ extern "C" zoa_status zoa_onebit_reduce(zoa_handle h, void *stream)
         return fail(h, ZOA_ERR_STATE, "zoa_onebit_reduce: nothing accumulated since the last sync (sum of learning rates is not positive)");
     if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, "zoa_onebit_reduce: the handle's device is not the current CUDA device");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const StateView st = view(h);
-    ZOA_CUDA(h, launch_compress(st, s));
-    ZOA_CUDA(h, launch_reduce(st, h->c, gamma_sum, s));
-    h->n_launches += 2;
+    ZOA_CUDA(h, run_compress(h, s));
+    ZOA_CUDA(h, run_server(h, gamma_sum, s));
     h->gamma_sum = 0.0;
     h->t_sync = h->t_last;
     h->n_syncs += 1;
@@ -285,8 +372,7 @@ extern "C" zoa_status zoa_onebit_reduce(zoa_handle h, void *stream)
 extern "C" zoa_status zoa_onebit_compress(zoa_handle h, void *stream)
 {
     if (!h) return ZOA_ERR_ARG;
-    ZOA_CUDA(h, launch_compress(view(h), static_cast<cudaStream_t>(stream)));
-    h->n_launches += 1;
+    ZOA_CUDA(h, run_compress(h, static_cast<cudaStream_t>(stream)));
     return ZOA_OK;
 }
 
@@ -296,8 +382,7 @@ extern "C" zoa_status zoa_onebit_average(zoa_handle h, void *stream)
     const float gamma_sum = (float)h->gamma_sum;
     if (!(h->gamma_sum > 0.0) || !(gamma_sum > 0.f) || !std::isfinite(gamma_sum))
         return fail(h, ZOA_ERR_STATE, "zoa_onebit_average: nothing accumulated since the last sync (sum of learning rates is not positive)");
-    ZOA_CUDA(h, launch_reduce(view(h), h->c, gamma_sum, static_cast<cudaStream_t>(stream)));
-    h->n_launches += 1;
+    ZOA_CUDA(h, run_server(h, gamma_sum, static_cast<cudaStream_t>(stream)));
     h->gamma_sum = 0.0;
     h->t_sync = h->t_last;
     h->n_syncs += 1;
@@ -318,6 +403,20 @@ extern "C" zoa_status zoa_step_sync(zoa_handle h, const float *const *grads, flo
     commit_variance(h);
     const bool do_var = zoa_var_due(h, t) == 1;
     const StateView st = view(h);
+    if (h->large_chunk) {
+        // No single block can hold a chunk: the local step is written out, then compressed.
+        ZOA_CUDA(h, launch_local_step(st, gp, h->c, lr, do_var, aligned, h->sm_count, s));
+        h->n_launches += 1;
+        ZOA_CUDA(h, run_compress(h, s));
+        ZOA_CUDA(h, run_server(h, gamma_sum, s));
+        if (do_var) { h->v_pending = true; h->n_var_updates += 1; }
+        h->gamma_sum = 0.0;
+        h->t_last = t;
+        h->t_sync = t;
+        h->n_steps += 1;
+        h->n_syncs += 1;
+        return ZOA_OK;
+    }
     const int stages = h->use_pipeline ? pipeline_stages(st, aligned) : 0;
     long long var_first = 0;     // coordinates from here on still need lines 14-15
     if (stages > 0) {
@@ -361,8 +460,16 @@ extern "C" zoa_status zoa_alg2_step(zoa_handle h, const float *const *grads, flo
     if (rc != ZOA_OK) return rc;
     commit_variance(h);
     const bool full = zoa_var_due(h, t) == 1;
-    ZOA_CUDA(h, launch_alg2(view(h), gp, h->c, lr, full, aligned, h->sm_count, static_cast<cudaStream_t>(stream)));
-    h->n_launches += 1;
+    if (h->large_chunk && !full) {
+        int launches = 0;
+        cudaStream_t s = static_cast<cudaStream_t>(stream);
+        ZOA_CUDA(h, launch_large_compress(view(h), gp, true, aligned, h->partials, &launches, s));
+        ZOA_CUDA(h, launch_large_server(view(h), h->c, 2, lr, h->partials, &launches, s));
+        h->n_launches += launches;
+    } else {
+        ZOA_CUDA(h, launch_alg2(view(h), gp, h->c, lr, full, aligned, h->sm_count, static_cast<cudaStream_t>(stream)));
+        h->n_launches += 1;
+    }
     if (full) { h->v_pending = true; h->n_var_updates += 1; } else h->n_syncs += 1;
     h->t_last = t;
     h->n_steps += 1;

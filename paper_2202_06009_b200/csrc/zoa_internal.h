@@ -19,6 +19,13 @@ cudaError_t launch_step_sync(const StateView &st, const GradPtrs &g, const Const
 cudaError_t launch_alg2(const StateView &st, const GradPtrs &g, const Consts &c, float gamma, bool full_precision,
                         bool g_aligned, int sm_count, cudaStream_t s);
 
+// Chunks larger than kMaxChunk (up to the whole vector): multi-pass kernels, zoa_kernels.cu.
+long long large_chunk_segments(const StateView &st);
+cudaError_t launch_large_compress(const StateView &st, const GradPtrs &g, bool from_grads, bool g_aligned,
+                                  double *partials, int *launches, cudaStream_t s);
+cudaError_t launch_large_server(const StateView &st, const Consts &c, int mode, float scalar, double *partials,
+                                int *launches, cudaStream_t s);
+
 // Pipelined (bulk-copy ring) form of the fused sync step, zoa_pipeline.cu.
 int pipeline_stages(const StateView &st, bool g_aligned);
 cudaError_t launch_step_sync_pipelined(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,

@@ -474,6 +474,191 @@ __global__ void __launch_bounds__(512, 2) alg2_compressed_kernel(StateView st, G
 }
 
 // ---------------------------------------------------------------------------
+// Large chunks (chunk > 16384, up to the whole vector = Eq. 3 as printed): a chunk no
+// longer fits one block, so each l1 norm is taken in two steps - one binary64 partial
+// sum per segment of 4096 coordinates, then a fixed-order sum of a chunk's partials -
+// and the values being compressed are recomputed instead of kept.
+// ---------------------------------------------------------------------------
+constexpr int kSegment = 4096;
+
+struct SegGeom {
+    long long c;     // chunk
+    long long j0;    // first coordinate of the segment
+    int len;         // live coordinates in the segment (0 if it lies beyond the chunk's end)
+    int chunk_len;   // true length of the chunk
+};
+__device__ __forceinline__ SegGeom seg_geom(const StateView &st, long long seg, long long segs_per_chunk)
+{
+    SegGeom g;
+    g.c = seg / segs_per_chunk;
+    const long long s = seg % segs_per_chunk;
+    const long long c0 = g.c * st.chunk;
+    const long long rest = st.n - c0;
+    const long long clen = rest < st.chunk ? rest : (long long)st.chunk;
+    g.chunk_len = (int)clen;
+    const long long start = s * kSegment;
+    const long long live = clen - start;
+    g.len = live <= 0 ? 0 : (live < kSegment ? (int)live : kSegment);
+    g.j0 = c0 + start;
+    return g;
+}
+
+// What a worker compresses, four coordinates from j: its source buffer plus its error.
+template <bool FROM_GRADS>
+__device__ __forceinline__ float4 lc_worker_input(const StateView &st, const GradPtrs &g, int i, long long j, int g_aligned)
+{
+    const long long row = (long long)i * st.n_pad + j;
+    const float4 a = FROM_GRADS ? ld_grad4(g.p[i], j, st.n, g_aligned) : ld4(st.u + row);
+    const float4 e = ld4(st.dw + row);
+    return make_float4(f_add(a.x, e.x), f_add(a.y, e.y), f_add(a.z, e.z), f_add(a.w, e.w));
+}
+
+// partials[i][seg] = sum |z| over segment `seg` of worker i = blockIdx.y.
+template <bool FROM_GRADS>
+__global__ void __launch_bounds__(512)
+lc_partial_l1_kernel(StateView st, GradPtrs g, int g_aligned, long long segs_per_chunk, long long n_segs, double *partials)
+{
+    __shared__ double scratch[34];
+    const SegGeom sg = seg_geom(st, blockIdx.x, segs_per_chunk);
+    const int i = blockIdx.y;
+    double l1 = 0.0;
+    for (int idx = 4 * threadIdx.x; idx < sg.len; idx += 4 * blockDim.x) {
+        const float4 z = lc_worker_input<FROM_GRADS>(st, g, i, sg.j0 + idx, g_aligned);
+        const float zz[4] = {z.x, z.y, z.z, z.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            if (idx + k < sg.len) l1 += fabs((double)zz[k]);
+    }
+    const double total = block_sum(l1, scratch);
+    if (threadIdx.x == 0) partials[(long long)i * n_segs + blockIdx.x] = total;
+}
+
+// scales[row][c] = (sum of the chunk's partials, in segment order per lane then a fixed tree) / len.
+__global__ void lc_scales_kernel(StateView st, const double *partials, long long segs_per_chunk, long long n_segs,
+                                 float *scales)
+{
+    const long long c = blockIdx.x;
+    const int row = blockIdx.y;
+    const double *p = partials + (long long)row * n_segs + c * segs_per_chunk;
+    double sum = 0.0;
+    for (long long s = threadIdx.x; s < segs_per_chunk; s += 32) sum += p[s];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    if (threadIdx.x == 0) {
+        const long long rest = st.n - c * st.chunk;
+        const int len = (int)(rest < st.chunk ? rest : (long long)st.chunk);
+        scales[(long long)row * st.n_chunks + c] = chunk_scale(sum, len);
+    }
+}
+
+// Worker side of Algorithm 3 once the magnitudes are known: bits, errors.
+template <bool FROM_GRADS>
+__global__ void __launch_bounds__(512)
+lc_compress_apply_kernel(StateView st, GradPtrs g, int g_aligned, long long segs_per_chunk)
+{
+    const SegGeom sg = seg_geom(st, blockIdx.x, segs_per_chunk);
+    const int i = blockIdx.y;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    const float scale = st.scales_w[(long long)i * st.n_chunks + sg.c];
+    for (int base = warp * 128; base < sg.len; base += n_warps * 128) {
+        const int idx = base + 4 * lane;
+        float z[4] = {0.f, 0.f, 0.f, 0.f}, hat[4];
+        if (idx < sg.len) {
+            const float4 z4 = lc_worker_input<FROM_GRADS>(st, g, i, sg.j0 + idx, g_aligned);
+            z[0] = z4.x; z[1] = z4.y; z[2] = z4.z; z[3] = z4.w;
+        }
+        const uint32_t word = compress_tile(z, hat, scale, idx, sg.len);
+        if (idx < sg.len) st4(st.dw + (long long)i * st.n_pad + sg.j0 + idx, make_float4(z[0], z[1], z[2], z[3]));
+        if (lane < 4 && base + 32 * lane < sg.len)
+            st.words_w[(long long)i * st.words_stride + ((sg.j0 + base) >> 5) + lane] = word;
+    }
+}
+
+// Server input of Algorithm 3 for four coordinates from j, from what the workers sent.
+__device__ __forceinline__ void lc_server_input(const StateView &st, const float *scales_sm, long long j, int valid, float a[4])
+{
+    double A[4] = {0.0, 0.0, 0.0, 0.0};
+    const long long word_idx = j >> 5;
+    const int shift = (int)(j & 31);
+    for (int i = 0; i < st.W; ++i) {   // worker order
+        const uint32_t nib = st.words_w[(long long)i * st.words_stride + word_idx] >> shift;
+        const double s = (double)scales_sm[i];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) A[k] += ((nib >> k) & 1u) ? s : -s;
+    }
+    const float4 e4 = ld4(st.ds + j);
+    const float ee[4] = {e4.x, e4.y, e4.z, e4.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) a[k] = k < valid ? server_input(A[k], st.W, ee[k]) : 0.0f;
+}
+
+// partials[W][seg] = sum |mean of the compressed buffers + server error| over the segment.
+__global__ void __launch_bounds__(512)
+lc_server_partial_kernel(StateView st, long long segs_per_chunk, long long n_segs, double *partials)
+{
+    __shared__ double scratch[34];
+    __shared__ float scales_sm[kMaxWorkers];
+    const SegGeom sg = seg_geom(st, blockIdx.x, segs_per_chunk);
+    for (int i = threadIdx.x; i < st.W; i += blockDim.x) scales_sm[i] = st.scales_w[(long long)i * st.n_chunks + sg.c];
+    __syncthreads();
+    double l1 = 0.0;
+    for (int idx = 4 * threadIdx.x; idx < sg.len; idx += 4 * blockDim.x) {
+        float a[4];
+        lc_server_input(st, scales_sm, sg.j0 + idx, sg.len - idx, a);
+        l1 += fabs((double)a[0]) + fabs((double)a[1]) + fabs((double)a[2]) + fabs((double)a[3]);
+    }
+    const double total = block_sum(l1, scratch);
+    if (threadIdx.x == 0) partials[(long long)st.W * n_segs + blockIdx.x] = total;
+}
+
+// Server compression and what follows it.  MODE 1: lines 8-10 of Algorithm 1.
+// MODE 2: lines 10-11 of Algorithm 2 (momentum and model driven by the received gradient).
+template <int MODE>
+__global__ void __launch_bounds__(512)
+lc_server_apply_kernel(StateView st, Consts c, float gamma_or_sum, long long segs_per_chunk)
+{
+    __shared__ float scales_sm[kMaxWorkers];
+    const SegGeom sg = seg_geom(st, blockIdx.x, segs_per_chunk);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    for (int i = threadIdx.x; i < st.W; i += blockDim.x) scales_sm[i] = st.scales_w[(long long)i * st.n_chunks + sg.c];
+    __syncthreads();
+    const float scale = st.scales_s[sg.c];
+    ChunkGeom cg;           // the segment seen as a short chunk, for server_tile
+    cg.c0 = sg.j0;
+    cg.len = sg.len;
+    for (int base = warp * 128; base < sg.len; base += n_warps * 128) {
+        const int idx = base + 4 * lane;
+        float a[4] = {0.f, 0.f, 0.f, 0.f};
+        if (idx < sg.len) lc_server_input(st, scales_sm, sg.j0 + idx, sg.len - idx, a);
+        if (MODE == 1) {
+            server_tile(st, c, cg, base, lane, a, scale, gamma_or_sum);
+        } else {
+            float gb[4];
+            const uint32_t word = compress_tile(a, gb, scale, idx, sg.len);
+            if (lane < 4 && base + 32 * lane < sg.len) st.words_s[((sg.j0 + base) >> 5) + lane] = word;
+            if (idx >= sg.len) continue;
+            const long long j = sg.j0 + idx;
+            st4(st.ds + j, make_float4(a[0], a[1], a[2], a[3]));
+            const float4 v4 = ld4(st.v + j);
+            const float d[4] = {denom(c, v4.x), denom(c, v4.y), denom(c, v4.z), denom(c, v4.w)};
+            for (int i = 0; i < st.W; ++i) {
+                const long long row = (long long)i * st.n_pad + j;
+                const float4 m4 = ld4(st.m + row), x4 = ld4(st.x + row);
+                const float mm[4] = {m4.x, m4.y, m4.z, m4.w}, xx[4] = {x4.x, x4.y, x4.z, x4.w};
+                float mo[4], xo[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    mo[k] = momentum(c, mm[k], gb[k]);
+                    xo[k] = f_sub(xx[k], f_div(f_mul(gamma_or_sum, mo[k]), d[k]));
+                }
+                st4(st.m + row, make_float4(mo[0], mo[1], mo[2], mo[3]));
+                st4(st.x + row, make_float4(xo[0], xo[1], xo[2], xo[3]));
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
 // Launchers
 // ---------------------------------------------------------------------------
 static int block_threads_for_chunk(int chunk)
@@ -565,6 +750,46 @@ cudaError_t launch_step_sync(const StateView &st, const GradPtrs &g, const Const
 {
     step_sync_kernel<<<(unsigned)count, block_threads_for_chunk(st.chunk), step_sync_smem(st.chunk), s>>>(
         st, g, c, gamma, gamma_sum, g_aligned, first_chunk);
+    return cudaGetLastError();
+}
+
+}  // namespace zoa
+
+namespace zoa {
+
+long long large_chunk_segments(const StateView &st)
+{
+    const long long span = st.chunk < st.n ? (long long)st.chunk : st.n;
+    return (span + kSegment - 1) / kSegment;
+}
+
+// Worker side of Algorithm 3 for chunks too large for one block.  from_grads: compress
+// g + delta (Algorithm 2) instead of u + delta (Algorithm 1).  partials: [W + 1][n_chunks * segments].
+cudaError_t launch_large_compress(const StateView &st, const GradPtrs &g, bool from_grads, bool g_aligned,
+                                  double *partials, int *launches, cudaStream_t s)
+{
+    const long long spc = large_chunk_segments(st), n_segs = spc * st.n_chunks;
+    const dim3 grid((unsigned)n_segs, (unsigned)st.W);
+    if (from_grads) lc_partial_l1_kernel<true><<<grid, 512, 0, s>>>(st, g, g_aligned, spc, n_segs, partials);
+    else lc_partial_l1_kernel<false><<<grid, 512, 0, s>>>(st, g, g_aligned, spc, n_segs, partials);
+    lc_scales_kernel<<<dim3((unsigned)st.n_chunks, (unsigned)st.W), 32, 0, s>>>(st, partials, spc, n_segs, st.scales_w);
+    if (from_grads) lc_compress_apply_kernel<true><<<grid, 512, 0, s>>>(st, g, g_aligned, spc);
+    else lc_compress_apply_kernel<false><<<grid, 512, 0, s>>>(st, g, g_aligned, spc);
+    *launches += 3;
+    return cudaGetLastError();
+}
+
+// Server side.  mode 1: Algorithm 1 lines 8-10 (scalar = sum of learning rates); mode 2: Algorithm 2
+// lines 10-11 (scalar = learning rate).
+cudaError_t launch_large_server(const StateView &st, const Consts &c, int mode, float scalar, double *partials,
+                                int *launches, cudaStream_t s)
+{
+    const long long spc = large_chunk_segments(st), n_segs = spc * st.n_chunks;
+    lc_server_partial_kernel<<<(unsigned)n_segs, 512, 0, s>>>(st, spc, n_segs, partials);
+    lc_scales_kernel<<<dim3((unsigned)st.n_chunks, 1), 32, 0, s>>>(st, partials + (long long)st.W * n_segs, spc, n_segs, st.scales_s);
+    if (mode == 1) lc_server_apply_kernel<1><<<(unsigned)n_segs, 512, 0, s>>>(st, c, scalar, spc);
+    else lc_server_apply_kernel<2><<<(unsigned)n_segs, 512, 0, s>>>(st, c, scalar, spc);
+    *launches += 3;
     return cudaGetLastError();
 }
 

@@ -38,7 +38,7 @@ def test_validation_before_any_cuda_call():
     h = ctypes.c_void_p()
     for args in ((0, 2, 0.9, 0.999, 1e-8, 64), (10, 0, 0.9, 0.999, 1e-8, 64), (10, 65, 0.9, 0.999, 1e-8, 64),
                  (10, 2, 1.0, 0.999, 1e-8, 64), (10, 2, 0.9, -0.1, 1e-8, 64), (10, 2, 0.9, 0.999, 0.0, 64),
-                 (10, 2, 0.9, 0.999, 1e-8, 33), (10, 2, 0.9, 0.999, 1e-8, 16), (10, 2, 0.9, 0.999, 1e-8, 32768)):
+                 (10, 2, 0.9, 0.999, 1e-8, 33), (10, 2, 0.9, 0.999, 1e-8, 16), (10, 2, 0.9, 0.999, 1e-8, (1 << 30) + 32)):
         assert B.lib.zoa_create(ctypes.byref(h), *args) == B.ERR_ARG
         assert h.value is None and B.lib.zoa_last_error(None)
     assert B.lib.zoa_destroy(None) == B.ERR_ARG
@@ -53,3 +53,25 @@ def test_product_has_no_route_to_the_oracle():
         for f in files:
             if f.endswith((".py", ".cu", ".cuh", ".h")):
                 assert "oracle" not in open(os.path.join(dirpath, f)).read().replace("test oracle", ""), f
+
+
+def test_paper_schedules():
+    """The T_v gap rule and the T_u interval rule of the paragraph "Policy for T_v and T_u",
+    checked against values worked out by hand from the rules."""
+    from paper_2202_06009_b200 import binding as B
+    # kappa = 16: sixteen gaps of 1, sixteen of 2, sixteen of 4, ...
+    steps = B.zoa_policy_var_steps(16, 200)
+    assert steps[:17] == list(range(17))
+    assert steps[17:33] == list(range(18, 49, 2)) and steps[33] == 52 and steps[34] == 56
+    gaps = [b - a for a, b in zip(steps, steps[1:])]
+    assert gaps[:16] == [1] * 16 and gaps[16:32] == [2] * 16 and set(gaps[32:48]) <= {4}
+    assert steps[-1] < 200
+    assert B.zoa_policy_var_steps(1, 40) == [0, 1, 3, 7, 15, 31]        # gaps 1, 2, 4, 8, 16
+    assert B.zoa_policy_var_steps(16, 0) == []
+    # BERT: interval 1 through the 12.5K warm-up, x2 every 32678 steps, clipped at 16
+    b, k = B.zoa_policy_sync_pieces(12500, 32678, 16)
+    assert k == [1, 2, 4, 8, 16]
+    assert b == [0, 12500 + 32678, 12500 + 2 * 32678, 12500 + 3 * 32678, 12500 + 4 * 32678]
+    assert B.zoa_policy_sync_pieces(10, 5, 1) == ([0], [1])
+    assert B.zoa_policy_sync_pieces(0, 4, 12) == ([0, 4, 8, 12, 16], [1, 2, 4, 8, 12])
+    assert B.lib.zoa_policy_sync_pieces(0, 0, 4, None, None, 0) == 0      # bad arguments

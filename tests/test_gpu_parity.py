@@ -283,7 +283,7 @@ def test_argument_and_state_errors():
     with pytest.raises(ZoaError) as e:
         Zoa(100, 0)
     assert e.value.status == B.ERR_ARG
-    for kw in (dict(chunk=48), dict(chunk=16), dict(chunk=32768), dict(beta1=1.0), dict(eps=0.0)):
+    for kw in (dict(chunk=48), dict(chunk=16), dict(chunk=(1 << 30) + 32), dict(beta1=1.0), dict(eps=0.0)):
         with pytest.raises(ZoaError):
             Zoa(100, 2, **kw)
     z = Zoa(100, 2, chunk=32)
@@ -403,3 +403,43 @@ def test_alg2_unaligned_and_interleaved_variance_steps():
             p.compare(f"t={t}", wire=False)
     finally:
         p.close()
+
+
+# --------------------------------------------------------------------------
+# Chunks larger than one block can hold, up to the whole vector (Eq. 3 as printed)
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("mode", ["fused", "two_call", "alg2"])
+@pytest.mark.parametrize("W,chunk,n", [(3, 32768, 2 * 32768 + 5000), (4, 1 << 20, 300001), (2, 20000 * 32, 20000 * 32),
+                                       (5, 16384 + 32, 3 * (16384 + 32) + 17), (16, 1 << 22, 70000)])
+def test_large_chunks_and_whole_vector_scale(W, chunk, n, mode):
+    """chunk > 16384 goes through the multi-pass kernels; chunk >= n is the paper's compressor
+    with one magnitude for the whole vector."""
+    rng = np.random.default_rng(W + n)
+    p = Pair(n, W, chunk, var_steps=(0, 2), sync=((0, 3), (1, 2)), x0=rng.standard_normal(n) * 0.02)
+    try:
+        for t in range(6):
+            g = _grads(rng, W, n)
+            if mode == "alg2":
+                p.gpu.alg2_step(list(torch.from_numpy(g).cuda()), 1e-3, t)
+                torch.cuda.synchronize()
+                p.cpu.alg2_step(g, np.float32(1e-3), t in (0, 2))
+                p.compare(f"t={t}", wire=t not in (0, 2))
+            else:
+                p.step(g, 1e-3, t, mode)
+                p.compare(f"t={t}", wire=p.gpu.sync_due(t))
+        p.padding_is_zero()
+        if chunk >= n:
+            assert p.gpu.read("scales_s").size == 1
+    finally:
+        p.close()
+
+
+def test_paper_schedules_on_a_handle():
+    z = Zoa(64, 1, chunk=32)
+    try:
+        B.zoa_set_var_policy_doubling(z.h, 2, 1000)
+        B.zoa_set_sync_policy_doubling(z.h, 10, 5, 4, True)      # interval 1 until step 15, 2 until 20, then 4
+        assert [t for t in range(30) if z.sync_due(t)] == list(range(15)) + [15, 17, 19] + [20, 24, 28]
+        assert [t for t in range(40) if z.var_due(t)] == [0, 1, 2, 4, 6, 10, 14]     # nothing from step 15 on
+    finally:
+        z.close()
