@@ -28,34 +28,34 @@ DRAM_TRAFFIC_RATIO = 0.995   # measured DRAM bytes / algorithmic bytes, see prof
 
 
 # ---- byte model: what the method must move, per launch -------------------------
-def sync_step_bytes(n, W, chunk):
+def sync_step_bytes(n, W, chunk, g_bytes=4):
     """Fused sync step: per parameter and worker read g, m, u, delta (16 B), write
     delta, x, m, u (16 B) and 1 sign bit, plus one scale per chunk; per parameter
     read delta_bar, v, x_sync (12 B), write delta_bar, x_sync (8 B) and 1 sign bit."""
     n_chunks = -(-n // chunk)
-    return n * W * (32 + 1 / 8) + n_chunks * W * 4 + n * (20 + 1 / 8) + n_chunks * 4
+    return n * W * (28 + g_bytes + 1 / 8) + n_chunks * W * 4 + n * (20 + 1 / 8) + n_chunks * 4
 
 
-def local_step_bytes(n, W):
+def local_step_bytes(n, W, g_bytes=4):
     """Local step: per parameter and worker read g, m, x, u and write m, x, u (28 B); v read once."""
-    return n * W * 28 + n * 4
+    return n * W * (24 + g_bytes) + n * 4
 
 
 def variance_bytes(n, W):
     return n * W * 4 + n * 8
 
 
-def alg2_compressed_bytes(n, W, chunk):
+def alg2_compressed_bytes(n, W, chunk, g_bytes=4):
     """Algorithm 2, compressed step: per parameter and worker read g, delta, m, x (16 B), write
     delta, m, x (12 B) and 1 sign bit + a scale per chunk; per parameter read delta_bar, v,
     write delta_bar (12 B) and 1 sign bit."""
     n_chunks = -(-n // chunk)
-    return n * W * (28 + 1 / 8) + n_chunks * W * 4 + n * (12 + 1 / 8) + n_chunks * 4
+    return n * W * (24 + g_bytes + 1 / 8) + n_chunks * W * 4 + n * (12 + 1 / 8) + n_chunks * 4
 
 
-def alg2_full_bytes(n, W):
+def alg2_full_bytes(n, W, g_bytes=4):
     """Algorithm 2, T_v step: per parameter and worker read g, m, x, write m, x (20 B); v in and out."""
-    return n * W * 20 + n * 8
+    return n * W * (16 + g_bytes) + n * 8
 
 
 def measured_hbm_peak():
@@ -187,11 +187,25 @@ def run_ours(args, wl):
     stream = synth.GradientStream(wl, "cuda", seed)
     from paper_2202_06009_b200 import binding as B
 
+    gdt = {"f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloat16}[args.grad_dtype]
+    g_bytes = 4 if gdt == torch.float32 else 2
+    opt.set_grad_dtype(gdt)
+    g16 = None if g_bytes == 4 else [torch.empty(wl.n, device="cuda", dtype=gdt) for _ in range(wl.W)]
+
+    def batch(t):
+        """The step's gradients, resident in device memory in the dtype the handle expects (untimed)."""
+        bufs = stream.fill(t)
+        if g16 is None:
+            return bufs
+        for dst, src in zip(g16, bufs):
+            dst.copy_(src)
+        return g16
+
     K, Wu = args.steps, max(args.warmup, 3)
     for t in range(Wu):                                   # warm-up: the first steps of the schedule
-        opt.step_auto(stream.fill(t), wl.lr_at(t), t)
+        opt.step_auto(batch(t), wl.lr_at(t), t)
     # also warm the local-step kernel, then rewind the step counter (timing does not depend on values)
-    opt.step(stream.bufs, wl.lr, Wu)
+    opt.step(batch(Wu), wl.lr, Wu)
     B.zoa_set_scalars(opt.h, 0.0, 0, -1)
     barrier()
 
@@ -202,7 +216,7 @@ def run_ours(args, wl):
         barrier()
         wall0 = time.perf_counter()
         for t in range(K):
-            bufs = stream.fill(t)                         # untimed: the batch is resident before the step starts
+            bufs = batch(t)                               # untimed: the batch is resident before the step starts
             ev[t][0].record()
             if args.algorithm == "alg2":
                 opt.alg2_step(bufs, wl.lr_at(t), t)
@@ -226,12 +240,12 @@ def run_ours(args, wl):
     for k, m in zip(kinds, ms):
         by_kind.setdefault(k, []).append(m)
     peak, peak_kind = measured_hbm_peak()
-    bytes_of = {"sync": sync_step_bytes(wl.n, wl.W, wl.chunk), "local": local_step_bytes(wl.n, wl.W)}
+    bytes_of = {"sync": sync_step_bytes(wl.n, wl.W, wl.chunk, g_bytes), "local": local_step_bytes(wl.n, wl.W, g_bytes)}
     # the variance update needs nothing beyond writing v_{t+1}: g and v are read anyway
     bytes_of["sync+var"] = bytes_of["sync"] + wl.n * 4
     bytes_of["local+var"] = bytes_of["local"] + wl.n * 4
-    bytes_of["alg2_compressed"] = alg2_compressed_bytes(wl.n, wl.W, wl.chunk)
-    bytes_of["alg2_full"] = alg2_full_bytes(wl.n, wl.W)
+    bytes_of["alg2_compressed"] = alg2_compressed_bytes(wl.n, wl.W, wl.chunk, g_bytes)
+    bytes_of["alg2_full"] = alg2_full_bytes(wl.n, wl.W, g_bytes)
     step_types = {k: {"count": len(v), "ms": statistics.mean(v), "algorithmic_GB": bytes_of[k] / 1e9,
                       "GBps": bytes_of[k] / 1e6 / statistics.mean(v)} for k, v in by_kind.items()}
     total_bytes = sum(bytes_of[k] for k in kinds)
@@ -257,7 +271,7 @@ def run_ours(args, wl):
     e2e = None
     if args.e2e_steps > 0 and args.algorithm == "alg1":
         ke = max(1, min(args.e2e_steps, K))
-        host_g = torch.empty(wl.n, dtype=torch.float32).pin_memory()
+        host_g = torch.empty(wl.n, dtype=gdt).pin_memory()
         host_g.copy_(stream.bufs[0])
         host_x = torch.empty(wl.n, dtype=torch.float32).pin_memory()
         B.zoa_set_scalars(opt.h, 0.0, 0, -1)
@@ -276,7 +290,7 @@ def run_ours(args, wl):
             dist.all_reduce(tt, op=dist.ReduceOp.MAX)
             e_ms = float(tt.item())
         e2e = {"value": wl.n * wl.W * ke * world / (e_ms / 1e3), "unit": UNIT,
-               "h2d_bytes_per_step": wl.n * wl.W * 4, "d2h_bytes_per_step": wl.n * 4, "steps": ke,
+               "h2d_bytes_per_step": wl.n * wl.W * g_bytes, "d2h_bytes_per_step": wl.n * 4, "steps": ke,
                "ms_per_step": e_ms / ke,
                "how": "zoa_step_host: W copies from pinned host memory (one pinned buffer serves every "
                       "worker), the step, worker 0's model copied back"}
@@ -290,7 +304,7 @@ def run_ours(args, wl):
         line = {"metric": METRIC, "value": wl.n * wl.W * K * world / (total_ms / 1e3), "unit": UNIT,
                 "n_gpus": world, "steps": K, "warmup": Wu, "ms_per_step": total_ms / K,
                 "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
-                "data": "synthetic",
+                "data": "synthetic", "grad_dtype": args.grad_dtype,
                 "config": {"workload": wl.name, "n_params": wl.n, "W": wl.W, "chunk": wl.chunk,
                            "algorithm": "Algorithm 1 (0/1 Adam)" if args.algorithm == "alg1" else
                                         "Algorithm 2 (gradients through the 1-bit AllReduce, full precision on T_v steps)",
@@ -384,6 +398,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--scale", type=int, default=1, help="shrink every tensor by this factor (profiling captures)")
     ap.add_argument("--no-pipeline", action="store_true", help="fused sync step through the chunk-per-block kernel")
+    ap.add_argument("--grad-dtype", default="f32", choices=["f32", "f16", "bf16"],
+                    help="element type of the gradient buffers (state and arithmetic stay f32)")
     ap.add_argument("--chunk", type=int, default=0,
                     help="override the workload's chunk (e.g. 1073741824 = one magnitude for the whole vector, Eq. 3 as printed)")
     ap.add_argument("--algorithm", default="alg1", choices=["alg1", "alg2"],

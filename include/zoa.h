@@ -125,10 +125,11 @@ int zoa_var_due(zoa_handle h, int64_t t);
 /* Algorithm 1 lines 3-5 for every worker, and lines 14-15 when t is in T_v
  * (the new variance takes effect from the next step on, so that a following
  * zoa_onebit_reduce still uses v_t as line 9 does).
- * grads: (host) array of W (device) pointers, n_params floats each, worker i's
- * gradient at step t; 16-byte aligned pointers take the vector path.
+ * grads: (host) array of W (device) pointers, n_params elements each (binary32
+ * unless ZOA_OPT_GRAD_TYPE says otherwise), worker i's gradient at step t;
+ * 16-byte aligned pointers take the vector path.
  * lr is gamma_t; t must be larger than at the previous step. */
-zoa_status zoa_step(zoa_handle h, const float *const *grads, float lr, int64_t t, void *stream);
+zoa_status zoa_step(zoa_handle h, const void *const *grads, float lr, int64_t t, void *stream);
 
 /* Algorithm 1 lines 7-11 with Algorithm 3 inside: compresses u + delta per
  * worker (Eq. 3 per chunk), averages, compresses again on the "server" with its
@@ -147,7 +148,7 @@ zoa_status zoa_onebit_average(zoa_handle h, void *stream);
 
 /* zoa_step followed by zoa_onebit_reduce, same results bit for bit, in one
  * pass over memory that never writes the half-step values. */
-zoa_status zoa_step_sync(zoa_handle h, const float *const *grads, float lr, int64_t t,
+zoa_status zoa_step_sync(zoa_handle h, const void *const *grads, float lr, int64_t t,
                          void *stream);
 
 /* One iteration of Algorithm 2 (the frozen-variance framework that exchanges
@@ -160,11 +161,11 @@ zoa_status zoa_step_sync(zoa_handle h, const float *const *grads, float lr, int6
  * momentum just computed (the convention that makes this the no-local-step case
  * of Algorithm 1).  u, x_sync and the sum of learning rates are not touched.
  * Arguments and errors as zoa_step. */
-zoa_status zoa_alg2_step(zoa_handle h, const float *const *grads, float lr, int64_t t, void *stream);
+zoa_status zoa_alg2_step(zoa_handle h, const void *const *grads, float lr, int64_t t, void *stream);
 
 /* One iteration of Algorithm 1 under the handle's own policies: zoa_step_sync
  * if t is in T_u, else zoa_step. */
-zoa_status zoa_step_auto(zoa_handle h, const float *const *grads, float lr, int64_t t,
+zoa_status zoa_step_auto(zoa_handle h, const void *const *grads, float lr, int64_t t,
                          void *stream);
 
 /* The same iteration with gradients in (host) memory: host_grads is an array
@@ -172,7 +173,7 @@ zoa_status zoa_step_auto(zoa_handle h, const float *const *grads, float lr, int6
  * Copies them to a device staging area the handle allocates on first use,
  * runs zoa_step_auto, and, if host_x_out is not NULL, copies worker 0's model
  * back (n_params floats).  All on `stream`; does not synchronise. */
-zoa_status zoa_step_host(zoa_handle h, const float *const *host_grads, float lr, int64_t t,
+zoa_status zoa_step_host(zoa_handle h, const void *const *host_grads, float lr, int64_t t,
                          float *host_x_out, void *stream);
 
 /* Borrowed (device) pointer to one row of a state buffer and its length in
@@ -206,8 +207,15 @@ zoa_status zoa_check_device(zoa_handle h);
  * undefined and zoa_check_device reports ZOA_ERR_DEVICE.
  * ZOA_OPT_TEST_STOP_AFTER_TILES (default 0 = off): for testing that error path
  * only - the copy-issuing lane of every block stops after this many tiles, so
- * the waits of the other threads run out after the limit. */
-enum { ZOA_OPT_PIPELINE = 1, ZOA_OPT_WAIT_LIMIT_MS = 2, ZOA_OPT_TEST_STOP_AFTER_TILES = 3 };
+ * the waits of the other threads run out after the limit.
+ * ZOA_OPT_GRAD_TYPE (default ZOA_GRAD_F32): element type of the buffers passed as
+ * `grads` / `host_grads` from now on: binary32, binary16 (IEEE half) or bfloat16.
+ * 16-bit gradients are converted to binary32 exactly when they are loaded; all
+ * arithmetic and all state stay binary32, so the results equal those of the same
+ * values passed as binary32.  (The paper trains in FP16; its communication buffer
+ * u is still formed in the optimizer's precision.) */
+enum { ZOA_OPT_PIPELINE = 1, ZOA_OPT_WAIT_LIMIT_MS = 2, ZOA_OPT_TEST_STOP_AFTER_TILES = 3, ZOA_OPT_GRAD_TYPE = 4 };
+enum { ZOA_GRAD_F32 = 0, ZOA_GRAD_F16 = 1, ZOA_GRAD_BF16 = 2 };
 zoa_status zoa_set_option(zoa_handle h, int option, int value);
 
 /* Text of the last error on this handle (or of the last failed zoa_create if h

@@ -197,7 +197,8 @@ def zoa_get_stats(h):
     return {name: getattr(s, name) for name, _ in Stats._fields_}
 
 
-OPT_PIPELINE, OPT_WAIT_LIMIT_MS, OPT_TEST_STOP_AFTER_TILES = 1, 2, 3
+OPT_PIPELINE, OPT_WAIT_LIMIT_MS, OPT_TEST_STOP_AFTER_TILES, OPT_GRAD_TYPE = 1, 2, 3, 4
+GRAD_F32, GRAD_F16, GRAD_BF16 = 0, 1, 2
 
 
 def zoa_set_option(h, option, value):

@@ -27,6 +27,7 @@ struct zoa_handle_s {
     unsigned long long *sched = nullptr;   // device [2]: chunk counter of the persistent kernel, finished blocks
     double *partials = nullptr;    // device [W + 1][n_chunks * segments]: per-segment l1 sums, chunk > 16384 only
     bool large_chunk = false;
+    int grad_type = 0;             // 0 binary32, 1 binary16, 2 bfloat16: how `grads` buffers are read
     bool use_pipeline = true;      // bulk-copy ring form of the fused sync step where the shape allows
     int wait_limit_ms = 2000;      // bound on every device-side wait
     long long test_stop_after_tiles = 0;   // error-path test hook, see zoa_set_option
@@ -274,8 +275,8 @@ extern "C" int zoa_var_due(zoa_handle h, int64_t t)
 // Checks shared by the step entry points; fills the pointer pack.
 static bool on_own_device(zoa_handle h);
 
-static zoa_status check_step_args(zoa_handle h, const float *const *grads, float lr, int64_t t, GradPtrs *gp,
-                                  bool *aligned, const char *who)
+static zoa_status check_step_args(zoa_handle h, const void *const *grads, float lr, int64_t t, GradPtrs *gp,
+                                  int *aligned, const char *who)
 {
     if (!h) return ZOA_ERR_ARG;
     if (!grads) return fail(h, ZOA_ERR_ARG, std::string(who) + ": grads is NULL");
@@ -283,13 +284,14 @@ static zoa_status check_step_args(zoa_handle h, const float *const *grads, float
     if (t < 0) return fail(h, ZOA_ERR_ARG, std::string(who) + ": t is negative");
     if (t <= h->t_last) return fail(h, ZOA_ERR_STATE, std::string(who) + ": t must increase from step to step");
     if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, std::string(who) + ": the handle's device is not the current CUDA device");
-    *aligned = true;
+    bool all_aligned = true;
     for (int i = 0; i < h->W; ++i) {
         if (!grads[i]) return fail(h, ZOA_ERR_ARG, std::string(who) + ": a gradient pointer is NULL");
-        gp->p[i] = grads[i];
-        if (reinterpret_cast<uintptr_t>(grads[i]) & 15u) *aligned = false;
+        gp->p[i] = static_cast<const float *>(grads[i]);
+        if (reinterpret_cast<uintptr_t>(grads[i]) & 15u) all_aligned = false;
     }
     for (int i = h->W; i < kMaxWorkers; ++i) gp->p[i] = nullptr;
+    *aligned = (all_aligned ? kGradAligned : 0) | (h->grad_type << 1);   // the format code ld_grad4 takes
     return ZOA_OK;
 }
 
@@ -336,10 +338,10 @@ static cudaError_t run_server(zoa_handle h, float gamma_sum, cudaStream_t s)
     return e;
 }
 
-extern "C" zoa_status zoa_step(zoa_handle h, const float *const *grads, float lr, int64_t t, void *stream)
+extern "C" zoa_status zoa_step(zoa_handle h, const void *const *grads, float lr, int64_t t, void *stream)
 {
     GradPtrs gp;
-    bool aligned;
+    int aligned;   // gradient format code: alignment bit and element type
     zoa_status rc = check_step_args(h, grads, lr, t, &gp, &aligned, "zoa_step");
     if (rc != ZOA_OK) return rc;
     commit_variance(h);
@@ -389,10 +391,10 @@ extern "C" zoa_status zoa_onebit_average(zoa_handle h, void *stream)
     return ZOA_OK;
 }
 
-extern "C" zoa_status zoa_step_sync(zoa_handle h, const float *const *grads, float lr, int64_t t, void *stream)
+extern "C" zoa_status zoa_step_sync(zoa_handle h, const void *const *grads, float lr, int64_t t, void *stream)
 {
     GradPtrs gp;
-    bool aligned;
+    int aligned;   // gradient format code: alignment bit and element type
     zoa_status rc = check_step_args(h, grads, lr, t, &gp, &aligned, "zoa_step_sync");
     if (rc != ZOA_OK) return rc;
     const double total = h->gamma_sum + (double)lr;
@@ -423,7 +425,7 @@ extern "C" zoa_status zoa_step_sync(zoa_handle h, const float *const *grads, flo
         // Full chunks through the bulk-copy ring; a ragged last chunk through the chunk-per-block kernel.
         const long long n_full = h->n / h->chunk;
         bool var_fused = false;
-        ZOA_CUDA(h, launch_step_sync_pipelined(st, gp, h->c, lr, gamma_sum, do_var, stages, h->sm_count,
+        ZOA_CUDA(h, launch_step_sync_pipelined(st, gp, h->c, lr, gamma_sum, do_var, aligned, stages, h->sm_count,
                                                h->error_flag, h->sched, (unsigned long long)h->wait_limit_ms * 1000000ull,
                                                h->test_stop_after_tiles, &var_fused, s));
         h->n_launches += 1;
@@ -452,10 +454,10 @@ extern "C" zoa_status zoa_step_sync(zoa_handle h, const float *const *grads, flo
     return ZOA_OK;
 }
 
-extern "C" zoa_status zoa_alg2_step(zoa_handle h, const float *const *grads, float lr, int64_t t, void *stream)
+extern "C" zoa_status zoa_alg2_step(zoa_handle h, const void *const *grads, float lr, int64_t t, void *stream)
 {
     GradPtrs gp;
-    bool aligned;
+    int aligned;   // gradient format code: alignment bit and element type
     zoa_status rc = check_step_args(h, grads, lr, t, &gp, &aligned, "zoa_alg2_step");
     if (rc != ZOA_OK) return rc;
     commit_variance(h);
@@ -476,13 +478,13 @@ extern "C" zoa_status zoa_alg2_step(zoa_handle h, const float *const *grads, flo
     return ZOA_OK;
 }
 
-extern "C" zoa_status zoa_step_auto(zoa_handle h, const float *const *grads, float lr, int64_t t, void *stream)
+extern "C" zoa_status zoa_step_auto(zoa_handle h, const void *const *grads, float lr, int64_t t, void *stream)
 {
     if (!h) return ZOA_ERR_ARG;
     return zoa_sync_due(h, t) == 1 ? zoa_step_sync(h, grads, lr, t, stream) : zoa_step(h, grads, lr, t, stream);
 }
 
-extern "C" zoa_status zoa_step_host(zoa_handle h, const float *const *host_grads, float lr, int64_t t,
+extern "C" zoa_status zoa_step_host(zoa_handle h, const void *const *host_grads, float lr, int64_t t,
                                     float *host_x_out, void *stream)
 {
     if (!h) return ZOA_ERR_ARG;
@@ -496,10 +498,10 @@ extern "C" zoa_status zoa_step_host(zoa_handle h, const float *const *host_grads
         cudaError_t e = cudaMalloc(reinterpret_cast<void **>(&h->staging), (size_t)h->W * h->n_pad * sizeof(float));
         if (e != cudaSuccess) { h->staging = nullptr; cudaGetLastError(); return fail_cuda(h, e, "zoa_step_host: staging area"); }
     }
-    const float *dev[kMaxWorkers];
+    const void *dev[kMaxWorkers];
     for (int i = 0; i < h->W; ++i) {
         float *dst = h->staging + (size_t)i * h->n_pad;
-        ZOA_CUDA(h, cudaMemcpyAsync(dst, host_grads[i], (size_t)h->n * sizeof(float), cudaMemcpyHostToDevice, s));
+        ZOA_CUDA(h, cudaMemcpyAsync(dst, host_grads[i], (size_t)h->n * (h->grad_type ? 2 : 4), cudaMemcpyHostToDevice, s));
         dev[i] = dst;
     }
     zoa_status rc = zoa_step_auto(h, dev, lr, t, stream);
@@ -614,6 +616,10 @@ extern "C" zoa_status zoa_set_option(zoa_handle h, int option, int value)
     if (!h) return ZOA_ERR_ARG;
     switch (option) {
     case ZOA_OPT_PIPELINE: h->use_pipeline = value != 0; return ZOA_OK;
+    case ZOA_OPT_GRAD_TYPE:
+        if (value < ZOA_GRAD_F32 || value > ZOA_GRAD_BF16) return fail(h, ZOA_ERR_ARG, "zoa_set_option: unknown gradient type");
+        h->grad_type = value;
+        return ZOA_OK;
     case ZOA_OPT_WAIT_LIMIT_MS:
         if (value < 1 || value > 60000) return fail(h, ZOA_ERR_ARG, "zoa_set_option: wait limit must be 1..60000 ms");
         h->wait_limit_ms = value;

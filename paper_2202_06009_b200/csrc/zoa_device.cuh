@@ -3,6 +3,8 @@
 // binary64 sum and the sign-bit packing.
 #pragma once
 
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -81,17 +83,47 @@ __device__ __forceinline__ float4 ld4_stream(const float *p)
 }
 __device__ __forceinline__ void st4_stream(float *p, float4 v) { __stcs(reinterpret_cast<float4 *>(p), v); }
 
+// How the W gradient buffers are to be read: bit 0 = every pointer is aligned for the
+// vector path (16 bytes for binary32, 8 for the 16-bit types), bits 1-2 = element type.
+// Gradients in binary16 / bfloat16 are converted to binary32 exactly on load; all
+// arithmetic and all state stay binary32.
+constexpr int kGradAligned = 1;
+constexpr int kGradF32 = 0, kGradF16 = 1 << 1, kGradBF16 = 2 << 1, kGradTypeMask = 3 << 1;
+
+__device__ __forceinline__ float grad16_to_float(unsigned short bits, int fmt)
+{
+    return (fmt & kGradTypeMask) == kGradBF16 ? __uint_as_float((unsigned)bits << 16)
+                                              : __half2float(__ushort_as_half(bits));
+}
+__device__ __forceinline__ float4 grad16x4_to_float4(uint2 raw, int fmt)
+{
+    return make_float4(grad16_to_float((unsigned short)(raw.x & 0xFFFFu), fmt), grad16_to_float((unsigned short)(raw.x >> 16), fmt),
+                       grad16_to_float((unsigned short)(raw.y & 0xFFFFu), fmt), grad16_to_float((unsigned short)(raw.y >> 16), fmt));
+}
+
 // Four consecutive gradient values starting at j (j % 4 == 0); the user's buffer
 // has exactly n elements and may be unaligned, so the ragged end and the
-// unaligned case go through guarded scalar loads (zero beyond n).
-__device__ __forceinline__ float4 ld_grad4(const float *g, long long j, long long n, bool aligned)
+// unaligned case go through guarded scalar loads (zero beyond n).  `fmt` as above
+// (0 and 1 are plain binary32, unaligned and aligned).
+__device__ __forceinline__ float4 ld_grad4(const float *g, long long j, long long n, int fmt)
 {
-    if (aligned && j + 4 <= n) return ld4_stream(g + j);
+    const bool aligned = fmt & kGradAligned;
+    if ((fmt & kGradTypeMask) == kGradF32) {
+        if (aligned && j + 4 <= n) return ld4_stream(g + j);
+        float4 r;
+        r.x = j + 0 < n ? g[j + 0] : 0.f;
+        r.y = j + 1 < n ? g[j + 1] : 0.f;
+        r.z = j + 2 < n ? g[j + 2] : 0.f;
+        r.w = j + 3 < n ? g[j + 3] : 0.f;
+        return r;
+    }
+    const unsigned short *h = reinterpret_cast<const unsigned short *>(g);
+    if (aligned && j + 4 <= n) return grad16x4_to_float4(__ldcs(reinterpret_cast<const uint2 *>(h + j)), fmt);
     float4 r;
-    r.x = j + 0 < n ? g[j + 0] : 0.f;
-    r.y = j + 1 < n ? g[j + 1] : 0.f;
-    r.z = j + 2 < n ? g[j + 2] : 0.f;
-    r.w = j + 3 < n ? g[j + 3] : 0.f;
+    r.x = j + 0 < n ? grad16_to_float(h[j + 0], fmt) : 0.f;
+    r.y = j + 1 < n ? grad16_to_float(h[j + 1], fmt) : 0.f;
+    r.z = j + 2 < n ? grad16_to_float(h[j + 2], fmt) : 0.f;
+    r.w = j + 3 < n ? grad16_to_float(h[j + 3], fmt) : 0.f;
     return r;
 }
 

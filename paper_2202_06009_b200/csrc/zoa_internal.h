@@ -8,28 +8,28 @@ namespace zoa {
 cudaError_t configure_kernels();
 
 cudaError_t launch_local_step(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
-                              bool do_var, bool g_aligned, int sm_count, cudaStream_t s);
-cudaError_t launch_variance(const StateView &st, const GradPtrs &g, const Consts &c, bool g_aligned,
+                              bool do_var, int g_aligned, int sm_count, cudaStream_t s);
+cudaError_t launch_variance(const StateView &st, const GradPtrs &g, const Consts &c, int g_aligned,
                             long long first, int sm_count, cudaStream_t s);
 cudaError_t launch_compress(const StateView &st, cudaStream_t s);
 cudaError_t launch_reduce(const StateView &st, const Consts &c, float gamma_sum, cudaStream_t s);
 cudaError_t launch_step_sync(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
-                             float gamma_sum, bool g_aligned, long long first_chunk, long long count, cudaStream_t s);
+                             float gamma_sum, int g_aligned, long long first_chunk, long long count, cudaStream_t s);
 
 cudaError_t launch_alg2(const StateView &st, const GradPtrs &g, const Consts &c, float gamma, bool full_precision,
-                        bool g_aligned, int sm_count, cudaStream_t s);
+                        int g_aligned, int sm_count, cudaStream_t s);
 
 // Chunks larger than kMaxChunk (up to the whole vector): multi-pass kernels, zoa_kernels.cu.
 long long large_chunk_segments(const StateView &st);
-cudaError_t launch_large_compress(const StateView &st, const GradPtrs &g, bool from_grads, bool g_aligned,
+cudaError_t launch_large_compress(const StateView &st, const GradPtrs &g, bool from_grads, int g_aligned,
                                   double *partials, int *launches, cudaStream_t s);
 cudaError_t launch_large_server(const StateView &st, const Consts &c, int mode, float scalar, double *partials,
                                 int *launches, cudaStream_t s);
 
 // Pipelined (bulk-copy ring) form of the fused sync step, zoa_pipeline.cu.
-int pipeline_stages(const StateView &st, bool g_aligned);
+int pipeline_stages(const StateView &st, int grad_fmt);
 cudaError_t launch_step_sync_pipelined(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
-                                       float gamma_sum, bool do_var, int stages, int sm_count, int *error_flag,
+                                       float gamma_sum, bool do_var, int grad_fmt, int stages, int sm_count, int *error_flag,
                                        unsigned long long *sched, unsigned long long wait_limit_ns,
                                        long long test_stop_after_tiles, bool *var_fused, cudaStream_t s);
 

@@ -685,7 +685,7 @@ static int elementwise_grid(long long n4, int /*sm_count*/)
 }
 
 cudaError_t launch_local_step(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
-                              bool do_var, bool g_aligned, int sm_count, cudaStream_t s)
+                              bool do_var, int g_aligned, int sm_count, cudaStream_t s)
 {
     const int grid = elementwise_grid((st.n + 3) / 4, sm_count);
     if (do_var)
@@ -696,7 +696,7 @@ cudaError_t launch_local_step(const StateView &st, const GradPtrs &g, const Cons
 }
 
 // Lines 14-15 for the coordinates [first, n); first is a multiple of 4.
-cudaError_t launch_variance(const StateView &st, const GradPtrs &g, const Consts &c, bool g_aligned,
+cudaError_t launch_variance(const StateView &st, const GradPtrs &g, const Consts &c, int g_aligned,
                             long long first, int sm_count, cudaStream_t s)
 {
     const long long first4 = first >> 2;
@@ -721,7 +721,7 @@ cudaError_t configure_kernels()
 }
 
 cudaError_t launch_alg2(const StateView &st, const GradPtrs &g, const Consts &c, float gamma, bool full_precision,
-                        bool g_aligned, int sm_count, cudaStream_t s)
+                        int g_aligned, int sm_count, cudaStream_t s)
 {
     if (full_precision)
         alg2_full_kernel<<<elementwise_grid((st.n + 3) / 4, sm_count), 256, 0, s>>>(st, g, c, gamma, g_aligned);
@@ -746,7 +746,7 @@ cudaError_t launch_reduce(const StateView &st, const Consts &c, float gamma_sum,
 
 // The chunks [first_chunk, first_chunk + count) of a sync step, one block each.
 cudaError_t launch_step_sync(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
-                             float gamma_sum, bool g_aligned, long long first_chunk, long long count, cudaStream_t s)
+                             float gamma_sum, int g_aligned, long long first_chunk, long long count, cudaStream_t s)
 {
     step_sync_kernel<<<(unsigned)count, block_threads_for_chunk(st.chunk), step_sync_smem(st.chunk), s>>>(
         st, g, c, gamma, gamma_sum, g_aligned, first_chunk);
@@ -765,7 +765,7 @@ long long large_chunk_segments(const StateView &st)
 
 // Worker side of Algorithm 3 for chunks too large for one block.  from_grads: compress
 // g + delta (Algorithm 2) instead of u + delta (Algorithm 1).  partials: [W + 1][n_chunks * segments].
-cudaError_t launch_large_compress(const StateView &st, const GradPtrs &g, bool from_grads, bool g_aligned,
+cudaError_t launch_large_compress(const StateView &st, const GradPtrs &g, bool from_grads, int g_aligned,
                                   double *partials, int *launches, cudaStream_t s)
 {
     const long long spc = large_chunk_segments(st), n_segs = spc * st.n_chunks;

@@ -39,6 +39,7 @@ struct PipeArgs {
     int stages;
     int *error_flag;  // device int, set non-zero when a wait ran out
     unsigned long long *sched;  // device: [0] next chunk to hand out, [1] blocks that have finished
+    int grad_fmt;                      // kGradF32 / kGradF16 / kGradBF16 (| kGradAligned, always set here)
     unsigned long long wait_limit_ns;  // how long a thread waits on an mbarrier before it gives up
     long long test_stop_after_tiles;   // > 0: each producer stops after this many tiles (error-path test)
 };
@@ -220,8 +221,9 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
                     const long long off = c0 + (long long)t * kTile;
                     if (i < W) {
                         const long long row = (long long)i * st.n_pad + off;
-                        mbar_arrive_expect_tx(full, 4 * kTileBytes);
-                        bulk_load(dst, a.g.p[i] + off, kTileBytes, full);
+                        const uint32_t g_elem = (a.grad_fmt & kGradTypeMask) == kGradF32 ? 4u : 2u;
+                        mbar_arrive_expect_tx(full, 3 * kTileBytes + kTile * g_elem);
+                        bulk_load(dst, reinterpret_cast<const char *>(a.g.p[i]) + off * g_elem, kTile * g_elem, full);
                         bulk_load(dst + kTileBytes, st.m + row, kTileBytes, full);
                         bulk_load(dst + 2 * kTileBytes, st.u + row, kTileBytes, full);
                         bulk_load(dst + 3 * kTileBytes, st.dw + row, kTileBytes, full);
@@ -316,7 +318,10 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
                 const float *stage = reinterpret_cast<const float *>(ring + (size_t)s * kStageBytes);
                 float4 g4 = make_float4(0.f, 0.f, 0.f, 0.f), m4 = g4, u4 = g4, e4 = g4;
                 if (ready) {
-                    g4 = ld4(stage + pos);
+                    if ((a.grad_fmt & kGradTypeMask) == kGradF32)
+                        g4 = ld4(stage + pos);
+                    else   // 16-bit gradients fill the first half of the slot
+                        g4 = grad16x4_to_float4(*reinterpret_cast<const uint2 *>(reinterpret_cast<const unsigned short *>(stage) + pos), a.grad_fmt);
                     m4 = ld4(stage + kTile + pos);
                     u4 = ld4(stage + 2 * kTile + pos);
                     e4 = ld4(stage + 3 * kTile + pos);
@@ -460,9 +465,9 @@ static size_t pipeline_fixed_smem(int W, int chunk)
 }
 
 // How many ring stages fit (0 = the pipelined kernel does not apply to this shape).
-int pipeline_stages(const StateView &st, bool g_aligned)
+int pipeline_stages(const StateView &st, int grad_fmt)
 {
-    if (!g_aligned) return 0;
+    if (!(grad_fmt & kGradAligned)) return 0;
     if (st.chunk != kTile && st.chunk != 2 * kTile && st.chunk != 4 * kTile) return 0;
     if (st.n / st.chunk < 1) return 0;
     const int tiles = st.chunk / kTile;
@@ -494,7 +499,7 @@ static cudaError_t launch_pipe(const PipeArgs &a, int grid, size_t smem, cudaStr
 // Runs the full chunks [0, n / chunk) of a sync step; the ragged last chunk, if any, is the caller's.
 // *var_fused tells whether lines 14-15 were done here too.
 cudaError_t launch_step_sync_pipelined(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
-                                       float gamma_sum, bool do_var, int stages, int sm_count, int *error_flag,
+                                       float gamma_sum, bool do_var, int grad_fmt, int stages, int sm_count, int *error_flag,
                                        unsigned long long *sched, unsigned long long wait_limit_ns,
                                        long long test_stop_after_tiles, bool *var_fused, cudaStream_t s)
 {
@@ -504,6 +509,7 @@ cudaError_t launch_step_sync_pipelined(const StateView &st, const GradPtrs &g, c
     a.stages = stages;
     a.error_flag = error_flag;
     a.sched = sched;
+    a.grad_fmt = grad_fmt;
     a.wait_limit_ns = wait_limit_ns;
     a.test_stop_after_tiles = test_stop_after_tiles;
     const int grid = (int)(a.n_full_chunks < sm_count ? a.n_full_chunks : sm_count);

@@ -18,14 +18,17 @@ def _stream():
     return torch.cuda.current_stream().cuda_stream
 
 
-def _grad_ptrs(grads, n, W):
+_GRAD_TYPES = {torch.float32: B.GRAD_F32, torch.float16: B.GRAD_F16, torch.bfloat16: B.GRAD_BF16}
+
+
+def _grad_ptrs(grads, n, W, dtype=torch.float32):
     if isinstance(grads, torch.Tensor):
         grads = list(grads)
     if len(grads) != W:
         raise ValueError(f"expected {W} gradient tensors, got {len(grads)}")
     for g in grads:
-        if not (g.is_cuda and g.dtype == torch.float32 and g.is_contiguous() and g.numel() == n):
-            raise ValueError("each gradient must be a contiguous float32 CUDA tensor of n_params elements")
+        if not (g.is_cuda and g.dtype == dtype and g.is_contiguous() and g.numel() == n):
+            raise ValueError(f"each gradient must be a contiguous {dtype} CUDA tensor of n_params elements")
     return [g.data_ptr() for g in grads]
 
 
@@ -34,6 +37,7 @@ class Zoa:
         self.n, self.W, self.chunk = int(n_params), int(W), int(chunk)
         self.n_chunks = (self.n + self.chunk - 1) // self.chunk
         self.h = B.zoa_create(self.n, self.W, beta1, beta2, eps, self.chunk)
+        self.grad_dtype = torch.float32
 
     def close(self):
         if self.h is not None:
@@ -67,6 +71,11 @@ class Zoa:
         """Fused sync step through the bulk-copy ring kernel (default) or the chunk-per-block one."""
         B.zoa_set_option(self.h, B.OPT_PIPELINE, int(bool(on)))
 
+    def set_grad_dtype(self, dtype):
+        """Gradients arrive as torch.float32 (default), torch.float16 or torch.bfloat16."""
+        B.zoa_set_option(self.h, B.OPT_GRAD_TYPE, _GRAD_TYPES[dtype])
+        self.grad_dtype = dtype
+
     def sync_due(self, t):
         return B.zoa_sync_due(self.h, t) == 1
 
@@ -75,7 +84,7 @@ class Zoa:
 
     # -- Algorithm 1 --------------------------------------------------------
     def step(self, grads, lr, t):
-        B.zoa_step(self.h, _grad_ptrs(grads, self.n, self.W), lr, t, _stream())
+        B.zoa_step(self.h, _grad_ptrs(grads, self.n, self.W, self.grad_dtype), lr, t, _stream())
 
     def onebit_reduce(self):
         B.zoa_onebit_reduce(self.h, _stream())
@@ -99,13 +108,13 @@ class Zoa:
         return t.view(torch.int32) if words else t
 
     def step_sync(self, grads, lr, t):
-        B.zoa_step_sync(self.h, _grad_ptrs(grads, self.n, self.W), lr, t, _stream())
+        B.zoa_step_sync(self.h, _grad_ptrs(grads, self.n, self.W, self.grad_dtype), lr, t, _stream())
 
     def step_auto(self, grads, lr, t):
-        B.zoa_step_auto(self.h, _grad_ptrs(grads, self.n, self.W), lr, t, _stream())
+        B.zoa_step_auto(self.h, _grad_ptrs(grads, self.n, self.W, self.grad_dtype), lr, t, _stream())
 
     def alg2_step(self, grads, lr, t):
-        B.zoa_alg2_step(self.h, _grad_ptrs(grads, self.n, self.W), lr, t, _stream())
+        B.zoa_alg2_step(self.h, _grad_ptrs(grads, self.n, self.W, self.grad_dtype), lr, t, _stream())
 
     def step_host(self, host_grads, lr, t, host_x_out=None):
         ptrs = [g.data_ptr() for g in host_grads]

@@ -443,3 +443,59 @@ def test_paper_schedules_on_a_handle():
         assert [t for t in range(40) if z.var_due(t)] == [0, 1, 2, 4, 6, 10, 14]     # nothing from step 15 on
     finally:
         z.close()
+
+
+# --------------------------------------------------------------------------
+# 16-bit gradients (the paper trains in FP16): converted exactly on load
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
+@pytest.mark.parametrize("mode", ["fused", "two_call", "alg2"])
+@pytest.mark.parametrize("W,chunk,n,offset", [(4, 2048, 9 * 2048 + 77, 0), (3, 4096, 5 * 4096 + 1852, 0), (2, 8192, 3 * 8192, 0),
+                                              (3, 1024, 5000, 0), (2, 4096, 3 * 4096 + 5, 1), (2, 32768, 70000, 0)])
+def test_sixteen_bit_gradients(dtype, mode, W, chunk, n, offset):
+    """The oracle is given the binary32 values of the very same 16-bit numbers; the GPU reads
+    the 16-bit buffers.  `offset` shifts the buffers by one element (unaligned path)."""
+    rng = np.random.default_rng(W * chunk + n)
+    p = Pair(n, W, chunk, var_steps=(0, 2), sync=((0, 3), (1, 2)), x0=rng.standard_normal(n) * 0.02)
+    try:
+        p.gpu.set_grad_dtype(dtype)
+        for t in range(5):
+            backing = torch.from_numpy(_grads(rng, W, n + offset)).cuda().to(dtype)
+            g16 = [backing[i, offset:offset + n] for i in range(W)]
+            if offset == 0:
+                g16 = [g.clone() for g in g16]
+            g32 = torch.stack([g.float() for g in g16]).cpu().numpy()
+            sync, var = p.gpu.sync_due(t), p.gpu.var_due(t)
+            if mode == "alg2":
+                p.gpu.alg2_step(g16, 1e-3, t)
+                p.cpu.alg2_step(g32, np.float32(1e-3), var)
+            else:
+                if mode == "fused":
+                    p.gpu.step_auto(g16, 1e-3, t)
+                else:
+                    p.gpu.step(g16, 1e-3, t)
+                    if sync:
+                        p.gpu.onebit_reduce()
+                p.cpu.step(g32, np.float32(1e-3), t, sync, var)
+            torch.cuda.synchronize()
+            p.compare(f"t={t}", wire=False)
+        p.gpu.check_device()
+    finally:
+        p.close()
+
+
+def test_sixteen_bit_host_gradients():
+    rng = np.random.default_rng(9)
+    n, W, chunk = 3 * 2048 + 100, 2, 2048
+    a, b = Zoa(n, W, chunk=chunk), Zoa(n, W, chunk=chunk)
+    try:
+        a.set_grad_dtype(torch.bfloat16), b.set_grad_dtype(torch.bfloat16)
+        for t in range(3):
+            g = torch.from_numpy(_grads(rng, W, n)).to(torch.bfloat16).pin_memory()
+            out = torch.empty(n).pin_memory()
+            a.step_host(list(g), 1e-3, t, out)
+            b.step_auto(list(g.cuda()), 1e-3, t)
+            torch.cuda.synchronize()
+            assert np.array_equal(out.numpy(), b.read("x", 0))
+    finally:
+        a.close(), b.close()
