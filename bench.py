@@ -45,6 +45,16 @@ def variance_bytes(n, W):
     return n * W * 4 + n * 8
 
 
+def two_call_sync_bytes(n, W, chunk, g_bytes=4):
+    """zoa_step then zoa_onebit_reduce: the local step writes m, x, u (24 + g B in, 12 B out),
+    the compress kernel reads u, delta and writes delta and the packed form (12 1/8 B), the
+    reduce kernel reads the packed form and writes m, x, u (12 1/8 B) plus the per-parameter
+    server traffic (20 1/8 B)."""
+    n_chunks = -(-n // chunk)
+    return (local_step_bytes(n, W, g_bytes) + n * W * (12 + 1 / 8) + 4 * n_chunks * W
+            + n * W * (12 + 1 / 8) + 4 * n_chunks * W + n * (20 + 1 / 8) + 4 * n_chunks)
+
+
 def alg2_compressed_bytes(n, W, chunk, g_bytes=4):
     """Algorithm 2, compressed step: per parameter and worker read g, delta, m, x (16 B), write
     delta, m, x (12 B) and 1 sign bit + a scale per chunk; per parameter read delta_bar, v,
@@ -221,6 +231,10 @@ def run_ours(args, wl):
             if args.algorithm == "alg2":
                 opt.alg2_step(bufs, wl.lr_at(t), t)
                 kinds.append("alg2_full" if wl.in_T_v(t) else "alg2_compressed")
+            elif args.two_call and wl.in_T_u(t):
+                opt.step(bufs, wl.lr_at(t), t)
+                opt.onebit_reduce()
+                kinds.append("two_call_sync" + ("+var" if wl.in_T_v(t) else ""))
             else:
                 opt.step_auto(bufs, wl.lr_at(t), t)
                 kinds.append(("sync" if wl.in_T_u(t) else "local") + ("+var" if wl.in_T_v(t) else ""))
@@ -244,17 +258,20 @@ def run_ours(args, wl):
     # the variance update needs nothing beyond writing v_{t+1}: g and v are read anyway
     bytes_of["sync+var"] = bytes_of["sync"] + wl.n * 4
     bytes_of["local+var"] = bytes_of["local"] + wl.n * 4
+    bytes_of["two_call_sync"] = two_call_sync_bytes(wl.n, wl.W, wl.chunk, g_bytes)
+    bytes_of["two_call_sync+var"] = bytes_of["two_call_sync"] + wl.n * 4
     bytes_of["alg2_compressed"] = alg2_compressed_bytes(wl.n, wl.W, wl.chunk, g_bytes)
     bytes_of["alg2_full"] = alg2_full_bytes(wl.n, wl.W, g_bytes)
     step_types = {k: {"count": len(v), "ms": statistics.mean(v), "algorithmic_GB": bytes_of[k] / 1e9,
                       "GBps": bytes_of[k] / 1e6 / statistics.mean(v)} for k, v in by_kind.items()}
     total_bytes = sum(bytes_of[k] for k in kinds)
-    dominant = next((k for k in ("sync", "sync+var", "alg2_compressed") if k in by_kind), kinds[0])
+    dominant = next((k for k in ("sync", "sync+var", "two_call_sync", "alg2_compressed") if k in by_kind), kinds[0])
     achieved = bytes_of[dominant] / 1e6 / statistics.mean(by_kind[dominant])
     sync_kernel = "step_sync_kernel" if args.no_pipeline else "step_sync_pipelined_kernel"
     if wl.chunk > 16384:
         sync_kernel = "local_step_kernel + lc_* (multi-pass large-chunk kernels)"
-    kernel_of = {"sync": sync_kernel, "sync+var": sync_kernel, "alg2_compressed": "alg2_compressed_kernel",
+    kernel_of = {"sync": sync_kernel, "sync+var": sync_kernel,
+                 "two_call_sync": "local_step_kernel + compress_kernel + reduce_kernel", "alg2_compressed": "alg2_compressed_kernel",
                  "alg2_full": "alg2_full_kernel"}
     roofline = {"bound": "hbm", "kernel": kernel_of.get(dominant, "local_step_kernel"),
                 "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
@@ -398,6 +415,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--scale", type=int, default=1, help="shrink every tensor by this factor (profiling captures)")
     ap.add_argument("--no-pipeline", action="store_true", help="fused sync step through the chunk-per-block kernel")
+    ap.add_argument("--two-call", action="store_true",
+                    help="sync steps as zoa_step + zoa_onebit_reduce (three kernels) instead of the fused call")
     ap.add_argument("--grad-dtype", default="f32", choices=["f32", "f16", "bf16"],
                     help="element type of the gradient buffers (state and arithmetic stay f32)")
     ap.add_argument("--chunk", type=int, default=0,
