@@ -1,12 +1,17 @@
-// The zoa kernels, chunk-per-block form: correct for every shape the API
-// accepts (any chunk that is a multiple of 32, a ragged last chunk, unaligned
-// gradient pointers).
+// The zoa kernels other than the bulk-copy ring kernel (zoa_pipeline.cu).
 //
-//   local_step_kernel   Algorithm 1 lines 3-5 (+ lines 14-15 on T_v steps)
-//   variance_kernel     Algorithm 1 lines 14-15 alone
-//   compress_kernel     Algorithm 3 worker side (Eq. 3 per chunk, error feedback)
-//   reduce_kernel       Algorithm 3 server side + Algorithm 1 lines 8-10
-//   step_sync_kernel    all of the above for a sync step, one pass over memory
+// Elementwise, one float4 per thread:
+//   local_step_kernel        Algorithm 1 lines 3-5 (+ lines 14-15 on T_v steps)
+//   variance_kernel          Algorithm 1 lines 14-15 alone
+//   alg2_full_kernel         Algorithm 2 on a T_v step (full-precision exchange)
+// One block per chunk (any chunk that is a multiple of 32 up to 16384, ragged last
+// chunk, unaligned or 16-bit gradient buffers):
+//   compress_kernel          Algorithm 3 worker side (Eq. 3 per chunk, error feedback)
+//   reduce_kernel            Algorithm 3 server side + Algorithm 1 lines 8-10
+//   step_sync_kernel         a whole sync step of Algorithm 1 in one pass over memory
+//   alg2_compressed_kernel   Algorithm 2 on any other step (gradients through Algorithm 3)
+// Chunks larger than a block can hold, up to the whole vector (Eq. 3 as printed):
+//   lc_* kernels             per-segment partial l1 sums, fixed-order chunk sums, apply passes
 #include "zoa_internal.h"
 
 namespace zoa {
@@ -15,10 +20,13 @@ namespace zoa {
 // Local step: elementwise, one thread per 4 coordinates, loop over workers so
 // that v is read once and the gradient mean for the variance comes for free.
 // ---------------------------------------------------------------------------
-template <bool DO_VAR>
+// GFMT: the gradient format when it is known at compile time (the aligned cases, which are
+// the fast path), or -1 to read it from the argument.
+template <bool DO_VAR, int GFMT>
 __global__ void __launch_bounds__(256)
-local_step_kernel(StateView st, GradPtrs g, Consts c, float gamma, int g_aligned)
+local_step_kernel(StateView st, GradPtrs g, Consts c, float gamma, int g_fmt_arg)
 {
+    const int g_aligned = GFMT >= 0 ? GFMT : g_fmt_arg;
     const long long n4 = (st.n + 3) >> 2;
     const long long stride = (long long)gridDim.x * blockDim.x;
     for (long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x; q < n4; q += stride) {
@@ -673,7 +681,7 @@ static int block_threads_for_chunk(int chunk)
     return p;
 }
 
-static int elementwise_grid(long long n4, int /*sm_count*/)
+static int elementwise_grid(long long n4)
 {
     // One float4 per thread and as many blocks as that takes: SMs do not all get the same
     // share of DRAM bandwidth, and the hardware block scheduler evens that out, where a
@@ -687,11 +695,15 @@ static int elementwise_grid(long long n4, int /*sm_count*/)
 cudaError_t launch_local_step(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
                               bool do_var, int g_aligned, int sm_count, cudaStream_t s)
 {
-    const int grid = elementwise_grid((st.n + 3) / 4, sm_count);
-    if (do_var)
-        local_step_kernel<true><<<grid, 256, 0, s>>>(st, g, c, gamma, g_aligned);
-    else
-        local_step_kernel<false><<<grid, 256, 0, s>>>(st, g, c, gamma, g_aligned);
+    const int grid = elementwise_grid((st.n + 3) / 4);
+#define ZOA_LOCAL(VAR, FMT) local_step_kernel<VAR, FMT><<<grid, 256, 0, s>>>(st, g, c, gamma, g_aligned)
+    switch (g_aligned) {
+    case kGradF32 | kGradAligned: if (do_var) ZOA_LOCAL(true, kGradF32 | kGradAligned); else ZOA_LOCAL(false, kGradF32 | kGradAligned); break;
+    case kGradF16 | kGradAligned: if (do_var) ZOA_LOCAL(true, kGradF16 | kGradAligned); else ZOA_LOCAL(false, kGradF16 | kGradAligned); break;
+    case kGradBF16 | kGradAligned: if (do_var) ZOA_LOCAL(true, kGradBF16 | kGradAligned); else ZOA_LOCAL(false, kGradBF16 | kGradAligned); break;
+    default: if (do_var) ZOA_LOCAL(true, -1); else ZOA_LOCAL(false, -1); break;
+    }
+#undef ZOA_LOCAL
     return cudaGetLastError();
 }
 
@@ -700,7 +712,7 @@ cudaError_t launch_variance(const StateView &st, const GradPtrs &g, const Consts
                             long long first, int sm_count, cudaStream_t s)
 {
     const long long first4 = first >> 2;
-    variance_kernel<<<elementwise_grid((st.n + 3) / 4 - first4, sm_count), 256, 0, s>>>(st, g, c, g_aligned, first4);
+    variance_kernel<<<elementwise_grid((st.n + 3) / 4 - first4), 256, 0, s>>>(st, g, c, g_aligned, first4);
     return cudaGetLastError();
 }
 
@@ -724,7 +736,7 @@ cudaError_t launch_alg2(const StateView &st, const GradPtrs &g, const Consts &c,
                         int g_aligned, int sm_count, cudaStream_t s)
 {
     if (full_precision)
-        alg2_full_kernel<<<elementwise_grid((st.n + 3) / 4, sm_count), 256, 0, s>>>(st, g, c, gamma, g_aligned);
+        alg2_full_kernel<<<elementwise_grid((st.n + 3) / 4), 256, 0, s>>>(st, g, c, gamma, g_aligned);
     else
         alg2_compressed_kernel<<<(unsigned)st.n_chunks, block_threads_for_chunk(st.chunk), step_sync_smem(st.chunk), s>>>(
             st, g, c, gamma, g_aligned);

@@ -149,23 +149,7 @@ __device__ __forceinline__ uint32_t pack_group(const bool b[4])
     return __reduce_or_sync(0xFFu << (lane & 24), nib << ((lane & 7) * 4));
 }
 
-#ifdef ZOA_PIPE_PROFILE
-__device__ unsigned long long g_pipe_prof[256][8];
-#define PROF_T0() const long long prof_t0_ = clock64()
-#define PROF_ADD(slot) do { if (tid == 0) prof[slot] += clock64() - prof_t0_; } while (0)
-#else
-#define PROF_T0() do {} while (0)
-#define PROF_ADD(slot) do {} while (0)
-#endif
-
 }  // namespace
-
-#ifdef ZOA_PIPE_PROFILE
-extern "C" int zoa_debug_read_pipe_profile(unsigned long long *out)
-{
-    return (int)cudaMemcpyFromSymbol(out, g_pipe_prof, sizeof(g_pipe_prof));
-}
-#endif
 
 template <int TILES, bool DO_VAR>
 __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const __grid_constant__ PipeArgs a)
@@ -259,10 +243,6 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
     }
 
     // -------------------------------- consumers --------------------------------
-#ifdef ZOA_PIPE_PROFILE
-    unsigned long long prof[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-    const long long prof_start = clock64();
-#endif
     int s = 0;
     uint32_t phase = 0;
     int flip = 0;
@@ -312,9 +292,7 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
             double l1 = 0.0;
 #pragma unroll
             for (int t = 0; t < TILES; ++t) {
-                PROF_T0();
                 const bool ready = mbar_wait(smem_addr(&sh->full[s]), phase, abort_flag, a.error_flag, a.wait_limit_ns);
-                PROF_ADD(0);
                 const float *stage = reinterpret_cast<const float *>(ring + (size_t)s * kStageBytes);
                 float4 g4 = make_float4(0.f, 0.f, 0.f, 0.f), m4 = g4, u4 = g4, e4 = g4;
                 if (ready) {
@@ -339,9 +317,7 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
                     if (DO_VAR) G[t][k] += (double)gg[k];
                 }
             }
-            float scale;
-            { PROF_T0(); scale = chunk_scale(consumer_sum(l1, sh, flip), st.chunk); PROF_ADD(1); }
-            PROF_T0();
+            const float scale = chunk_scale(consumer_sum(l1, sh, flip), st.chunk);
             const long long row = (long long)i * st.n_pad + c0;
 #pragma unroll
             for (int t = 0; t < TILES; ++t) {
@@ -362,7 +338,6 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
             if (lane == 0) my_scales[i] = scale;
             if (tid == 0) st.scales_w[(long long)i * st.n_chunks + chunk] = scale;
             if (DEFER && c0_prev >= 0) store_prev_worker(i);
-            PROF_ADD(2);
         }
         __syncwarp();   // bits_s and my_scales were written by lanes of this warp
 
@@ -447,12 +422,6 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
     }
     if (c0_prev >= 0)
         for (int i = 0; i < W; ++i) store_prev_worker(i);   // the block's last chunk
-#ifdef ZOA_PIPE_PROFILE
-    if (tid == 0) {
-        prof[7] = clock64() - prof_start;
-        for (int k = 0; k < 8; ++k) g_pipe_prof[blockIdx.x][k] = prof[k];
-    }
-#endif
 }
 
 // ---------------------------------------------------------------------------

@@ -499,3 +499,17 @@ def test_sixteen_bit_host_gradients():
             assert np.array_equal(out.numpy(), b.read("x", 0))
     finally:
         a.close(), b.close()
+
+
+def test_create_destroy_returns_device_memory():
+    torch.cuda.empty_cache()
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    for _ in range(20):
+        z = Zoa(1 << 22, 4, chunk=4096)            # ~340 MB of state each
+        z.step_sync(list(torch.zeros(4, 1 << 22, device="cuda")), 1e-3, 0)
+        z.close()
+    torch.cuda.empty_cache()
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free0 - free1 < 64 << 20, f"{(free0 - free1) >> 20} MiB did not come back"
