@@ -419,7 +419,10 @@ extern "C" zoa_status zoa_step_sync(zoa_handle h, const void *const *grads, floa
         h->n_syncs += 1;
         return ZOA_OK;
     }
-    const int stages = h->use_pipeline ? pipeline_stages(st, aligned) : 0;
+    // The persistent kernel pays off once every SM has a few chunks to stream; below that the
+    // one-block-per-chunk kernel starts faster (measured on the 512-chunk configuration).
+    const bool enough_chunks = h->n / h->chunk >= 4ll * h->sm_count;
+    const int stages = h->use_pipeline && enough_chunks ? pipeline_stages(st, aligned) : 0;
     long long var_first = 0;     // coordinates from here on still need lines 14-15
     if (stages > 0) {
         // Full chunks through the bulk-copy ring; a ragged last chunk through the chunk-per-block kernel.
@@ -469,8 +472,21 @@ extern "C" zoa_status zoa_alg2_step(zoa_handle h, const void *const *grads, floa
         ZOA_CUDA(h, launch_large_server(view(h), h->c, 2, lr, h->partials, &launches, s));
         h->n_launches += launches;
     } else {
-        ZOA_CUDA(h, launch_alg2(view(h), gp, h->c, lr, full, aligned, h->sm_count, static_cast<cudaStream_t>(stream)));
-        h->n_launches += 1;
+        cudaStream_t s = static_cast<cudaStream_t>(stream);
+        const StateView st = view(h);
+        const bool enough_chunks = h->n / h->chunk >= 4ll * h->sm_count;
+        const int stages = (!full && h->use_pipeline && enough_chunks) ? alg2_pipeline_stages(st, aligned) : 0;
+        long long first = 0;
+        if (stages > 0) {   // full chunks through the bulk-copy ring, a ragged last chunk through the block kernel
+            ZOA_CUDA(h, launch_alg2_pipelined(st, gp, h->c, lr, aligned, stages, h->sm_count, h->error_flag, h->sched,
+                                              (unsigned long long)h->wait_limit_ms * 1000000ull, h->test_stop_after_tiles, s));
+            h->n_launches += 1;
+            first = h->n / h->chunk;
+        }
+        if (full || first < h->n_chunks) {
+            ZOA_CUDA(h, launch_alg2(st, gp, h->c, lr, full, aligned, first, h->n_chunks - first, s));
+            h->n_launches += 1;
+        }
     }
     if (full) { h->v_pending = true; h->n_var_updates += 1; } else h->n_syncs += 1;
     h->t_last = t;

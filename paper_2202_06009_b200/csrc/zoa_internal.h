@@ -17,7 +17,7 @@ cudaError_t launch_step_sync(const StateView &st, const GradPtrs &g, const Const
                              float gamma_sum, int g_aligned, long long first_chunk, long long count, cudaStream_t s);
 
 cudaError_t launch_alg2(const StateView &st, const GradPtrs &g, const Consts &c, float gamma, bool full_precision,
-                        int g_aligned, int sm_count, cudaStream_t s);
+                        int g_aligned, long long first_chunk, long long count, cudaStream_t s);
 
 // Chunks larger than kMaxChunk (up to the whole vector): multi-pass kernels, zoa_kernels.cu.
 long long large_chunk_segments(const StateView &st);
@@ -32,5 +32,10 @@ cudaError_t launch_step_sync_pipelined(const StateView &st, const GradPtrs &g, c
                                        float gamma_sum, bool do_var, int grad_fmt, int stages, int sm_count, int *error_flag,
                                        unsigned long long *sched, unsigned long long wait_limit_ns,
                                        long long test_stop_after_tiles, bool *var_fused, cudaStream_t s);
+
+int alg2_pipeline_stages(const StateView &st, int grad_fmt);
+cudaError_t launch_alg2_pipelined(const StateView &st, const GradPtrs &g, const Consts &c, float gamma, int grad_fmt,
+                                  int stages, int sm_count, int *error_flag, unsigned long long *sched,
+                                  unsigned long long wait_limit_ns, long long test_stop_after_tiles, cudaStream_t s);
 
 }  // namespace zoa

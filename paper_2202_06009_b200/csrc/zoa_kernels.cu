@@ -377,13 +377,14 @@ alg2_full_kernel(StateView st, GradPtrs g, Consts c, float gamma, int g_aligned)
 // Any other step of Algorithm 2 for chunk blockIdx.x (lines 7, 10-11): the
 // gradients go through the error-feedback 1-bit AllReduce (Algorithm 3), the
 // decompressed mean drives momentum and model on every worker.
-__global__ void __launch_bounds__(512, 2) alg2_compressed_kernel(StateView st, GradPtrs g, Consts c, float gamma, int g_aligned)
+__global__ void __launch_bounds__(512, 2) alg2_compressed_kernel(StateView st, GradPtrs g, Consts c, float gamma, int g_aligned, long long chunk_offset)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     double *scratch = reinterpret_cast<double *>(smem_raw);
     double *A_s = scratch + 34;
     float *z_s = reinterpret_cast<float *>(A_s + st.chunk);
-    const ChunkGeom cg = chunk_geom(st, blockIdx.x);
+    const long long chunk_id = chunk_offset + blockIdx.x;
+    const ChunkGeom cg = chunk_geom(st, chunk_id);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
 
     for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
@@ -420,7 +421,7 @@ __global__ void __launch_bounds__(512, 2) alg2_compressed_kernel(StateView st, G
             if (lane < 4 && base + 32 * lane < cg.len)
                 st.words_w[(long long)i * st.words_stride + ((cg.c0 + base) >> 5) + lane] = word;
         }
-        if (threadIdx.x == 0) st.scales_w[(long long)i * st.n_chunks + blockIdx.x] = scale;
+        if (threadIdx.x == 0) st.scales_w[(long long)i * st.n_chunks + chunk_id] = scale;
     }
     double l1 = 0.0;
     for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
@@ -478,7 +479,7 @@ __global__ void __launch_bounds__(512, 2) alg2_compressed_kernel(StateView st, G
                 }
         }
     }
-    if (threadIdx.x == 0) st.scales_s[blockIdx.x] = scale;
+    if (threadIdx.x == 0) st.scales_s[chunk_id] = scale;
 }
 
 // ---------------------------------------------------------------------------
@@ -732,14 +733,16 @@ cudaError_t configure_kernels()
     return cudaFuncSetAttribute(step_sync_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)step_sync_smem(kMaxChunk));
 }
 
+// A step of Algorithm 2: the whole vector at full precision, or the chunks
+// [first_chunk, first_chunk + count) through the 1-bit AllReduce.
 cudaError_t launch_alg2(const StateView &st, const GradPtrs &g, const Consts &c, float gamma, bool full_precision,
-                        int g_aligned, int sm_count, cudaStream_t s)
+                        int g_aligned, long long first_chunk, long long count, cudaStream_t s)
 {
     if (full_precision)
         alg2_full_kernel<<<elementwise_grid((st.n + 3) / 4), 256, 0, s>>>(st, g, c, gamma, g_aligned);
     else
-        alg2_compressed_kernel<<<(unsigned)st.n_chunks, block_threads_for_chunk(st.chunk), step_sync_smem(st.chunk), s>>>(
-            st, g, c, gamma, g_aligned);
+        alg2_compressed_kernel<<<(unsigned)count, block_threads_for_chunk(st.chunk), step_sync_smem(st.chunk), s>>>(
+            st, g, c, gamma, g_aligned, first_chunk);
     return cudaGetLastError();
 }
 

@@ -28,7 +28,8 @@ constexpr int kThreads = kConsumers + 32;       // + one producer warp
 constexpr int kTile = 4 * kConsumers;           // coordinates per ring stage and array
 constexpr int kTileBytes = kTile * 4;
 constexpr int kStageBytes = 4 * kTileBytes;     // g, m, u, delta  |  delta_bar, v, x_sync, (unused)
-constexpr int kMaxStages = 6;
+constexpr int kSyncStages = 6;                  // ring depth of the fused sync kernel (32 KB stages)
+constexpr int kMaxStages = 12;                  // of the Algorithm 2 kernel (16 KB stages)
 
 struct PipeArgs {
     StateView st;
@@ -425,6 +426,234 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
 }
 
 // ---------------------------------------------------------------------------
+// Algorithm 2, compressed step, in the same style: per chunk the ring carries W x TILES
+// tiles of (g_i, delta_i), TILES tiles of (delta_bar, v), then W x TILES tiles of (m_i, x_i).
+// The received gradient g_bar and the denominators sqrt(v + eps) stay in registers
+// between the server part and the update of the W workers' momentum and model.
+// ---------------------------------------------------------------------------
+constexpr int kStage2Bytes = 2 * kTileBytes;
+
+template <int TILES>
+__global__ void __launch_bounds__(kThreads, 1) alg2_pipelined_kernel(const __grid_constant__ PipeArgs a)
+{
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    PipeShared *sh = reinterpret_cast<PipeShared *>(smem_raw);
+    const StateView &st = a.st;
+    const int W = st.W;
+    const int words_per_chunk = st.chunk >> 5;
+    uint32_t *bits_s = reinterpret_cast<uint32_t *>(smem_raw + 1024);
+    float *scales_s = reinterpret_cast<float *>(bits_s + W * words_per_chunk);
+    unsigned char *ring = smem_raw + ((1024 + (size_t)W * words_per_chunk * 4 + (size_t)kConsumerWarps * W * 4 + 1023) & ~(size_t)1023);
+    const int R = a.stages;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    volatile int *abort_flag = &sh->abort;
+
+    if (tid == 0) {
+        for (int s = 0; s < R; ++s) {
+            mbar_init(smem_addr(&sh->full[s]), 1);
+            mbar_init(smem_addr(&sh->empty[s]), kConsumerWarps);
+        }
+        sh->abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+
+    if (warp == kConsumerWarps) {
+        // ------------------------------ producer ------------------------------
+        if (lane != 0) return;
+        int s = 0;
+        uint32_t phase = 0;
+        long long issued = 0;
+        bool ok = true;
+        const uint32_t g_elem = (a.grad_fmt & kGradTypeMask) == kGradF32 ? 4u : 2u;
+        for (long long k = 0; ok; ++k) {
+            const long long chunk = (long long)atomicAdd(&a.sched[0], 1ull);
+            const bool last = chunk >= a.n_full_chunks;
+            if (!mbar_wait(smem_addr(&sh->empty[s]), phase ^ 1u, abort_flag, a.error_flag, a.wait_limit_ns)) { ok = false; break; }
+            sh->chunk_queue[k % (kMaxStages + 2)] = last ? -1 : chunk;
+            if (last) {
+                mbar_arrive(smem_addr(&sh->full[s]));
+                break;
+            }
+            const long long c0 = chunk * st.chunk;
+            for (int i = 0; ok && i <= 2 * W; ++i) {        // i < W: (g, delta); i == W: (delta_bar, v); i > W: (m, x)
+                for (int t = 0; t < TILES; ++t) {
+                    const uint32_t full = smem_addr(&sh->full[s]);
+                    if (!mbar_wait(smem_addr(&sh->empty[s]), phase ^ 1u, abort_flag, a.error_flag, a.wait_limit_ns)) { ok = false; break; }
+                    const uint32_t dst = smem_addr(ring + (size_t)s * kStage2Bytes);
+                    const long long off = c0 + (long long)t * kTile;
+                    if (i < W) {
+                        mbar_arrive_expect_tx(full, kTileBytes + kTile * g_elem);
+                        bulk_load(dst, reinterpret_cast<const char *>(a.g.p[i]) + off * g_elem, kTile * g_elem, full);
+                        bulk_load(dst + kTileBytes, st.dw + (long long)i * st.n_pad + off, kTileBytes, full);
+                    } else if (i == W) {
+                        mbar_arrive_expect_tx(full, 2 * kTileBytes);
+                        bulk_load(dst, st.ds + off, kTileBytes, full);
+                        bulk_load(dst + kTileBytes, st.v + off, kTileBytes, full);
+                    } else {
+                        const long long row = (long long)(i - W - 1) * st.n_pad + off;
+                        mbar_arrive_expect_tx(full, 2 * kTileBytes);
+                        bulk_load(dst, st.m + row, kTileBytes, full);
+                        bulk_load(dst + kTileBytes, st.x + row, kTileBytes, full);
+                    }
+                    ++issued;
+                    if (++s == R) { s = 0; phase ^= 1u; }
+                    if (a.test_stop_after_tiles > 0 && issued >= a.test_stop_after_tiles) { ok = false; break; }
+                }
+            }
+        }
+        if (!ok) {
+            const long long outstanding = issued < R ? issued : R;
+            for (long long k = 1; k <= outstanding; ++k) {
+                const long long q = issued - k;
+                const uint32_t bar = smem_addr(&sh->full[q % R]);
+                const uint32_t par = (uint32_t)((q / R) & 1);
+                const unsigned long long start = global_timer_ns();
+                while (!mbar_try_wait(bar, par) && global_timer_ns() - start < a.wait_limit_ns) {}
+            }
+        }
+        if (atomicAdd(&a.sched[1], 1ull) == gridDim.x - 1) {
+            a.sched[0] = 0;
+            a.sched[1] = 0;
+        }
+        return;
+    }
+
+    // -------------------------------- consumers --------------------------------
+    int s = 0;
+    uint32_t phase = 0;
+    int flip = 0;
+    const int pos = 4 * tid;
+    const int word_in_tile = pos >> 5;
+    const bool group_leader = (lane & 7) == 0;
+    float *my_scales = scales_s + warp * W;
+    const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
+
+    // Waits for the next stage, hands back its two slots, and releases it once the warp has read them.
+    auto next_tile = [&](float4 &slot0, float4 &slot1, bool slot0_is_grad) {
+        const bool ready = mbar_wait(smem_addr(&sh->full[s]), phase, abort_flag, a.error_flag, a.wait_limit_ns);
+        const float *stage = reinterpret_cast<const float *>(ring + (size_t)s * kStage2Bytes);
+        slot0 = zero4;
+        slot1 = zero4;
+        if (ready) {
+            if (slot0_is_grad && (a.grad_fmt & kGradTypeMask) != kGradF32)
+                slot0 = grad16x4_to_float4(*reinterpret_cast<const uint2 *>(reinterpret_cast<const unsigned short *>(stage) + pos), a.grad_fmt);
+            else
+                slot0 = ld4(stage + pos);
+            slot1 = ld4(stage + kTile + pos);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_addr(&sh->empty[s]));
+        if (++s == R) { s = 0; phase ^= 1u; }
+    };
+
+    for (long long k = 0;; ++k) {
+        const bool gave_up = !mbar_wait(smem_addr(&sh->full[s]), phase, abort_flag, a.error_flag, a.wait_limit_ns);
+        if (consumer_any(gave_up)) break;
+        const long long chunk = sh->chunk_queue[k % (kMaxStages + 2)];
+        if (chunk < 0) break;
+        const long long c0 = chunk * st.chunk;
+
+        // ---- workers: compress g + delta (Algorithm 3, worker side) ----
+        for (int i = 0; i < W; ++i) {
+            float z[TILES][4];
+            double l1 = 0.0;
+#pragma unroll
+            for (int t = 0; t < TILES; ++t) {
+                float4 g4, e4;
+                next_tile(g4, e4, true);
+                z[t][0] = f_add(g4.x, e4.x); z[t][1] = f_add(g4.y, e4.y);
+                z[t][2] = f_add(g4.z, e4.z); z[t][3] = f_add(g4.w, e4.w);
+                l1 += fabs((double)z[t][0]) + fabs((double)z[t][1]) + fabs((double)z[t][2]) + fabs((double)z[t][3]);
+            }
+            const float scale = chunk_scale(consumer_sum(l1, sh, flip), st.chunk);
+            const long long row = (long long)i * st.n_pad + c0;
+#pragma unroll
+            for (int t = 0; t < TILES; ++t) {
+                bool b[4];
+                float e[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    b[q] = z[t][q] >= 0.0f;
+                    e[q] = f_sub(z[t][q], b[q] ? scale : -scale);
+                }
+                st4_stream(st.dw + row + t * kTile + pos, make_float4(e[0], e[1], e[2], e[3]));
+                const uint32_t word = pack_group(b);
+                if (group_leader) {
+                    bits_s[i * words_per_chunk + t * (kTile / 32) + word_in_tile] = word;
+                    st.words_w[(long long)i * st.words_stride + ((c0 + t * kTile) >> 5) + word_in_tile] = word;
+                }
+            }
+            if (lane == 0) my_scales[i] = scale;
+            if (tid == 0) st.scales_w[(long long)i * st.n_chunks + chunk] = scale;
+        }
+        __syncwarp();
+
+        // ---- server: mean + server error, compress again; keep g_bar and the denominators ----
+        float gbar[TILES][4], dn[TILES][4];
+        double l1 = 0.0;
+#pragma unroll
+        for (int t = 0; t < TILES; ++t) {
+            float4 d4, v4;
+            next_tile(d4, v4, false);
+            const float dd[4] = {d4.x, d4.y, d4.z, d4.w}, vv[4] = {v4.x, v4.y, v4.z, v4.w};
+            double A[4] = {0.0, 0.0, 0.0, 0.0};
+            const int shift = (lane & 7) * 4;
+            for (int i = 0; i < W; ++i) {
+                const uint32_t nib = bits_s[i * words_per_chunk + t * (kTile / 32) + word_in_tile] >> shift;
+                const double sc = (double)my_scales[i];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) A[q] += ((nib >> q) & 1u) ? sc : -sc;
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                gbar[t][q] = server_input(A[q], W, dd[q]);       // the server's input for now
+                dn[t][q] = denom(a.c, vv[q]);
+                l1 += fabs((double)gbar[t][q]);
+            }
+        }
+        const float scale = chunk_scale(consumer_sum(l1, sh, flip), st.chunk);
+#pragma unroll
+        for (int t = 0; t < TILES; ++t) {
+            bool b[4];
+            float e[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                b[q] = gbar[t][q] >= 0.0f;
+                const float hat = b[q] ? scale : -scale;
+                e[q] = f_sub(gbar[t][q], hat);
+                gbar[t][q] = hat;                                // line 7: what every worker receives
+            }
+            const uint32_t word = pack_group(b);
+            if (group_leader) st.words_s[((c0 + t * kTile) >> 5) + word_in_tile] = word;
+            st4_stream(st.ds + c0 + t * kTile + pos, make_float4(e[0], e[1], e[2], e[3]));
+        }
+        if (tid == 0) st.scales_s[chunk] = scale;
+
+        // ---- every worker: momentum and model (lines 10-11) ----
+        for (int i = 0; i < W; ++i) {
+#pragma unroll
+            for (int t = 0; t < TILES; ++t) {
+                float4 m4, x4;
+                next_tile(m4, x4, false);
+                const float mm[4] = {m4.x, m4.y, m4.z, m4.w}, xx[4] = {x4.x, x4.y, x4.z, x4.w};
+                float mo[4], xo[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    mo[q] = momentum(a.c, mm[q], gbar[t][q]);
+                    xo[q] = f_sub(xx[q], f_div(f_mul(a.gamma, mo[q]), dn[t][q]));
+                }
+                const long long row = (long long)i * st.n_pad + c0 + t * kTile + pos;
+                st4_stream(st.m + row, make_float4(mo[0], mo[1], mo[2], mo[3]));
+                st4_stream(st.x + row, make_float4(xo[0], xo[1], xo[2], xo[3]));
+            }
+        }
+        __syncwarp();
+    }
+}
+
+// ---------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------
 static size_t pipeline_fixed_smem(int W, int chunk)
@@ -444,7 +673,7 @@ int pipeline_stages(const StateView &st, int grad_fmt)
     const size_t fixed = pipeline_fixed_smem(st.W, st.chunk);
     if (fixed + (size_t)(tiles + 1) * kStageBytes > budget) return 0;
     int stages = (int)((budget - fixed) / kStageBytes);
-    if (stages > kMaxStages) stages = kMaxStages;
+    if (stages > kSyncStages) stages = kSyncStages;
     return stages >= tiles + 1 ? stages : 0;
 }
 
@@ -489,6 +718,63 @@ cudaError_t launch_step_sync_pipelined(const StateView &st, const GradPtrs &g, c
     case 1: return do_var ? launch_pipe<1, true>(a, grid, smem, s) : launch_pipe<1, false>(a, grid, smem, s);
     case 2: return do_var ? launch_pipe<2, true>(a, grid, smem, s) : launch_pipe<2, false>(a, grid, smem, s);
     case 4: return do_var ? launch_pipe<4, true>(a, grid, smem, s) : launch_pipe<4, false>(a, grid, smem, s);
+    default: return cudaErrorInvalidValue;
+    }
+}
+
+}  // namespace zoa
+
+namespace zoa {
+
+int alg2_pipeline_stages(const StateView &st, int grad_fmt)
+{
+    if (!(grad_fmt & kGradAligned)) return 0;
+    if (st.chunk != kTile && st.chunk != 2 * kTile && st.chunk != 4 * kTile) return 0;
+    if (st.n / st.chunk < 1) return 0;
+    const size_t budget = 227 * 1024;
+    const size_t fixed = pipeline_fixed_smem(st.W, st.chunk);
+    if (fixed + 2 * (size_t)kStage2Bytes > budget) return 0;
+    int stages = (int)((budget - fixed) / kStage2Bytes);
+    return stages > kMaxStages ? kMaxStages : stages;
+}
+
+template <int TILES>
+static cudaError_t launch_alg2_pipe(const PipeArgs &a, int grid, size_t smem, cudaStream_t s)
+{
+    auto kern = alg2_pipelined_kernel<TILES>;
+    static bool configured[64] = {false};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64 || !configured[dev]) {
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) configured[dev] = true;
+    }
+    kern<<<grid, kThreads, smem, s>>>(a);
+    return cudaGetLastError();
+}
+
+// The full chunks of a compressed step of Algorithm 2; a ragged last chunk is the caller's.
+cudaError_t launch_alg2_pipelined(const StateView &st, const GradPtrs &g, const Consts &c, float gamma, int grad_fmt,
+                                  int stages, int sm_count, int *error_flag, unsigned long long *sched,
+                                  unsigned long long wait_limit_ns, long long test_stop_after_tiles, cudaStream_t s)
+{
+    PipeArgs a;
+    a.st = st; a.g = g; a.c = c; a.gamma = gamma; a.gamma_sum = 0.f;
+    a.n_full_chunks = st.n / st.chunk;
+    a.stages = stages;
+    a.error_flag = error_flag;
+    a.sched = sched;
+    a.grad_fmt = grad_fmt;
+    a.wait_limit_ns = wait_limit_ns;
+    a.test_stop_after_tiles = test_stop_after_tiles;
+    const int grid = (int)(a.n_full_chunks < sm_count ? a.n_full_chunks : sm_count);
+    const size_t smem = pipeline_fixed_smem(st.W, st.chunk) + (size_t)stages * kStage2Bytes;
+    switch (st.chunk / kTile) {
+    case 1: return launch_alg2_pipe<1>(a, grid, smem, s);
+    case 2: return launch_alg2_pipe<2>(a, grid, smem, s);
+    case 4: return launch_alg2_pipe<4>(a, grid, smem, s);
     default: return cudaErrorInvalidValue;
     }
 }

@@ -513,3 +513,34 @@ def test_create_destroy_returns_device_memory():
     torch.cuda.synchronize()
     free1, _ = torch.cuda.mem_get_info()
     assert free0 - free1 < 64 << 20, f"{(free0 - free1) >> 20} MiB did not come back"
+
+
+@pytest.mark.parametrize("W,chunk,n_chunks,tail,dtype", [(5, 4096, 301, 1852, torch.float32), (3, 2048, 700, 0, torch.float32),
+                                                         (4, 8192, 160, 704, torch.bfloat16), (16, 4096, 40, 5, torch.float16),
+                                                         (64, 2048, 20, 33, torch.float32)])
+def test_alg2_ring_kernel_equals_block_kernel(W, chunk, n_chunks, tail, dtype):
+    rng = np.random.default_rng(W + chunk)
+    n = n_chunks * chunk + tail
+    x0 = torch.from_numpy((rng.standard_normal(n) * 0.02).astype(np.float32))
+    a, b = Zoa(n, W, chunk=chunk), Zoa(n, W, chunk=chunk)
+    try:
+        b.set_pipeline(False)
+        for z in (a, b):
+            z.set_params(x0)
+            z.set_policies((0,), (0,), (1,))
+            z.set_grad_dtype(dtype)
+        g = torch.empty(W, n, device="cuda")
+        for t in range(4):
+            g.normal_(generator=torch.Generator("cuda").manual_seed(t + 5))
+            gg = list(g.to(dtype))
+            a.alg2_step(gg, 1e-3, t)
+            b.alg2_step(gg, 1e-3, t)
+            torch.cuda.synchronize()
+            a.check_device()
+            for name in ("x", "m", "delta_w", "words_w", "scales_w"):
+                for i in (0, W // 2, W - 1):
+                    assert np.array_equal(a.read(name, i), b.read(name, i)), (name, i, t)
+            for name in ("v", "delta_s", "words_s", "scales_s"):
+                assert np.array_equal(a.read(name), b.read(name)), (name, t)
+    finally:
+        a.close(), b.close()
