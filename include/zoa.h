@@ -198,10 +198,11 @@ zoa_status zoa_get_stats(zoa_handle h, zoa_stats *out);
  * of this handle failed since the last check. */
 zoa_status zoa_check_device(zoa_handle h);
 
-/* Tuning switches.  ZOA_OPT_PIPELINE (default 1): run the fused sync step as the
- * persistent bulk-copy-ring kernel where the shape allows (chunk 2048, 4096 or
- * 8192, 16-byte aligned gradients); 0 forces the chunk-per-block kernel.  The
- * results are the same bit for bit.
+/* Tuning switches.  ZOA_OPT_PIPELINE (default 1): run the fused sync step and the
+ * compressed step of Algorithm 2 as the persistent bulk-copy-ring kernels where
+ * the shape allows (chunk 2048, 4096 or 8192, 16-byte aligned gradients) and the
+ * problem has at least four chunks per SM; 2: wherever the shape allows; 0: always
+ * the chunk-per-block kernels.  The results are the same bit for bit.
  * ZOA_OPT_WAIT_LIMIT_MS (default 2000): how long a kernel thread waits for an
  * asynchronous copy before it gives up; the kernel then ends early, the state is
  * undefined and zoa_check_device reports ZOA_ERR_DEVICE.

@@ -28,7 +28,7 @@ struct zoa_handle_s {
     double *partials = nullptr;    // device [W + 1][n_chunks * segments]: per-segment l1 sums, chunk > 16384 only
     bool large_chunk = false;
     int grad_type = 0;             // 0 binary32, 1 binary16, 2 bfloat16: how `grads` buffers are read
-    bool use_pipeline = true;      // bulk-copy ring form of the fused sync step where the shape allows
+    int use_pipeline = 1;          // ring kernels: 0 never, 1 where the shape allows and the problem is large enough, 2 wherever the shape allows
     int wait_limit_ms = 2000;      // bound on every device-side wait
     long long test_stop_after_tiles = 0;   // error-path test hook, see zoa_set_option
     bool v_pending = false;        // v_nxt holds v_{t+1}; it becomes v at the next step
@@ -421,7 +421,7 @@ extern "C" zoa_status zoa_step_sync(zoa_handle h, const void *const *grads, floa
     }
     // The persistent kernel pays off once every SM has a few chunks to stream; below that the
     // one-block-per-chunk kernel starts faster (measured on the 512-chunk configuration).
-    const bool enough_chunks = h->n / h->chunk >= 4ll * h->sm_count;
+    const bool enough_chunks = h->use_pipeline == 2 || h->n / h->chunk >= 4ll * h->sm_count;
     const int stages = h->use_pipeline && enough_chunks ? pipeline_stages(st, aligned) : 0;
     long long var_first = 0;     // coordinates from here on still need lines 14-15
     if (stages > 0) {
@@ -474,7 +474,7 @@ extern "C" zoa_status zoa_alg2_step(zoa_handle h, const void *const *grads, floa
     } else {
         cudaStream_t s = static_cast<cudaStream_t>(stream);
         const StateView st = view(h);
-        const bool enough_chunks = h->n / h->chunk >= 4ll * h->sm_count;
+        const bool enough_chunks = h->use_pipeline == 2 || h->n / h->chunk >= 4ll * h->sm_count;
         const int stages = (!full && h->use_pipeline && enough_chunks) ? alg2_pipeline_stages(st, aligned) : 0;
         long long first = 0;
         if (stages > 0) {   // full chunks through the bulk-copy ring, a ragged last chunk through the block kernel
@@ -631,7 +631,10 @@ extern "C" zoa_status zoa_set_option(zoa_handle h, int option, int value)
 {
     if (!h) return ZOA_ERR_ARG;
     switch (option) {
-    case ZOA_OPT_PIPELINE: h->use_pipeline = value != 0; return ZOA_OK;
+    case ZOA_OPT_PIPELINE:
+        if (value < 0 || value > 2) return fail(h, ZOA_ERR_ARG, "zoa_set_option: ZOA_OPT_PIPELINE takes 0, 1 or 2");
+        h->use_pipeline = value;
+        return ZOA_OK;
     case ZOA_OPT_GRAD_TYPE:
         if (value < ZOA_GRAD_F32 || value > ZOA_GRAD_BF16) return fail(h, ZOA_ERR_ARG, "zoa_set_option: unknown gradient type");
         h->grad_type = value;

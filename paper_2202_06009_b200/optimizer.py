@@ -67,9 +67,10 @@ class Zoa:
         B.zoa_set_var_steps(self.h, list(var_steps))
         B.zoa_set_sync_policy(self.h, list(sync_boundaries), list(sync_intervals))
 
-    def set_pipeline(self, on):
-        """Fused sync step through the bulk-copy ring kernel (default) or the chunk-per-block one."""
-        B.zoa_set_option(self.h, B.OPT_PIPELINE, int(bool(on)))
+    def set_pipeline(self, mode):
+        """Ring kernels: False = never, True = where shape and problem size allow (default),
+        "force" = wherever the shape allows."""
+        B.zoa_set_option(self.h, B.OPT_PIPELINE, 2 if mode == "force" else int(bool(mode)))
 
     def set_grad_dtype(self, dtype):
         """Gradients arrive as torch.float32 (default), torch.float16 or torch.bfloat16."""

@@ -28,6 +28,7 @@ class Pair:
     def __init__(self, n, W, chunk, beta1=0.9, beta2=0.999, eps=1e-8, var_steps=(), sync=((0,), (1,)), x0=None):
         self.n, self.W, self.chunk = n, W, chunk
         self.gpu = Zoa(n, W, beta1, beta2, eps, chunk)
+        self.gpu.set_pipeline("force")          # small test problems still go through the ring kernels
         self.gpu.set_policies(var_steps, sync[0], sync[1])
         self.cpu = zo.Oracle(n, W, chunk, beta1, beta2, eps, dtype=np.float32)
         if x0 is not None:

@@ -90,6 +90,7 @@ def test_pipelined_kernel_equals_chunk_per_block_kernel(W, chunk, n_chunks, tail
     x0 = torch.from_numpy((rng.standard_normal(n) * 0.02).astype(np.float32))
     a, b = Zoa(n, W, chunk=chunk), Zoa(n, W, chunk=chunk)
     try:
+        a.set_pipeline("force")
         b.set_pipeline(False)
         for z in (a, b):
             z.set_params(x0)
@@ -343,6 +344,7 @@ def test_device_wait_runs_out_and_is_reported():
     z = Zoa(n, W, chunk=chunk)
     try:
         g = list(torch.randn(W, n, device="cuda"))
+        z.set_pipeline("force")
         z.step_sync(g, 1e-3, 0)
         z.check_device()                                  # the normal path works
         B.zoa_set_option(z.h, B.OPT_WAIT_LIMIT_MS, 100)
@@ -524,6 +526,7 @@ def test_alg2_ring_kernel_equals_block_kernel(W, chunk, n_chunks, tail, dtype):
     x0 = torch.from_numpy((rng.standard_normal(n) * 0.02).astype(np.float32))
     a, b = Zoa(n, W, chunk=chunk), Zoa(n, W, chunk=chunk)
     try:
+        a.set_pipeline("force")
         b.set_pipeline(False)
         for z in (a, b):
             z.set_params(x0)
