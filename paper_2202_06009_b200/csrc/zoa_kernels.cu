@@ -750,8 +750,8 @@ cudaError_t launch_compress(const StateView &st, cudaStream_t s)
 {
     const dim3 grid((unsigned)st.n_chunks, (unsigned)st.W);
     // 16 coordinates per thread here (measured: 256-thread blocks move chunk 4096 at 6.7 TB/s, 512-thread ones at 6.0)
-    int thr = block_threads_for_chunk(st.chunk) / 2;
-    if (thr < 128) thr = 128;
+    int thr = 128;
+    while (thr < st.chunk / 16 && thr < 512) thr <<= 1;
     compress_kernel<<<grid, thr, compress_smem(st.chunk), s>>>(st);
     return cudaGetLastError();
 }
