@@ -146,6 +146,34 @@ zoa_status zoa_onebit_reduce(zoa_handle h, void *stream);
 zoa_status zoa_onebit_compress(zoa_handle h, void *stream);
 zoa_status zoa_onebit_average(zoa_handle h, void *stream);
 
+/* Building blocks for the paper's own mapping, one worker per GPU (Algorithm 3:
+ * every worker sends its packed buffer to the server, the server sends its
+ * packed result to every worker).  Each GPU holds a handle for its own
+ * worker(s) and is the server for a contiguous range of chunks; the
+ * collectives run between these calls (paper_2202_06009_b200/distributed.py
+ * drives them with torch.distributed):
+ *   zoa_step, zoa_onebit_compress          local step, pack u + delta (words_w, scales_w)
+ *   -- all-to-all of each range's words and scales --
+ *   zoa_dist_server_range                  server side for this GPU's chunk range
+ *   -- all-gather of words_s / scales_s into every handle's own buffers --
+ *   zoa_dist_apply                         lines 8-11 of Algorithm 1 from words_s / scales_s
+ * zoa_dist_server_range: words_all / scales_all (device) hold, for each of the
+ * W_total workers in worker order, the packed words and the magnitudes of the
+ * chunks [first_chunk, first_chunk + n_chunks), rows words_stride / scales_stride
+ * elements apart, starting at the range's first word / chunk.  It updates the
+ * server error of that range and writes that range of words_s / scales_s.
+ * Chunks above 16384 are not supported here.
+ * zoa_dist_variance: lines 14-15 of Algorithm 1 when the mean gradient g_bar
+ * (device, n_params floats) comes from a collective; call it after zoa_step on a
+ * step in T_v for which the handle's own T_v list is empty.  A collective's
+ * binary32 sum is not the binary64 worker-order sum of the single-GPU path, so v
+ * (and through it x) can differ from it in the last bits. */
+zoa_status zoa_dist_server_range(zoa_handle h, const uint32_t *words_all, size_t words_stride,
+                                 const float *scales_all, size_t scales_stride, int W_total,
+                                 int64_t first_chunk, int64_t n_chunks, void *stream);
+zoa_status zoa_dist_apply(zoa_handle h, void *stream);
+zoa_status zoa_dist_variance(zoa_handle h, const float *g_bar, void *stream);
+
 /* zoa_step followed by zoa_onebit_reduce, same results bit for bit, in one
  * pass over memory that never writes the half-step values. */
 zoa_status zoa_step_sync(zoa_handle h, const void *const *grads, float lr, int64_t t,

@@ -51,6 +51,9 @@ def _load():
         "zoa_onebit_reduce": ([H, p], C.c_int),
         "zoa_onebit_compress": ([H, p], C.c_int),
         "zoa_onebit_average": ([H, p], C.c_int),
+        "zoa_dist_server_range": ([H, p, C.c_size_t, p, C.c_size_t, C.c_int, C.c_int64, C.c_int64, p], C.c_int),
+        "zoa_dist_apply": ([H, p], C.c_int),
+        "zoa_dist_variance": ([H, p, p], C.c_int),
         "zoa_step_sync": ([H, C.POINTER(p), C.c_float, C.c_int64, p], C.c_int),
         "zoa_step_auto": ([H, C.POINTER(p), C.c_float, C.c_int64, p], C.c_int),
         "zoa_alg2_step": ([H, C.POINTER(p), C.c_float, C.c_int64, p], C.c_int),
@@ -155,6 +158,19 @@ def zoa_onebit_compress(h, stream=0):
 
 def zoa_onebit_average(h, stream=0):
     _check(h, lib.zoa_onebit_average(h, stream))
+
+
+def zoa_dist_server_range(h, words_ptr, words_stride, scales_ptr, scales_stride, W_total, first_chunk, n_chunks, stream=0):
+    _check(h, lib.zoa_dist_server_range(h, words_ptr, words_stride, scales_ptr, scales_stride, W_total,
+                                        first_chunk, n_chunks, stream))
+
+
+def zoa_dist_apply(h, stream=0):
+    _check(h, lib.zoa_dist_apply(h, stream))
+
+
+def zoa_dist_variance(h, g_bar_ptr, stream=0):
+    _check(h, lib.zoa_dist_variance(h, g_bar_ptr, stream))
 
 
 def zoa_step_sync(h, grad_ptrs, lr, t, stream=0):

@@ -391,6 +391,54 @@ extern "C" zoa_status zoa_onebit_average(zoa_handle h, void *stream)
     return ZOA_OK;
 }
 
+// ---- one worker per GPU: the pieces between the collectives ------------------------------------
+
+extern "C" zoa_status zoa_dist_server_range(zoa_handle h, const uint32_t *words_all, size_t words_stride,
+                                            const float *scales_all, size_t scales_stride, int W_total,
+                                            int64_t first_chunk, int64_t n_chunks, void *stream)
+{
+    if (!h) return ZOA_ERR_ARG;
+    if (h->large_chunk) return fail(h, ZOA_ERR_ARG, "zoa_dist_server_range: chunk must be at most 16384");
+    if (W_total < 1 || W_total > kMaxWorkers) return fail(h, ZOA_ERR_ARG, "zoa_dist_server_range: W_total must be in [1, 64]");
+    if (first_chunk < 0 || n_chunks < 0 || first_chunk + n_chunks > h->n_chunks)
+        return fail(h, ZOA_ERR_ARG, "zoa_dist_server_range: chunk range outside the vector");
+    if (n_chunks == 0) return ZOA_OK;
+    if (!words_all || !scales_all) return fail(h, ZOA_ERR_ARG, "zoa_dist_server_range: NULL buffer");
+    if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, "zoa_dist_server_range: the handle's device is not the current CUDA device");
+    ZOA_CUDA(h, launch_dist_server(view(h), words_all, (long long)words_stride, scales_all, (long long)scales_stride,
+                                   W_total, first_chunk, n_chunks, static_cast<cudaStream_t>(stream)));
+    h->n_launches += 1;
+    return ZOA_OK;
+}
+
+extern "C" zoa_status zoa_dist_apply(zoa_handle h, void *stream)
+{
+    if (!h) return ZOA_ERR_ARG;
+    const float gamma_sum = (float)h->gamma_sum;
+    if (!(h->gamma_sum > 0.0) || !(gamma_sum > 0.f) || !std::isfinite(gamma_sum))
+        return fail(h, ZOA_ERR_STATE, "zoa_dist_apply: nothing accumulated since the last sync (sum of learning rates is not positive)");
+    if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, "zoa_dist_apply: the handle's device is not the current CUDA device");
+    ZOA_CUDA(h, launch_dist_apply(view(h), h->c, gamma_sum, static_cast<cudaStream_t>(stream)));
+    h->n_launches += 1;
+    h->gamma_sum = 0.0;
+    h->t_sync = h->t_last;
+    h->n_syncs += 1;
+    return ZOA_OK;
+}
+
+extern "C" zoa_status zoa_dist_variance(zoa_handle h, const float *g_bar, void *stream)
+{
+    if (!h) return ZOA_ERR_ARG;
+    if (!g_bar) return fail(h, ZOA_ERR_ARG, "zoa_dist_variance: g_bar is NULL");
+    if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, "zoa_dist_variance: the handle's device is not the current CUDA device");
+    if (h->v_pending) return fail(h, ZOA_ERR_STATE, "zoa_dist_variance: a variance update is already pending for this step");
+    ZOA_CUDA(h, launch_dist_variance(view(h), h->c, g_bar, static_cast<cudaStream_t>(stream)));
+    h->n_launches += 1;
+    h->v_pending = true;
+    h->n_var_updates += 1;
+    return ZOA_OK;
+}
+
 extern "C" zoa_status zoa_step_sync(zoa_handle h, const void *const *grads, float lr, int64_t t, void *stream)
 {
     GradPtrs gp;

@@ -33,6 +33,13 @@ cudaError_t launch_step_sync_pipelined(const StateView &st, const GradPtrs &g, c
                                        unsigned long long *sched, unsigned long long wait_limit_ns,
                                        long long test_stop_after_tiles, bool *var_fused, cudaStream_t s);
 
+// One worker per GPU: the kernels between the collectives.
+cudaError_t launch_dist_server(const StateView &st, const uint32_t *words_in, long long words_in_stride,
+                               const float *scales_in, long long scales_in_stride, int W_total,
+                               long long first_chunk, long long count, cudaStream_t s);
+cudaError_t launch_dist_apply(const StateView &st, const Consts &c, float gamma_sum, cudaStream_t s);
+cudaError_t launch_dist_variance(const StateView &st, const Consts &c, const float *g_bar, cudaStream_t s);
+
 int alg2_pipeline_stages(const StateView &st, int grad_fmt);
 cudaError_t launch_alg2_pipelined(const StateView &st, const GradPtrs &g, const Consts &c, float gamma, int grad_fmt,
                                   int stages, int sm_count, int *error_flag, unsigned long long *sched,

@@ -330,6 +330,110 @@ __global__ void step_sync_kernel(StateView st, GradPtrs g, Consts c, float gamma
 }
 
 // ---------------------------------------------------------------------------
+// One worker per GPU (the paper's own mapping: workers send packed buffers to the server
+// that owns a range of chunks, the server sends its packed result to every worker).
+// The collectives run between these two kernels; see distributed.py.
+// ---------------------------------------------------------------------------
+
+// Server side of Algorithm 3 alone for chunk first_chunk + blockIdx.x, reading packed buffers
+// gathered from W_total workers: words_in[w][range words], scales_in[w][range chunks], both
+// starting at the range's first chunk.  Writes the server error, words_s and scales_s.
+__global__ void dist_server_kernel(StateView st, const uint32_t *words_in, long long words_in_stride,
+                                   const float *scales_in, long long scales_in_stride, int W_total,
+                                   long long first_chunk)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    double *scratch = reinterpret_cast<double *>(smem_raw);
+    float *scales = reinterpret_cast<float *>(smem_raw + 34 * sizeof(double));
+    float *a_s = scales + kMaxWorkers;
+    const long long chunk_id = first_chunk + blockIdx.x;
+    const ChunkGeom cg = chunk_geom(st, chunk_id);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    const long long range_word0 = (first_chunk * st.chunk) >> 5;
+
+    for (int i = threadIdx.x; i < W_total; i += blockDim.x) scales[i] = scales_in[(long long)i * scales_in_stride + blockIdx.x];
+    __syncthreads();
+    double l1 = 0.0;
+    for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
+        const int idx = base + 4 * lane;
+        if (idx < cg.len) {
+            double A[4] = {0.0, 0.0, 0.0, 0.0};
+            const long long word_idx = ((cg.c0 + idx) >> 5) - range_word0;
+            const int shift = idx & 31;
+            for (int i = 0; i < W_total; ++i) {  // worker order
+                const uint32_t nib = words_in[(long long)i * words_in_stride + word_idx] >> shift;
+                const double sc = (double)scales[i];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) A[k] += ((nib >> k) & 1u) ? sc : -sc;
+            }
+            const float4 e4 = ld4(st.ds + cg.c0 + idx);
+            const float ee[4] = {e4.x, e4.y, e4.z, e4.w};
+            float a[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                a[k] = idx + k < cg.len ? server_input(A[k], W_total, ee[k]) : 0.0f;
+                l1 += fabs((double)a[k]);
+            }
+            st4(a_s + idx, make_float4(a[0], a[1], a[2], a[3]));
+        }
+    }
+    const float scale = chunk_scale(block_sum(l1, scratch), cg.len);
+    for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
+        const int idx = base + 4 * lane;
+        float a[4] = {0.f, 0.f, 0.f, 0.f}, hat[4];
+        if (idx < cg.len) {
+            const float4 a4 = ld4(a_s + idx);
+            a[0] = a4.x; a[1] = a4.y; a[2] = a4.z; a[3] = a4.w;
+        }
+        const uint32_t word = compress_tile(a, hat, scale, idx, cg.len);
+        if (lane < 4 && base + 32 * lane < cg.len) st.words_s[((cg.c0 + base) >> 5) + lane] = word;
+        if (idx < cg.len) st4(st.ds + cg.c0 + idx, make_float4(a[0], a[1], a[2], a[3]));
+    }
+    if (threadIdx.x == 0) st.scales_s[chunk_id] = scale;
+}
+
+// Lines 8-10 of Algorithm 1 from the server's packed result (words_s, scales_s of the whole
+// vector): m = u_bar / sum(gamma), x = x_sync - u_bar / sqrt(v + eps), u = 0, on this GPU's workers.
+__global__ void __launch_bounds__(256)
+dist_apply_kernel(StateView st, Consts c, float gamma_sum)
+{
+    const long long n4 = (st.n + 3) >> 2;
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x; q < n4; q += stride) {
+        const long long j = q << 2;
+        const uint32_t nib = st.words_s[j >> 5] >> (j & 31);
+        const float scale = st.scales_s[j / st.chunk];
+        const float4 v4 = ld4(st.v + j), xs4 = ld4(st.xs + j);
+        const float vv[4] = {v4.x, v4.y, v4.z, v4.w}, xs[4] = {xs4.x, xs4.y, xs4.z, xs4.w};
+        float mo[4], xo[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const bool valid = j + k < st.n;
+            const float hat = ((nib >> k) & 1u) ? scale : -scale;
+            mo[k] = valid ? f_div(hat, gamma_sum) : 0.0f;                       // line 8
+            xo[k] = valid ? f_sub(xs[k], f_div(hat, denom(c, vv[k]))) : 0.0f;   // line 9
+        }
+        const float4 m4 = make_float4(mo[0], mo[1], mo[2], mo[3]), x4 = make_float4(xo[0], xo[1], xo[2], xo[3]);
+        st4(st.xs + j, x4);
+        for (int i = 0; i < st.W; ++i) {
+            const long long row = (long long)i * st.n_pad + j;
+            st4(st.m + row, m4);
+            st4(st.x + row, x4);
+            st4(st.u + row, make_float4(0.f, 0.f, 0.f, 0.f));                   // line 10
+        }
+    }
+}
+
+// Lines 14-15 of Algorithm 1 when the mean gradient comes from a collective: v_{t+1} from g_bar.
+__global__ void __launch_bounds__(256)
+dist_variance_kernel(StateView st, Consts c, const float *g_bar)
+{
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long j = (long long)blockIdx.x * blockDim.x + threadIdx.x; j < st.n; j += stride)
+        st.v_next[j] = variance(c, st.v[j], g_bar[j]);
+}
+
+// ---------------------------------------------------------------------------
 // Algorithm 2: the frozen-variance framework that exchanges gradients instead of
 // accumulated updates (1-bit Adam when T_v is an initial run of steps).
 // ---------------------------------------------------------------------------
@@ -808,6 +912,40 @@ cudaError_t launch_large_server(const StateView &st, const Consts &c, int mode, 
     if (mode == 1) lc_server_apply_kernel<1><<<(unsigned)n_segs, 512, 0, s>>>(st, c, scalar, spc);
     else lc_server_apply_kernel<2><<<(unsigned)n_segs, 512, 0, s>>>(st, c, scalar, spc);
     *launches += 3;
+    return cudaGetLastError();
+}
+
+}  // namespace zoa
+
+namespace zoa {
+
+cudaError_t launch_dist_server(const StateView &st, const uint32_t *words_in, long long words_in_stride,
+                               const float *scales_in, long long scales_in_stride, int W_total,
+                               long long first_chunk, long long count, cudaStream_t s)
+{
+    static bool configured[64] = {false};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64 || !configured[dev]) {
+        e = cudaFuncSetAttribute(dist_server_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)reduce_smem(kMaxChunk));
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) configured[dev] = true;
+    }
+    dist_server_kernel<<<(unsigned)count, block_threads_for_chunk(st.chunk), reduce_smem(st.chunk), s>>>(
+        st, words_in, words_in_stride, scales_in, scales_in_stride, W_total, first_chunk);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_dist_apply(const StateView &st, const Consts &c, float gamma_sum, cudaStream_t s)
+{
+    dist_apply_kernel<<<elementwise_grid((st.n + 3) / 4), 256, 0, s>>>(st, c, gamma_sum);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_dist_variance(const StateView &st, const Consts &c, const float *g_bar, cudaStream_t s)
+{
+    dist_variance_kernel<<<elementwise_grid((st.n + 255) / 256 * 64), 256, 0, s>>>(st, c, g_bar);
     return cudaGetLastError();
 }
 

@@ -1,0 +1,58 @@
+"""The exchange of the one-worker-per-GPU mapping on CPU: three gloo ranks send each chunk
+range's packed words and magnitudes to the rank that serves it (all-to-all) and spread the
+servers' results back (all-gather); every word must land where the plan says."""
+import os
+import sys
+
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _worker(rank, world, port, n, chunk, out_dir):
+    sys.path.insert(0, ROOT)
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from paper_2202_06009_b200.distributed import ExchangePlan, exchange_packed, gather_server
+    plan = ExchangePlan.make(n, chunk, world)
+    n_words, n_chunks = (n + 31) // 32, -(-n // chunk)
+    # cover: ranges tile the vector, word ranges follow the chunk ranges
+    assert plan.chunks[0].start == 0 and plan.chunks[-1].stop == n_chunks
+    assert all(a.stop == b.start for a, b in zip(plan.chunks, plan.chunks[1:]))
+    assert all(a.stop == b.start for a, b in zip(plan.words, plan.words[1:])) and plan.words[-1].stop == n_words
+    assert all(w.start == c.start * chunk // 32 for w, c in zip(plan.words, plan.chunks))
+    # worker -> server: word k of worker r carries (r, k)
+    words = torch.arange(n_words, dtype=torch.int32) + rank * 1_000_000
+    scales = torch.arange(n_chunks, dtype=torch.float32) + rank * 1000.0
+    recv_words, recv_scales = exchange_packed(plan, rank, words, scales)
+    mine_w, mine_c = plan.words[rank], plan.chunks[rank]
+    for w in range(world):
+        assert torch.equal(recv_words[w], torch.arange(mine_w.start, mine_w.stop, dtype=torch.int32) + w * 1_000_000)
+        assert torch.equal(recv_scales[w], torch.arange(mine_c.start, mine_c.stop, dtype=torch.float32) + w * 1000.0)
+    # server -> workers: each server's range carries its rank
+    words_s = torch.full((n_words,), -1, dtype=torch.int32)
+    scales_s = torch.full((n_chunks,), -1.0)
+    words_s[mine_w.start:mine_w.stop] = rank
+    scales_s[mine_c.start:mine_c.stop] = float(rank)
+    gather_server(plan, rank, words_s, scales_s)
+    for r in range(world):
+        assert (words_s[plan.words[r].start:plan.words[r].stop] == r).all()
+        assert (scales_s[plan.chunks[r].start:plan.chunks[r].stop] == float(r)).all()
+    dist.barrier()
+    if rank == 0:
+        open(os.path.join(out_dir, "ok"), "w").write("ok")
+    dist.destroy_process_group()
+
+
+def test_packed_exchange_three_ranks(tmp_path):
+    port = 29700 + os.getpid() % 2000
+    mp.spawn(_worker, args=(3, port, 10 * 256 + 77, 256, str(tmp_path)), nprocs=3, join=True)
+    assert (tmp_path / "ok").exists()
+
+
+def test_packed_exchange_more_ranks_than_chunks(tmp_path):
+    port = 31700 + os.getpid() % 2000
+    mp.spawn(_worker, args=(4, port, 3 * 64 + 5, 64, str(tmp_path)), nprocs=4, join=True)
+    assert (tmp_path / "ok").exists()

@@ -1,0 +1,102 @@
+"""One worker per GPU, checked on one GPU: the ranks are emulated as separate handles in one
+process (each with a single worker and its own server range), the collectives by plain copies
+between their buffers; the result must equal the single handle that holds all W workers, bit
+for bit.  A second test runs the real driver, collectives included, as a one-rank NCCL job."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2202_06009_b200 import Zoa
+from paper_2202_06009_b200.distributed import WorkerPerGpu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("W,chunk,n", [(3, 1024, 7 * 1024 + 100), (4, 4096, 9 * 4096), (5, 256, 3 * 256 + 7), (2, 2048, 2048 * 5 + 33)])
+def test_emulated_ranks_equal_the_single_handle(W, chunk, n):
+    rng = np.random.default_rng(W * n)
+    var_steps, sync = (0, 1, 3), ((0, 3), (1, 2))
+    x0 = torch.from_numpy((rng.standard_normal(n) * 0.02).astype(np.float32))
+    ref = Zoa(n, W, chunk=chunk)
+    ranks = [WorkerPerGpu(n, chunk, r, W, var_steps, *sync) for r in range(W)]
+    try:
+        ref.set_params(x0)
+        ref.set_policies(var_steps, *sync)
+        for w in ranks:
+            w.opt.set_params(x0)
+        for t in range(7):
+            g = torch.from_numpy(rng.standard_normal((W, n)).astype(np.float32)).cuda()
+            ref.step_auto(list(g), 1e-3, t)
+            for r, w in enumerate(ranks):
+                w.opt.step([g[r]], 1e-3, t)
+            if t in var_steps:                       # stands in for the all-reduce: the same worker-order binary64 mean
+                acc = g[0].double()
+                for i in range(1, W):
+                    acc = acc + g[i].double()
+                g_bar = (acc / W).float()
+                for w in ranks:
+                    w.variance(g_bar)
+            if ref.sync_due(t):
+                packs = [w.pack() for w in ranks]
+                torch.cuda.synchronize()
+                served = []
+                for r, w in enumerate(ranks):        # stands in for the all-to-all
+                    wr, cr = w.plan.words[r], w.plan.chunks[r]
+                    recv_words = torch.stack([p[0][wr.start:wr.stop] for p in packs]).contiguous()
+                    recv_scales = torch.stack([p[1][cr.start:cr.stop] for p in packs]).contiguous()
+                    served.append(w.serve(recv_words, recv_scales))
+                torch.cuda.synchronize()
+                for r, w in enumerate(ranks):        # stands in for the all-gather
+                    wr, cr = w.plan.words[r], w.plan.chunks[r]
+                    for q, other in enumerate(ranks):
+                        if q != r:
+                            served[q][0][wr.start:wr.stop] = served[r][0][wr.start:wr.stop]
+                            served[q][1][cr.start:cr.stop] = served[r][1][cr.start:cr.stop]
+                for w in ranks:
+                    w.apply()
+            torch.cuda.synchronize()
+            for r, w in enumerate(ranks):
+                for name in ("x", "m", "u", "delta_w"):
+                    assert np.array_equal(w.opt.read(name, 0), ref.read(name, r)), (name, r, t)
+                assert np.array_equal(w.opt.read("v"), ref.read("v")), ("v", r, t)
+                assert np.array_equal(w.opt.read("x_sync"), ref.read("x_sync")), ("x_sync", r, t)
+                cr = w.plan.chunks[r]
+                lo, hi = cr.start * chunk, min(cr.stop * chunk, n)
+                if hi > lo:
+                    assert np.array_equal(w.opt.read("delta_s", 0, lo, hi - lo), ref.read("delta_s", 0, lo, hi - lo)), ("delta_s", r, t)
+                if ref.sync_due(t):
+                    assert np.array_equal(w.opt.read("words_s"), ref.read("words_s")), ("words_s", r, t)
+                    assert np.array_equal(w.opt.read("scales_s"), ref.read("scales_s")), ("scales_s", r, t)
+    finally:
+        ref.close()
+        for w in ranks:
+            w.close()
+
+
+def test_driver_with_real_collectives_one_rank():
+    """world_size 1 over NCCL: every collective of WorkerPerGpu.step runs for real; W = 1 must
+    equal the plain single-worker handle."""
+    import torch.distributed as dist
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    os.environ.setdefault("MASTER_PORT", str(29900 + os.getpid() % 1000))
+    dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", 0))
+    rng = np.random.default_rng(3)
+    n, chunk = 6 * 1024 + 50, 1024
+    ref = Zoa(n, 1, chunk=chunk)
+    w = WorkerPerGpu(n, chunk, 0, 1, var_steps=(0, 2), sync_boundaries=(0, 2), sync_intervals=(1, 2))
+    try:
+        ref.set_policies((0, 2), (0, 2), (1, 2))
+        for t in range(5):
+            g = torch.from_numpy(rng.standard_normal((1, n)).astype(np.float32)).cuda()
+            ref.step_auto(list(g), 1e-3, t)
+            w.step(g[0], 1e-3, t)
+            torch.cuda.synchronize()
+            for name in ("x", "m", "u", "delta_w"):
+                assert np.array_equal(w.opt.read(name, 0), ref.read(name, 0)), (name, t)
+            assert np.array_equal(w.opt.read("v"), ref.read("v")) and np.array_equal(w.opt.read("delta_s"), ref.read("delta_s"))
+    finally:
+        ref.close()
+        w.close()
+        dist.destroy_process_group()
