@@ -13,9 +13,10 @@ FLOAT_STATES = ("x", "m", "u", "delta_w")
 def assert_close(got, want, what):
     got, want = np.asarray(got, np.float64), np.asarray(want, np.float64)
     assert got.shape == want.shape, what
-    both_nan = np.isnan(got) & np.isnan(want)
-    err = np.abs(got - want)
-    bad = ~(err <= ATOL + RTOL * np.abs(want)) & ~both_nan
+    same = (np.isnan(got) & np.isnan(want)) | (got == want)      # NaN with NaN, equal infinities
+    with np.errstate(invalid="ignore"):
+        err = np.abs(got - want)
+        bad = ~(err <= ATOL + RTOL * np.abs(want)) & ~same
     if bad.any():
         k = int(np.argmax(np.where(bad, err, 0)))
         raise AssertionError(f"{what}: {int(bad.sum())} of {got.size} outside tolerance; worst at {k}: "

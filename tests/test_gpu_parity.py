@@ -547,3 +547,55 @@ def test_alg2_ring_kernel_equals_block_kernel(W, chunk, n_chunks, tail, dtype):
                 assert np.array_equal(a.read(name), b.read(name)), (name, t)
     finally:
         a.close(), b.close()
+
+
+@pytest.mark.parametrize("mode", ["fused", "two_call"])
+def test_nonfinite_gradients_propagate_like_the_oracle(mode):
+    """NaN and infinities do not trap or hang: the affected chunks turn NaN on both sides in the
+    same places, the others stay exact."""
+    rng = np.random.default_rng(13)
+    W, chunk, n = 3, 2048, 5 * 2048 + 9
+    p = Pair(n, W, chunk, var_steps=(0,), x0=rng.standard_normal(n) * 0.02)
+    try:
+        for t in range(3):
+            g = _grads(rng, W, n)
+            if t == 1:
+                g[0, 5] = np.nan                # chunk 0 of worker 0
+                g[1, 2 * 2048 + 7] = np.inf     # chunk 2 of worker 1
+                g[2, n - 1] = -np.inf           # the ragged last chunk
+            with np.errstate(invalid="ignore", over="ignore"):
+                p.step(g, 1e-3, t, mode)
+            p.compare(f"t={t}", wire=False)
+            for i in range(W):
+                assert np.array_equal(p.gpu.read("words_w", i), p.cpu.words_worker[i]), (t, i)
+        assert np.isnan(p.gpu.read("delta_w", 0)[:2048]).all()
+        assert np.isfinite(p.gpu.read("x", 0)[2048:2 * 2048]).all()      # an untouched chunk
+    finally:
+        p.close()
+
+
+def test_zero_learning_rate_steps():
+    rng = np.random.default_rng(14)
+    W, chunk, n = 2, 1024, 3000
+    p = Pair(n, W, chunk, var_steps=(0,), sync=((0,), (3,)), x0=rng.standard_normal(n) * 0.02)
+    try:
+        for t, lr in enumerate([1e-3, 0.0, 0.0, 2e-3, 0.0, 1e-3, 1e-3]):
+            p.step(_grads(rng, W, n), lr, t, "fused")
+            p.compare(f"t={t}", wire=False)
+    finally:
+        p.close()
+
+
+@pytest.mark.parametrize("W,chunk,n_chunks", [(64, 8192, 3), (64, 4096, 5), (48, 8192, 4)])
+def test_many_workers_ring_or_fallback(W, chunk, n_chunks):
+    """W = 64 with chunk 8192 does not leave room for the ring in shared memory and takes the
+    block kernel; chunk 4096 does fit.  Either way the oracle decides."""
+    rng = np.random.default_rng(W + chunk)
+    n = n_chunks * chunk + 100
+    p = Pair(n, W, chunk, var_steps=(0,), x0=rng.standard_normal(n) * 0.02)
+    try:
+        for t in range(2):
+            p.step(_grads(rng, W, n), 1e-3, t, "fused")
+            p.compare(f"t={t}")
+    finally:
+        p.close()

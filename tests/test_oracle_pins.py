@@ -435,3 +435,27 @@ def test_alg2_one_bit_adam_special_case():
             assert np.array_equal(o.x[i], o.x[0]) and np.array_equal(o.m[i], o.m[0])
     np.testing.assert_allclose(received, g[T0:].mean(axis=1).sum(axis=0) - (o.delta.mean(axis=0) + o.delta_bar),
                                rtol=0, atol=1e-11)
+
+
+def test_alg1_minimises_a_noisy_quadratic():
+    """Sanity of signs and scales end to end: on f(x) = |x|^2 / 2 with noisy gradients, 0/1 Adam
+    with 1-bit syncs and local steps drives the loss down about as far as Adam does (the paper's
+    claim is the same convergence rate as Adam)."""
+    rng = np.random.default_rng(41)
+    n, d, T = 4, 512, 400
+    x0 = rng.standard_normal(d)
+
+    def run(compressor, sync_every, var_until):
+        # eps = 1 keeps the very first steps, which divide by sqrt(v_0 + eps) with v_0 = 0, well scaled
+        o = zo.Oracle(d, n, 128, eps=1.0, dtype=np.float64, compressor=compressor)
+        o.set_params(x0)
+        for t in range(T):
+            g = o.x + 0.3 * rng.standard_normal((n, d))        # gradient of |x|^2/2 at each worker's model, plus noise
+            o.step(g, 0.02, t, t % sync_every == 0, t < var_until)
+        return 0.5 * float((o.x.mean(axis=0) ** 2).sum())
+
+    f0 = 0.5 * float((x0 ** 2).sum())
+    adam = run(zo.IDENTITY, 1, T)
+    zero_one = run(zo.ONEBIT, 4, 100)
+    assert adam < 0.02 * f0
+    assert zero_one < 0.05 * f0
