@@ -599,3 +599,15 @@ def test_many_workers_ring_or_fallback(W, chunk, n_chunks):
             p.compare(f"t={t}")
     finally:
         p.close()
+
+
+def test_allocation_failure_is_reported_and_leaves_the_context_usable():
+    with pytest.raises(ZoaError) as e:
+        Zoa(1 << 36, 64, chunk=4096)                  # 70 TB of state
+    assert e.value.status == B.ERR_ALLOC
+    z = Zoa(4096, 2, chunk=1024)                      # the device still works
+    try:
+        z.step_sync(list(torch.ones(2, 4096, device="cuda")), 1e-3, 0)
+        z.check_device()
+    finally:
+        z.close()
