@@ -222,8 +222,10 @@ zoa_status zoa_set_scalars(zoa_handle h, double gamma_sum, int64_t t_sync, int64
 
 zoa_status zoa_get_stats(zoa_handle h, zoa_stats *out);
 
-/* Waits for the device and reports ZOA_ERR_DEVICE / ZOA_ERR_CUDA if any kernel
- * of this handle failed since the last check. */
+/* Waits for the device and reports ZOA_ERR_CUDA if a CUDA error is pending,
+ * ZOA_ERR_DEVICE if a kernel of this handle gave up on a bounded wait since the
+ * last check, or if one of the guard areas that surround every device buffer of
+ * the handle no longer holds its pattern (a kernel wrote out of bounds). */
 zoa_status zoa_check_device(zoa_handle h);
 
 /* Tuning switches.  ZOA_OPT_PIPELINE (default 1): run the fused sync step and the

@@ -71,7 +71,7 @@
  *                       frozen v equals damped momentum SGD (torch.optim.SGD);
  *                       x = x_{t'} - u / sqrt(v + eps) between syncs;
  *                       hand-worked power-of-two fixture of one sync step;
- *                       sign and scale symmetries.
+ *                       sign and scale symmetries; a noisy quadratic is minimised.
  *  zo_alg2_step        identity compressor equals the closed form of Adam and
  *                       equals zo_alg1_step with T_u = all steps; T_v = the first
  *                       T0 steps is Adam for T0 steps and then keeps v; hand-worked

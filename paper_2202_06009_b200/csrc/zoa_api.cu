@@ -38,6 +38,8 @@ struct zoa_handle_s {
     double gamma_sum = 0.0;
     int64_t t_sync = 0, t_last = -1;
     int64_t n_steps = 0, n_syncs = 0, n_var_updates = 0, n_launches = 0;
+    struct Guarded { char *ptr; size_t bytes, padded; };
+    std::vector<Guarded> guarded;  // every device buffer: user pointer, payload bytes, payload rounded up to 256
     std::string err;
 };
 
@@ -70,20 +72,52 @@ static StateView view(zoa_handle h)
     return st;
 }
 
+// Every device buffer sits between two guard areas filled with a fixed pattern; zoa_check_device
+// verifies them, so a kernel that writes outside a buffer is caught without a memory checker.
+static const size_t kGuardBytes = 256;
+static const unsigned char kGuardByte = 0xA5;
+
 static void free_all(zoa_handle h)
 {
-    void *ptrs[] = {h->x, h->m, h->u, h->dw, h->v_cur, h->v_nxt, h->ds, h->xs,
-                    h->words_w, h->words_s, h->scales_w, h->scales_s, h->staging, h->error_flag, h->sched, h->partials};
-    for (void *p : ptrs)
-        if (p) cudaFree(p);
+    for (auto &b : h->guarded) cudaFree(b.ptr - kGuardBytes);
+    h->guarded.clear();
+    if (h->staging) cudaFree(h->staging);
+}
+
+static cudaError_t alloc_guarded(zoa_handle h, void **p, size_t bytes)
+{
+    char *base = nullptr;
+    const size_t payload = (bytes + 255) / 256 * 256;
+    cudaError_t e = cudaMalloc(reinterpret_cast<void **>(&base), payload + 2 * kGuardBytes);
+    if (e != cudaSuccess) { *p = nullptr; return e; }
+    e = cudaMemset(base, kGuardByte, payload + 2 * kGuardBytes);          // guards and the rounding slack
+    if (e == cudaSuccess && bytes) e = cudaMemset(base + kGuardBytes, 0, bytes);   // the payload itself starts at zero
+    if (e != cudaSuccess) { cudaFree(base); *p = nullptr; return e; }
+    *p = base + kGuardBytes;
+    h->guarded.push_back({base + kGuardBytes, bytes, payload});
+    return cudaSuccess;
+}
+
+// True if every guard area still holds its pattern.
+static cudaError_t guards_intact(zoa_handle h, bool *intact)
+{
+    unsigned char host[3 * 256];
+    *intact = true;
+    for (auto &b : h->guarded) {
+        const size_t tail = b.padded - b.bytes + kGuardBytes;   // rounding slack + the guard after it
+        cudaError_t e = cudaMemcpy(host, b.ptr - kGuardBytes, kGuardBytes, cudaMemcpyDeviceToHost);
+        if (e == cudaSuccess) e = cudaMemcpy(host + kGuardBytes, b.ptr + b.bytes, tail, cudaMemcpyDeviceToHost);
+        if (e != cudaSuccess) return e;
+        for (size_t k = 0; k < kGuardBytes + tail; ++k)
+            if (host[k] != kGuardByte) *intact = false;
+    }
+    return cudaSuccess;
 }
 
 template <typename T>
-static cudaError_t alloc_zero(T **p, size_t count)
+static cudaError_t alloc_zero(zoa_handle h, T **p, size_t count)
 {
-    cudaError_t e = cudaMalloc(reinterpret_cast<void **>(p), count * sizeof(T));
-    if (e != cudaSuccess) { *p = nullptr; return e; }
-    return cudaMemset(*p, 0, count * sizeof(T));
+    return alloc_guarded(h, reinterpret_cast<void **>(p), count * sizeof(T));
 }
 
 extern "C" zoa_status zoa_create(zoa_handle *out, size_t n_params, int W, float beta1, float beta2,
@@ -117,18 +151,18 @@ extern "C" zoa_status zoa_create(zoa_handle *out, size_t n_params, int W, float 
     h->c.eps = eps;
 
     const size_t rows = (size_t)W * (size_t)h->n_pad, row = (size_t)h->n_pad;
-    if ((e = alloc_zero(&h->x, rows)) == cudaSuccess && (e = alloc_zero(&h->m, rows)) == cudaSuccess &&
-        (e = alloc_zero(&h->u, rows)) == cudaSuccess && (e = alloc_zero(&h->dw, rows)) == cudaSuccess &&
-        (e = alloc_zero(&h->v_cur, row)) == cudaSuccess && (e = alloc_zero(&h->v_nxt, row)) == cudaSuccess &&
-        (e = alloc_zero(&h->ds, row)) == cudaSuccess && (e = alloc_zero(&h->xs, row)) == cudaSuccess &&
-        (e = alloc_zero(&h->words_w, (size_t)W * h->words_stride)) == cudaSuccess &&
-        (e = alloc_zero(&h->words_s, (size_t)h->words_stride)) == cudaSuccess &&
-        (e = alloc_zero(&h->scales_w, (size_t)W * h->n_chunks)) == cudaSuccess &&
-        (e = alloc_zero(&h->scales_s, (size_t)h->n_chunks)) == cudaSuccess &&
-        (e = alloc_zero(&h->error_flag, 1)) == cudaSuccess && (e = alloc_zero(&h->sched, 2)) == cudaSuccess) {
+    if ((e = alloc_zero(h, &h->x, rows)) == cudaSuccess && (e = alloc_zero(h, &h->m, rows)) == cudaSuccess &&
+        (e = alloc_zero(h, &h->u, rows)) == cudaSuccess && (e = alloc_zero(h, &h->dw, rows)) == cudaSuccess &&
+        (e = alloc_zero(h, &h->v_cur, row)) == cudaSuccess && (e = alloc_zero(h, &h->v_nxt, row)) == cudaSuccess &&
+        (e = alloc_zero(h, &h->ds, row)) == cudaSuccess && (e = alloc_zero(h, &h->xs, row)) == cudaSuccess &&
+        (e = alloc_zero(h, &h->words_w, (size_t)W * h->words_stride)) == cudaSuccess &&
+        (e = alloc_zero(h, &h->words_s, (size_t)h->words_stride)) == cudaSuccess &&
+        (e = alloc_zero(h, &h->scales_w, (size_t)W * h->n_chunks)) == cudaSuccess &&
+        (e = alloc_zero(h, &h->scales_s, (size_t)h->n_chunks)) == cudaSuccess &&
+        (e = alloc_zero(h, &h->error_flag, 1)) == cudaSuccess && (e = alloc_zero(h, &h->sched, 2)) == cudaSuccess) {
         h->large_chunk = chunk > kMaxChunk;
         if (h->large_chunk)
-            e = alloc_zero(&h->partials, (size_t)(W + 1) * (size_t)h->n_chunks * (size_t)large_chunk_segments(view(h)));
+            e = alloc_zero(h, &h->partials, (size_t)(W + 1) * (size_t)h->n_chunks * (size_t)large_chunk_segments(view(h)));
         if (e == cudaSuccess) e = cudaDeviceSynchronize();
     }
     if (e != cudaSuccess) {
@@ -665,6 +699,9 @@ extern "C" zoa_status zoa_check_device(zoa_handle h)
     if (!h) return ZOA_ERR_ARG;
     ZOA_CUDA(h, cudaDeviceSynchronize());
     ZOA_CUDA(h, cudaGetLastError());
+    bool intact = true;
+    ZOA_CUDA(h, guards_intact(h, &intact));
+    if (!intact) return fail(h, ZOA_ERR_DEVICE, "a kernel wrote outside one of the handle's buffers (guard area overwritten)");
     int flag = 0;
     ZOA_CUDA(h, cudaMemcpy(&flag, h->error_flag, sizeof(int), cudaMemcpyDeviceToHost));
     if (flag) {

@@ -38,7 +38,10 @@ class Pair:
             self.cpu.set_params(x0)
 
     def close(self):
-        self.gpu.close()
+        try:
+            self.gpu.check_device()      # also verifies the guard areas around every state buffer
+        finally:
+            self.gpu.close()
 
     def step(self, g, lr, t, mode):
         """g: float32 array [W][n] (numpy).  mode: 'fused' (zoa_step_auto) or 'two_call'."""
