@@ -350,7 +350,7 @@ static cudaError_t run_compress(zoa_handle h, cudaStream_t s)
     cudaError_t e;
     if (h->large_chunk) {
         GradPtrs none{};
-        e = launch_large_compress(view(h), none, false, true, h->partials, &launches, s);
+        e = launch_large_compress(view(h), none, h->c, 0.f, 0, kGradAligned, h->partials, &launches, s);
     } else {
         e = launch_compress(view(h), s);
         launches = 1;
@@ -488,12 +488,18 @@ extern "C" zoa_status zoa_step_sync(zoa_handle h, const void *const *grads, floa
     const bool do_var = zoa_var_due(h, t) == 1;
     const StateView st = view(h);
     if (h->large_chunk) {
-        // No single block can hold a chunk: the local step is written out, then compressed.
-        ZOA_CUDA(h, launch_local_step(st, gp, h->c, lr, do_var, aligned, h->sm_count, s));
-        h->n_launches += 1;
-        ZOA_CUDA(h, run_compress(h, s));
+        // No single block can hold a chunk: the multi-pass kernels form the half-step buffer on the
+        // fly (twice), so m, x, u are written once, by the server pass.
+        int launches = 0;
+        ZOA_CUDA(h, launch_large_compress(st, gp, h->c, lr, 2, aligned, h->partials, &launches, s));
+        h->n_launches += launches;
         ZOA_CUDA(h, run_server(h, gamma_sum, s));
-        if (do_var) { h->v_pending = true; h->n_var_updates += 1; }
+        if (do_var) {
+            ZOA_CUDA(h, launch_variance(st, gp, h->c, aligned, 0, h->sm_count, s));
+            h->n_launches += 1;
+            h->v_pending = true;
+            h->n_var_updates += 1;
+        }
         h->gamma_sum = 0.0;
         h->t_last = t;
         h->t_sync = t;
@@ -550,7 +556,7 @@ extern "C" zoa_status zoa_alg2_step(zoa_handle h, const void *const *grads, floa
     if (h->large_chunk && !full) {
         int launches = 0;
         cudaStream_t s = static_cast<cudaStream_t>(stream);
-        ZOA_CUDA(h, launch_large_compress(view(h), gp, true, aligned, h->partials, &launches, s));
+        ZOA_CUDA(h, launch_large_compress(view(h), gp, h->c, lr, 1, aligned, h->partials, &launches, s));
         ZOA_CUDA(h, launch_large_server(view(h), h->c, 2, lr, h->partials, &launches, s));
         h->n_launches += launches;
     } else {

@@ -21,8 +21,8 @@ cudaError_t launch_alg2(const StateView &st, const GradPtrs &g, const Consts &c,
 
 // Chunks larger than kMaxChunk (up to the whole vector): multi-pass kernels, zoa_kernels.cu.
 long long large_chunk_segments(const StateView &st);
-cudaError_t launch_large_compress(const StateView &st, const GradPtrs &g, bool from_grads, int g_aligned,
-                                  double *partials, int *launches, cudaStream_t s);
+cudaError_t launch_large_compress(const StateView &st, const GradPtrs &g, const Consts &c, float gamma, int src,
+                                  int g_aligned, double *partials, int *launches, cudaStream_t s);
 cudaError_t launch_large_server(const StateView &st, const Consts &c, int mode, float scalar, double *partials,
                                 int *launches, cudaStream_t s);
 

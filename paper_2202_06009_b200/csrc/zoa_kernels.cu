@@ -618,27 +618,40 @@ __device__ __forceinline__ SegGeom seg_geom(const StateView &st, long long seg, 
     return g;
 }
 
-// What a worker compresses, four coordinates from j: its source buffer plus its error.
-template <bool FROM_GRADS>
-__device__ __forceinline__ float4 lc_worker_input(const StateView &st, const GradPtrs &g, int i, long long j, int g_aligned)
+// What a worker compresses, four coordinates from j.  SRC 0: u + delta (zoa_onebit_reduce);
+// SRC 1: g + delta (Algorithm 2); SRC 2: the half-step buffer formed on the fly,
+// (u + gamma m_{t+1/2}) + delta with m_{t+1/2} = beta1 m + (1 - beta1) g (fused sync step).
+template <int SRC>
+__device__ __forceinline__ float4 lc_worker_input(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
+                                                  int i, long long j, int g_aligned)
 {
     const long long row = (long long)i * st.n_pad + j;
-    const float4 a = FROM_GRADS ? ld_grad4(g.p[i], j, st.n, g_aligned) : ld4(st.u + row);
     const float4 e = ld4(st.dw + row);
+    float4 a;
+    if (SRC == 0) {
+        a = ld4(st.u + row);
+    } else if (SRC == 1) {
+        a = ld_grad4(g.p[i], j, st.n, g_aligned);
+    } else {
+        const float4 g4 = ld_grad4(g.p[i], j, st.n, g_aligned), m4 = ld4(st.m + row), u4 = ld4(st.u + row);
+        a = make_float4(f_add(u4.x, f_mul(gamma, momentum(c, m4.x, g4.x))), f_add(u4.y, f_mul(gamma, momentum(c, m4.y, g4.y))),
+                        f_add(u4.z, f_mul(gamma, momentum(c, m4.z, g4.z))), f_add(u4.w, f_mul(gamma, momentum(c, m4.w, g4.w))));
+    }
     return make_float4(f_add(a.x, e.x), f_add(a.y, e.y), f_add(a.z, e.z), f_add(a.w, e.w));
 }
 
 // partials[i][seg] = sum |z| over segment `seg` of worker i = blockIdx.y.
-template <bool FROM_GRADS>
+template <int SRC>
 __global__ void __launch_bounds__(512)
-lc_partial_l1_kernel(StateView st, GradPtrs g, int g_aligned, long long segs_per_chunk, long long n_segs, double *partials)
+lc_partial_l1_kernel(StateView st, GradPtrs g, Consts c, float gamma, int g_aligned, long long segs_per_chunk,
+                     long long n_segs, double *partials)
 {
     __shared__ double scratch[34];
     const SegGeom sg = seg_geom(st, blockIdx.x, segs_per_chunk);
     const int i = blockIdx.y;
     double l1 = 0.0;
     for (int idx = 4 * threadIdx.x; idx < sg.len; idx += 4 * blockDim.x) {
-        const float4 z = lc_worker_input<FROM_GRADS>(st, g, i, sg.j0 + idx, g_aligned);
+        const float4 z = lc_worker_input<SRC>(st, g, c, gamma, i, sg.j0 + idx, g_aligned);
         const float zz[4] = {z.x, z.y, z.z, z.w};
 #pragma unroll
         for (int k = 0; k < 4; ++k)
@@ -667,9 +680,9 @@ __global__ void lc_scales_kernel(StateView st, const double *partials, long long
 }
 
 // Worker side of Algorithm 3 once the magnitudes are known: bits, errors.
-template <bool FROM_GRADS>
+template <int SRC>
 __global__ void __launch_bounds__(512)
-lc_compress_apply_kernel(StateView st, GradPtrs g, int g_aligned, long long segs_per_chunk)
+lc_compress_apply_kernel(StateView st, GradPtrs g, Consts c, float gamma, int g_aligned, long long segs_per_chunk)
 {
     const SegGeom sg = seg_geom(st, blockIdx.x, segs_per_chunk);
     const int i = blockIdx.y;
@@ -679,7 +692,7 @@ lc_compress_apply_kernel(StateView st, GradPtrs g, int g_aligned, long long segs
         const int idx = base + 4 * lane;
         float z[4] = {0.f, 0.f, 0.f, 0.f}, hat[4];
         if (idx < sg.len) {
-            const float4 z4 = lc_worker_input<FROM_GRADS>(st, g, i, sg.j0 + idx, g_aligned);
+            const float4 z4 = lc_worker_input<SRC>(st, g, c, gamma, i, sg.j0 + idx, g_aligned);
             z[0] = z4.x; z[1] = z4.y; z[2] = z4.z; z[3] = z4.w;
         }
         const uint32_t word = compress_tile(z, hat, scale, idx, sg.len);
@@ -887,18 +900,21 @@ long long large_chunk_segments(const StateView &st)
     return (span + kSegment - 1) / kSegment;
 }
 
-// Worker side of Algorithm 3 for chunks too large for one block.  from_grads: compress
-// g + delta (Algorithm 2) instead of u + delta (Algorithm 1).  partials: [W + 1][n_chunks * segments].
-cudaError_t launch_large_compress(const StateView &st, const GradPtrs &g, bool from_grads, int g_aligned,
-                                  double *partials, int *launches, cudaStream_t s)
+// Worker side of Algorithm 3 for chunks too large for one block.  src 0: compress u + delta;
+// 1: g + delta (Algorithm 2); 2: the half-step buffer formed on the fly from g, m, u (fused sync
+// step; m, x, u are then written by the server pass only).  partials: [W + 1][n_chunks * segments].
+cudaError_t launch_large_compress(const StateView &st, const GradPtrs &g, const Consts &c, float gamma, int src,
+                                  int g_aligned, double *partials, int *launches, cudaStream_t s)
 {
     const long long spc = large_chunk_segments(st), n_segs = spc * st.n_chunks;
     const dim3 grid((unsigned)n_segs, (unsigned)st.W);
-    if (from_grads) lc_partial_l1_kernel<true><<<grid, 512, 0, s>>>(st, g, g_aligned, spc, n_segs, partials);
-    else lc_partial_l1_kernel<false><<<grid, 512, 0, s>>>(st, g, g_aligned, spc, n_segs, partials);
+    if (src == 0) lc_partial_l1_kernel<0><<<grid, 512, 0, s>>>(st, g, c, gamma, g_aligned, spc, n_segs, partials);
+    else if (src == 1) lc_partial_l1_kernel<1><<<grid, 512, 0, s>>>(st, g, c, gamma, g_aligned, spc, n_segs, partials);
+    else lc_partial_l1_kernel<2><<<grid, 512, 0, s>>>(st, g, c, gamma, g_aligned, spc, n_segs, partials);
     lc_scales_kernel<<<dim3((unsigned)st.n_chunks, (unsigned)st.W), 32, 0, s>>>(st, partials, spc, n_segs, st.scales_w);
-    if (from_grads) lc_compress_apply_kernel<true><<<grid, 512, 0, s>>>(st, g, g_aligned, spc);
-    else lc_compress_apply_kernel<false><<<grid, 512, 0, s>>>(st, g, g_aligned, spc);
+    if (src == 0) lc_compress_apply_kernel<0><<<grid, 512, 0, s>>>(st, g, c, gamma, g_aligned, spc);
+    else if (src == 1) lc_compress_apply_kernel<1><<<grid, 512, 0, s>>>(st, g, c, gamma, g_aligned, spc);
+    else lc_compress_apply_kernel<2><<<grid, 512, 0, s>>>(st, g, c, gamma, g_aligned, spc);
     *launches += 3;
     return cudaGetLastError();
 }
