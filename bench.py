@@ -312,7 +312,7 @@ def run_ours(args, wl):
                "h2d_bytes_per_step": wl.n * wl.W * g_bytes, "d2h_bytes_per_step": wl.n * 4, "steps": ke,
                "ms_per_step": e_ms / ke,
                "how": "zoa_step_host: W copies from pinned host memory (one pinned buffer serves every "
-                      "worker), the step, worker 0's model copied back"}
+                      "worker) in eight chunk ranges overlapped with the step's kernels, worker 0's model copied back"}
     opt.close()
 
     if rank == 0:

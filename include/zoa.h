@@ -200,7 +200,11 @@ zoa_status zoa_step_auto(zoa_handle h, const void *const *grads, float lr, int64
  * of W (host) pointers of n_params floats (pinned memory copies fastest).
  * Copies them to a device staging area the handle allocates on first use,
  * runs zoa_step_auto, and, if host_x_out is not NULL, copies worker 0's model
- * back (n_params floats).  All on `stream`; does not synchronise. */
+ * back (n_params floats).  Large problems are cut into eight chunk ranges so
+ * that the copies of one range (on a stream of the handle's own) overlap the
+ * kernels and the result copy of the previous one (on `stream`); everything is
+ * ordered with `stream`, which therefore tells when the step and host_x_out are
+ * done.  Does not synchronise. */
 zoa_status zoa_step_host(zoa_handle h, const void *const *host_grads, float lr, int64_t t,
                          float *host_x_out, void *stream);
 

@@ -23,6 +23,8 @@ struct zoa_handle_s {
     uint32_t *words_w = nullptr, *words_s = nullptr;
     float *scales_w = nullptr, *scales_s = nullptr;
     float *staging = nullptr;      // [W][n_pad], device copy of host gradients (zoa_step_host)
+    cudaStream_t copy_stream = nullptr;                 // host-to-device copies of zoa_step_host run here ...
+    std::vector<cudaEvent_t> copy_events;               // ... and these order them with the caller's stream
     int *error_flag = nullptr;     // device int: a kernel gave up on a bounded wait
     unsigned long long *sched = nullptr;   // device [2]: chunk counter of the persistent kernel, finished blocks
     double *partials = nullptr;    // device [W + 1][n_chunks * segments]: per-segment l1 sums, chunk > 16384 only
@@ -82,6 +84,10 @@ static void free_all(zoa_handle h)
     for (auto &b : h->guarded) cudaFree(b.ptr - kGuardBytes);
     h->guarded.clear();
     if (h->staging) cudaFree(h->staging);
+    for (cudaEvent_t e : h->copy_events) cudaEventDestroy(e);
+    h->copy_events.clear();
+    if (h->copy_stream) cudaStreamDestroy(h->copy_stream);
+    h->copy_stream = nullptr;
 }
 
 static cudaError_t alloc_guarded(zoa_handle h, void **p, size_t bytes)
@@ -372,6 +378,52 @@ static cudaError_t run_server(zoa_handle h, float gamma_sum, cudaStream_t s)
     return e;
 }
 
+// Lines 3-5 (+ 14-15) for the chunks [c0, c1).
+static zoa_status run_local_range(zoa_handle h, const StateView &st, const GradPtrs &gp, float lr, bool do_var, int fmt,
+                                  long long c0, long long c1, cudaStream_t s)
+{
+    const long long e0 = c0 * h->chunk, e1 = std::min<long long>(c1 * (long long)h->chunk, h->n);
+    ZOA_CUDA(h, launch_local_step(st, gp, h->c, lr, do_var, fmt, e0, e1, s));
+    h->n_launches += 1;
+    return ZOA_OK;
+}
+
+// A whole sync step (chunks up to 16384) for the chunks [c0, c1): the bulk-copy ring for the
+// full chunks where it applies, the chunk-per-block kernel for the rest, the variance update
+// fused or beside it.
+static zoa_status run_sync_range(zoa_handle h, const StateView &st, const GradPtrs &gp, float lr, float gamma_sum,
+                                 bool do_var, int fmt, long long c0, long long c1, cudaStream_t s)
+{
+    const long long e0 = c0 * h->chunk, e1 = std::min<long long>(c1 * (long long)h->chunk, h->n);
+    const bool ragged = c1 == h->n_chunks && h->n % h->chunk != 0;
+    const long long n_full = c1 - c0 - (ragged ? 1 : 0);
+    // The persistent kernel pays off once every SM has a few chunks to stream; below that the
+    // one-block-per-chunk kernel starts faster (measured on a 512-chunk problem).
+    const bool enough_chunks = h->use_pipeline == 2 || n_full >= 4ll * h->sm_count;
+    const int stages = h->use_pipeline && enough_chunks && n_full > 0 ? pipeline_stages(st, fmt) : 0;
+    long long var_first = e0;     // coordinates from here to e1 still need lines 14-15
+    if (stages > 0) {
+        bool var_fused = false;
+        ZOA_CUDA(h, launch_step_sync_pipelined(st, gp, h->c, lr, gamma_sum, do_var, fmt, c0, n_full, stages, h->sm_count,
+                                               h->error_flag, h->sched, (unsigned long long)h->wait_limit_ms * 1000000ull,
+                                               h->test_stop_after_tiles, &var_fused, s));
+        h->n_launches += 1;
+        if (ragged) {
+            ZOA_CUDA(h, launch_step_sync(st, gp, h->c, lr, gamma_sum, fmt, c0 + n_full, 1, s));
+            h->n_launches += 1;
+        }
+        if (var_fused) var_first = (c0 + n_full) * h->chunk;
+    } else {
+        ZOA_CUDA(h, launch_step_sync(st, gp, h->c, lr, gamma_sum, fmt, c0, c1 - c0, s));
+        h->n_launches += 1;
+    }
+    if (do_var && var_first < e1) {
+        ZOA_CUDA(h, launch_variance(st, gp, h->c, fmt, var_first, e1, s));
+        h->n_launches += 1;
+    }
+    return ZOA_OK;
+}
+
 extern "C" zoa_status zoa_step(zoa_handle h, const void *const *grads, float lr, int64_t t, void *stream)
 {
     GradPtrs gp;
@@ -380,8 +432,8 @@ extern "C" zoa_status zoa_step(zoa_handle h, const void *const *grads, float lr,
     if (rc != ZOA_OK) return rc;
     commit_variance(h);
     const bool do_var = zoa_var_due(h, t) == 1;
-    ZOA_CUDA(h, launch_local_step(view(h), gp, h->c, lr, do_var, aligned, h->sm_count, static_cast<cudaStream_t>(stream)));
-    h->n_launches += 1;
+    rc = run_local_range(h, view(h), gp, lr, do_var, aligned, 0, h->n_chunks, static_cast<cudaStream_t>(stream));
+    if (rc != ZOA_OK) return rc;
     h->gamma_sum += (double)lr;
     if (do_var) { h->v_pending = true; h->n_var_updates += 1; }
     h->t_last = t;
@@ -495,7 +547,7 @@ extern "C" zoa_status zoa_step_sync(zoa_handle h, const void *const *grads, floa
         h->n_launches += launches;
         ZOA_CUDA(h, run_server(h, gamma_sum, s));
         if (do_var) {
-            ZOA_CUDA(h, launch_variance(st, gp, h->c, aligned, 0, h->sm_count, s));
+            ZOA_CUDA(h, launch_variance(st, gp, h->c, aligned, 0, h->n, s));
             h->n_launches += 1;
             h->v_pending = true;
             h->n_var_updates += 1;
@@ -507,33 +559,9 @@ extern "C" zoa_status zoa_step_sync(zoa_handle h, const void *const *grads, floa
         h->n_syncs += 1;
         return ZOA_OK;
     }
-    // The persistent kernel pays off once every SM has a few chunks to stream; below that the
-    // one-block-per-chunk kernel starts faster (measured on the 512-chunk configuration).
-    const bool enough_chunks = h->use_pipeline == 2 || h->n / h->chunk >= 4ll * h->sm_count;
-    const int stages = h->use_pipeline && enough_chunks ? pipeline_stages(st, aligned) : 0;
-    long long var_first = 0;     // coordinates from here on still need lines 14-15
-    if (stages > 0) {
-        // Full chunks through the bulk-copy ring; a ragged last chunk through the chunk-per-block kernel.
-        const long long n_full = h->n / h->chunk;
-        bool var_fused = false;
-        ZOA_CUDA(h, launch_step_sync_pipelined(st, gp, h->c, lr, gamma_sum, do_var, aligned, stages, h->sm_count,
-                                               h->error_flag, h->sched, (unsigned long long)h->wait_limit_ms * 1000000ull,
-                                               h->test_stop_after_tiles, &var_fused, s));
-        h->n_launches += 1;
-        if (n_full < h->n_chunks) {
-            ZOA_CUDA(h, launch_step_sync(st, gp, h->c, lr, gamma_sum, aligned, n_full, h->n_chunks - n_full, s));
-            h->n_launches += 1;
-        }
-        var_first = var_fused ? n_full * h->chunk : 0;
-    } else {
-        ZOA_CUDA(h, launch_step_sync(st, gp, h->c, lr, gamma_sum, aligned, 0, h->n_chunks, s));
-        h->n_launches += 1;
-    }
+    rc = run_sync_range(h, st, gp, lr, gamma_sum, do_var, aligned, 0, h->n_chunks, s);
+    if (rc != ZOA_OK) return rc;
     if (do_var) {
-        if (var_first < h->n) {
-            ZOA_CUDA(h, launch_variance(st, gp, h->c, aligned, var_first, h->sm_count, s));
-            h->n_launches += 1;
-        }
         h->v_pending = true;
         h->n_var_updates += 1;
     }
@@ -595,23 +623,71 @@ extern "C" zoa_status zoa_step_host(zoa_handle h, const void *const *host_grads,
     if (!host_grads) return fail(h, ZOA_ERR_ARG, "zoa_step_host: host_grads is NULL");
     for (int i = 0; i < h->W; ++i)
         if (!host_grads[i]) return fail(h, ZOA_ERR_ARG, "zoa_step_host: a gradient pointer is NULL");
-    if (!std::isfinite(lr) || t < 0) return fail(h, ZOA_ERR_ARG, "zoa_step_host: bad lr or t");
-    if (t <= h->t_last) return fail(h, ZOA_ERR_STATE, "zoa_step_host: t must increase from step to step");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (!h->staging) {
         cudaError_t e = cudaMalloc(reinterpret_cast<void **>(&h->staging), (size_t)h->W * h->n_pad * sizeof(float));
         if (e != cudaSuccess) { h->staging = nullptr; cudaGetLastError(); return fail_cuda(h, e, "zoa_step_host: staging area"); }
     }
     const void *dev[kMaxWorkers];
-    for (int i = 0; i < h->W; ++i) {
-        float *dst = h->staging + (size_t)i * h->n_pad;
-        ZOA_CUDA(h, cudaMemcpyAsync(dst, host_grads[i], (size_t)h->n * (h->grad_type ? 2 : 4), cudaMemcpyHostToDevice, s));
-        dev[i] = dst;
+    for (int i = 0; i < h->W; ++i) dev[i] = h->staging + (size_t)i * h->n_pad;
+    const size_t g_bytes = h->grad_type ? 2 : 4;
+
+    // Large chunks are not cut into ranges, and small problems are not worth it: copy, then step.
+    const int kSegments = 8;
+    if (h->large_chunk || h->n_chunks < 64 * kSegments) {
+        for (int i = 0; i < h->W; ++i)
+            ZOA_CUDA(h, cudaMemcpyAsync(const_cast<void *>(dev[i]), host_grads[i], (size_t)h->n * g_bytes, cudaMemcpyHostToDevice, s));
+        zoa_status rc = zoa_step_auto(h, dev, lr, t, stream);
+        if (rc != ZOA_OK) return rc;
+        if (host_x_out)
+            ZOA_CUDA(h, cudaMemcpyAsync(host_x_out, h->x, (size_t)h->n * sizeof(float), cudaMemcpyDeviceToHost, s));
+        return ZOA_OK;
     }
-    zoa_status rc = zoa_step_auto(h, dev, lr, t, stream);
+
+    // Otherwise the vector is cut into chunk ranges: the copies of range k+1 (on the handle's own copy
+    // stream) run while the kernels of range k and the copy of its part of the result (on the
+    // caller's stream) do, so the step costs little more than moving the gradients over the bus.
+    GradPtrs gp;
+    int fmt;
+    zoa_status rc = check_step_args(h, dev, lr, t, &gp, &fmt, "zoa_step_host");
     if (rc != ZOA_OK) return rc;
-    if (host_x_out)
-        ZOA_CUDA(h, cudaMemcpyAsync(host_x_out, h->x, (size_t)h->n * sizeof(float), cudaMemcpyDeviceToHost, s));
+    const bool do_sync = zoa_sync_due(h, t) == 1;
+    const double total = h->gamma_sum + (double)lr;
+    const float gamma_sum = (float)total;
+    if (do_sync && (!(total > 0.0) || !(gamma_sum > 0.f) || !std::isfinite(gamma_sum)))
+        return fail(h, ZOA_ERR_STATE, "zoa_step_host: sum of learning rates since the last sync is not positive");
+    if (!h->copy_stream) ZOA_CUDA(h, cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking));
+    while ((int)h->copy_events.size() < kSegments + 1) {
+        cudaEvent_t e;
+        ZOA_CUDA(h, cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+        h->copy_events.push_back(e);
+    }
+    // the staging area may still be read by the caller's stream (the previous step)
+    ZOA_CUDA(h, cudaEventRecord(h->copy_events[kSegments], s));
+    ZOA_CUDA(h, cudaStreamWaitEvent(h->copy_stream, h->copy_events[kSegments], 0));
+    commit_variance(h);
+    const bool do_var = zoa_var_due(h, t) == 1;
+    const StateView st = view(h);
+    for (int k = 0; k < kSegments; ++k) {
+        const long long c0 = h->n_chunks * k / kSegments, c1 = h->n_chunks * (k + 1) / kSegments;
+        const long long e0 = c0 * h->chunk, e1 = std::min<long long>(c1 * (long long)h->chunk, h->n);
+        for (int i = 0; i < h->W; ++i)
+            ZOA_CUDA(h, cudaMemcpyAsync(reinterpret_cast<char *>(const_cast<void *>(dev[i])) + (size_t)e0 * g_bytes,
+                                        static_cast<const char *>(host_grads[i]) + (size_t)e0 * g_bytes,
+                                        (size_t)(e1 - e0) * g_bytes, cudaMemcpyHostToDevice, h->copy_stream));
+        ZOA_CUDA(h, cudaEventRecord(h->copy_events[k], h->copy_stream));
+        ZOA_CUDA(h, cudaStreamWaitEvent(s, h->copy_events[k], 0));
+        rc = do_sync ? run_sync_range(h, st, gp, lr, gamma_sum, do_var, fmt, c0, c1, s)
+                     : run_local_range(h, st, gp, lr, do_var, fmt, c0, c1, s);
+        if (rc != ZOA_OK) return rc;
+        if (host_x_out)
+            ZOA_CUDA(h, cudaMemcpyAsync(host_x_out + e0, h->x + e0, (size_t)(e1 - e0) * sizeof(float), cudaMemcpyDeviceToHost, s));
+    }
+    if (do_var) { h->v_pending = true; h->n_var_updates += 1; }
+    h->gamma_sum = do_sync ? 0.0 : total;
+    h->t_last = t;
+    if (do_sync) { h->t_sync = t; h->n_syncs += 1; }
+    h->n_steps += 1;
     return ZOA_OK;
 }
 

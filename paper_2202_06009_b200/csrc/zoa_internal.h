@@ -8,9 +8,9 @@ namespace zoa {
 cudaError_t configure_kernels();
 
 cudaError_t launch_local_step(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
-                              bool do_var, int g_aligned, int sm_count, cudaStream_t s);
+                              bool do_var, int g_aligned, long long first, long long end, cudaStream_t s);
 cudaError_t launch_variance(const StateView &st, const GradPtrs &g, const Consts &c, int g_aligned,
-                            long long first, int sm_count, cudaStream_t s);
+                            long long first, long long end, cudaStream_t s);
 cudaError_t launch_compress(const StateView &st, cudaStream_t s);
 cudaError_t launch_reduce(const StateView &st, const Consts &c, float gamma_sum, cudaStream_t s);
 cudaError_t launch_step_sync(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
@@ -29,7 +29,8 @@ cudaError_t launch_large_server(const StateView &st, const Consts &c, int mode, 
 // Pipelined (bulk-copy ring) form of the fused sync step, zoa_pipeline.cu.
 int pipeline_stages(const StateView &st, int grad_fmt);
 cudaError_t launch_step_sync_pipelined(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
-                                       float gamma_sum, bool do_var, int grad_fmt, int stages, int sm_count, int *error_flag,
+                                       float gamma_sum, bool do_var, int grad_fmt, long long first_chunk, long long n_chunks, int stages,
+                                       int sm_count, int *error_flag,
                                        unsigned long long *sched, unsigned long long wait_limit_ns,
                                        long long test_stop_after_tiles, bool *var_fused, cudaStream_t s);
 

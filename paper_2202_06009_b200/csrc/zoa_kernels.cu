@@ -26,12 +26,11 @@ namespace zoa {
 // pays (measured 5.9 -> 6.4 TB/s); with binary32 gradients it does not (6.7 -> 6.4 TB/s).
 template <bool DO_VAR, int GFMT>
 __global__ void __launch_bounds__(256, (GFMT > 0 && (GFMT & kGradTypeMask) != kGradF32) ? 5 : 4)
-local_step_kernel(StateView st, GradPtrs g, Consts c, float gamma, int g_fmt_arg)
+local_step_kernel(StateView st, GradPtrs g, Consts c, float gamma, int g_fmt_arg, long long first4, long long end4)
 {
     const int g_aligned = GFMT >= 0 ? GFMT : g_fmt_arg;
-    const long long n4 = (st.n + 3) >> 2;
     const long long stride = (long long)gridDim.x * blockDim.x;
-    for (long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x; q < n4; q += stride) {
+    for (long long q = first4 + (long long)blockIdx.x * blockDim.x + threadIdx.x; q < end4; q += stride) {   // float4 groups [first4, end4)
         const long long j = q << 2;
         const float4 v4 = ld4(st.v + j);
         const float d[4] = {denom(c, v4.x), denom(c, v4.y), denom(c, v4.z), denom(c, v4.w)};
@@ -68,11 +67,10 @@ local_step_kernel(StateView st, GradPtrs g, Consts c, float gamma, int g_fmt_arg
 }
 
 __global__ void __launch_bounds__(256)
-variance_kernel(StateView st, GradPtrs g, Consts c, int g_aligned, long long first4)
+variance_kernel(StateView st, GradPtrs g, Consts c, int g_aligned, long long first4, long long end4)
 {
-    const long long n4 = (st.n + 3) >> 2;
     const long long stride = (long long)gridDim.x * blockDim.x;
-    for (long long q = first4 + (long long)blockIdx.x * blockDim.x + threadIdx.x; q < n4; q += stride) {
+    for (long long q = first4 + (long long)blockIdx.x * blockDim.x + threadIdx.x; q < end4; q += stride) {
         const long long j = q << 2;
         double G[4] = {0.0, 0.0, 0.0, 0.0};
         for (int i = 0; i < st.W; ++i) {
@@ -812,11 +810,13 @@ static int elementwise_grid(long long n4)
     return (int)(blocks < 1 ? 1 : blocks);
 }
 
+// Lines 3-5 (and 14-15 if do_var) for the coordinates [first, end); first is a multiple of 4.
 cudaError_t launch_local_step(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
-                              bool do_var, int g_aligned, int sm_count, cudaStream_t s)
+                              bool do_var, int g_aligned, long long first, long long end, cudaStream_t s)
 {
-    const int grid = elementwise_grid((st.n + 3) / 4);
-#define ZOA_LOCAL(VAR, FMT) local_step_kernel<VAR, FMT><<<grid, 256, 0, s>>>(st, g, c, gamma, g_aligned)
+    const long long first4 = first >> 2, end4 = (end + 3) >> 2;
+    const int grid = elementwise_grid(end4 - first4);
+#define ZOA_LOCAL(VAR, FMT) local_step_kernel<VAR, FMT><<<grid, 256, 0, s>>>(st, g, c, gamma, g_aligned, first4, end4)
     switch (g_aligned) {
     case kGradF32 | kGradAligned: if (do_var) ZOA_LOCAL(true, kGradF32 | kGradAligned); else ZOA_LOCAL(false, kGradF32 | kGradAligned); break;
     case kGradF16 | kGradAligned: if (do_var) ZOA_LOCAL(true, kGradF16 | kGradAligned); else ZOA_LOCAL(false, kGradF16 | kGradAligned); break;
@@ -827,12 +827,12 @@ cudaError_t launch_local_step(const StateView &st, const GradPtrs &g, const Cons
     return cudaGetLastError();
 }
 
-// Lines 14-15 for the coordinates [first, n); first is a multiple of 4.
+// Lines 14-15 for the coordinates [first, end); first is a multiple of 4.
 cudaError_t launch_variance(const StateView &st, const GradPtrs &g, const Consts &c, int g_aligned,
-                            long long first, int sm_count, cudaStream_t s)
+                            long long first, long long end, cudaStream_t s)
 {
-    const long long first4 = first >> 2;
-    variance_kernel<<<elementwise_grid((st.n + 3) / 4 - first4), 256, 0, s>>>(st, g, c, g_aligned, first4);
+    const long long first4 = first >> 2, end4 = (end + 3) >> 2;
+    variance_kernel<<<elementwise_grid(end4 - first4), 256, 0, s>>>(st, g, c, g_aligned, first4, end4);
     return cudaGetLastError();
 }
 

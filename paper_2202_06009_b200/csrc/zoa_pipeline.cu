@@ -36,6 +36,7 @@ struct PipeArgs {
     GradPtrs g;
     Consts c;
     float gamma, gamma_sum;
+    long long first_chunk;    // the launch covers the full chunks [first_chunk, first_chunk + n_full_chunks)
     long long n_full_chunks;
     int stages;
     int *error_flag;  // device int, set non-zero when a wait ran out
@@ -186,8 +187,9 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
         long long issued = 0;
         bool ok = true;
         for (long long k = 0; ok; ++k) {
-            const long long chunk = (long long)atomicAdd(&a.sched[0], 1ull);
-            const bool last = chunk >= a.n_full_chunks;
+            const long long taken = (long long)atomicAdd(&a.sched[0], 1ull);
+            const bool last = taken >= a.n_full_chunks;
+            const long long chunk = a.first_chunk + taken;
             // The chunk id travels to the consumers through shared memory; the arrive on the
             // first tile's barrier below publishes it.  The queue cannot wrap onto an unread
             // entry: the producer is at most `stages` tiles, hence chunks, ahead.
@@ -468,8 +470,9 @@ __global__ void __launch_bounds__(kThreads, 1) alg2_pipelined_kernel(const __gri
         bool ok = true;
         const uint32_t g_elem = (a.grad_fmt & kGradTypeMask) == kGradF32 ? 4u : 2u;
         for (long long k = 0; ok; ++k) {
-            const long long chunk = (long long)atomicAdd(&a.sched[0], 1ull);
-            const bool last = chunk >= a.n_full_chunks;
+            const long long taken = (long long)atomicAdd(&a.sched[0], 1ull);
+            const bool last = taken >= a.n_full_chunks;
+            const long long chunk = a.first_chunk + taken;
             if (!mbar_wait(smem_addr(&sh->empty[s]), phase ^ 1u, abort_flag, a.error_flag, a.wait_limit_ns)) { ok = false; break; }
             sh->chunk_queue[k % (kMaxStages + 2)] = last ? -1 : chunk;
             if (last) {
@@ -694,16 +697,17 @@ static cudaError_t launch_pipe(const PipeArgs &a, int grid, size_t smem, cudaStr
     return cudaGetLastError();
 }
 
-// Runs the full chunks [0, n / chunk) of a sync step; the ragged last chunk, if any, is the caller's.
+// Runs the full chunks [first_chunk, first_chunk + n_chunks) of a sync step; a ragged last chunk is the caller's.
 // *var_fused tells whether lines 14-15 were done here too.
 cudaError_t launch_step_sync_pipelined(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
-                                       float gamma_sum, bool do_var, int grad_fmt, int stages, int sm_count, int *error_flag,
-                                       unsigned long long *sched, unsigned long long wait_limit_ns,
+                                       float gamma_sum, bool do_var, int grad_fmt, long long first_chunk, long long n_chunks, int stages,
+                                       int sm_count, int *error_flag, unsigned long long *sched, unsigned long long wait_limit_ns,
                                        long long test_stop_after_tiles, bool *var_fused, cudaStream_t s)
 {
     PipeArgs a;
     a.st = st; a.g = g; a.c = c; a.gamma = gamma; a.gamma_sum = gamma_sum;
-    a.n_full_chunks = st.n / st.chunk;
+    a.first_chunk = first_chunk;
+    a.n_full_chunks = n_chunks;
     a.stages = stages;
     a.error_flag = error_flag;
     a.sched = sched;
@@ -762,6 +766,7 @@ cudaError_t launch_alg2_pipelined(const StateView &st, const GradPtrs &g, const 
 {
     PipeArgs a;
     a.st = st; a.g = g; a.c = c; a.gamma = gamma; a.gamma_sum = 0.f;
+    a.first_chunk = 0;
     a.n_full_chunks = st.n / st.chunk;
     a.stages = stages;
     a.error_flag = error_flag;

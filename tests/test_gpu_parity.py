@@ -280,6 +280,36 @@ def test_host_gradient_entry_point():
         a.close(), b.close()
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_host_entry_point_in_overlapped_segments(dtype):
+    """Large enough to be cut into eight chunk ranges with the copies overlapping the kernels:
+    every state must equal the plain device path, over sync, local and variance steps."""
+    rng = np.random.default_rng(21)
+    n, W, chunk = 700 * 1024 + 100, 3, 1024
+    a, b = Zoa(n, W, chunk=chunk), Zoa(n, W, chunk=chunk)
+    try:
+        for z in (a, b):
+            z.set_pipeline("force")
+            z.set_policies((0, 1, 4), (0, 2), (1, 3))
+            z.set_grad_dtype(dtype)
+        out = torch.empty(n).pin_memory()
+        for t in range(7):
+            g = torch.from_numpy(_grads(rng, W, n)).to(dtype).pin_memory()
+            a.step_host(list(g), 1e-3, t, out)
+            b.step_auto(list(g.cuda()), 1e-3, t)
+            torch.cuda.synchronize()
+            assert np.array_equal(out.numpy(), b.read("x", 0)), t
+            for name in ("x", "m", "u", "delta_w"):
+                for i in range(W):
+                    assert np.array_equal(a.read(name, i), b.read(name, i)), (name, i, t)
+            for name in ("v", "delta_s", "x_sync", "words_s", "scales_s"):
+                assert np.array_equal(a.read(name), b.read(name)), (name, t)
+        assert a.stats()["n_syncs"] == b.stats()["n_syncs"] and a.stats()["t_sync"] == b.stats()["t_sync"]
+        a.check_device()
+    finally:
+        a.close(), b.close()
+
+
 def test_argument_and_state_errors():
     with pytest.raises(ZoaError) as e:
         Zoa(100, 0)
