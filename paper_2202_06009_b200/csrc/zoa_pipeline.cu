@@ -151,6 +151,87 @@ __device__ __forceinline__ uint32_t pack_group(const bool b[4])
     return __reduce_or_sync(0xFFu << (lane & 24), nib << ((lane & 7) * 4));
 }
 
+// Set-up shared by the ring kernels: stage barriers and the abort flag, then a block barrier.
+__device__ __forceinline__ void ring_init(PipeShared *sh, int stages)
+{
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) {
+            mbar_init(smem_addr(&sh->full[s]), 1);
+            mbar_init(smem_addr(&sh->empty[s]), kConsumerWarps);
+        }
+        sh->abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+}
+
+// The copy-issuing lane's side of the ring: which stage comes next, chunk ids from the global
+// counter, and the orderly way out when a wait runs out.
+struct RingProducer {
+    const PipeArgs &a;
+    PipeShared *sh;
+    unsigned char *ring;
+    int stage_bytes;
+    int s = 0;
+    uint32_t phase = 0;
+    long long issued = 0;
+    bool ok = true;
+
+    __device__ RingProducer(const PipeArgs &args, PipeShared *shared, unsigned char *ring_base, int bytes)
+        : a(args), sh(shared), ring(ring_base), stage_bytes(bytes) {}
+
+    // Waits until the consumers have released the current stage.
+    __device__ __forceinline__ bool stage_free()
+    {
+        if (!ok) return false;
+        if (!mbar_wait(smem_addr(&sh->empty[s]), phase ^ 1u, &sh->abort, a.error_flag, a.wait_limit_ns)) ok = false;
+        return ok;
+    }
+    // Takes the k-th chunk of this block from the global counter and tells the consumers: the id
+    // travels through shared memory and the arrive on the chunk's first tile publishes it.  The queue
+    // cannot wrap onto an unread entry: the producer is at most `stages` tiles, hence chunks, ahead.
+    // Returns false when no chunk is left (the consumers are told) or a wait ran out.
+    __device__ __forceinline__ bool next_chunk(long long k, long long *chunk)
+    {
+        const long long taken = (long long)atomicAdd(&a.sched[0], 1ull);
+        const bool last = taken >= a.n_full_chunks;
+        *chunk = a.first_chunk + taken;
+        if (!stage_free()) return false;
+        sh->chunk_queue[k % (kMaxStages + 2)] = last ? -1 : *chunk;
+        if (last) mbar_arrive(smem_addr(&sh->full[s]));   // an empty "tile": wakes the consumers to read the -1
+        return !last;
+    }
+    __device__ __forceinline__ uint32_t stage_addr() const { return smem_addr(ring + (size_t)s * stage_bytes); }
+    __device__ __forceinline__ uint32_t full_barrier() const { return smem_addr(&sh->full[s]); }
+    // The current stage's copies have been issued.
+    __device__ __forceinline__ void advance()
+    {
+        ++issued;
+        if (++s == a.stages) { s = 0; phase ^= 1u; }
+        if (a.test_stop_after_tiles > 0 && issued >= a.test_stop_after_tiles) ok = false;
+    }
+    // After the last chunk, or after giving up: let copies still in flight land before the block's
+    // shared memory is released, and let the last block to finish rearm the counters.
+    __device__ __forceinline__ void finish()
+    {
+        if (!ok) {
+            const long long R = a.stages, outstanding = issued < R ? issued : R;
+            for (long long k = 1; k <= outstanding; ++k) {
+                const long long q = issued - k;                      // sequence number of an issued tile
+                const uint32_t bar = smem_addr(&sh->full[q % R]);
+                const uint32_t par = (uint32_t)((q / R) & 1);
+                const unsigned long long start = global_timer_ns();
+                while (!mbar_try_wait(bar, par) && global_timer_ns() - start < a.wait_limit_ns) {}
+            }
+        }
+        if (atomicAdd(&a.sched[1], 1ull) == gridDim.x - 1) {
+            a.sched[0] = 0;
+            a.sched[1] = 0;
+        }
+    }
+};
+
 }  // namespace
 
 template <int TILES, bool DO_VAR>
@@ -168,47 +249,22 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     volatile int *abort_flag = &sh->abort;
 
-    if (tid == 0) {
-        for (int s = 0; s < R; ++s) {
-            mbar_init(smem_addr(&sh->full[s]), 1);
-            mbar_init(smem_addr(&sh->empty[s]), kConsumerWarps);
-        }
-        sh->abort = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-    __syncthreads();
+    ring_init(sh, R);
 
     if (warp == kConsumerWarps) {
         // ------------------------------ producer ------------------------------
         if (lane != 0) return;
-        int s = 0;
-        uint32_t phase = 0;
-        long long issued = 0;
-        bool ok = true;
-        for (long long k = 0; ok; ++k) {
-            const long long taken = (long long)atomicAdd(&a.sched[0], 1ull);
-            const bool last = taken >= a.n_full_chunks;
-            const long long chunk = a.first_chunk + taken;
-            // The chunk id travels to the consumers through shared memory; the arrive on the
-            // first tile's barrier below publishes it.  The queue cannot wrap onto an unread
-            // entry: the producer is at most `stages` tiles, hence chunks, ahead.
-            if (!mbar_wait(smem_addr(&sh->empty[s]), phase ^ 1u, abort_flag, a.error_flag, a.wait_limit_ns)) { ok = false; break; }
-            sh->chunk_queue[k % (kMaxStages + 2)] = last ? -1 : chunk;
-            if (last) {
-                mbar_arrive(smem_addr(&sh->full[s]));       // an empty "tile": wakes the consumers to read the -1
-                break;
-            }
+        RingProducer p(a, sh, ring, kStageBytes);
+        const uint32_t g_elem = (a.grad_fmt & kGradTypeMask) == kGradF32 ? 4u : 2u;
+        long long chunk;
+        for (long long k = 0; p.ok && p.next_chunk(k, &chunk); ++k) {
             const long long c0 = chunk * st.chunk;
-            for (int i = 0; ok && i <= W; ++i) {            // i == W: the server's tiles
-                for (int t = 0; t < TILES; ++t) {
-                    const uint32_t full = smem_addr(&sh->full[s]);
-                    if (!mbar_wait(smem_addr(&sh->empty[s]), phase ^ 1u, abort_flag, a.error_flag, a.wait_limit_ns)) { ok = false; break; }
-                    const uint32_t dst = smem_addr(ring + (size_t)s * kStageBytes);
+            for (int i = 0; p.ok && i <= W; ++i) {          // i == W: the server's tiles
+                for (int t = 0; t < TILES && p.stage_free(); ++t) {
+                    const uint32_t full = p.full_barrier(), dst = p.stage_addr();
                     const long long off = c0 + (long long)t * kTile;
                     if (i < W) {
                         const long long row = (long long)i * st.n_pad + off;
-                        const uint32_t g_elem = (a.grad_fmt & kGradTypeMask) == kGradF32 ? 4u : 2u;
                         mbar_arrive_expect_tx(full, 3 * kTileBytes + kTile * g_elem);
                         bulk_load(dst, reinterpret_cast<const char *>(a.g.p[i]) + off * g_elem, kTile * g_elem, full);
                         bulk_load(dst + kTileBytes, st.m + row, kTileBytes, full);
@@ -220,28 +276,11 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
                         bulk_load(dst + kTileBytes, st.v + off, kTileBytes, full);
                         bulk_load(dst + 2 * kTileBytes, st.xs + off, kTileBytes, full);
                     }
-                    ++issued;
-                    if (++s == R) { s = 0; phase ^= 1u; }
-                    if (a.test_stop_after_tiles > 0 && issued >= a.test_stop_after_tiles) { ok = false; break; }
+                    p.advance();
                 }
             }
         }
-        if (!ok) {
-            // Aborted: let the copies still in flight land before the block's shared memory is released.
-            const long long outstanding = issued < R ? issued : R;
-            for (long long k = 1; k <= outstanding; ++k) {
-                const long long q = issued - k;                      // sequence number of an issued tile
-                const uint32_t bar = smem_addr(&sh->full[q % R]);
-                const uint32_t par = (uint32_t)((q / R) & 1);
-                const unsigned long long start = global_timer_ns();
-                while (!mbar_try_wait(bar, par) && global_timer_ns() - start < a.wait_limit_ns) {}
-            }
-        }
-        // The last block to finish taking chunks rearms the counters for the next launch.
-        if (atomicAdd(&a.sched[1], 1ull) == gridDim.x - 1) {
-            a.sched[0] = 0;
-            a.sched[1] = 0;
-        }
+        p.finish();
         return;
     }
 
@@ -450,41 +489,19 @@ __global__ void __launch_bounds__(kThreads, 1) alg2_pipelined_kernel(const __gri
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     volatile int *abort_flag = &sh->abort;
 
-    if (tid == 0) {
-        for (int s = 0; s < R; ++s) {
-            mbar_init(smem_addr(&sh->full[s]), 1);
-            mbar_init(smem_addr(&sh->empty[s]), kConsumerWarps);
-        }
-        sh->abort = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-    __syncthreads();
+    ring_init(sh, R);
 
     if (warp == kConsumerWarps) {
         // ------------------------------ producer ------------------------------
         if (lane != 0) return;
-        int s = 0;
-        uint32_t phase = 0;
-        long long issued = 0;
-        bool ok = true;
+        RingProducer p(a, sh, ring, kStage2Bytes);
         const uint32_t g_elem = (a.grad_fmt & kGradTypeMask) == kGradF32 ? 4u : 2u;
-        for (long long k = 0; ok; ++k) {
-            const long long taken = (long long)atomicAdd(&a.sched[0], 1ull);
-            const bool last = taken >= a.n_full_chunks;
-            const long long chunk = a.first_chunk + taken;
-            if (!mbar_wait(smem_addr(&sh->empty[s]), phase ^ 1u, abort_flag, a.error_flag, a.wait_limit_ns)) { ok = false; break; }
-            sh->chunk_queue[k % (kMaxStages + 2)] = last ? -1 : chunk;
-            if (last) {
-                mbar_arrive(smem_addr(&sh->full[s]));
-                break;
-            }
+        long long chunk;
+        for (long long k = 0; p.ok && p.next_chunk(k, &chunk); ++k) {
             const long long c0 = chunk * st.chunk;
-            for (int i = 0; ok && i <= 2 * W; ++i) {        // i < W: (g, delta); i == W: (delta_bar, v); i > W: (m, x)
-                for (int t = 0; t < TILES; ++t) {
-                    const uint32_t full = smem_addr(&sh->full[s]);
-                    if (!mbar_wait(smem_addr(&sh->empty[s]), phase ^ 1u, abort_flag, a.error_flag, a.wait_limit_ns)) { ok = false; break; }
-                    const uint32_t dst = smem_addr(ring + (size_t)s * kStage2Bytes);
+            for (int i = 0; p.ok && i <= 2 * W; ++i) {      // i < W: (g, delta); i == W: (delta_bar, v); i > W: (m, x)
+                for (int t = 0; t < TILES && p.stage_free(); ++t) {
+                    const uint32_t full = p.full_barrier(), dst = p.stage_addr();
                     const long long off = c0 + (long long)t * kTile;
                     if (i < W) {
                         mbar_arrive_expect_tx(full, kTileBytes + kTile * g_elem);
@@ -500,26 +517,11 @@ __global__ void __launch_bounds__(kThreads, 1) alg2_pipelined_kernel(const __gri
                         bulk_load(dst, st.m + row, kTileBytes, full);
                         bulk_load(dst + kTileBytes, st.x + row, kTileBytes, full);
                     }
-                    ++issued;
-                    if (++s == R) { s = 0; phase ^= 1u; }
-                    if (a.test_stop_after_tiles > 0 && issued >= a.test_stop_after_tiles) { ok = false; break; }
+                    p.advance();
                 }
             }
         }
-        if (!ok) {
-            const long long outstanding = issued < R ? issued : R;
-            for (long long k = 1; k <= outstanding; ++k) {
-                const long long q = issued - k;
-                const uint32_t bar = smem_addr(&sh->full[q % R]);
-                const uint32_t par = (uint32_t)((q / R) & 1);
-                const unsigned long long start = global_timer_ns();
-                while (!mbar_try_wait(bar, par) && global_timer_ns() - start < a.wait_limit_ns) {}
-            }
-        }
-        if (atomicAdd(&a.sched[1], 1ull) == gridDim.x - 1) {
-            a.sched[0] = 0;
-            a.sched[1] = 0;
-        }
+        p.finish();
         return;
     }
 
