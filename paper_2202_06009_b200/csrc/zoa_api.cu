@@ -8,6 +8,8 @@
 #include <string>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "../../include/zoa.h"
 #include "zoa_internal.h"
 
@@ -43,6 +45,12 @@ struct zoa_handle_s {
     struct Guarded { char *ptr; size_t bytes, padded; };
     std::vector<Guarded> guarded;  // every device buffer: user pointer, payload bytes, payload rounded up to 256
     std::string err;
+};
+
+// Named range around an entry point, for profilers (costs a pointer test when none is attached).
+struct TraceRange {
+    explicit TraceRange(const char *name) { nvtxRangePushA(name); }
+    ~TraceRange() { nvtxRangePop(); }
 };
 
 static std::string g_create_error;
@@ -426,6 +434,7 @@ static zoa_status run_sync_range(zoa_handle h, const StateView &st, const GradPt
 
 extern "C" zoa_status zoa_step(zoa_handle h, const void *const *grads, float lr, int64_t t, void *stream)
 {
+    TraceRange trace("zoa_step");
     GradPtrs gp;
     int aligned;   // gradient format code: alignment bit and element type
     zoa_status rc = check_step_args(h, grads, lr, t, &gp, &aligned, "zoa_step");
@@ -443,6 +452,7 @@ extern "C" zoa_status zoa_step(zoa_handle h, const void *const *grads, float lr,
 
 extern "C" zoa_status zoa_onebit_reduce(zoa_handle h, void *stream)
 {
+    TraceRange trace("zoa_onebit_reduce");
     if (!h) return ZOA_ERR_ARG;
     const float gamma_sum = (float)h->gamma_sum;
     if (!(h->gamma_sum > 0.0) || !(gamma_sum > 0.f) || !std::isfinite(gamma_sum))
@@ -527,6 +537,7 @@ extern "C" zoa_status zoa_dist_variance(zoa_handle h, const float *g_bar, void *
 
 extern "C" zoa_status zoa_step_sync(zoa_handle h, const void *const *grads, float lr, int64_t t, void *stream)
 {
+    TraceRange trace("zoa_step_sync");
     GradPtrs gp;
     int aligned;   // gradient format code: alignment bit and element type
     zoa_status rc = check_step_args(h, grads, lr, t, &gp, &aligned, "zoa_step_sync");
@@ -575,6 +586,7 @@ extern "C" zoa_status zoa_step_sync(zoa_handle h, const void *const *grads, floa
 
 extern "C" zoa_status zoa_alg2_step(zoa_handle h, const void *const *grads, float lr, int64_t t, void *stream)
 {
+    TraceRange trace("zoa_alg2_step");
     GradPtrs gp;
     int aligned;   // gradient format code: alignment bit and element type
     zoa_status rc = check_step_args(h, grads, lr, t, &gp, &aligned, "zoa_alg2_step");
@@ -619,6 +631,7 @@ extern "C" zoa_status zoa_step_auto(zoa_handle h, const void *const *grads, floa
 extern "C" zoa_status zoa_step_host(zoa_handle h, const void *const *host_grads, float lr, int64_t t,
                                     float *host_x_out, void *stream)
 {
+    TraceRange trace("zoa_step_host");
     if (!h) return ZOA_ERR_ARG;
     if (!host_grads) return fail(h, ZOA_ERR_ARG, "zoa_step_host: host_grads is NULL");
     for (int i = 0; i < h->W; ++i)
