@@ -393,7 +393,7 @@ def run_worker_per_gpu(args, wl):
 # ---- kernel sweep: worker compression and W-way decompress-average on flat vectors ---------
 def run_sweep(args):
     """Times zoa_onebit_compress (Algorithm 3, worker side) and zoa_onebit_average (server
-    side + lines 8-10 of Algorithm 1) alone, for n = 2^20 .. 2^30 in powers of 4,
+    side + the post-sync updates of Algorithm 1) alone, for n = 2^20 .. 2^30 in powers of 4,
     W in {2,4,8,16}, chunk in {1024,4096,16384}; inputs N(0,1) with 1 % of the elements
     scaled by 100.  One JSON line per combination."""
     import torch

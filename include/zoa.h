@@ -63,7 +63,7 @@ typedef struct {
     double gamma_sum;       /* learning rates accumulated into u since the last sync */
 } zoa_stats;
 
-/* Algorithm 1, "Require" line: creates the state for a d = n_params
+/* The inputs of Algorithm 1 (its "Require" clause): creates the state for a d = n_params
  * dimensional model on W workers with m_0 = v_0 = u_0 = 0, both compression
  * errors 0 (Algorithm 3), x_0 = 0 until zoa_set_params, t' = 0, on the current
  * CUDA device.  chunk is the number of consecutive coordinates that share one
@@ -122,26 +122,27 @@ zoa_status zoa_set_sync_policy(zoa_handle h, const int64_t *boundaries, const in
 int zoa_sync_due(zoa_handle h, int64_t t);
 int zoa_var_due(zoa_handle h, int64_t t);
 
-/* Algorithm 1 lines 3-5 for every worker, and lines 14-15 when t is in T_v
+/* Algorithm 1: the momentum, model and buffer updates for every worker, and the
+ * variance update (full-precision mean of the gradients, then v) when t is in T_v
  * (the new variance takes effect from the next step on, so that a following
- * zoa_onebit_reduce still uses v_t as line 9 does).
+ * zoa_onebit_reduce still uses v_t as the algorithm's model sync does).
  * grads: (host) array of W (device) pointers, n_params elements each (binary32
  * unless ZOA_OPT_GRAD_TYPE says otherwise), worker i's gradient at step t;
  * 16-byte aligned pointers take the vector path.
  * lr is gamma_t; t must be larger than at the previous step. */
 zoa_status zoa_step(zoa_handle h, const void *const *grads, float lr, int64_t t, void *stream);
 
-/* Algorithm 1 lines 7-11 with Algorithm 3 inside: compresses u + delta per
+/* Algorithm 1's sync branch (t in T_u) with Algorithm 3 inside: compresses u + delta per
  * worker (Eq. 3 per chunk), averages, compresses again on the "server" with its
  * own error, then m = u_bar / sum(gamma), x = x_sync - u_bar / sqrt(v_t + eps),
  * u = 0 on every worker.  ZOA_ERR_STATE if nothing was accumulated since the
- * last sync (the divisor of line 8 would be zero). */
+ * last sync (the divisor of the momentum approximation would be zero). */
 zoa_status zoa_onebit_reduce(zoa_handle h, void *stream);
 
 /* The two halves of zoa_onebit_reduce, for callers that want to time or
  * interleave them: zoa_onebit_compress is the worker side of Algorithm 3 (packs
  * u + delta of every worker into words_w / scales_w, keeps the errors);
- * zoa_onebit_average is the server side and lines 8-11 of Algorithm 1 (reads
+ * zoa_onebit_average is the server side and the rest of Algorithm 1's sync branch (reads
  * words_w / scales_w).  compress then average == zoa_onebit_reduce. */
 zoa_status zoa_onebit_compress(zoa_handle h, void *stream);
 zoa_status zoa_onebit_average(zoa_handle h, void *stream);
@@ -156,14 +157,14 @@ zoa_status zoa_onebit_average(zoa_handle h, void *stream);
  *   -- all-to-all of each range's words and scales --
  *   zoa_dist_server_range                  server side for this GPU's chunk range
  *   -- all-gather of words_s / scales_s into every handle's own buffers --
- *   zoa_dist_apply                         lines 8-11 of Algorithm 1 from words_s / scales_s
+ *   zoa_dist_apply                         rest of Algorithm 1's sync branch from words_s / scales_s
  * zoa_dist_server_range: words_all / scales_all (device) hold, for each of the
  * W_total workers in worker order, the packed words and the magnitudes of the
  * chunks [first_chunk, first_chunk + n_chunks), rows words_stride / scales_stride
  * elements apart, starting at the range's first word / chunk.  It updates the
  * server error of that range and writes that range of words_s / scales_s.
  * Chunks above 16384 are not supported here.
- * zoa_dist_variance: lines 14-15 of Algorithm 1 when the mean gradient g_bar
+ * zoa_dist_variance: the variance update of Algorithm 1 when the mean gradient g_bar
  * (device, n_params floats) comes from a collective; call it after zoa_step on a
  * step in T_v for which the handle's own T_v list is empty.  A collective's
  * binary32 sum is not the binary64 worker-order sum of the single-GPU path, so v

@@ -27,19 +27,20 @@
  * once at the end.
  *
  * Readings taken where the paper is silent, ambiguous or misprinted:
- *  R1  Lines 4-5 of Algorithm 1 print m_t, the momentum before line 3.  Read
- *      literally with a sync at every step, line 8 overwrites m_{t+1} with the
+ *  R1  The model and buffer updates of Algorithm 1 print m_t, the momentum before
+ *      the momentum update.  Read literally with a sync at every step, the
+ *      momentum approximation of the sync branch overwrites m_{t+1} with the
  *      mean of m_t, so the gradient never enters m and the model never moves.
  *      The derivation in Section 4 (u_t = sum_k gamma_k m_k with m_k the
  *      momentum of step k) and the non-sync branch m_{t+1} = m_{t+1/2} need
  *      m_{t+1/2}.  We use m_{t+1/2}; `literal_momentum` = 1 selects the printed
  *      form so that a test can show it is degenerate.
- *  R2  The divisor on line 8, sum_{h=t'}^{t} gamma_h, is taken as the sum of
+ *  R2  The divisor of the momentum approximation, sum_{h=t'}^{t} gamma_h, is taken as the sum of
  *      the gamma_h that were actually accumulated into u since u was last
  *      reset (the inclusive printed range would count gamma_{t'} twice).
- *  R3  x_{t'} on line 9 is the model produced by the sync at step t' (x_0
+ *  R3  x_{t'} in the model sync is the model produced by the sync at step t' (x_0
  *      before the first sync).
- *  R4  The server line of Algorithm 3 prints \hat z_{t+1} inside C[.] and
+ *  R4  The server step of Algorithm 3 prints \hat z_{t+1} inside C[.] and
  *      \hat z_t in the error update; both are the buffers just received.
  *  R5  C[.] is applied per chunk of `chunk` consecutive coordinates of the flat
  *      vector, the last chunk dividing by its true length.  chunk >= d gives
@@ -49,7 +50,7 @@
  *  R7  Wire format: coordinate j is bit (j mod 32), least significant first,
  *      of 32-bit word floor(j/32); unused bits of the last word are 0; one
  *      scale per chunk.
- *  R8  Line 9 uses v_t; line 15 assigns v_{t+1} afterwards.
+ *  R8  The model sync uses v_t; the variance update assigns v_{t+1} afterwards.
  *  R9  Algorithm 2 also prints m_t in its model update.  It is introduced as the
  *      special case of Algorithm 1 without local steps, so it takes the same
  *      convention as R1: the momentum just computed.  (With the identity
@@ -106,7 +107,7 @@ typedef struct {
     int64_t chunk;            /* coordinates sharing one scale (R5) */
     real beta1, beta2, eps;
     int32_t compressor;       /* ZO_COMPRESSOR_* */
-    int32_t literal_momentum; /* R1: 1 = use m_t on lines 4-5 as printed */
+    int32_t literal_momentum; /* R1: 1 = use m_t in the model and buffer updates, as printed */
     real *x;                  /* [n][d] local models x^(i) */
     real *m;                  /* [n][d] momentum m^(i) */
     real *u;                  /* [n][d] auxiliary buffer u^(i) */
@@ -194,7 +195,7 @@ void ZO(zo_allreduce)(const real *g, int32_t n, int64_t d, real *g_bar)
     }
 }
 
-/* Algorithm 1, lines 3-5: momentum, local model step, buffer accumulation. */
+/* Algorithm 1, first half of an iteration: momentum update, local model update, buffer update. */
 void ZO(zo_alg1_half_step)(ZO(zo_state) *st, const real *g, real gamma)
 {
     const real one_minus_beta1 = (real)1 - st->beta1;
@@ -202,63 +203,63 @@ void ZO(zo_alg1_half_step)(ZO(zo_state) *st, const real *g, real gamma)
         for (int64_t j = 0; j < st->d; ++j) {
             size_t k = (size_t)i * st->d + j;
             real m_prev = st->m[k];
-            real m_half = st->beta1 * m_prev + one_minus_beta1 * g[k];     /* line 3 */
+            real m_half = st->beta1 * m_prev + one_minus_beta1 * g[k];     /* momentum update */
             real m_used = st->literal_momentum ? m_prev : m_half;          /* R1 */
             real step = gamma * m_used;
-            st->x[k] = st->x[k] - step / ZO(zo_sqrt)(st->v[j] + st->eps);    /* line 4 */
-            st->u[k] = st->u[k] + step;                                    /* line 5 */
+            st->x[k] = st->x[k] - step / ZO(zo_sqrt)(st->v[j] + st->eps);    /* model update */
+            st->u[k] = st->u[k] + step;                                    /* buffer update */
             st->m[k] = m_half;
         }
     st->gamma_sum += (double)gamma;                                        /* R2 */
 }
 
-/* Algorithm 1, lines 7-11.  Returns 0, or -1 when nothing was accumulated
- * since the last sync (the divisor of line 8 would be zero). */
+/* Algorithm 1, the sync branch (t in T_u).  Returns 0, or -1 when nothing was accumulated
+ * since the last sync (the divisor of the momentum approximation would be zero). */
 int ZO(zo_alg1_sync)(ZO(zo_state) *st, int64_t t)
 {
     if (!(st->gamma_sum > 0.0)) return -1;
     const real gamma_sum = (real)st->gamma_sum;
-    ZO(zo_onebit_allreduce)(st, st->u);                                    /* line 7 */
+    ZO(zo_onebit_allreduce)(st, st->u);                                    /* 1-bit AllReduce */
     for (int64_t j = 0; j < st->d; ++j) {
-        real m_next = st->u_bar[j] / gamma_sum;                            /* line 8 */
-        real x_next = st->x_sync[j] - st->u_bar[j] / ZO(zo_sqrt)(st->v[j] + st->eps); /* line 9 */
+        real m_next = st->u_bar[j] / gamma_sum;                            /* momentum approximation */
+        real x_next = st->x_sync[j] - st->u_bar[j] / ZO(zo_sqrt)(st->v[j] + st->eps); /* model sync */
         for (int i = 0; i < st->n; ++i) {
             size_t k = (size_t)i * st->d + j;
             st->m[k] = m_next;
             st->x[k] = x_next;
-            st->u[k] = (real)0;                                            /* line 10 */
+            st->u[k] = (real)0;                                            /* buffer reset */
         }
         st->x_sync[j] = x_next;                                            /* R3 */
     }
     st->gamma_sum = 0.0;
-    st->t_sync = t;                                                        /* line 11 */
+    st->t_sync = t;                                                        /* t' = t */
     return 0;
 }
 
-/* Algorithm 1, lines 14-15. */
+/* Algorithm 1, the variance branch (t in T_v). */
 void ZO(zo_alg1_variance)(ZO(zo_state) *st, const real *g, real *g_bar_scratch)
 {
     const real one_minus_beta2 = (real)1 - st->beta2;
-    ZO(zo_allreduce)(g, st->n, st->d, g_bar_scratch);                      /* line 14 */
+    ZO(zo_allreduce)(g, st->n, st->d, g_bar_scratch);                      /* full-precision AllReduce */
     for (int64_t j = 0; j < st->d; ++j) {
         real g_bar = g_bar_scratch[j];
-        st->v[j] = st->beta2 * st->v[j] + one_minus_beta2 * (g_bar * g_bar); /* line 15 */
+        st->v[j] = st->beta2 * st->v[j] + one_minus_beta2 * (g_bar * g_bar); /* variance update */
     }
 }
 
-/* One iteration t of Algorithm 1 (lines 2-19) given the gradients g^(i)_t.
+/* One whole iteration t of Algorithm 1 given the gradients g^(i)_t.
  * g_bar_scratch is [d]. */
 int ZO(zo_alg1_step)(ZO(zo_state) *st, const real *g, real gamma, int64_t t,
                      int in_T_u, int in_T_v, real *g_bar_scratch)
 {
     int rc = 0;
     ZO(zo_alg1_half_step)(st, g, gamma);
-    if (in_T_u) rc = ZO(zo_alg1_sync)(st, t);   /* else line 13: keep the half-step values */
-    if (in_T_v) ZO(zo_alg1_variance)(st, g, g_bar_scratch); /* else line 18: v stays (R8) */
+    if (in_T_u) rc = ZO(zo_alg1_sync)(st, t);   /* else: keep the half-step values */
+    if (in_T_v) ZO(zo_alg1_variance)(st, g, g_bar_scratch); /* else: v stays (R8) */
     return rc;
 }
 
-/* One iteration t of Algorithm 2 (lines 2-11).  On a T_v step the workers
+/* One whole iteration t of Algorithm 2.  On a T_v step the workers
  * exchange full-precision gradients (Algorithm 4) and the variance moves; on
  * any other step they exchange 1-bit compressed gradients (Algorithm 3).
  * Momentum and model are the same on every worker; they are kept per worker
@@ -268,21 +269,21 @@ void ZO(zo_alg2_step)(ZO(zo_state) *st, const real *g, real gamma, int in_T_v, r
     const real one_minus_beta1 = (real)1 - st->beta1, one_minus_beta2 = (real)1 - st->beta2;
     const real *g_bar = g_bar_scratch;
     if (in_T_v) {
-        ZO(zo_allreduce)(g, st->n, st->d, g_bar_scratch);                  /* line 4 */
+        ZO(zo_allreduce)(g, st->n, st->d, g_bar_scratch);                  /* model update */
     } else {
-        ZO(zo_onebit_allreduce)(st, g);                                    /* line 7 */
+        ZO(zo_onebit_allreduce)(st, g);                                    /* 1-bit AllReduce */
         g_bar = st->u_bar;
     }
     for (int i = 0; i < st->n; ++i)
         for (int64_t j = 0; j < st->d; ++j) {
             size_t k = (size_t)i * st->d + j;
             real m_prev = st->m[k];
-            real m_next = st->beta1 * m_prev + one_minus_beta1 * g_bar[j]; /* line 10 */
+            real m_next = st->beta1 * m_prev + one_minus_beta1 * g_bar[j]; /* buffer reset */
             real m_used = st->literal_momentum ? m_prev : m_next;          /* R9 */
-            st->x[k] = st->x[k] - (gamma * m_used) / ZO(zo_sqrt)(st->v[j] + st->eps); /* line 11 */
+            st->x[k] = st->x[k] - (gamma * m_used) / ZO(zo_sqrt)(st->v[j] + st->eps); /* t' = t */
             st->m[k] = m_next;
         }
     if (in_T_v)
         for (int64_t j = 0; j < st->d; ++j)
-            st->v[j] = st->beta2 * st->v[j] + one_minus_beta2 * (g_bar[j] * g_bar[j]); /* line 5 */
+            st->v[j] = st->beta2 * st->v[j] + one_minus_beta2 * (g_bar[j] * g_bar[j]); /* buffer update */
 }

@@ -386,7 +386,7 @@ static cudaError_t run_server(zoa_handle h, float gamma_sum, cudaStream_t s)
     return e;
 }
 
-// Lines 3-5 (+ 14-15) for the chunks [c0, c1).
+// The local updates of Algorithm 1 (+ the variance update) for the chunks [c0, c1).
 static zoa_status run_local_range(zoa_handle h, const StateView &st, const GradPtrs &gp, float lr, bool do_var, int fmt,
                                   long long c0, long long c1, cudaStream_t s)
 {
@@ -409,7 +409,7 @@ static zoa_status run_sync_range(zoa_handle h, const StateView &st, const GradPt
     // one-block-per-chunk kernel starts faster (measured on a 512-chunk problem).
     const bool enough_chunks = h->use_pipeline == 2 || n_full >= 4ll * h->sm_count;
     const int stages = h->use_pipeline && enough_chunks && n_full > 0 ? pipeline_stages(st, fmt) : 0;
-    long long var_first = e0;     // coordinates from here to e1 still need lines 14-15
+    long long var_first = e0;     // coordinates from here to e1 still need the variance update
     if (stages > 0) {
         bool var_fused = false;
         ZOA_CUDA(h, launch_step_sync_pipelined(st, gp, h->c, lr, gamma_sum, do_var, fmt, c0, n_full, stages, h->sm_count,

@@ -45,14 +45,14 @@ __device__ __forceinline__ float f_mul(float a, float b) { return __fmul_rn(a, b
 __device__ __forceinline__ float f_div(float a, float b) { return __fdiv_rn(a, b); }
 __device__ __forceinline__ float f_sqrt(float a) { return __fsqrt_rn(a); }
 
-// Algorithm 1 line 3: m_{t+1/2} = beta1 m_t + (1 - beta1) g_t.
+// Momentum update of Algorithm 1: m_{t+1/2} = beta1 m_t + (1 - beta1) g_t.
 __device__ __forceinline__ float momentum(const Consts &c, float m, float g)
 {
     return f_add(f_mul(c.b1, m), f_mul(c.ob1, g));
 }
-// Denominator of lines 4 and 9: sqrt(v_t + eps).
+// Denominator of both model updates of Algorithm 1: sqrt(v_t + eps).
 __device__ __forceinline__ float denom(const Consts &c, float v) { return f_sqrt(f_add(v, c.eps)); }
-// Algorithm 1 line 15: v_{t+1} = beta2 v_t + (1 - beta2) g_bar^2.
+// Variance update of Algorithm 1: v_{t+1} = beta2 v_t + (1 - beta2) g_bar^2.
 __device__ __forceinline__ float variance(const Consts &c, float v, float g_bar)
 {
     return f_add(f_mul(c.b2, v), f_mul(c.ob2, f_mul(g_bar, g_bar)));

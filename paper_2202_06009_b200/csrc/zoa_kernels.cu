@@ -1,13 +1,13 @@
 // The zoa kernels other than the bulk-copy ring kernel (zoa_pipeline.cu).
 //
 // Elementwise, one float4 per thread:
-//   local_step_kernel        Algorithm 1 lines 3-5 (+ lines 14-15 on T_v steps)
-//   variance_kernel          Algorithm 1 lines 14-15 alone
+//   local_step_kernel        Algorithm 1: momentum, model and buffer updates (+ variance update on T_v steps)
+//   variance_kernel          Algorithm 1: the variance update alone
 //   alg2_full_kernel         Algorithm 2 on a T_v step (full-precision exchange)
 // One block per chunk (any chunk that is a multiple of 32 up to 16384, ragged last
 // chunk, unaligned or 16-bit gradient buffers):
 //   compress_kernel          Algorithm 3 worker side (Eq. 3 per chunk, error feedback)
-//   reduce_kernel            Algorithm 3 server side + Algorithm 1 lines 8-10
+//   reduce_kernel            Algorithm 3 server side + Algorithm 1: momentum approximation, model sync, buffer reset
 //   step_sync_kernel         a whole sync step of Algorithm 1 in one pass over memory
 //   alg2_compressed_kernel   Algorithm 2 on any other step (gradients through Algorithm 3)
 // Chunks larger than a block can hold, up to the whole vector (Eq. 3 as printed):
@@ -46,10 +46,10 @@ local_step_kernel(StateView st, GradPtrs g, Consts c, float gamma, int g_fmt_arg
             float mo[4], xo[4], uo[4];
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                mo[k] = momentum(c, mm[k], gg[k]);              // line 3
+                mo[k] = momentum(c, mm[k], gg[k]);              // momentum update
                 const float s = f_mul(gamma, mo[k]);
-                xo[k] = f_sub(xx[k], f_div(s, d[k]));           // line 4
-                uo[k] = f_add(uu[k], s);                        // line 5
+                xo[k] = f_sub(xx[k], f_div(s, d[k]));           // model update
+                uo[k] = f_add(uu[k], s);                        // buffer update
                 if (DO_VAR) G[k] += (double)gg[k];
             }
             st4(st.m + row, make_float4(mo[0], mo[1], mo[2], mo[3]));
@@ -60,7 +60,7 @@ local_step_kernel(StateView st, GradPtrs g, Consts c, float gamma, int g_fmt_arg
             const float vv[4] = {v4.x, v4.y, v4.z, v4.w};
             float vo[4];
 #pragma unroll
-            for (int k = 0; k < 4; ++k) vo[k] = variance(c, vv[k], mean_round(G[k], st.W));  // lines 14-15
+            for (int k = 0; k < 4; ++k) vo[k] = variance(c, vv[k], mean_round(G[k], st.W));  // variance update
             st4(st.v_next + j, make_float4(vo[0], vo[1], vo[2], vo[3]));
         }
     }
@@ -158,7 +158,7 @@ __global__ void compress_kernel(StateView st)
     if (threadIdx.x == 0) st.scales_w[(long long)i * st.n_chunks + blockIdx.x] = scale;
 }
 
-// Server side of Algorithm 3 and lines 8-10 of Algorithm 1 for one tile whose
+// Server side of Algorithm 3 and the post-sync updates of Algorithm 1 for one tile whose
 // server input a[k] is known: compress it, keep the server error, rebuild m and x,
 // clear u, on every worker.  `scale` is the chunk's server magnitude.
 __device__ __forceinline__ void server_tile(const StateView &st, const Consts &c, const ChunkGeom &cg,
@@ -177,8 +177,8 @@ __device__ __forceinline__ void server_tile(const StateView &st, const Consts &c
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
         const bool valid = idx + k < cg.len;
-        mo[k] = valid ? f_div(hat[k], gamma_sum) : 0.0f;                        // line 8
-        xo[k] = valid ? f_sub(xs[k], f_div(hat[k], denom(c, vv[k]))) : 0.0f;    // line 9
+        mo[k] = valid ? f_div(hat[k], gamma_sum) : 0.0f;                        // momentum approximation
+        xo[k] = valid ? f_sub(xs[k], f_div(hat[k], denom(c, vv[k]))) : 0.0f;    // model sync
     }
     const float4 m4 = make_float4(mo[0], mo[1], mo[2], mo[3]);
     const float4 x4 = make_float4(xo[0], xo[1], xo[2], xo[3]);
@@ -188,7 +188,7 @@ __device__ __forceinline__ void server_tile(const StateView &st, const Consts &c
         const long long row = (long long)i * st.n_pad + j;
         st4(st.m + row, m4);
         st4(st.x + row, x4);
-        st4(st.u + row, zero);                                                   // line 10
+        st4(st.u + row, zero);                                                   // buffer reset
     }
 }
 
@@ -242,9 +242,9 @@ __global__ void reduce_kernel(StateView st, Consts c, float gamma_sum)
     if (threadIdx.x == 0) st.scales_s[blockIdx.x] = scale;
 }
 
-// A whole sync step for chunk blockIdx.x: lines 3-5 in registers, worker
-// compression, server, lines 8-10.  The half-step m, x, u never reach memory;
-// x is not even read (line 9 rebuilds it from x_sync).
+// A whole sync step for chunk blockIdx.x: the local updates in registers, worker
+// compression, server, the post-sync updates.  The half-step m, x, u never reach memory;
+// x is not even read (the model sync rebuilds it from x_sync).
 __global__ void step_sync_kernel(StateView st, GradPtrs g, Consts c, float gamma, float gamma_sum,
                                  int g_aligned, long long chunk_offset)
 {
@@ -275,7 +275,7 @@ __global__ void step_sync_kernel(StateView st, GradPtrs g, Consts c, float gamma
                 float z[4];
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
-                    const float s = f_mul(gamma, momentum(c, mm[k], gg[k]));     // lines 3, 5
+                    const float s = f_mul(gamma, momentum(c, mm[k], gg[k]));     // momentum update, buffer update
                     z[k] = f_add(f_add(uu[k], s), ee[k]);                        // u_{t+1/2} + delta
                     l1 += fabs((double)z[k]);
                 }
@@ -392,7 +392,7 @@ __global__ void dist_server_kernel(StateView st, const uint32_t *words_in, long 
     if (threadIdx.x == 0) st.scales_s[chunk_id] = scale;
 }
 
-// Lines 8-10 of Algorithm 1 from the server's packed result (words_s, scales_s of the whole
+// The post-sync updates of Algorithm 1 from the server's packed result (words_s, scales_s of the whole
 // vector): m = u_bar / sum(gamma), x = x_sync - u_bar / sqrt(v + eps), u = 0, on this GPU's workers.
 __global__ void __launch_bounds__(256)
 dist_apply_kernel(StateView st, Consts c, float gamma_sum)
@@ -410,8 +410,8 @@ dist_apply_kernel(StateView st, Consts c, float gamma_sum)
         for (int k = 0; k < 4; ++k) {
             const bool valid = j + k < st.n;
             const float hat = ((nib >> k) & 1u) ? scale : -scale;
-            mo[k] = valid ? f_div(hat, gamma_sum) : 0.0f;                       // line 8
-            xo[k] = valid ? f_sub(xs[k], f_div(hat, denom(c, vv[k]))) : 0.0f;   // line 9
+            mo[k] = valid ? f_div(hat, gamma_sum) : 0.0f;                       // momentum approximation
+            xo[k] = valid ? f_sub(xs[k], f_div(hat, denom(c, vv[k]))) : 0.0f;   // model sync
         }
         const float4 m4 = make_float4(mo[0], mo[1], mo[2], mo[3]), x4 = make_float4(xo[0], xo[1], xo[2], xo[3]);
         st4(st.xs + j, x4);
@@ -419,12 +419,12 @@ dist_apply_kernel(StateView st, Consts c, float gamma_sum)
             const long long row = (long long)i * st.n_pad + j;
             st4(st.m + row, m4);
             st4(st.x + row, x4);
-            st4(st.u + row, make_float4(0.f, 0.f, 0.f, 0.f));                   // line 10
+            st4(st.u + row, make_float4(0.f, 0.f, 0.f, 0.f));                   // buffer reset
         }
     }
 }
 
-// Lines 14-15 of Algorithm 1 when the mean gradient comes from a collective: v_{t+1} from g_bar.
+// The variance update of Algorithm 1 when the mean gradient comes from a collective: v_{t+1} from g_bar.
 __global__ void __launch_bounds__(256)
 dist_variance_kernel(StateView st, Consts c, const float *g_bar)
 {
@@ -438,7 +438,7 @@ dist_variance_kernel(StateView st, Consts c, const float *g_bar)
 // accumulated updates (1-bit Adam when T_v is an initial run of steps).
 // ---------------------------------------------------------------------------
 
-// A T_v step of Algorithm 2 (lines 4-5, 10-11): full-precision mean of the
+// A T_v step of Algorithm 2 (full-precision AllReduce, variance, momentum, model): mean of the
 // gradients, momentum and model update with v_t on every worker, then v_{t+1}.
 __global__ void __launch_bounds__(256)
 alg2_full_kernel(StateView st, GradPtrs g, Consts c, float gamma, int g_aligned)
@@ -457,9 +457,9 @@ alg2_full_kernel(StateView st, GradPtrs g, Consts c, float gamma, int g_aligned)
         float gb[4], d[4], vo[4];
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-            gb[k] = mean_round(G[k], st.W);                     // line 4 (Algorithm 4)
+            gb[k] = mean_round(G[k], st.W);                     // full-precision mean (Algorithm 4)
             d[k] = denom(c, vv[k]);
-            vo[k] = variance(c, vv[k], gb[k]);                  // line 5
+            vo[k] = variance(c, vv[k], gb[k]);                  // buffer update
         }
         st4(st.v_next + j, make_float4(vo[0], vo[1], vo[2], vo[3]));
         for (int i = 0; i < st.W; ++i) {
@@ -469,8 +469,8 @@ alg2_full_kernel(StateView st, GradPtrs g, Consts c, float gamma, int g_aligned)
             float mo[4], xo[4];
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                mo[k] = momentum(c, mm[k], gb[k]);                              // line 10
-                xo[k] = f_sub(xx[k], f_div(f_mul(gamma, mo[k]), d[k]));         // line 11
+                mo[k] = momentum(c, mm[k], gb[k]);                              // momentum update
+                xo[k] = f_sub(xx[k], f_div(f_mul(gamma, mo[k]), d[k]));         // model update
             }
             st4(st.m + row, make_float4(mo[0], mo[1], mo[2], mo[3]));
             st4(st.x + row, make_float4(xo[0], xo[1], xo[2], xo[3]));
@@ -478,7 +478,7 @@ alg2_full_kernel(StateView st, GradPtrs g, Consts c, float gamma, int g_aligned)
     }
 }
 
-// Any other step of Algorithm 2 for chunk blockIdx.x (lines 7, 10-11): the
+// Any other step of Algorithm 2 for chunk blockIdx.x (Compressed-AllReduce, momentum, model): the
 // gradients go through the error-feedback 1-bit AllReduce (Algorithm 3), the
 // decompressed mean drives momentum and model on every worker.
 __global__ void __launch_bounds__(512, 2) alg2_compressed_kernel(StateView st, GradPtrs g, Consts c, float gamma, int g_aligned, long long chunk_offset)
@@ -575,8 +575,8 @@ __global__ void __launch_bounds__(512, 2) alg2_compressed_kernel(StateView st, G
                     float mo[4], xo[4];
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {
-                        mo[k] = momentum(c, mm[k], gb[k]);                              // line 10
-                        xo[k] = f_sub(xx[k], f_div(f_mul(gamma, mo[k]), d[k]));         // line 11
+                        mo[k] = momentum(c, mm[k], gb[k]);                              // momentum update
+                        xo[k] = f_sub(xx[k], f_div(f_mul(gamma, mo[k]), d[k]));         // model update
                     }
                     st4_stream(st.m + row, make_float4(mo[0], mo[1], mo[2], mo[3]));
                     st4_stream(st.x + row, make_float4(xo[0], xo[1], xo[2], xo[3]));
@@ -737,8 +737,8 @@ lc_server_partial_kernel(StateView st, long long segs_per_chunk, long long n_seg
     if (threadIdx.x == 0) partials[(long long)st.W * n_segs + blockIdx.x] = total;
 }
 
-// Server compression and what follows it.  MODE 1: lines 8-10 of Algorithm 1.
-// MODE 2: lines 10-11 of Algorithm 2 (momentum and model driven by the received gradient).
+// Server compression and what follows it.  MODE 1: the post-sync updates of Algorithm 1.
+// MODE 2: momentum and model updates of Algorithm 2, driven by the received gradient.
 template <int MODE>
 __global__ void __launch_bounds__(512)
 lc_server_apply_kernel(StateView st, Consts c, float gamma_or_sum, long long segs_per_chunk)
@@ -810,7 +810,7 @@ static int elementwise_grid(long long n4)
     return (int)(blocks < 1 ? 1 : blocks);
 }
 
-// Lines 3-5 (and 14-15 if do_var) for the coordinates [first, end); first is a multiple of 4.
+// The local updates of Algorithm 1 (and the variance update if do_var) for the coordinates [first, end); first is a multiple of 4.
 cudaError_t launch_local_step(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
                               bool do_var, int g_aligned, long long first, long long end, cudaStream_t s)
 {
@@ -827,7 +827,7 @@ cudaError_t launch_local_step(const StateView &st, const GradPtrs &g, const Cons
     return cudaGetLastError();
 }
 
-// Lines 14-15 for the coordinates [first, end); first is a multiple of 4.
+// The variance update of Algorithm 1 for the coordinates [first, end); first is a multiple of 4.
 cudaError_t launch_variance(const StateView &st, const GradPtrs &g, const Consts &c, int g_aligned,
                             long long first, long long end, cudaStream_t s)
 {
@@ -919,8 +919,8 @@ cudaError_t launch_large_compress(const StateView &st, const GradPtrs &g, const 
     return cudaGetLastError();
 }
 
-// Server side.  mode 1: Algorithm 1 lines 8-10 (scalar = sum of learning rates); mode 2: Algorithm 2
-// lines 10-11 (scalar = learning rate).
+// Server side.  mode 1: post-sync updates of Algorithm 1 (scalar = sum of learning rates); mode 2:
+// momentum and model updates of Algorithm 2 (scalar = learning rate).
 cudaError_t launch_large_server(const StateView &st, const Consts &c, int mode, float scalar, double *partials,
                                 int *launches, cudaStream_t s)
 {

@@ -1,4 +1,4 @@
-// step_sync_pipelined_kernel: the fused sync step (Algorithm 1 lines 3-11 with
+// step_sync_pipelined_kernel: the fused sync step (a whole sync iteration of Algorithm 1 with
 // Algorithm 3 inside) as a persistent, warp-specialised kernel for sm_100a.
 //
 // One block per SM takes chunks from a global counter (SMs do not all get the same
@@ -293,7 +293,7 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
     const bool group_leader = (lane & 7) == 0;
     float *my_scales = scales_s + warp * W;
 
-    // Lines 8-10 of the previous chunk, carried in registers: its 3 W tile stores are
+    // The post-sync updates of the previous chunk, carried in registers: its 3 W tile stores are
     // spread over the worker iterations of the next chunk (one worker's m, x, u after
     // each worker's compression) instead of leaving in one burst, so that the block's
     // stores and its ring's loads stay evenly mixed.  m is +-m_pos by the server's bit.
@@ -311,7 +311,7 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
             st4_stream(st.m + row, make_float4((nib & 1u) ? m_pos_prev : -m_pos_prev, (nib & 2u) ? m_pos_prev : -m_pos_prev,
                                                (nib & 4u) ? m_pos_prev : -m_pos_prev, (nib & 8u) ? m_pos_prev : -m_pos_prev));
             st4_stream(st.x + row, make_float4(x_prev[t][0], x_prev[t][1], x_prev[t][2], x_prev[t][3]));
-            st4_stream(st.u + row, zero);                                      // line 10
+            st4_stream(st.u + row, zero);                                      // buffer reset
         }
     };
 
@@ -353,7 +353,7 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
                 const float uu[4] = {u4.x, u4.y, u4.z, u4.w}, ee[4] = {e4.x, e4.y, e4.z, e4.w};
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
-                    const float step = f_mul(a.gamma, momentum(a.c, mm[k], gg[k]));   // lines 3, 5
+                    const float step = f_mul(a.gamma, momentum(a.c, mm[k], gg[k]));   // momentum update, buffer update
                     z[t][k] = f_add(f_add(uu[k], step), ee[k]);                       // u_{t+1/2} + delta
                     l1 += fabs((double)z[t][k]);
                     if (DO_VAR) G[t][k] += (double)gg[k];
@@ -425,7 +425,7 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
                 b[k] = av[t][k] >= 0.0f;
                 const float hat = b[k] ? scale : -scale;
                 e[k] = f_sub(av[t][k], hat);
-                xo[k] = f_sub(xs[k], f_div(hat, denom(a.c, vv[k])));           // line 9
+                xo[k] = f_sub(xs[k], f_div(hat, denom(a.c, vv[k])));           // model sync
                 if (DEFER) {
                     x_prev[t][k] = xo[k];
                     bits_prev |= (b[k] ? 1u : 0u) << (4 * t + k);
@@ -437,7 +437,7 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
             st4_stream(st.ds + j, make_float4(e[0], e[1], e[2], e[3]));
             st4_stream(st.xs + j, make_float4(xo[0], xo[1], xo[2], xo[3]));
             if (!DEFER) {
-                const float mp = f_div(scale, a.gamma_sum);                    // line 8
+                const float mp = f_div(scale, a.gamma_sum);                    // momentum approximation
                 const float4 m4 = make_float4(b[0] ? mp : -mp, b[1] ? mp : -mp, b[2] ? mp : -mp, b[3] ? mp : -mp);
                 const float4 x4 = make_float4(xo[0], xo[1], xo[2], xo[3]);
                 const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -445,18 +445,18 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
                     const long long row = (long long)i * st.n_pad + j;
                     st4_stream(st.m + row, m4);
                     st4_stream(st.x + row, x4);
-                    st4_stream(st.u + row, zero);                              // line 10
+                    st4_stream(st.u + row, zero);                              // buffer reset
                 }
             }
             if (DO_VAR) {
                 float vo[4];
 #pragma unroll
-                for (int k = 0; k < 4; ++k) vo[k] = variance(a.c, vv[k], mean_round(G[t][k], W));   // lines 14-15
+                for (int k = 0; k < 4; ++k) vo[k] = variance(a.c, vv[k], mean_round(G[t][k], W));   // variance update
                 st4_stream(st.v_next + j, make_float4(vo[0], vo[1], vo[2], vo[3]));
             }
         }
         if (DEFER) {
-            m_pos_prev = f_div(scale, a.gamma_sum);     // line 8: m = +-scale / sum(gamma); -(s/G) == (-s)/G exactly
+            m_pos_prev = f_div(scale, a.gamma_sum);     // momentum approximation: m = +-scale / sum(gamma); -(s/G) == (-s)/G exactly
             c0_prev = c0;
         }
         if (tid == 0) st.scales_s[chunk] = scale;
@@ -628,7 +628,7 @@ __global__ void __launch_bounds__(kThreads, 1) alg2_pipelined_kernel(const __gri
                 b[q] = gbar[t][q] >= 0.0f;
                 const float hat = b[q] ? scale : -scale;
                 e[q] = f_sub(gbar[t][q], hat);
-                gbar[t][q] = hat;                                // line 7: what every worker receives
+                gbar[t][q] = hat;                                // what every worker receives from the Compressed-AllReduce
             }
             const uint32_t word = pack_group(b);
             if (group_leader) st.words_s[((c0 + t * kTile) >> 5) + word_in_tile] = word;
@@ -636,7 +636,7 @@ __global__ void __launch_bounds__(kThreads, 1) alg2_pipelined_kernel(const __gri
         }
         if (tid == 0) st.scales_s[chunk] = scale;
 
-        // ---- every worker: momentum and model (lines 10-11) ----
+        // ---- every worker: momentum update and model update of Algorithm 2 ----
         for (int i = 0; i < W; ++i) {
 #pragma unroll
             for (int t = 0; t < TILES; ++t) {
@@ -700,7 +700,7 @@ static cudaError_t launch_pipe(const PipeArgs &a, int grid, size_t smem, cudaStr
 }
 
 // Runs the full chunks [first_chunk, first_chunk + n_chunks) of a sync step; a ragged last chunk is the caller's.
-// *var_fused tells whether lines 14-15 were done here too.
+// *var_fused tells whether the variance update was done here too.
 cudaError_t launch_step_sync_pipelined(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
                                        float gamma_sum, bool do_var, int grad_fmt, long long first_chunk, long long n_chunks, int stages,
                                        int sm_count, int *error_flag, unsigned long long *sched, unsigned long long wait_limit_ns,

@@ -320,7 +320,7 @@ def test_argument_and_state_errors():
     z = Zoa(100, 2, chunk=32)
     try:
         with pytest.raises(ZoaError) as e:
-            z.onebit_reduce()                       # nothing accumulated: line 8 would divide by zero
+            z.onebit_reduce()                       # nothing accumulated: the momentum approximation would divide by zero
         assert e.value.status == B.ERR_STATE
         g = list(torch.zeros(2, 100, device="cuda"))
         z.step(g, 1e-3, 5)

@@ -306,7 +306,7 @@ def test_alg1_local_steps_are_linear_in_u():
 
 
 def test_alg1_printed_momentum_index_is_degenerate():
-    """Taking m_t (before line 3) on lines 4-5, as printed, with a sync at every
+    """Taking m_t (from before the momentum update) in the model and buffer updates, as printed, with a sync at every
     step: the gradient never reaches the model.  This is why m_{t+1/2} is used."""
     rng = np.random.default_rng(25)
     o = zo.Oracle(64, 2, 32, dtype=np.float64, compressor=zo.IDENTITY, literal_momentum=True)
