@@ -124,12 +124,17 @@ class Zoa:
 
     # -- state access (synchronous copies) ----------------------------------------
     def read(self, name, worker=0, offset=0, count=None):
+        """Copies `count` elements of a state row to a numpy array (default: the live part of the row:
+        n parameters, ceil(n / 32) words or n_chunks magnitudes)."""
         which = _NAMES[name]
-        _, row_len = B.zoa_get_buffer(self.h, which, worker)
         if count is None:
-            count = {True: (self.n + 31) // 32}.get(which in B.WORD_BUFFERS,
-                                                      self.n_chunks if name.startswith("scales") else self.n)
-            count -= offset
+            if which in B.WORD_BUFFERS:
+                live = (self.n + 31) // 32
+            elif name.startswith("scales"):
+                live = self.n_chunks
+            else:
+                live = self.n
+            count = live - offset
         out = np.empty(count, np.uint32 if which in B.WORD_BUFFERS else np.float32)
         B.zoa_copy_out(self.h, which, worker, offset, count, out.ctypes.data)
         return out
