@@ -364,8 +364,9 @@ def test_policies_match_the_workload_tables():
         z.close()
 
 
-def test_device_wait_runs_out_and_is_reported():
-    """Error path of the ring kernel without any fault: the copy-issuing lane of every block
+@pytest.mark.parametrize("algorithm", ["alg1", "alg2"])
+def test_device_wait_runs_out_and_is_reported(algorithm):
+    """Error path of the ring kernels without any fault: the copy-issuing lane of every block
     stops after three tiles (test hook), the other threads' bounded waits run out after
     100 ms, the kernel ends by itself, zoa_check_device reports ZOA_ERR_DEVICE, and the
     context and the handle stay usable."""
@@ -375,19 +376,20 @@ def test_device_wait_runs_out_and_is_reported():
     try:
         g = list(torch.randn(W, n, device="cuda"))
         z.set_pipeline("force")
-        z.step_sync(g, 1e-3, 0)
+        step = z.step_sync if algorithm == "alg1" else z.alg2_step
+        step(g, 1e-3, 0)
         z.check_device()                                  # the normal path works
         B.zoa_set_option(z.h, B.OPT_WAIT_LIMIT_MS, 100)
         B.zoa_set_option(z.h, B.OPT_TEST_STOP_AFTER_TILES, 3)
         t0 = time.perf_counter()
-        z.step_sync(g, 1e-3, 1)
+        step(g, 1e-3, 1)
         with pytest.raises(ZoaError) as e:
             z.check_device()
         assert e.value.status == B.ERR_DEVICE
         assert time.perf_counter() - t0 < 5.0             # bounded: a few wait limits, not a hang
         B.zoa_set_option(z.h, B.OPT_TEST_STOP_AFTER_TILES, 0)
         B.zoa_set_option(z.h, B.OPT_WAIT_LIMIT_MS, 2000)
-        z.step_sync(g, 1e-3, 2)
+        step(g, 1e-3, 2)
         z.check_device()                                  # flag cleared, chunk counter rearmed
     finally:
         z.close()
