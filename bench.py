@@ -463,7 +463,8 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="bert_large")
+    ap.add_argument("--workload", default="bert_large",
+                    help="tiny | bert_base | bert_large (default, the headline) | gpt2_1p5b | all (one line each)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-sample", type=int, default=1 << 22, help="parameters in the oracle's timed sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -502,6 +503,18 @@ def main():
         return run_reference(args, wl)
 
     from paper_2202_06009_b200 import synth
+    if args.workload == "all":      # one JSON line per shaped workload, BERT-Large (the headline) last
+        import copy
+        for name in ("bert_base", "gpt2_1p5b", "bert_large"):
+            sub = copy.copy(args)
+            sub.workload, sub.steps = name, None
+            sub.no_cpu_baseline = args.no_cpu_baseline or name != "bert_large"
+            wl = synth.WORKLOADS[name]()
+            sub.steps = wl.steps
+            run_ours(sub, wl)
+            import torch
+            torch.cuda.empty_cache()
+        return
     wl = synth.WORKLOADS[args.workload]()
     if args.scale > 1:
         wl = synth.scaled(wl, args.scale)

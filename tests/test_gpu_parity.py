@@ -137,13 +137,14 @@ def test_special_values(mode):
         p.close()
 
 
-def test_tiny_config_full_run():
+@pytest.mark.parametrize("seed", [synth.DEFAULT_SEED, 7, 123456789])
+def test_tiny_config_full_run(seed):
     """The small configuration in full: 2^20 parameters, W = 4, chunk 2048, 64 steps,
     T_v = {0,1,2,4,8,16}, sync every step until 16 then every other step; every
-    state compared after every step."""
+    state compared after every step; three seeds."""
     wl = synth.tiny()
-    stream = synth.GradientStream(wl, "cuda")
-    x0 = synth.initial_params(wl, "cuda")
+    stream = synth.GradientStream(wl, "cuda", seed)
+    x0 = synth.initial_params(wl, "cuda", seed)
     p = Pair(wl.n, wl.W, wl.chunk, wl.beta1, wl.beta2, wl.eps, wl.var_steps,
              (wl.sync_boundaries, wl.sync_intervals), x0=x0.cpu().numpy())
     try:
