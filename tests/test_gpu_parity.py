@@ -37,7 +37,7 @@ def test_ragged_sizes(n, mode):
         p.close()
 
 
-@pytest.mark.parametrize("W,chunk,n", [(1, 32, 1000), (2, 64, 4096 + 5), (5, 96, 96 * 7 + 3), (4, 1024, 20000),
+@pytest.mark.parametrize("W,chunk,n", [(1, 32, 1000), (1, 2048, 2048 * 6 + 5), (1, 8192, 8192 * 3), (2, 64, 4096 + 5), (5, 96, 96 * 7 + 3), (4, 1024, 20000),
                                        (8, 4096, 3 * 4096 + 1852), (16, 4096, 2 * 4096 + 77), (4, 8192, 8192 * 2 + 704),
                                        (2, 16384, 16384 * 2 + 100), (64, 256, 1500), (3, 4000, 9000)])
 @pytest.mark.parametrize("mode", ["fused", "two_call"])
