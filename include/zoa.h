@@ -43,7 +43,8 @@ typedef enum {
     ZOA_ERR_ALLOC = 2,  /* device or host memory could not be had */
     ZOA_ERR_CUDA = 3,   /* a CUDA call or an earlier kernel failed; see zoa_last_error */
     ZOA_ERR_STATE = 4,  /* calls out of order: t not increasing, reduce with nothing accumulated */
-    ZOA_ERR_DEVICE = 5  /* a kernel gave up on a bounded wait; state is undefined */
+    ZOA_ERR_DEVICE = 5, /* a kernel gave up on a bounded wait or wrote out of bounds; state is undefined */
+    ZOA_ERR_NONFINITE = 6 /* zoa_check_finite found NaN or infinite values */
 } zoa_status;
 
 typedef enum {
@@ -232,6 +233,12 @@ zoa_status zoa_get_stats(zoa_handle h, zoa_stats *out);
  * last check, or if one of the guard areas that surround every device buffer of
  * the handle no longer holds its pattern (a kernel wrote out of bounds). */
 zoa_status zoa_check_device(zoa_handle h);
+
+/* Debug scan (synchronous, reads every float state buffer once): counts the NaN
+ * and infinite values in x, m, u, both errors, v and x_sync; returns
+ * ZOA_ERR_NONFINITE if there are any.  n_nonfinite may be NULL.  A non-finite
+ * gradient spreads through the l1 norm to its whole chunk at the next sync. */
+zoa_status zoa_check_finite(zoa_handle h, int64_t *n_nonfinite);
 
 /* Tuning switches.  ZOA_OPT_PIPELINE (default 1): run the fused sync step and the
  * compressed step of Algorithm 2 as the persistent bulk-copy-ring kernels where

@@ -10,7 +10,7 @@ import os
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libzoa.so")
 
-OK, ERR_ARG, ERR_ALLOC, ERR_CUDA, ERR_STATE, ERR_DEVICE = range(6)
+OK, ERR_ARG, ERR_ALLOC, ERR_CUDA, ERR_STATE, ERR_DEVICE, ERR_NONFINITE = range(7)
 (BUF_X, BUF_M, BUF_U, BUF_DELTA_W, BUF_V, BUF_DELTA_S, BUF_X_SYNC,
  BUF_WORDS_W, BUF_SCALES_W, BUF_WORDS_S, BUF_SCALES_S) = range(11)
 WORD_BUFFERS = (BUF_WORDS_W, BUF_WORDS_S)
@@ -64,6 +64,7 @@ def _load():
         "zoa_set_scalars": ([H, C.c_double, C.c_int64, C.c_int64], C.c_int),
         "zoa_get_stats": ([H, C.POINTER(Stats)], C.c_int),
         "zoa_check_device": ([H], C.c_int),
+        "zoa_check_finite": ([H, C.POINTER(C.c_int64)], C.c_int),
         "zoa_last_error": ([H], C.c_char_p),
         "zoa_set_option": ([H, C.c_int, C.c_int], C.c_int),
         "zoa_onebit_allreduce_static": ([C.POINTER(p), C.POINTER(p), p, p, C.c_size_t, C.c_int, C.c_int, p], C.c_int),
@@ -219,6 +220,15 @@ GRAD_F32, GRAD_F16, GRAD_BF16 = 0, 1, 2
 
 def zoa_set_option(h, option, value):
     _check(h, lib.zoa_set_option(h, option, value))
+
+
+def zoa_check_finite(h):
+    """Number of NaN / infinite values in the float state (0 = clean); never raises for a non-zero count."""
+    n = C.c_int64()
+    status = lib.zoa_check_finite(h, C.byref(n))
+    if status not in (OK, ERR_NONFINITE):
+        _check(h, status)
+    return n.value
 
 
 def zoa_check_device(h):

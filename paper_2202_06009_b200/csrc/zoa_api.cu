@@ -807,6 +807,24 @@ extern "C" zoa_status zoa_check_device(zoa_handle h)
     return ZOA_OK;
 }
 
+extern "C" zoa_status zoa_check_finite(zoa_handle h, int64_t *n_nonfinite)
+{
+    if (!h) return ZOA_ERR_ARG;
+    if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, "zoa_check_finite: the handle's device is not the current CUDA device");
+    ZOA_CUDA(h, cudaDeviceSynchronize());
+    ZOA_CUDA(h, cudaMemset(h->sched, 0, 2 * sizeof(unsigned long long)));      // borrowed as the counter; it is 0 between launches
+    const long long rows = (long long)h->W * h->n_pad;
+    const float *bufs[] = {h->x, h->m, h->u, h->dw, h->v_pending ? h->v_nxt : h->v_cur, h->ds, h->xs};
+    const long long counts[] = {rows, rows, rows, rows, h->n_pad, h->n_pad, h->n_pad};
+    for (int k = 0; k < 7; ++k) ZOA_CUDA(h, launch_count_nonfinite(bufs[k], counts[k], h->sched, h->sm_count, nullptr));
+    unsigned long long bad = 0;
+    ZOA_CUDA(h, cudaMemcpy(&bad, h->sched, sizeof(bad), cudaMemcpyDeviceToHost));
+    ZOA_CUDA(h, cudaMemset(h->sched, 0, 2 * sizeof(unsigned long long)));
+    if (n_nonfinite) *n_nonfinite = (int64_t)bad;
+    if (bad) return fail(h, ZOA_ERR_NONFINITE, "the optimizer state holds NaN or infinite values");
+    return ZOA_OK;
+}
+
 extern "C" zoa_status zoa_set_option(zoa_handle h, int option, int value)
 {
     if (!h) return ZOA_ERR_ARG;

@@ -41,6 +41,8 @@ cudaError_t launch_dist_server(const StateView &st, const uint32_t *words_in, lo
 cudaError_t launch_dist_apply(const StateView &st, const Consts &c, float gamma_sum, cudaStream_t s);
 cudaError_t launch_dist_variance(const StateView &st, const Consts &c, const float *g_bar, cudaStream_t s);
 
+cudaError_t launch_count_nonfinite(const float *p, long long count, unsigned long long *out, int sm_count, cudaStream_t s);
+
 int alg2_pipeline_stages(const StateView &st, int grad_fmt);
 cudaError_t launch_alg2_pipelined(const StateView &st, const GradPtrs &g, const Consts &c, float gamma, int grad_fmt,
                                   int stages, int sm_count, int *error_flag, unsigned long long *sched,

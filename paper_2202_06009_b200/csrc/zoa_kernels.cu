@@ -784,6 +784,18 @@ lc_server_apply_kernel(StateView st, Consts c, float gamma_or_sum, long long seg
     }
 }
 
+// Debug scan: how many of p[0..count) are NaN or infinite.
+__global__ void __launch_bounds__(256) count_nonfinite_kernel(const float *p, long long count, unsigned long long *out)
+{
+    unsigned long long bad = 0;
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long j = (long long)blockIdx.x * blockDim.x + threadIdx.x; j < count; j += stride)
+        bad += !isfinite(p[j]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) bad += __shfl_xor_sync(0xffffffffu, bad, o);
+    if ((threadIdx.x & 31) == 0 && bad) atomicAdd(out, bad);
+}
+
 // ---------------------------------------------------------------------------
 // Launchers
 // ---------------------------------------------------------------------------
@@ -964,6 +976,18 @@ cudaError_t launch_dist_apply(const StateView &st, const Consts &c, float gamma_
 cudaError_t launch_dist_variance(const StateView &st, const Consts &c, const float *g_bar, cudaStream_t s)
 {
     dist_variance_kernel<<<elementwise_grid((st.n + 255) / 256 * 64), 256, 0, s>>>(st, c, g_bar);
+    return cudaGetLastError();
+}
+
+}  // namespace zoa
+
+namespace zoa {
+
+cudaError_t launch_count_nonfinite(const float *p, long long count, unsigned long long *out, int sm_count, cudaStream_t s)
+{
+    long long blocks = (count + 255) / 256;
+    if (blocks > (long long)sm_count * 32) blocks = (long long)sm_count * 32;
+    count_nonfinite_kernel<<<(unsigned)(blocks < 1 ? 1 : blocks), 256, 0, s>>>(p, count, out);
     return cudaGetLastError();
 }
 

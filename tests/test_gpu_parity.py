@@ -339,6 +339,7 @@ def test_argument_and_state_errors():
         with pytest.raises(ZoaError):
             z.read("x", worker=2)
         z.check_device()
+        assert B.zoa_check_finite(z.h) == 0
         s = z.stats()
         assert s["n_steps"] == 1 and s["n_syncs"] == 1 and s["n_launches"] == 3
         assert s["bits_per_worker"] == 100 + 32 * 4
@@ -601,6 +602,7 @@ def test_nonfinite_gradients_propagate_like_the_oracle(mode):
             p.compare(f"t={t}", wire=False)
             for i in range(W):
                 assert np.array_equal(p.gpu.read("words_w", i), p.cpu.words_worker[i]), (t, i)
+        assert B.zoa_check_finite(p.gpu.h) > 0
         assert np.isnan(p.gpu.read("delta_w", 0)[:2048]).all()
         assert np.isfinite(p.gpu.read("x", 0)[2048:2 * 2048]).all()      # an untouched chunk
     finally:
