@@ -262,7 +262,7 @@ def run_ours(args, wl):
     bytes_of["two_call_sync+var"] = bytes_of["two_call_sync"] + wl.n * 4
     bytes_of["alg2_compressed"] = alg2_compressed_bytes(wl.n, wl.W, wl.chunk, g_bytes)
     bytes_of["alg2_full"] = alg2_full_bytes(wl.n, wl.W, g_bytes)
-    step_types = {k: {"count": len(v), "ms": statistics.mean(v), "algorithmic_GB": bytes_of[k] / 1e9,
+    step_types = {k: {"count": len(v), "ms": statistics.mean(v), "ms_median": statistics.median(v), "algorithmic_GB": bytes_of[k] / 1e9,
                       "GBps": bytes_of[k] / 1e6 / statistics.mean(v)} for k, v in by_kind.items()}
     total_bytes = sum(bytes_of[k] for k in kinds)
     dominant = next((k for k in ("sync", "sync+var", "two_call_sync", "alg2_compressed") if k in by_kind), kinds[0])
