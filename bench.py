@@ -178,11 +178,14 @@ def run_ours(args, wl):
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    # Under torchrun the process group is set up even for one rank, so that the barrier and the
+    # max-over-ranks reduction of the N > 1 launch are the same code at every N.
+    use_dist = world > 1 or ("MASTER_ADDR" in os.environ and "RANK" in os.environ)
+    if use_dist:
+        dist.init_process_group("nccl", rank=rank, world_size=world, device_id=torch.device("cuda", local_rank))
 
     def barrier():
-        if world > 1:
+        if use_dist:
             dist.barrier()
         torch.cuda.synchronize()
 
@@ -244,7 +247,7 @@ def run_ours(args, wl):
     opt.check_device()
     ms = [a.elapsed_time(b) for a, b in ev]
     total_ms = sum(ms)
-    if world > 1:
+    if use_dist:
         tt = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
         dist.all_reduce(tt, op=dist.ReduceOp.MAX)
         total_ms = float(tt.item())
@@ -304,7 +307,7 @@ def run_ours(args, wl):
         b.record()
         barrier()
         e_ms = a.elapsed_time(b)
-        if world > 1:
+        if use_dist:
             tt = torch.tensor([e_ms], device="cuda", dtype=torch.float64)
             dist.all_reduce(tt, op=dist.ReduceOp.MAX)
             e_ms = float(tt.item())
@@ -334,7 +337,7 @@ def run_ours(args, wl):
                 "step_types": step_types, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e,
                 "gpu_launches": launches, "clocks": clocks.summary(), "wall_s_timed_region": wall}
         print(json.dumps(line))
-    if world > 1:
+    if use_dist:
         dist.destroy_process_group()
 
 
