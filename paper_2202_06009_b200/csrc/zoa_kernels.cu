@@ -245,9 +245,12 @@ __global__ void reduce_kernel(StateView st, Consts c, float gamma_sum)
 // A whole sync step for chunk blockIdx.x: the local updates in registers, worker
 // compression, server, the post-sync updates.  The half-step m, x, u never reach memory;
 // x is not even read (the model sync rebuilds it from x_sync).
+// GFMT as in local_step_kernel (aligned binary32 at compile time, or -1 for the argument).
+template <int GFMT>
 __global__ void step_sync_kernel(StateView st, GradPtrs g, Consts c, float gamma, float gamma_sum,
-                                 int g_aligned, long long chunk_offset)
+                                 int g_fmt_arg, long long chunk_offset)
 {
+    const int g_aligned = GFMT >= 0 ? GFMT : g_fmt_arg;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     double *scratch = reinterpret_cast<double *>(smem_raw);                      // 34 doubles
     double *A_s = scratch + 34;                                                  // [chunk]
@@ -440,9 +443,12 @@ dist_variance_kernel(StateView st, Consts c, const float *g_bar)
 
 // A T_v step of Algorithm 2 (full-precision AllReduce, variance, momentum, model): mean of the
 // gradients, momentum and model update with v_t on every worker, then v_{t+1}.
+// GFMT as in local_step_kernel: the gradient format when known at compile time, else -1.
+template <int GFMT>
 __global__ void __launch_bounds__(256)
-alg2_full_kernel(StateView st, GradPtrs g, Consts c, float gamma, int g_aligned)
+alg2_full_kernel(StateView st, GradPtrs g, Consts c, float gamma, int g_fmt_arg)
 {
+    const int g_aligned = GFMT >= 0 ? GFMT : g_fmt_arg;
     const long long n4 = (st.n + 3) >> 2;
     const long long stride = (long long)gridDim.x * blockDim.x;
     for (long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x; q < n4; q += stride) {
@@ -861,7 +867,9 @@ cudaError_t configure_kernels()
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(alg2_compressed_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)step_sync_smem(kMaxChunk));
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(step_sync_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)step_sync_smem(kMaxChunk));
+    e = cudaFuncSetAttribute(step_sync_kernel<kGradF32 | kGradAligned>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)step_sync_smem(kMaxChunk));
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(step_sync_kernel<-1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)step_sync_smem(kMaxChunk));
 }
 
 // A step of Algorithm 2: the whole vector at full precision, or the chunks
@@ -869,9 +877,15 @@ cudaError_t configure_kernels()
 cudaError_t launch_alg2(const StateView &st, const GradPtrs &g, const Consts &c, float gamma, bool full_precision,
                         int g_aligned, long long first_chunk, long long count, cudaStream_t s)
 {
-    if (full_precision)
-        alg2_full_kernel<<<elementwise_grid((st.n + 3) / 4), 256, 0, s>>>(st, g, c, gamma, g_aligned);
-    else
+    if (full_precision) {
+        const int grid = elementwise_grid((st.n + 3) / 4);
+        switch (g_aligned) {
+        case kGradF32 | kGradAligned: alg2_full_kernel<kGradF32 | kGradAligned><<<grid, 256, 0, s>>>(st, g, c, gamma, g_aligned); break;
+        case kGradF16 | kGradAligned: alg2_full_kernel<kGradF16 | kGradAligned><<<grid, 256, 0, s>>>(st, g, c, gamma, g_aligned); break;
+        case kGradBF16 | kGradAligned: alg2_full_kernel<kGradBF16 | kGradAligned><<<grid, 256, 0, s>>>(st, g, c, gamma, g_aligned); break;
+        default: alg2_full_kernel<-1><<<grid, 256, 0, s>>>(st, g, c, gamma, g_aligned); break;
+        }
+    } else
         alg2_compressed_kernel<<<(unsigned)count, block_threads_for_chunk(st.chunk), step_sync_smem(st.chunk), s>>>(
             st, g, c, gamma, g_aligned, first_chunk);
     return cudaGetLastError();
@@ -897,8 +911,14 @@ cudaError_t launch_reduce(const StateView &st, const Consts &c, float gamma_sum,
 cudaError_t launch_step_sync(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
                              float gamma_sum, int g_aligned, long long first_chunk, long long count, cudaStream_t s)
 {
-    step_sync_kernel<<<(unsigned)count, block_threads_for_chunk(st.chunk), step_sync_smem(st.chunk), s>>>(
-        st, g, c, gamma, gamma_sum, g_aligned, first_chunk);
+    // Above 8192 coordinates the chunk's shared memory leaves room for one block per SM only, and
+    // 1024 threads then beat 512 (chunk 16384, BERT-Large-shaped: 33.9 against 40.0 ms).
+    const int threads = st.chunk > 8192 ? 1024 : block_threads_for_chunk(st.chunk);
+    const size_t smem = step_sync_smem(st.chunk);
+    if (g_aligned == (kGradF32 | kGradAligned))
+        step_sync_kernel<kGradF32 | kGradAligned><<<(unsigned)count, threads, smem, s>>>(st, g, c, gamma, gamma_sum, g_aligned, first_chunk);
+    else
+        step_sync_kernel<-1><<<(unsigned)count, threads, smem, s>>>(st, g, c, gamma, gamma_sum, g_aligned, first_chunk);
     return cudaGetLastError();
 }
 

@@ -11,7 +11,7 @@ from helpers import Pair
 
 pytestmark = pytest.mark.gpu
 
-CHUNKS = [32, 64, 96, 256, 1024, 2048, 2048, 4096, 4096, 8192, 16384, 16416, 32768, 1 << 20]
+CHUNKS = [32, 64, 96, 256, 1024, 2048, 2048, 4096, 4096, 8192, 12288, 16384, 16416, 32768, 1 << 20]
 DTYPES = [torch.float32, torch.float32, torch.float16, torch.bfloat16]
 
 
