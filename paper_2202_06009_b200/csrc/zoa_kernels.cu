@@ -894,16 +894,24 @@ cudaError_t launch_alg2(const StateView &st, const GradPtrs &g, const Consts &c,
 cudaError_t launch_compress(const StateView &st, cudaStream_t s)
 {
     const dim3 grid((unsigned)st.n_chunks, (unsigned)st.W);
-    // 16 coordinates per thread here (measured: 256-thread blocks move chunk 4096 at 6.7 TB/s, 512-thread ones at 6.0)
+    // 16 coordinates per thread here (measured: 256-thread blocks move chunk 4096 at 6.7 TB/s,
+    // 512-thread ones at 6.0; at chunk 16384, 1024 threads 5.6 against 5.4 for 512)
     int thr = 128;
-    while (thr < st.chunk / 16 && thr < 512) thr <<= 1;
+    while (thr < st.chunk / 16 && thr < 1024) thr <<= 1;
     compress_kernel<<<grid, thr, compress_smem(st.chunk), s>>>(st);
     return cudaGetLastError();
 }
 
 cudaError_t launch_reduce(const StateView &st, const Consts &c, float gamma_sum, cudaStream_t s)
 {
-    reduce_kernel<<<(unsigned)st.n_chunks, block_threads_for_chunk(st.chunk), reduce_smem(st.chunk), s>>>(st, c, gamma_sum);
+    // With few workers a block has little to move between its barriers, and smaller blocks
+    // (more of them per SM) do better: measured at chunk 4096, n = 2^28, W = 2: 4.75 TB/s with
+    // 512 threads, 5.21 with 256, 5.76 with 128; W = 4: 5.46, 6.07, 6.06; W = 16: 5.94, 5.91, 5.80.
+    // At chunk 16384, 512 threads are best at every W.
+    const int per_thread = st.W <= 2 ? 32 : 16;
+    int thr = 128;
+    while (thr < st.chunk / per_thread && thr < 512) thr <<= 1;
+    reduce_kernel<<<(unsigned)st.n_chunks, thr, reduce_smem(st.chunk), s>>>(st, c, gamma_sum);
     return cudaGetLastError();
 }
 
