@@ -193,7 +193,7 @@ __device__ __forceinline__ void server_tile(const StateView &st, const Consts &c
 }
 
 // Server side for chunk blockIdx.x, reading what compress_kernel sent.
-__global__ void reduce_kernel(StateView st, Consts c, float gamma_sum)
+__global__ void __launch_bounds__(512, 3) reduce_kernel(StateView st, Consts c, float gamma_sum)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     double *scratch = reinterpret_cast<double *>(smem_raw);
