@@ -646,3 +646,33 @@ def test_allocation_failure_is_reported_and_leaves_the_context_usable():
         z.check_device()
     finally:
         z.close()
+
+
+def test_work_is_ordered_on_the_callers_stream():
+    """Gradients are produced late on a non-blocking side stream and consumed by the steps
+    enqueued behind them on the same stream; nothing synchronises in between, so a kernel
+    launched on any other stream would read the stale buffers."""
+    n, W, chunk = 6 * 4096 + 100, 3, 4096
+    rng = np.random.default_rng(77)
+    p = Pair(n, W, chunk, var_steps=(0, 2), sync=((0,), (2,)), x0=rng.standard_normal(n) * 0.02)
+    side = torch.cuda.Stream()
+    gdev = torch.zeros((W, n), device="cuda")
+    staged = [torch.from_numpy(rng.standard_normal((W, n)).astype(np.float32)).cuda() for _ in range(4)]
+    torch.cuda.synchronize()
+    try:
+        with torch.cuda.stream(side):
+            for t in range(4):
+                torch.cuda._sleep(20_000_000)            # ~10 ms: the copy below lands well after the host has moved on
+                gdev.copy_(staged[t], non_blocking=True)
+                if t >= 2:
+                    p.gpu.step_auto(list(gdev), 1e-3, t)
+                else:
+                    p.gpu.step(list(gdev), 1e-3, t)
+                    if p.gpu.sync_due(t):
+                        p.gpu.onebit_reduce()
+        side.synchronize()
+        for t in range(4):
+            assert p.cpu.step(staged[t].cpu().numpy(), np.float32(1e-3), t, p.gpu.sync_due(t), p.gpu.var_due(t)) == 0
+        p.compare("side stream")
+    finally:
+        p.close()
