@@ -367,8 +367,14 @@ def run_worker_per_gpu(args, wl):
                          wl.shared, wl.noise, wl.noise_kind, wl.tensor_scale)
     stream = synth.GradientStream(one, "cuda", synth.DEFAULT_SEED + rank)
     K, Wu = args.steps, max(args.warmup, 3)
+    if args.exchange == "push":          # the kernels store into the peers' buffers themselves
+        from paper_2202_06009_b200.distributed import PeerTable
+        peers = PeerTable.symmetric(w)
+        step = lambda g, lr, t: w.step_pushed(g, lr, t, peers, dist.barrier)
+    else:
+        step = w.step
     for t in range(Wu):
-        w.step(stream.fill(t)[0], wl.lr_at(t), t)
+        step(stream.fill(t)[0], wl.lr_at(t), t)
     from paper_2202_06009_b200 import binding as B
     B.zoa_set_scalars(w.opt.h, 0.0, 0, -1)
     dist.barrier(); torch.cuda.synchronize()
@@ -376,7 +382,7 @@ def run_worker_per_gpu(args, wl):
     for t in range(K):
         g = stream.fill(t)[0]
         ev[t][0].record()
-        w.step(g, wl.lr_at(t), t)
+        step(g, wl.lr_at(t), t)
         ev[t][1].record()
     dist.barrier(); torch.cuda.synchronize()
     total_ms = torch.tensor([sum(a.elapsed_time(b) for a, b in ev)], device="cuda", dtype=torch.float64)
@@ -389,7 +395,8 @@ def run_worker_per_gpu(args, wl):
                           "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": "f32",
                           "data": "synthetic",
                           "config": {"workload": wl.name, "n_params": wl.n, "W": world, "chunk": wl.chunk,
-                                     "parallelism": f"one worker per GPU x {world}, packed all-to-all + all-gather (NCCL)"},
+                                     "parallelism": f"one worker per GPU x {world}, " + ("packed buffers stored into the peers' memory by the kernels, two barriers"
+                                                                                         if args.exchange == "push" else "packed all-to-all + all-gather (NCCL)")},
                           "gpu_launches": launches}))
     dist.destroy_process_group()
 
@@ -477,6 +484,9 @@ def main():
     ap.add_argument("--mapping", default="simulated", choices=["simulated", "worker-per-gpu"],
                     help="simulated: W workers as state buffers on each GPU (the headline); worker-per-gpu: "
                          "the paper's own mapping, one worker per rank with the packed buffers exchanged")
+    ap.add_argument("--exchange", default="nccl", choices=["nccl", "push"],
+                    help="worker-per-gpu mapping: exchange the packed buffers with NCCL collectives, or let the "
+                         "kernels store them into the peers' buffers (symmetric memory) between two barriers")
     ap.add_argument("--two-call", action="store_true",
                     help="sync steps as zoa_step + zoa_onebit_reduce (three kernels) instead of the fused call")
     ap.add_argument("--grad-dtype", default="f32", choices=["f32", "f16", "bf16"],

@@ -176,6 +176,46 @@ zoa_status zoa_dist_server_range(zoa_handle h, const uint32_t *words_all, size_t
 zoa_status zoa_dist_apply(zoa_handle h, void *stream);
 zoa_status zoa_dist_variance(zoa_handle h, const float *g_bar, void *stream);
 
+/* The same round with the two exchanges done by the kernels themselves, as stores
+ * through peer pointers (NVLink), for handles that hold one worker each:
+ *   zoa_dist_step_pack_push   local updates of a sync step + worker side of Algorithm 3,
+ *                             the packed words and magnitudes of each chunk stored into
+ *                             the receive buffer of the rank that serves it
+ *   -- every rank waits until all ranks have finished that call --
+ *   zoa_dist_server_push      server side for this rank's chunk range, its packed result
+ *                             stored into every rank's whole-vector words_s / scales_s
+ *   -- every rank waits again --
+ *   zoa_dist_apply
+ * No kernel waits for another rank: the two waits belong to the caller (a
+ * stream-ordered barrier between the ranks).  world ranks; rank s serves the
+ * chunks [chunk_begin[s], chunk_begin[s+1]) (host array of world + 1 entries, from
+ * 0 to the number of chunks, not decreasing).  peer_words[s] / peer_scales[s]
+ * (host arrays of world device pointers) point at the first word / magnitude of
+ * that range inside the row that rank s keeps for the calling rank, i.e. inside
+ * the words_all / scales_all it will pass to zoa_dist_server_push; they may be
+ * NULL for ranks that serve no chunk.  zoa_dist_pack_push is the worker side
+ * alone, after zoa_step.  zoa_dist_step_pack_push takes the rank's gradient
+ * (device, n_params elements in the handle's gradient type) and stands for
+ * zoa_step on a sync step: the half-step momentum, model and buffer are formed
+ * in registers and not stored, since zoa_dist_apply overwrites all three; the
+ * variance update of a T_v step still goes through zoa_dist_variance.  The
+ * handle's own words_w / scales_w are written as well.  peer_words_s[r] /
+ * peer_scales_s[r] point at the first element of rank r's whole-vector buffers
+ * (n_pad/32 words, n_chunks magnitudes; the calling rank's own entry may be its
+ * own buffers or any other buffer of that size).  Errors: ZOA_ERR_ARG for a
+ * handle with more than one worker, chunks above 16384, a malformed table or a
+ * NULL pointer; ZOA_ERR_STATE as for zoa_step.  Nothing is allocated.  (The
+ * paper ships these buffers over the network; it describes no such kernels.) */
+zoa_status zoa_dist_pack_push(zoa_handle h, int world, const int64_t *chunk_begin,
+                              void *const *peer_words, void *const *peer_scales, void *stream);
+zoa_status zoa_dist_step_pack_push(zoa_handle h, const void *grad, float lr, int64_t t, int world,
+                                   const int64_t *chunk_begin, void *const *peer_words,
+                                   void *const *peer_scales, void *stream);
+zoa_status zoa_dist_server_push(zoa_handle h, const uint32_t *words_all, size_t words_stride,
+                                const float *scales_all, size_t scales_stride, int W_total,
+                                int64_t first_chunk, int64_t n_chunks, int world,
+                                void *const *peer_words_s, void *const *peer_scales_s, void *stream);
+
 /* zoa_step followed by zoa_onebit_reduce, same results bit for bit, in one
  * pass over memory that never writes the half-step values. */
 zoa_status zoa_step_sync(zoa_handle h, const void *const *grads, float lr, int64_t t,

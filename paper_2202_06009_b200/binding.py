@@ -54,6 +54,9 @@ def _load():
         "zoa_dist_server_range": ([H, p, C.c_size_t, p, C.c_size_t, C.c_int, C.c_int64, C.c_int64, p], C.c_int),
         "zoa_dist_apply": ([H, p], C.c_int),
         "zoa_dist_variance": ([H, p, p], C.c_int),
+        "zoa_dist_pack_push": ([H, C.c_int, C.POINTER(C.c_int64), C.POINTER(p), C.POINTER(p), p], C.c_int),
+        "zoa_dist_step_pack_push": ([H, p, C.c_float, C.c_int64, C.c_int, C.POINTER(C.c_int64), C.POINTER(p), C.POINTER(p), p], C.c_int),
+        "zoa_dist_server_push": ([H, p, C.c_size_t, p, C.c_size_t, C.c_int, C.c_int64, C.c_int64, C.c_int, C.POINTER(p), C.POINTER(p), p], C.c_int),
         "zoa_step_sync": ([H, C.POINTER(p), C.c_float, C.c_int64, p], C.c_int),
         "zoa_step_auto": ([H, C.POINTER(p), C.c_float, C.c_int64, p], C.c_int),
         "zoa_alg2_step": ([H, C.POINTER(p), C.c_float, C.c_int64, p], C.c_int),
@@ -172,6 +175,27 @@ def zoa_dist_apply(h, stream=0):
 
 def zoa_dist_variance(h, g_bar_ptr, stream=0):
     _check(h, lib.zoa_dist_variance(h, g_bar_ptr, stream))
+
+
+def _i64_array(values):
+    return (C.c_int64 * len(values))(*values)
+
+
+def zoa_dist_pack_push(h, chunk_begin, peer_words, peer_scales, stream=0):
+    world = len(peer_words)
+    _check(h, lib.zoa_dist_pack_push(h, world, _i64_array(chunk_begin), _ptr_array(peer_words), _ptr_array(peer_scales), stream))
+
+
+def zoa_dist_step_pack_push(h, grad_ptr, lr, t, chunk_begin, peer_words, peer_scales, stream=0):
+    world = len(peer_words)
+    _check(h, lib.zoa_dist_step_pack_push(h, grad_ptr, lr, t, world, _i64_array(chunk_begin), _ptr_array(peer_words),
+                                          _ptr_array(peer_scales), stream))
+
+
+def zoa_dist_server_push(h, words_ptr, words_stride, scales_ptr, scales_stride, W_total, first_chunk, n_chunks,
+                         peer_words_s, peer_scales_s, stream=0):
+    _check(h, lib.zoa_dist_server_push(h, words_ptr, words_stride, scales_ptr, scales_stride, W_total, first_chunk,
+                                       n_chunks, len(peer_words_s), _ptr_array(peer_words_s), _ptr_array(peer_scales_s), stream))
 
 
 def zoa_step_sync(h, grad_ptrs, lr, t, stream=0):

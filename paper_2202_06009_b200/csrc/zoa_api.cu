@@ -501,9 +501,102 @@ extern "C" zoa_status zoa_dist_server_range(zoa_handle h, const uint32_t *words_
     if (n_chunks == 0) return ZOA_OK;
     if (!words_all || !scales_all) return fail(h, ZOA_ERR_ARG, "zoa_dist_server_range: NULL buffer");
     if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, "zoa_dist_server_range: the handle's device is not the current CUDA device");
+    PeerOut none{};
     ZOA_CUDA(h, launch_dist_server(view(h), words_all, (long long)words_stride, scales_all, (long long)scales_stride,
-                                   W_total, first_chunk, n_chunks, static_cast<cudaStream_t>(stream)));
+                                   W_total, first_chunk, n_chunks, none, static_cast<cudaStream_t>(stream)));
     h->n_launches += 1;
+    return ZOA_OK;
+}
+
+extern "C" zoa_status zoa_dist_server_push(zoa_handle h, const uint32_t *words_all, size_t words_stride,
+                                           const float *scales_all, size_t scales_stride, int W_total,
+                                           int64_t first_chunk, int64_t n_chunks, int world,
+                                           void *const *peer_words_s, void *const *peer_scales_s, void *stream)
+{
+    if (!h) return ZOA_ERR_ARG;
+    if (h->large_chunk) return fail(h, ZOA_ERR_ARG, "zoa_dist_server_push: chunk must be at most 16384");
+    if (W_total < 1 || W_total > kMaxWorkers) return fail(h, ZOA_ERR_ARG, "zoa_dist_server_push: W_total must be in [1, 64]");
+    if (world < 1 || world > kMaxWorkers) return fail(h, ZOA_ERR_ARG, "zoa_dist_server_push: world must be in [1, 64]");
+    if (first_chunk < 0 || n_chunks < 0 || first_chunk + n_chunks > h->n_chunks)
+        return fail(h, ZOA_ERR_ARG, "zoa_dist_server_push: chunk range outside the vector");
+    if (!peer_words_s || !peer_scales_s) return fail(h, ZOA_ERR_ARG, "zoa_dist_server_push: NULL pointer table");
+    PeerOut out{};
+    out.world = world;
+    for (int r = 0; r < world; ++r) {
+        if (!peer_words_s[r] || !peer_scales_s[r]) return fail(h, ZOA_ERR_ARG, "zoa_dist_server_push: a peer pointer is NULL");
+        out.words_s[r] = static_cast<uint32_t *>(peer_words_s[r]);
+        out.scales_s[r] = static_cast<float *>(peer_scales_s[r]);
+    }
+    if (n_chunks == 0) return ZOA_OK;
+    if (!words_all || !scales_all) return fail(h, ZOA_ERR_ARG, "zoa_dist_server_push: NULL buffer");
+    if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, "zoa_dist_server_push: the handle's device is not the current CUDA device");
+    ZOA_CUDA(h, launch_dist_server(view(h), words_all, (long long)words_stride, scales_all, (long long)scales_stride,
+                                   W_total, first_chunk, n_chunks, out, static_cast<cudaStream_t>(stream)));
+    h->n_launches += 1;
+    return ZOA_OK;
+}
+
+// The table of a rank's destinations, checked: the ranges tile the chunks in rank order and
+// every rank that serves a chunk has both pointers.
+static zoa_status make_push_plan(zoa_handle h, int world, const int64_t *chunk_begin, void *const *peer_words,
+                                 void *const *peer_scales, PushPlan *plan, const char *who)
+{
+    if (h->W != 1) return fail(h, ZOA_ERR_ARG, std::string(who) + ": the handle must hold exactly one worker");
+    if (h->large_chunk) return fail(h, ZOA_ERR_ARG, std::string(who) + ": chunk must be at most 16384");
+    if (world < 1 || world > kMaxWorkers) return fail(h, ZOA_ERR_ARG, std::string(who) + ": world must be in [1, 64]");
+    if (!chunk_begin || !peer_words || !peer_scales) return fail(h, ZOA_ERR_ARG, std::string(who) + ": NULL table");
+    if (chunk_begin[0] != 0 || chunk_begin[world] != h->n_chunks)
+        return fail(h, ZOA_ERR_ARG, std::string(who) + ": chunk_begin must run from 0 to the number of chunks");
+    *plan = PushPlan{};
+    plan->world = world;
+    for (int r = 0; r < world; ++r) {
+        if (chunk_begin[r + 1] < chunk_begin[r]) return fail(h, ZOA_ERR_ARG, std::string(who) + ": chunk_begin must not decrease");
+        if (chunk_begin[r + 1] > chunk_begin[r] && (!peer_words[r] || !peer_scales[r]))
+            return fail(h, ZOA_ERR_ARG, std::string(who) + ": a rank that serves chunks has a NULL pointer");
+        plan->chunk_begin[r] = chunk_begin[r];
+        plan->words[r] = static_cast<uint32_t *>(peer_words[r]);
+        plan->scales[r] = static_cast<float *>(peer_scales[r]);
+    }
+    plan->chunk_begin[world] = chunk_begin[world];
+    return ZOA_OK;
+}
+
+extern "C" zoa_status zoa_dist_pack_push(zoa_handle h, int world, const int64_t *chunk_begin,
+                                         void *const *peer_words, void *const *peer_scales, void *stream)
+{
+    if (!h) return ZOA_ERR_ARG;
+    PushPlan plan;
+    zoa_status rc = make_push_plan(h, world, chunk_begin, peer_words, peer_scales, &plan, "zoa_dist_pack_push");
+    if (rc != ZOA_OK) return rc;
+    if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, "zoa_dist_pack_push: the handle's device is not the current CUDA device");
+    ZOA_CUDA(h, launch_dist_pack_push(view(h), nullptr, h->c, 0.f, 0, plan, static_cast<cudaStream_t>(stream)));
+    h->n_launches += 1;
+    return ZOA_OK;
+}
+
+extern "C" zoa_status zoa_dist_step_pack_push(zoa_handle h, const void *grad, float lr, int64_t t, int world,
+                                              const int64_t *chunk_begin, void *const *peer_words,
+                                              void *const *peer_scales, void *stream)
+{
+    TraceRange trace("zoa_dist_step_pack_push");
+    if (!h) return ZOA_ERR_ARG;
+    PushPlan plan;
+    zoa_status rc = make_push_plan(h, world, chunk_begin, peer_words, peer_scales, &plan, "zoa_dist_step_pack_push");
+    if (rc != ZOA_OK) return rc;
+    GradPtrs gp;
+    int fmt;
+    const void *grads[1] = {grad};
+    rc = check_step_args(h, grads, lr, t, &gp, &fmt, "zoa_dist_step_pack_push");
+    if (rc != ZOA_OK) return rc;
+    const double total = h->gamma_sum + (double)lr;
+    if (!(total > 0.0) || !((float)total > 0.f) || !std::isfinite((float)total))
+        return fail(h, ZOA_ERR_STATE, "zoa_dist_step_pack_push: sum of learning rates since the last sync is not positive");
+    commit_variance(h);
+    ZOA_CUDA(h, launch_dist_pack_push(view(h), gp.p[0], h->c, lr, fmt, plan, static_cast<cudaStream_t>(stream)));
+    h->n_launches += 1;
+    h->gamma_sum = total;
+    h->t_last = t;
+    h->n_steps += 1;
     return ZOA_OK;
 }
 

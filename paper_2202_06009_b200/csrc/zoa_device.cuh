@@ -38,6 +38,23 @@ struct StateView {
     int W, chunk;
 };
 
+// One worker per GPU: where a rank's packed buffers go.  Rank s serves the chunks
+// [chunk_begin[s], chunk_begin[s + 1]); words[s] / scales[s] point at the first word /
+// magnitude of that range inside a buffer that rank s can read (its own memory: the
+// pointer is a peer pointer for every other rank, and the stores cross NVLink).
+struct PushPlan {
+    int world;
+    long long chunk_begin[kMaxWorkers + 1];
+    uint32_t *words[kMaxWorkers];
+    float *scales[kMaxWorkers];
+};
+// Where a server's packed result goes: the whole-vector words_s / scales_s of every rank.
+struct PeerOut {
+    int world;
+    uint32_t *words_s[kMaxWorkers];
+    float *scales_s[kMaxWorkers];
+};
+
 // ---- binary32 arithmetic, one IEEE rounding per operation, never contracted ----
 __device__ __forceinline__ float f_add(float a, float b) { return __fadd_rn(a, b); }
 __device__ __forceinline__ float f_sub(float a, float b) { return __fsub_rn(a, b); }

@@ -341,9 +341,11 @@ __global__ void step_sync_kernel(StateView st, GradPtrs g, Consts c, float gamma
 // Server side of Algorithm 3 alone for chunk first_chunk + blockIdx.x, reading packed buffers
 // gathered from W_total workers: words_in[w][range words], scales_in[w][range chunks], both
 // starting at the range's first chunk.  Writes the server error, words_s and scales_s.
+// `out` lists where else the packed result of the range is to be stored (every rank's
+// words_s / scales_s, peer pointers included); out.world == 0 for none.
 __global__ void dist_server_kernel(StateView st, const uint32_t *words_in, long long words_in_stride,
                                    const float *scales_in, long long scales_in_stride, int W_total,
-                                   long long first_chunk)
+                                   long long first_chunk, PeerOut out)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     double *scratch = reinterpret_cast<double *>(smem_raw);
@@ -389,10 +391,78 @@ __global__ void dist_server_kernel(StateView st, const uint32_t *words_in, long 
             a[0] = a4.x; a[1] = a4.y; a[2] = a4.z; a[3] = a4.w;
         }
         const uint32_t word = compress_tile(a, hat, scale, idx, cg.len);
-        if (lane < 4 && base + 32 * lane < cg.len) st.words_s[((cg.c0 + base) >> 5) + lane] = word;
+        if (lane < 4 && base + 32 * lane < cg.len) {
+            const long long w = ((cg.c0 + base) >> 5) + lane;
+            st.words_s[w] = word;
+            for (int r = 0; r < out.world; ++r) out.words_s[r][w] = word;
+        }
         if (idx < cg.len) st4(st.ds + cg.c0 + idx, make_float4(a[0], a[1], a[2], a[3]));
     }
-    if (threadIdx.x == 0) st.scales_s[chunk_id] = scale;
+    if (threadIdx.x == 0) {
+        st.scales_s[chunk_id] = scale;
+        for (int r = 0; r < out.world; ++r) out.scales_s[r][chunk_id] = scale;
+    }
+}
+
+// Worker side of Algorithm 3 for the handle's single worker and chunk blockIdx.x, the packed
+// words and the magnitude stored straight into the receive buffer of the rank that serves the
+// chunk (and into the handle's own words_w / scales_w).  FUSED: the step is a sync step, so the
+// momentum and buffer updates of Algorithm 1 are formed in registers from g, m, u and only the
+// new compression error is written; otherwise u already holds the half-step buffer.
+template <bool FUSED, int GFMT>
+__global__ void dist_pack_push_kernel(StateView st, const float *g, Consts c, float gamma, int g_fmt_arg, PushPlan plan)
+{
+    const int g_fmt = GFMT >= 0 ? GFMT : g_fmt_arg;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    double *scratch = reinterpret_cast<double *>(smem_raw);        // 33 doubles
+    float *z_s = reinterpret_cast<float *>(smem_raw + 34 * sizeof(double));
+    const long long chunk_id = blockIdx.x;
+    const ChunkGeom cg = chunk_geom(st, chunk_id);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    int server = 0;
+    while (server + 1 < plan.world && chunk_id >= plan.chunk_begin[server + 1]) ++server;
+    const long long range_chunk0 = plan.chunk_begin[server];
+    const long long range_word0 = (range_chunk0 * st.chunk) >> 5;
+    uint32_t *words_out = plan.words[server];
+    float *scales_out = plan.scales[server];
+
+    double l1 = 0.0;
+    for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
+        const int idx = base + 4 * lane;
+        if (idx < cg.len) {
+            const long long j = cg.c0 + idx;
+            float4 u4 = ld4(st.u + j);
+            const float4 e4 = ld4(st.dw + j);
+            if (FUSED) {
+                const float4 g4 = ld_grad4(g, j, st.n, g_fmt), m4 = ld4(st.m + j);
+                u4 = make_float4(f_add(u4.x, f_mul(gamma, momentum(c, m4.x, g4.x))), f_add(u4.y, f_mul(gamma, momentum(c, m4.y, g4.y))),
+                                 f_add(u4.z, f_mul(gamma, momentum(c, m4.z, g4.z))), f_add(u4.w, f_mul(gamma, momentum(c, m4.w, g4.w))));
+            }
+            const float4 z4 = make_float4(f_add(u4.x, e4.x), f_add(u4.y, e4.y), f_add(u4.z, e4.z), f_add(u4.w, e4.w));
+            st4(z_s + idx, z4);
+            l1 += fabs((double)z4.x) + fabs((double)z4.y) + fabs((double)z4.z) + fabs((double)z4.w);
+        }
+    }
+    const float scale = chunk_scale(block_sum(l1, scratch), cg.len);
+    for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
+        const int idx = base + 4 * lane;
+        float z[4] = {0.f, 0.f, 0.f, 0.f}, hat[4];
+        if (idx < cg.len) {
+            const float4 z4 = ld4(z_s + idx);
+            z[0] = z4.x; z[1] = z4.y; z[2] = z4.z; z[3] = z4.w;
+        }
+        const uint32_t word = compress_tile(z, hat, scale, idx, cg.len);
+        if (idx < cg.len) st4(st.dw + cg.c0 + idx, make_float4(z[0], z[1], z[2], z[3]));
+        if (lane < 4 && base + 32 * lane < cg.len) {
+            const long long w = ((cg.c0 + base) >> 5) + lane;
+            st.words_w[w] = word;
+            words_out[w - range_word0] = word;
+        }
+    }
+    if (threadIdx.x == 0) {
+        st.scales_w[chunk_id] = scale;
+        scales_out[chunk_id - range_chunk0] = scale;
+    }
 }
 
 // The post-sync updates of Algorithm 1 from the server's packed result (words_s, scales_s of the whole
@@ -979,7 +1049,7 @@ namespace zoa {
 
 cudaError_t launch_dist_server(const StateView &st, const uint32_t *words_in, long long words_in_stride,
                                const float *scales_in, long long scales_in_stride, int W_total,
-                               long long first_chunk, long long count, cudaStream_t s)
+                               long long first_chunk, long long count, const PeerOut &out, cudaStream_t s)
 {
     static bool configured[64] = {false};
     int dev = 0;
@@ -991,7 +1061,34 @@ cudaError_t launch_dist_server(const StateView &st, const uint32_t *words_in, lo
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
     dist_server_kernel<<<(unsigned)count, block_threads_for_chunk(st.chunk), reduce_smem(st.chunk), s>>>(
-        st, words_in, words_in_stride, scales_in, scales_in_stride, W_total, first_chunk);
+        st, words_in, words_in_stride, scales_in, scales_in_stride, W_total, first_chunk, out);
+    return cudaGetLastError();
+}
+
+// Worker side of the 1-bit AllReduce for a single-worker handle with the packed result stored
+// through `plan`; g != nullptr: fused with the local updates of a sync step.
+cudaError_t launch_dist_pack_push(const StateView &st, const float *g, const Consts &c, float gamma, int g_fmt,
+                                  const PushPlan &plan, cudaStream_t s)
+{
+    static bool configured[64] = {false};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    const size_t max_smem = compress_smem(kMaxChunk);
+    if (dev < 0 || dev >= 64 || !configured[dev]) {
+        e = cudaFuncSetAttribute(dist_pack_push_kernel<false, -1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(dist_pack_push_kernel<true, -1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(dist_pack_push_kernel<true, kGradF32 | kGradAligned>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) configured[dev] = true;
+    }
+    int thr = 128;
+    while (thr < st.chunk / 16 && thr < 1024) thr <<= 1;
+    const unsigned grid = (unsigned)st.n_chunks;
+    const size_t smem = compress_smem(st.chunk);
+    if (!g) dist_pack_push_kernel<false, -1><<<grid, thr, smem, s>>>(st, nullptr, c, gamma, g_fmt, plan);
+    else if (g_fmt == (kGradF32 | kGradAligned)) dist_pack_push_kernel<true, kGradF32 | kGradAligned><<<grid, thr, smem, s>>>(st, g, c, gamma, g_fmt, plan);
+    else dist_pack_push_kernel<true, -1><<<grid, thr, smem, s>>>(st, g, c, gamma, g_fmt, plan);
     return cudaGetLastError();
 }
 

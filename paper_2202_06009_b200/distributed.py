@@ -15,6 +15,18 @@ same, instead of 4n bytes.  The collectives are torch.distributed's (NCCL over
 NVLink on GPUs); the arithmetic is the library's kernels.  The exchange itself
 (`ExchangePlan`, `exchange_packed`, `gather_server`) works on tensors of any
 device, which is how it is tested with the gloo backend.
+
+A second form lets the kernels do both exchanges themselves, as stores through
+peer pointers (`PeerTable`, `WorkerPerGpu.step_pushed`):
+
+    local updates + pack, stored into the servers' receive buffers   (zoa_dist_step_pack_push)
+    barrier between the ranks (stream-ordered)
+    server part, result stored into every rank's words_s / scales_s  (zoa_dist_server_push)
+    barrier
+    m, x, u from the packed result                                   (zoa_dist_apply)
+
+No kernel waits for another rank; on a sync step the half-step momentum, model and
+buffer are never written (32 bytes per parameter instead of 52).
 """
 from dataclasses import dataclass
 from typing import List, Sequence
@@ -89,6 +101,52 @@ def gather_server(plan: ExchangePlan, rank: int, words_s: torch.Tensor, scales_s
         scales_s[c.start:c.stop] = all_c[r, :len(c)]
 
 
+@dataclass
+class PeerTable:
+    """Device addresses through which every rank stores into the others' buffers.  Entry r belongs
+    to rank r: its receive buffers ([world][max_words] uint32, [world][max_chunks] float32; row w
+    is filled by worker w) and the whole-vector buffers that receive the servers' results."""
+    recv_words: List[int]
+    recv_scales: List[int]
+    words_s: List[int]
+    scales_s: List[int]
+    copy_back: bool = False     # words_s / scales_s above are staging buffers, not the handles' own
+
+    @staticmethod
+    def local(workers: Sequence["WorkerPerGpu"]) -> "PeerTable":
+        """All ranks live in this process (on one GPU): plain device pointers."""
+        for w in workers:
+            w.alloc_receive_buffers()
+        return PeerTable([w.recv_words.data_ptr() for w in workers], [w.recv_scales.data_ptr() for w in workers],
+                         [w.opt.device_view("words_s").data_ptr() for w in workers],
+                         [w.opt.device_view("scales_s").data_ptr() for w in workers])
+
+    @staticmethod
+    def symmetric(worker: "WorkerPerGpu", group=None) -> "PeerTable":
+        """One rank per process and GPU: the buffers are carved out of one block of torch's
+        symmetric memory, whose rendezvous hands every rank the others' addresses."""
+        import torch.distributed._symmetric_memory as symm_mem
+        plan, world = worker.plan, worker.world
+        mw, mc = plan.max_words(), plan.max_chunks()
+        total_w, total_c = (plan.n + 31) // 32, -(-plan.n // plan.chunk)
+        sizes = [world * mw, world * mc, total_w, total_c]          # 4-byte elements each
+        offsets = [0]
+        for sz in sizes:
+            offsets.append(offsets[-1] + (sz + 63) // 64 * 64)
+        block = symm_mem.empty(offsets[-1], dtype=torch.int32, device=torch.device("cuda", torch.cuda.current_device()))
+        block.zero_()
+        group = group if group is not None else dist.group.WORLD
+        handle = symm_mem.rendezvous(block, group=group)
+        worker.symmetric_block = block
+        worker.recv_words = block[offsets[0]:offsets[0] + sizes[0]].view(world, mw)
+        worker.recv_scales = block[offsets[1]:offsets[1] + sizes[1]].view(torch.float32).view(world, mc)
+        worker.staged_words_s = block[offsets[2]:offsets[2] + sizes[2]]
+        worker.staged_scales_s = block[offsets[3]:offsets[3] + sizes[3]].view(torch.float32)
+        bases = [int(p) for p in handle.buffer_ptrs]
+        return PeerTable([b + 4 * offsets[0] for b in bases], [b + 4 * offsets[1] for b in bases],
+                         [b + 4 * offsets[2] for b in bases], [b + 4 * offsets[3] for b in bases], copy_back=True)
+
+
 class WorkerPerGpu:
     """This rank's worker and server shard.  `var_steps` is T_v (kept here: the mean gradient of a
     T_v step comes from an all-reduce, not from the handle); the sync policy lives in the handle."""
@@ -102,6 +160,8 @@ class WorkerPerGpu:
         self.opt = Zoa(n_params, 1, beta1, beta2, eps, chunk)
         self.opt.set_policies((), sync_boundaries, sync_intervals)
         self.var_steps = frozenset(var_steps)
+        self.recv_words = self.recv_scales = None
+        self.staged_words_s = self.staged_scales_s = None
 
     def close(self):
         self.opt.close()
@@ -140,4 +200,59 @@ class WorkerPerGpu:
             recv_words, recv_scales = exchange_packed(self.plan, self.rank, words, scales, self.group)
             words_s, scales_s = self.serve(recv_words, recv_scales)
             gather_server(self.plan, self.rank, words_s, scales_s, self.group)
+            self.apply()
+
+    # -- the same round with the exchanges done by the kernels' own stores -------------
+    def alloc_receive_buffers(self):
+        if self.recv_words is None:
+            dev = torch.device("cuda", torch.cuda.current_device())
+            self.recv_words = torch.zeros((self.world, max(1, self.plan.max_words())), dtype=torch.int32, device=dev)
+            self.recv_scales = torch.zeros((self.world, max(1, self.plan.max_chunks())), dtype=torch.float32, device=dev)
+
+    def _push_tables(self, peers: PeerTable):
+        """This rank's row in every server's receive buffers (None where a rank serves nothing)."""
+        mw, mc = self.recv_words.shape[1], self.recv_scales.shape[1]
+        begin = [c.start for c in self.plan.chunks] + [self.plan.chunks[-1].stop]
+        words = [peers.recv_words[s] + 4 * self.rank * mw if len(self.plan.chunks[s]) else None for s in range(self.world)]
+        scales = [peers.recv_scales[s] + 4 * self.rank * mc if len(self.plan.chunks[s]) else None for s in range(self.world)]
+        return begin, words, scales
+
+    def push_pack(self, peers: PeerTable, grad: torch.Tensor = None, lr: float = 0.0, t: int = 0):
+        """Worker side, stored into the servers' receive buffers; with `grad` it also stands for the
+        local updates of the sync step t."""
+        from . import binding as B
+        begin, words, scales = self._push_tables(peers)
+        stream = torch.cuda.current_stream().cuda_stream
+        if grad is None:
+            B.zoa_dist_pack_push(self.opt.h, begin, words, scales, stream)
+        else:
+            B.zoa_dist_step_pack_push(self.opt.h, grad.data_ptr(), lr, t, begin, words, scales, stream)
+
+    def push_serve(self, peers: PeerTable):
+        from . import binding as B
+        c = self.plan.chunks[self.rank]
+        B.zoa_dist_server_push(self.opt.h, self.recv_words.data_ptr(), self.recv_words.stride(0),
+                               self.recv_scales.data_ptr(), self.recv_scales.stride(0), self.world, c.start, len(c),
+                               peers.words_s, peers.scales_s, torch.cuda.current_stream().cuda_stream)
+
+    def step_pushed(self, grad: torch.Tensor, lr: float, t: int, peers: PeerTable, barrier):
+        """One iteration of Algorithm 1 on this rank.  `barrier()` must order the ranks on the
+        current stream: nothing enqueued after it may start before every rank has finished what it
+        enqueued before (torch.distributed's NCCL barrier does)."""
+        if not self.opt.sync_due(t):
+            self.opt.step([grad], lr, t)
+        else:
+            self.push_pack(peers, grad, lr, t)
+        if t in self.var_steps:
+            g_bar = grad.clone()
+            dist.all_reduce(g_bar, op=dist.ReduceOp.SUM, group=self.group)
+            g_bar.div_(self.world)
+            self.variance(g_bar)
+        if self.opt.sync_due(t):
+            barrier()
+            self.push_serve(peers)
+            barrier()
+            if peers.copy_back:
+                self.opt.device_view("words_s")[:self.staged_words_s.numel()].copy_(self.staged_words_s)
+                self.opt.device_view("scales_s")[:self.staged_scales_s.numel()].copy_(self.staged_scales_s)
             self.apply()
