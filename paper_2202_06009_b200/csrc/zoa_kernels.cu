@@ -343,7 +343,7 @@ __global__ void step_sync_kernel(StateView st, GradPtrs g, Consts c, float gamma
 // starting at the range's first chunk.  Writes the server error, words_s and scales_s.
 // `out` lists where else the packed result of the range is to be stored (every rank's
 // words_s / scales_s, peer pointers included); out.world == 0 for none.
-__global__ void dist_server_kernel(StateView st, const uint32_t *words_in, long long words_in_stride,
+__global__ void __launch_bounds__(512, 3) dist_server_kernel(StateView st, const uint32_t *words_in, long long words_in_stride,
                                    const float *scales_in, long long scales_in_stride, int W_total,
                                    long long first_chunk, PeerOut out)
 {
@@ -1060,7 +1060,11 @@ cudaError_t launch_dist_server(const StateView &st, const uint32_t *words_in, lo
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    dist_server_kernel<<<(unsigned)count, block_threads_for_chunk(st.chunk), reduce_smem(st.chunk), s>>>(
+    // block size as for reduce_kernel: with few workers smaller blocks, more of them per SM
+    const int per_thread = W_total <= 2 ? 32 : 16;
+    int thr = 128;
+    while (thr < st.chunk / per_thread && thr < 512) thr <<= 1;
+    dist_server_kernel<<<(unsigned)count, thr, reduce_smem(st.chunk), s>>>(
         st, words_in, words_in_stride, scales_in, scales_in_stride, W_total, first_chunk, out);
     return cudaGetLastError();
 }
