@@ -14,6 +14,19 @@ from paper_2202_06009_b200.distributed import PeerTable, WorkerPerGpu
 pytestmark = pytest.mark.gpu
 
 
+def _one_rank_process_group():
+    """A one-rank NCCL group on a port nobody holds (each test makes and destroys its own)."""
+    import socket
+    import torch.distributed as dist
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", 0))
+    return dist
+
+
 @pytest.mark.parametrize("W,chunk,n", [(3, 1024, 7 * 1024 + 100), (4, 4096, 9 * 4096), (5, 256, 3 * 256 + 7), (2, 2048, 2048 * 5 + 33)])
 def test_emulated_ranks_equal_the_single_handle(W, chunk, n):
     rng = np.random.default_rng(W * n)
@@ -173,10 +186,7 @@ def test_peer_store_entry_points_reject_bad_tables():
 def test_pushed_driver_over_symmetric_memory_one_rank():
     """world_size 1 over NCCL with the buffers in torch's symmetric memory: the rendezvous, the
     address arithmetic of PeerTable.symmetric and the copy back into the handle run for real."""
-    import torch.distributed as dist
-    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-    os.environ.setdefault("MASTER_PORT", str(29900 + os.getpid() % 1000))
-    dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", 0))
+    dist = _one_rank_process_group()
     rng = np.random.default_rng(5)
     n, chunk = 6 * 1024 + 50, 1024
     ref = Zoa(n, 1, chunk=chunk)
@@ -204,10 +214,7 @@ def test_pushed_driver_over_symmetric_memory_one_rank():
 def test_driver_with_real_collectives_one_rank():
     """world_size 1 over NCCL: every collective of WorkerPerGpu.step runs for real; W = 1 must
     equal the plain single-worker handle."""
-    import torch.distributed as dist
-    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-    os.environ.setdefault("MASTER_PORT", str(29900 + os.getpid() % 1000))
-    dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", 0))
+    dist = _one_rank_process_group()
     rng = np.random.default_rng(3)
     n, chunk = 6 * 1024 + 50, 1024
     ref = Zoa(n, 1, chunk=chunk)
