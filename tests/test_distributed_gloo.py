@@ -11,6 +11,13 @@ import torch.multiprocessing as mp
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
+
+def _free_port():
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        return sock.getsockname()[1]
+
 def _worker(rank, world, port, n, chunk, out_dir):
     sys.path.insert(0, ROOT)
     os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
@@ -47,12 +54,12 @@ def _worker(rank, world, port, n, chunk, out_dir):
 
 
 def test_packed_exchange_three_ranks(tmp_path):
-    port = 29700 + os.getpid() % 2000
+    port = _free_port()
     mp.spawn(_worker, args=(3, port, 10 * 256 + 77, 256, str(tmp_path)), nprocs=3, join=True)
     assert (tmp_path / "ok").exists()
 
 
 def test_packed_exchange_more_ranks_than_chunks(tmp_path):
-    port = 31700 + os.getpid() % 2000
+    port = _free_port()
     mp.spawn(_worker, args=(4, port, 3 * 64 + 5, 64, str(tmp_path)), nprocs=4, join=True)
     assert (tmp_path / "ok").exists()

@@ -12,6 +12,13 @@ import torch.multiprocessing as mp
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
+
+def _free_port():
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        return sock.getsockname()[1]
+
 def _load_sharding():
     import importlib.util
     spec = importlib.util.spec_from_file_location("_sharding", os.path.join(ROOT, "paper_2202_06009_b200", "sharding.py"))
@@ -61,7 +68,7 @@ def _worker(rank, world, port, n, W, chunk, T, out_dir):
 
 
 def test_two_ranks_own_chunk_ranges(tmp_path):
-    port = 29500 + os.getpid() % 2000
+    port = _free_port()
     mp.spawn(_worker, args=(2, port, 5 * 256 + 77, 3, 256, 6, str(tmp_path)), nprocs=2, join=True)
     assert (tmp_path / "ok").exists()
 
