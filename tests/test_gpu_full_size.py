@@ -92,3 +92,9 @@ def test_bert_large_full_size_sampled_chunks():
 def test_gpt2_full_size_sampled_chunks():
     """1,557,611,200 parameters, W = 4, chunk 8192, Student-t noise; first 22 steps (sync, local and variance steps)."""
     _run(synth.gpt2_xl(), 22, {0, 3, 15, 16, 17, 19, 20, 21}, n_sample=24)
+
+
+def test_bert_base_full_size_sampled_chunks():
+    """110,106,428 parameters, W = 8, chunk 4096, all 200 steps of the schedule (sync every step,
+    every second, every fourth)."""
+    _run(synth.bert_base(), 200, {0, 1, 2, 31, 63, 64, 65, 66, 127, 128, 129, 130, 131, 132, 199})
