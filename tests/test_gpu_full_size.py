@@ -90,8 +90,8 @@ def test_bert_large_full_size_sampled_chunks():
 
 
 def test_gpt2_full_size_sampled_chunks():
-    """1,557,611,200 parameters, W = 4, chunk 8192, Student-t noise; first 22 steps (sync, local and variance steps)."""
-    _run(synth.gpt2_xl(), 22, {0, 3, 15, 16, 17, 19, 20, 21}, n_sample=24)
+    """1,557,611,200 parameters, W = 4, chunk 8192, Student-t noise; all 50 steps of the schedule."""
+    _run(synth.gpt2_xl(), 50, {0, 3, 15, 16, 17, 19, 20, 21, 32, 33, 36, 47, 48, 49}, n_sample=24)
 
 
 def test_bert_base_full_size_sampled_chunks():
