@@ -27,7 +27,7 @@ def _sample_chunks(wl, count, seed):
     return sorted(picks)[:count - 1] + [n_chunks - 1]    # the ragged last chunk stays last
 
 
-def _run(wl, steps, check_at, n_sample=40):
+def _run(wl, steps, check_at, n_sample=40, algorithm="alg1", grad_dtype=torch.float32):
     torch.cuda.empty_cache()
     free, _ = torch.cuda.mem_get_info()
     need = (5 * wl.W + 6) * wl.n * 4
@@ -46,15 +46,25 @@ def _run(wl, steps, check_at, n_sample=40):
         gpu.set_params(x0)
         del x0
         gpu.set_policies(wl.var_steps, wl.sync_boundaries, wl.sync_intervals)
+        gpu.set_grad_dtype(grad_dtype)
+        g16 = None if grad_dtype == torch.float32 else [torch.empty(wl.n, device="cuda", dtype=grad_dtype) for _ in range(wl.W)]
 
         def gather(name, worker=0):
             return np.concatenate([gpu.read(name, worker, a, b - a) for a, b in spans])
 
         for t in range(steps):
             bufs = stream.fill(t)
-            g = np.stack([b[idx].cpu().numpy() for b in bufs])
-            gpu.step_auto(bufs, wl.lr_at(t), t)
-            assert cpu.step(g, np.float32(wl.lr_at(t)), t, wl.in_T_u(t), wl.in_T_v(t)) == 0
+            if g16 is not None:                       # the oracle gets the binary32 values of the 16-bit numbers
+                for dst, src in zip(g16, bufs):
+                    dst.copy_(src)
+                bufs = g16
+            g = np.stack([b[idx].float().cpu().numpy() for b in bufs])
+            if algorithm == "alg2":
+                gpu.alg2_step(bufs, wl.lr_at(t), t)
+                cpu.alg2_step(g, np.float32(wl.lr_at(t)), wl.in_T_v(t))
+            else:
+                gpu.step_auto(bufs, wl.lr_at(t), t)
+                assert cpu.step(g, np.float32(wl.lr_at(t)), t, wl.in_T_u(t), wl.in_T_v(t)) == 0
             if t in check_at:
                 torch.cuda.synchronize()
                 for i in range(wl.W):
@@ -65,7 +75,7 @@ def _run(wl, steps, check_at, n_sample=40):
                 assert_close(gather("v"), cpu.v, f"t={t} v")
                 assert_close(gather("delta_s"), cpu.delta_bar, f"t={t} delta_s")
                 assert_close(gather("x_sync"), cpu.x_sync, f"t={t} x_sync")
-                if wl.in_T_u(t):
+                if wl.in_T_u(t) and algorithm == "alg1":
                     # packed words, bit-exact: oracle word k of sampled chunk j <-> GPU word (start_j/32 + k)
                     per = wl.chunk // 32
                     for j, (a, b) in enumerate(spans):
@@ -98,3 +108,16 @@ def test_bert_base_full_size_sampled_chunks():
     """110,106,428 parameters, W = 8, chunk 4096, all 200 steps of the schedule (sync every step,
     every second, every fourth)."""
     _run(synth.bert_base(), 200, {0, 1, 2, 31, 63, 64, 65, 66, 127, 128, 129, 130, 131, 132, 199})
+
+
+def test_bert_large_full_size_algorithm_2():
+    """The configuration `bench.py --algorithm alg2` times: full-precision steps on T_v, compressed
+    gradients through the ring kernel otherwise; first 20 steps."""
+    _run(synth.bert_large(), 20, {0, 1, 2, 3, 4, 5, 8, 9, 16, 17, 19}, n_sample=24, algorithm="alg2")
+
+
+def test_bert_large_full_size_bfloat16_gradients():
+    """The configuration `bench.py --grad-dtype bf16` times; first 12 steps and two local steps."""
+    wl = synth.bert_large()
+    wl.sync_boundaries, wl.sync_intervals = (0, 8), (1, 2)
+    _run(wl, 12, {0, 1, 2, 7, 8, 9, 10, 11}, n_sample=24, grad_dtype=torch.bfloat16)
