@@ -63,7 +63,12 @@ def _run(wl, steps, check_at, n_sample=40, algorithm="alg1", grad_dtype=torch.fl
                 gpu.alg2_step(bufs, wl.lr_at(t), t)
                 cpu.alg2_step(g, np.float32(wl.lr_at(t)), wl.in_T_v(t))
             else:
-                gpu.step_auto(bufs, wl.lr_at(t), t)
+                if algorithm == "two_call":
+                    gpu.step(bufs, wl.lr_at(t), t)
+                    if wl.in_T_u(t):
+                        gpu.onebit_reduce()
+                else:
+                    gpu.step_auto(bufs, wl.lr_at(t), t)
                 assert cpu.step(g, np.float32(wl.lr_at(t)), t, wl.in_T_u(t), wl.in_T_v(t)) == 0
             if t in check_at:
                 torch.cuda.synchronize()
@@ -75,7 +80,7 @@ def _run(wl, steps, check_at, n_sample=40, algorithm="alg1", grad_dtype=torch.fl
                 assert_close(gather("v"), cpu.v, f"t={t} v")
                 assert_close(gather("delta_s"), cpu.delta_bar, f"t={t} delta_s")
                 assert_close(gather("x_sync"), cpu.x_sync, f"t={t} x_sync")
-                if wl.in_T_u(t) and algorithm == "alg1":
+                if wl.in_T_u(t) and algorithm != "alg2":
                     # packed words, bit-exact: oracle word k of sampled chunk j <-> GPU word (start_j/32 + k)
                     per = wl.chunk // 32
                     for j, (a, b) in enumerate(spans):
@@ -121,3 +126,10 @@ def test_bert_large_full_size_bfloat16_gradients():
     wl = synth.bert_large()
     wl.sync_boundaries, wl.sync_intervals = (0, 8), (1, 2)
     _run(wl, 12, {0, 1, 2, 7, 8, 9, 10, 11}, n_sample=24, grad_dtype=torch.bfloat16)
+
+
+def test_bert_large_full_size_two_call_path():
+    """The configuration `bench.py --two-call` times: zoa_step, then zoa_onebit_reduce on sync steps."""
+    wl = synth.bert_large()
+    wl.sync_boundaries, wl.sync_intervals = (0, 4), (1, 2)
+    _run(wl, 8, {0, 1, 3, 4, 5, 6, 7}, n_sample=24, algorithm="two_call")
