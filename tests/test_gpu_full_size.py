@@ -133,3 +133,53 @@ def test_bert_large_full_size_two_call_path():
     wl = synth.bert_large()
     wl.sync_boundaries, wl.sync_intervals = (0, 4), (1, 2)
     _run(wl, 8, {0, 1, 3, 4, 5, 6, 7}, n_sample=24, algorithm="two_call")
+
+
+def test_bert_large_full_size_whole_vector_properties():
+    """What must hold for every coordinate after a sync step, checked over the whole vector with
+    plain torch operations (no sampling): all workers hold the same model, equal to x_sync; the
+    buffer is zero; the momentum is +-(server magnitude of the chunk) / (sum of learning rates)
+    with the sign the server's packed word carries; rows end in zero padding."""
+    wl = synth.bert_large()
+    torch.cuda.empty_cache()
+    free, _ = torch.cuda.mem_get_info()
+    if free < (5 * wl.W + 8) * wl.n * 4 * 1.03:
+        pytest.skip("not enough device memory")
+    stream = synth.GradientStream(wl, "cuda")
+    gpu = Zoa(wl.n, wl.W, wl.beta1, wl.beta2, wl.eps, wl.chunk)
+    try:
+        gpu.set_params(synth.initial_params(wl, "cuda"))
+        gpu.set_policies(wl.var_steps, (0, 2), (1, 2))
+        lrs = [1e-3, 5e-4, 2.5e-4, 1e-3, 7e-4]
+        for t in range(5):                                      # sync at 0, 1, 2, 4; local at 3: the last sync spans two steps
+            gpu.step_auto(stream.fill(t), lrs[t], t)
+        torch.cuda.synchronize()
+        n, chunk = wl.n, wl.chunk
+        gamma_sum = np.float32(np.float64(np.float32(lrs[3])) + np.float64(np.float32(lrs[4])))
+        x_sync = gpu.device_view("x_sync")
+        words = gpu.device_view("words_s")
+        scales = gpu.device_view("scales_s")
+        n_chunks = -(-n // chunk)
+        m_mag = scales[:n_chunks] / torch.tensor(gamma_sum, device="cuda")          # one IEEE division per chunk
+        for i in range(wl.W):
+            assert torch.equal(gpu.device_view("x", i), x_sync), f"x[{i}] differs from x_sync"
+            assert not gpu.device_view("u", i).any(), f"u[{i}] is not zero"
+        shifts = torch.arange(32, device="cuda", dtype=torch.int32)
+        span = 1 << 24                                          # coordinates per slice, a multiple of the chunk size
+        for lo in range(0, n, span):
+            hi = min(lo + span, n)
+            w = words[lo // 32:(hi + 31) // 32]
+            bits = ((w[:, None] >> shifts[None, :]) & 1).reshape(-1)[:hi - lo].bool()
+            mag = m_mag[lo // chunk:(hi + chunk - 1) // chunk].repeat_interleave(chunk)[:hi - lo]
+            want = torch.where(bits, mag, -mag)
+            for i in (0, wl.W // 2, wl.W - 1):
+                assert torch.equal(gpu.device_view("m", i)[lo:hi], want), f"m[{i}] in [{lo}, {hi})"
+        pad = (-n) % 128
+        if pad:
+            for name in ("x", "m", "u", "delta_w"):
+                assert not gpu.device_view(name, wl.W - 1)[n:n + pad].any()
+        gpu.check_device()
+    finally:
+        gpu.close()
+        del stream
+        torch.cuda.empty_cache()
