@@ -183,3 +183,97 @@ def test_bert_large_full_size_whole_vector_properties():
         gpu.close()
         del stream
         torch.cuda.empty_cache()
+
+
+def _unpack(words, count):
+    shifts = torch.arange(32, device=words.device, dtype=torch.int32)
+    return ((words[:, None] >> shifts[None, :]) & 1).reshape(-1)[:count].bool()
+
+
+def test_bert_base_full_size_every_coordinate_against_torch_arithmetic():
+    """Three sync steps of the BERT-Base-shaped configuration, every coordinate of every worker:
+    the step is worked out again from the state before it with plain torch operations (one IEEE
+    binary32 operation each, binary64 for the three reductions) and compared exactly; only the
+    per-chunk magnitudes get one unit in the last place, since a binary64 sum taken in another
+    order may round to the neighbouring binary32 value."""
+    wl = synth.bert_base()
+    n, W, chunk = wl.n, wl.W, wl.chunk
+    n_chunks, n_full = -(-n // chunk), n // chunk
+    f32 = lambda v: float(np.float32(v))
+    b1, b2, eps = f32(wl.beta1), f32(wl.beta2), f32(wl.eps)
+    ob1, ob2 = f32(np.float32(1) - np.float32(wl.beta1)), f32(np.float32(1) - np.float32(wl.beta2))
+    stream = synth.GradientStream(wl, "cuda")
+    gpu = Zoa(n, W, wl.beta1, wl.beta2, wl.eps, chunk)
+
+    def chunk_l1_scale(z):
+        """Eq. 3 magnitudes of a whole row: binary64 sums per chunk, one rounding."""
+        a = z[:n].abs().double()
+        s = a[:n_full * chunk].view(n_full, chunk).sum(1) / chunk
+        if n_chunks > n_full:
+            s = torch.cat([s, (a[n_full * chunk:].sum() / (n - n_full * chunk)).reshape(1)])
+        return s.float()
+
+    def per_coordinate(scales):
+        return scales.repeat_interleave(chunk)[:n]
+
+    def close_to_one_ulp(got, want, what):
+        bad = ~torch.isclose(got, want, rtol=1.3e-7, atol=0.0)
+        assert not bad.any(), f"{what}: {int(bad.sum())} magnitudes differ by more than one unit in the last place"
+
+    try:
+        gpu.set_params(synth.initial_params(wl, "cuda"))
+        gpu.set_policies((0, 1), (0,), (1,))
+        for t, lr in enumerate([1e-3, 5e-4, 2e-3]):
+            gamma = f32(lr)
+            before = {k: [gpu.device_view(k, i).clone() for i in range(W)] for k in ("m", "u", "delta_w")}
+            ds_old, xs_old = gpu.device_view("delta_s").clone(), gpu.device_view("x_sync").clone()
+            v_old = gpu.device_view("v").clone()
+            g = stream.fill(t)
+            gpu.step_auto(g, lr, t)
+            torch.cuda.synchronize()
+
+            A = torch.zeros(n, dtype=torch.float64, device="cuda")
+            for i in range(W):
+                m_half = before["m"][i][:n] * b1 + g[i] * ob1                      # momentum update
+                z = (before["u"][i][:n] + m_half * gamma) + before["delta_w"][i][:n]
+                s_gpu = gpu.device_view("scales_w", i)[:n_chunks]
+                close_to_one_ulp(s_gpu, chunk_l1_scale(z), f"t={t} scales_w[{i}]")
+                bits = z >= 0
+                assert torch.equal(_unpack(gpu.device_view("words_w", i), n), bits), f"t={t} words_w[{i}]"
+                s = per_coordinate(s_gpu)
+                z_hat = torch.where(bits, s, -s)
+                assert torch.equal(gpu.device_view("delta_w", i)[:n], z - z_hat), f"t={t} delta_w[{i}]"
+                A += z_hat.double()                                                 # worker order; exact in binary64
+                del m_half, z, bits, s, z_hat
+            a = (A / torch.tensor(float(W), dtype=torch.float64, device="cuda") + ds_old[:n].double()).float()
+            del A
+            s_gpu = gpu.device_view("scales_s")[:n_chunks]
+            close_to_one_ulp(s_gpu, chunk_l1_scale(a), f"t={t} scales_s")
+            bits = a >= 0
+            assert torch.equal(_unpack(gpu.device_view("words_s"), n), bits), f"t={t} words_s"
+            s = per_coordinate(s_gpu)
+            z_bar = torch.where(bits, s, -s)
+            assert torch.equal(gpu.device_view("delta_s")[:n], a - z_bar), f"t={t} delta_s"
+            x_new = xs_old[:n] - z_bar / (v_old[:n] + eps).sqrt()                    # model sync, with v_t
+            # momentum approximation (one step since the last sync); a tensor divisor, because torch
+            # turns division by a Python scalar into a multiplication by its reciprocal
+            m_new = z_bar / torch.tensor(gamma, device="cuda")
+            assert torch.equal(gpu.device_view("x_sync")[:n], x_new), f"t={t} x_sync"
+            for i in range(W):
+                assert torch.equal(gpu.device_view("x", i)[:n], x_new), f"t={t} x[{i}]"
+                assert torch.equal(gpu.device_view("m", i)[:n], m_new), f"t={t} m[{i}]"
+                assert not gpu.device_view("u", i).any(), f"t={t} u[{i}]"
+            if t in (0, 1):                                                           # variance update, effective from the next step
+                G = torch.zeros(n, dtype=torch.float64, device="cuda")
+                for i in range(W):
+                    G += g[i].double()
+                g_bar = (G / torch.tensor(float(W), dtype=torch.float64, device="cuda")).float()
+                assert torch.equal(gpu.device_view("v")[:n], v_old[:n] * b2 + (g_bar * g_bar) * ob2), f"t={t} v"
+            else:
+                assert torch.equal(gpu.device_view("v"), v_old), f"t={t} v changed outside T_v"
+            del before, a, bits, s, z_bar, x_new, m_new
+        gpu.check_device()
+    finally:
+        gpu.close()
+        del stream
+        torch.cuda.empty_cache()
