@@ -191,7 +191,8 @@ def _unpack(words, count):
 
 
 def test_bert_base_full_size_every_coordinate_against_torch_arithmetic():
-    """Three sync steps of the BERT-Base-shaped configuration, every coordinate of every worker:
+    """Four sync steps and a local step of the BERT-Base-shaped configuration (the last sync spans
+    two learning rates), every coordinate of every worker:
     the step is worked out again from the state before it with plain torch operations (one IEEE
     binary32 operation each, binary64 for the three reductions) and compared exactly; only the
     per-chunk magnitudes get one unit in the last place, since a binary64 sum taken in another
@@ -222,15 +223,33 @@ def test_bert_base_full_size_every_coordinate_against_torch_arithmetic():
 
     try:
         gpu.set_params(synth.initial_params(wl, "cuda"))
-        gpu.set_policies((0, 1), (0,), (1,))
-        for t, lr in enumerate([1e-3, 5e-4, 2e-3]):
+        gpu.set_policies((0, 1), (0, 2), (1, 2))                  # sync at t = 0, 1, 2, 4; t = 3 is a local step
+        lrs = [1e-3, 5e-4, 2e-3, 7e-4, 1e-3]
+        for t, lr in enumerate(lrs):
             gamma = f32(lr)
             before = {k: [gpu.device_view(k, i).clone() for i in range(W)] for k in ("m", "u", "delta_w")}
             ds_old, xs_old = gpu.device_view("delta_s").clone(), gpu.device_view("x_sync").clone()
             v_old = gpu.device_view("v").clone()
+            x_old = [gpu.device_view("x", i).clone() for i in range(W)] if t == 3 else None
             g = stream.fill(t)
             gpu.step_auto(g, lr, t)
             torch.cuda.synchronize()
+
+            if t == 3:                                                # local step: momentum, model and buffer updates
+                den = (v_old[:n] + eps).sqrt()
+                for i in range(W):
+                    m_half = before["m"][i][:n] * b1 + g[i] * ob1
+                    step = m_half * gamma
+                    assert torch.equal(gpu.device_view("m", i)[:n], m_half), f"t={t} m[{i}]"
+                    assert torch.equal(gpu.device_view("x", i)[:n], x_old[i][:n] - step / den), f"t={t} x[{i}]"
+                    assert torch.equal(gpu.device_view("u", i)[:n], before["u"][i][:n] + step), f"t={t} u[{i}]"
+                    assert torch.equal(gpu.device_view("delta_w", i), before["delta_w"][i]), f"t={t} delta_w[{i}]"
+                assert torch.equal(gpu.device_view("delta_s"), ds_old) and torch.equal(gpu.device_view("x_sync"), xs_old)
+                assert torch.equal(gpu.device_view("v"), v_old)
+                del before, x_old, den
+                continue
+            # sum of the learning rates since the last sync: binary64 sum of the binary32 values, rounded once
+            gamma_sum = f32(np.float64(np.float32(lrs[3])) + np.float64(np.float32(lrs[4]))) if t == 4 else gamma
 
             A = torch.zeros(n, dtype=torch.float64, device="cuda")
             for i in range(W):
@@ -255,9 +274,9 @@ def test_bert_base_full_size_every_coordinate_against_torch_arithmetic():
             z_bar = torch.where(bits, s, -s)
             assert torch.equal(gpu.device_view("delta_s")[:n], a - z_bar), f"t={t} delta_s"
             x_new = xs_old[:n] - z_bar / (v_old[:n] + eps).sqrt()                    # model sync, with v_t
-            # momentum approximation (one step since the last sync); a tensor divisor, because torch
+            # momentum approximation; a tensor divisor, because torch
             # turns division by a Python scalar into a multiplication by its reciprocal
-            m_new = z_bar / torch.tensor(gamma, device="cuda")
+            m_new = z_bar / torch.tensor(gamma_sum, device="cuda")
             assert torch.equal(gpu.device_view("x_sync")[:n], x_new), f"t={t} x_sync"
             for i in range(W):
                 assert torch.equal(gpu.device_view("x", i)[:n], x_new), f"t={t} x[{i}]"
