@@ -190,14 +190,13 @@ def _unpack(words, count):
     return ((words[:, None] >> shifts[None, :]) & 1).reshape(-1)[:count].bool()
 
 
-def test_bert_base_full_size_every_coordinate_against_torch_arithmetic():
-    """Four sync steps and a local step of the BERT-Base-shaped configuration (the last sync spans
-    two learning rates), every coordinate of every worker:
+def _every_coordinate_against_torch_arithmetic(wl):
+    """Four sync steps and a local step (the last sync spans two learning rates), every coordinate
+    of every worker:
     the step is worked out again from the state before it with plain torch operations (one IEEE
     binary32 operation each, binary64 for the three reductions) and compared exactly; only the
     per-chunk magnitudes get one unit in the last place, since a binary64 sum taken in another
     order may round to the neighbouring binary32 value."""
-    wl = synth.bert_base()
     n, W, chunk = wl.n, wl.W, wl.chunk
     n_chunks, n_full = -(-n // chunk), n // chunk
     f32 = lambda v: float(np.float32(v))
@@ -296,3 +295,13 @@ def test_bert_base_full_size_every_coordinate_against_torch_arithmetic():
         gpu.close()
         del stream
         torch.cuda.empty_cache()
+
+
+def test_bert_base_full_size_every_coordinate_against_torch_arithmetic():
+    _every_coordinate_against_torch_arithmetic(synth.bert_base())
+
+
+def test_gpt2_shaped_every_coordinate_against_torch_arithmetic():
+    """The GPT-2-shaped layout shrunk 8x (194,701,400 parameters, W = 4, chunk 8192, Student-t noise):
+    the four-tile ring kernel, with and without the fused variance update."""
+    _every_coordinate_against_torch_arithmetic(synth.scaled(synth.gpt2_xl(), 8))
