@@ -305,3 +305,84 @@ def test_gpt2_shaped_every_coordinate_against_torch_arithmetic():
     """The GPT-2-shaped layout shrunk 8x (194,701,400 parameters, W = 4, chunk 8192, Student-t noise):
     the four-tile ring kernel, with and without the fused variance update."""
     _every_coordinate_against_torch_arithmetic(synth.scaled(synth.gpt2_xl(), 8))
+
+
+def test_bert_base_full_size_algorithm_2_every_coordinate_against_torch_arithmetic():
+    """Algorithm 2 on the BERT-Base-shaped configuration: two full-precision steps (T_v) and two
+    compressed ones, every coordinate of every worker worked out again with plain torch operations."""
+    wl = synth.bert_base()
+    n, W, chunk = wl.n, wl.W, wl.chunk
+    n_chunks, n_full = -(-n // chunk), n // chunk
+    f32 = lambda v: float(np.float32(v))
+    b1, b2, eps = f32(wl.beta1), f32(wl.beta2), f32(wl.eps)
+    ob1, ob2 = f32(np.float32(1) - np.float32(wl.beta1)), f32(np.float32(1) - np.float32(wl.beta2))
+    W64 = torch.tensor(float(W), dtype=torch.float64, device="cuda")
+    stream = synth.GradientStream(wl, "cuda")
+    gpu = Zoa(n, W, wl.beta1, wl.beta2, wl.eps, chunk)
+
+    def chunk_l1_scale(z):
+        a = z[:n].abs().double()
+        s = a[:n_full * chunk].view(n_full, chunk).sum(1) / chunk
+        if n_chunks > n_full:
+            s = torch.cat([s, (a[n_full * chunk:].sum() / (n - n_full * chunk)).reshape(1)])
+        return s.float()
+
+    def one_ulp(got, want, what):
+        bad = ~torch.isclose(got, want, rtol=1.3e-7, atol=0.0)
+        assert not bad.any(), f"{what}: {int(bad.sum())} magnitudes differ by more than one unit in the last place"
+
+    try:
+        gpu.set_params(synth.initial_params(wl, "cuda"))
+        gpu.set_policies((0, 1), (0,), (1,))
+        for t, lr in enumerate([1e-3, 5e-4, 2e-3, 1e-3]):
+            gamma = f32(lr)
+            m_old = [gpu.device_view("m", i).clone() for i in range(W)]
+            x_old = [gpu.device_view("x", i).clone() for i in range(W)]
+            d_old = [gpu.device_view("delta_w", i).clone() for i in range(W)]
+            ds_old, v_old = gpu.device_view("delta_s").clone(), gpu.device_view("v").clone()
+            g = stream.fill(t)
+            gpu.alg2_step(g, lr, t)
+            torch.cuda.synchronize()
+            den = (v_old[:n] + eps).sqrt()
+            if t < 2:                                      # full-precision exchange, then the variance
+                G = torch.zeros(n, dtype=torch.float64, device="cuda")
+                for i in range(W):
+                    G += g[i].double()
+                g_bar = (G / W64).float()
+                assert torch.equal(gpu.device_view("v")[:n], v_old[:n] * b2 + (g_bar * g_bar) * ob2), f"t={t} v"
+                for i in range(W):
+                    assert torch.equal(gpu.device_view("delta_w", i), d_old[i]), f"t={t} delta_w[{i}]"
+                assert torch.equal(gpu.device_view("delta_s"), ds_old), f"t={t} delta_s"
+            else:                                          # gradients through the 1-bit AllReduce
+                A = torch.zeros(n, dtype=torch.float64, device="cuda")
+                for i in range(W):
+                    z = g[i] + d_old[i][:n]
+                    s_gpu = gpu.device_view("scales_w", i)[:n_chunks]
+                    one_ulp(s_gpu, chunk_l1_scale(z), f"t={t} scales_w[{i}]")
+                    bits = z >= 0
+                    assert torch.equal(_unpack(gpu.device_view("words_w", i), n), bits), f"t={t} words_w[{i}]"
+                    s = s_gpu.repeat_interleave(chunk)[:n]
+                    z_hat = torch.where(bits, s, -s)
+                    assert torch.equal(gpu.device_view("delta_w", i)[:n], z - z_hat), f"t={t} delta_w[{i}]"
+                    A += z_hat.double()
+                    del z, bits, s, z_hat
+                a = (A / W64 + ds_old[:n].double()).float()
+                s_gpu = gpu.device_view("scales_s")[:n_chunks]
+                one_ulp(s_gpu, chunk_l1_scale(a), f"t={t} scales_s")
+                bits = a >= 0
+                assert torch.equal(_unpack(gpu.device_view("words_s"), n), bits), f"t={t} words_s"
+                s = s_gpu.repeat_interleave(chunk)[:n]
+                g_bar = torch.where(bits, s, -s)
+                assert torch.equal(gpu.device_view("delta_s")[:n], a - g_bar), f"t={t} delta_s"
+                assert torch.equal(gpu.device_view("v"), v_old), f"t={t} v changed outside T_v"
+                del A, a, bits, s
+            for i in range(W):
+                m_new = m_old[i][:n] * b1 + g_bar * ob1
+                assert torch.equal(gpu.device_view("m", i)[:n], m_new), f"t={t} m[{i}]"
+                assert torch.equal(gpu.device_view("x", i)[:n], x_old[i][:n] - (m_new * gamma) / den), f"t={t} x[{i}]"
+            del m_old, x_old, d_old, g_bar, den
+        gpu.check_device()
+    finally:
+        gpu.close()
+        del stream
+        torch.cuda.empty_cache()
