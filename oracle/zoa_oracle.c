@@ -269,21 +269,21 @@ void ZO(zo_alg2_step)(ZO(zo_state) *st, const real *g, real gamma, int in_T_v, r
     const real one_minus_beta1 = (real)1 - st->beta1, one_minus_beta2 = (real)1 - st->beta2;
     const real *g_bar = g_bar_scratch;
     if (in_T_v) {
-        ZO(zo_allreduce)(g, st->n, st->d, g_bar_scratch);                  /* model update */
+        ZO(zo_allreduce)(g, st->n, st->d, g_bar_scratch);                  /* AllReduce (t in T_v) */
     } else {
-        ZO(zo_onebit_allreduce)(st, g);                                    /* 1-bit AllReduce */
+        ZO(zo_onebit_allreduce)(st, g);                                    /* Compressed-AllReduce (Algorithm 3) */
         g_bar = st->u_bar;
     }
     for (int i = 0; i < st->n; ++i)
         for (int64_t j = 0; j < st->d; ++j) {
             size_t k = (size_t)i * st->d + j;
             real m_prev = st->m[k];
-            real m_next = st->beta1 * m_prev + one_minus_beta1 * g_bar[j]; /* buffer reset */
+            real m_next = st->beta1 * m_prev + one_minus_beta1 * g_bar[j]; /* Update momentum */
             real m_used = st->literal_momentum ? m_prev : m_next;          /* R9 */
-            st->x[k] = st->x[k] - (gamma * m_used) / ZO(zo_sqrt)(st->v[j] + st->eps); /* t' = t */
+            st->x[k] = st->x[k] - (gamma * m_used) / ZO(zo_sqrt)(st->v[j] + st->eps); /* Update model (reads v_t) */
             st->m[k] = m_next;
         }
     if (in_T_v)
         for (int64_t j = 0; j < st->d; ++j)
-            st->v[j] = st->beta2 * st->v[j] + one_minus_beta2 * (g_bar[j] * g_bar[j]); /* buffer update */
+            st->v[j] = st->beta2 * st->v[j] + one_minus_beta2 * (g_bar[j] * g_bar[j]); /* Set v_{t+1} (else v_{t+1} = v_t) */
 }

@@ -535,7 +535,7 @@ alg2_full_kernel(StateView st, GradPtrs g, Consts c, float gamma, int g_fmt_arg)
         for (int k = 0; k < 4; ++k) {
             gb[k] = mean_round(G[k], st.W);                     // full-precision mean (Algorithm 4)
             d[k] = denom(c, vv[k]);
-            vo[k] = variance(c, vv[k], gb[k]);                  // buffer update
+            vo[k] = variance(c, vv[k], gb[k]);                  // set v_{t+1}
         }
         st4(st.v_next + j, make_float4(vo[0], vo[1], vo[2], vo[3]));
         for (int i = 0; i < st.W; ++i) {
@@ -545,8 +545,8 @@ alg2_full_kernel(StateView st, GradPtrs g, Consts c, float gamma, int g_fmt_arg)
             float mo[4], xo[4];
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                mo[k] = momentum(c, mm[k], gb[k]);                              // momentum update
-                xo[k] = f_sub(xx[k], f_div(f_mul(gamma, mo[k]), d[k]));         // model update
+                mo[k] = momentum(c, mm[k], gb[k]);                              // update momentum
+                xo[k] = f_sub(xx[k], f_div(f_mul(gamma, mo[k]), d[k]));         // update model (reads v_t)
             }
             st4(st.m + row, make_float4(mo[0], mo[1], mo[2], mo[3]));
             st4(st.x + row, make_float4(xo[0], xo[1], xo[2], xo[3]));
