@@ -1,13 +1,17 @@
 """One worker per GPU, checked on one GPU: the ranks are emulated as separate handles in one
 process (each with a single worker and its own server range), the collectives by plain copies
-between their buffers; the result must equal the single handle that holds all W workers, bit
-for bit.  A second test runs the real driver, collectives included, as a one-rank NCCL job."""
+between their buffers; the result must equal the CPU oracle of Algorithm 1 / Algorithm 3 (worker
+side on every rank, server side on the range each rank serves) within the parity tolerance with
+bit-exact packed words, and the single handle that holds all W workers bit for bit.  A second
+test runs the real driver, collectives included, as a one-rank NCCL job."""
 import os
 
 import numpy as np
 import pytest
 import torch
 
+from helpers import assert_close
+from oracle import zoa_oracle as zo
 from paper_2202_06009_b200 import Zoa
 from paper_2202_06009_b200.distributed import PeerTable, WorkerPerGpu
 
@@ -27,21 +31,47 @@ def _one_rank_process_group():
     return dist
 
 
+def _compare_ranks_with_oracle(ranks, cpu, chunk, n, t, synced, worker_wire=True):
+    """Every rank against the oracle that holds all the workers: rank r is worker r of Algorithm 1
+    and the server of Algorithm 3 for its own chunk range."""
+    for r, w in enumerate(ranks):
+        what = f"rank {r} t={t}"
+        assert_close(w.opt.read("x", 0), cpu.x[r], f"{what} x")
+        assert_close(w.opt.read("m", 0), cpu.m[r], f"{what} m")
+        assert_close(w.opt.read("u", 0), cpu.u[r], f"{what} u")
+        assert_close(w.opt.read("delta_w", 0), cpu.delta[r], f"{what} delta_w")
+        assert_close(w.opt.read("v"), cpu.v, f"{what} v")
+        assert_close(w.opt.read("x_sync"), cpu.x_sync, f"{what} x_sync")
+        cr = w.plan.chunks[r]
+        lo, hi = cr.start * chunk, min(cr.stop * chunk, n)
+        if hi > lo:
+            assert_close(w.opt.read("delta_s", 0, lo, hi - lo), cpu.delta_bar[lo:hi], f"{what} delta_s of the served range")
+        if synced:
+            if worker_wire:
+                assert np.array_equal(w.opt.read("words_w", 0), cpu.words_worker[r]), f"{what} words_w"
+                assert_close(w.opt.read("scales_w", 0), cpu.scales_worker[r], f"{what} scales_w")
+            assert np.array_equal(w.opt.read("words_s"), cpu.words_server), f"{what} words_s"
+            assert_close(w.opt.read("scales_s"), cpu.scales_server, f"{what} scales_s")
+
+
 @pytest.mark.parametrize("W,chunk,n", [(3, 1024, 7 * 1024 + 100), (4, 4096, 9 * 4096), (5, 256, 3 * 256 + 7), (2, 2048, 2048 * 5 + 33)])
 def test_emulated_ranks_equal_the_single_handle(W, chunk, n):
     rng = np.random.default_rng(W * n)
     var_steps, sync = (0, 1, 3), ((0, 3), (1, 2))
     x0 = torch.from_numpy((rng.standard_normal(n) * 0.02).astype(np.float32))
     ref = Zoa(n, W, chunk=chunk)
+    cpu = zo.Oracle(n, W, chunk, dtype=np.float32)
     ranks = [WorkerPerGpu(n, chunk, r, W, var_steps, *sync) for r in range(W)]
     try:
         ref.set_params(x0)
         ref.set_policies(var_steps, *sync)
+        cpu.set_params(x0.numpy())
         for w in ranks:
             w.opt.set_params(x0)
         for t in range(7):
             g = torch.from_numpy(rng.standard_normal((W, n)).astype(np.float32)).cuda()
             ref.step_auto(list(g), 1e-3, t)
+            assert cpu.step(g.cpu().numpy(), np.float32(1e-3), t, ref.sync_due(t), t in var_steps) == 0
             for r, w in enumerate(ranks):
                 w.opt.step([g[r]], 1e-3, t)
             if t in var_steps:                       # stands in for the all-reduce: the same worker-order binary64 mean
@@ -70,6 +100,7 @@ def test_emulated_ranks_equal_the_single_handle(W, chunk, n):
                 for w in ranks:
                     w.apply()
             torch.cuda.synchronize()
+            _compare_ranks_with_oracle(ranks, cpu, chunk, n, t, ref.sync_due(t))
             for r, w in enumerate(ranks):
                 for name in ("x", "m", "u", "delta_w"):
                     assert np.array_equal(w.opt.read(name, 0), ref.read(name, r)), (name, r, t)
@@ -116,10 +147,12 @@ def test_exchange_by_peer_stores_equals_the_single_handle(W, chunk, n, fused):
     var_steps, sync = (0, 1, 3), ((0, 3), (1, 2))
     x0 = torch.from_numpy((rng.standard_normal(n) * 0.02).astype(np.float32))
     ref = Zoa(n, W, chunk=chunk)
+    cpu = zo.Oracle(n, W, chunk, dtype=np.float32)
     ranks = [WorkerPerGpu(n, chunk, r, W, var_steps, *sync) for r in range(W)]
     try:
         ref.set_params(x0)
         ref.set_policies(var_steps, *sync)
+        cpu.set_params(x0.numpy())
         for w in ranks:
             w.opt.set_params(x0)
         peers = PeerTable.local(ranks)
@@ -127,6 +160,7 @@ def test_exchange_by_peer_stores_equals_the_single_handle(W, chunk, n, fused):
             g = torch.from_numpy(rng.standard_normal((W, n)).astype(np.float32)).cuda()
             ref.step_auto(list(g), 1e-3, t)
             synced = ref.sync_due(t)
+            assert cpu.step(g.cpu().numpy(), np.float32(1e-3), t, synced, t in var_steps) == 0
             for r, w in enumerate(ranks):
                 if synced and fused:
                     w.push_pack(peers, g[r], 1e-3, t)
@@ -148,6 +182,7 @@ def test_exchange_by_peer_stores_equals_the_single_handle(W, chunk, n, fused):
                 for w in ranks:
                     w.apply()
             torch.cuda.synchronize()
+            _compare_ranks_with_oracle(ranks, cpu, chunk, n, t, synced)
             _compare_ranks_with_single_handle(ranks, ref, chunk, n, t, synced)
         for w in ranks:
             w.opt.check_device()
@@ -190,6 +225,7 @@ def test_pushed_driver_over_symmetric_memory_one_rank():
     rng = np.random.default_rng(5)
     n, chunk = 6 * 1024 + 50, 1024
     ref = Zoa(n, 1, chunk=chunk)
+    cpu = zo.Oracle(n, 1, chunk, dtype=np.float32)
     w = WorkerPerGpu(n, chunk, 0, 1, var_steps=(0, 2), sync_boundaries=(0, 2), sync_intervals=(1, 2))
     try:
         try:
@@ -200,8 +236,10 @@ def test_pushed_driver_over_symmetric_memory_one_rank():
         for t in range(5):
             g = torch.from_numpy(rng.standard_normal((1, n)).astype(np.float32)).cuda()
             ref.step_auto(list(g), 1e-3, t)
-            w.step_pushed(g[0], 1e-3, t, peers, dist.barrier)
+            w.step_pushed(g[0], 1e-3, t, peers)      # default: the one-element all-reduce
             torch.cuda.synchronize()
+            assert cpu.step(g.cpu().numpy(), np.float32(1e-3), t, ref.sync_due(t), t in (0, 2)) == 0
+            _compare_ranks_with_oracle([w], cpu, chunk, n, t, ref.sync_due(t))
             for name in ("x", "m", "u", "delta_w"):
                 assert np.array_equal(w.opt.read(name, 0), ref.read(name, 0)), (name, t)
             assert np.array_equal(w.opt.read("v"), ref.read("v")) and np.array_equal(w.opt.read("delta_s"), ref.read("delta_s"))
@@ -218,6 +256,7 @@ def test_driver_with_real_collectives_one_rank():
     rng = np.random.default_rng(3)
     n, chunk = 6 * 1024 + 50, 1024
     ref = Zoa(n, 1, chunk=chunk)
+    cpu = zo.Oracle(n, 1, chunk, dtype=np.float32)
     w = WorkerPerGpu(n, chunk, 0, 1, var_steps=(0, 2), sync_boundaries=(0, 2), sync_intervals=(1, 2))
     try:
         ref.set_policies((0, 2), (0, 2), (1, 2))
@@ -226,6 +265,8 @@ def test_driver_with_real_collectives_one_rank():
             ref.step_auto(list(g), 1e-3, t)
             w.step(g[0], 1e-3, t)
             torch.cuda.synchronize()
+            assert cpu.step(g.cpu().numpy(), np.float32(1e-3), t, ref.sync_due(t), t in (0, 2)) == 0
+            _compare_ranks_with_oracle([w], cpu, chunk, n, t, ref.sync_due(t))
             for name in ("x", "m", "u", "delta_w"):
                 assert np.array_equal(w.opt.read(name, 0), ref.read(name, 0)), (name, t)
             assert np.array_equal(w.opt.read("v"), ref.read("v")) and np.array_equal(w.opt.read("delta_s"), ref.read("delta_s"))

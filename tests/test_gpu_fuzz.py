@@ -54,7 +54,9 @@ def _case(seed):
                     p.gpu.step_host(list(gdev.cpu().pin_memory()), lr, t)
                 assert p.cpu.step(gref, np.float32(lr), t, sync, var) == 0
             torch.cuda.synchronize()
-            p.compare(f"seed={seed} n={n} W={W} chunk={chunk} {algorithm} {dtype} t={t}", wire=False)
+            # packed words (bit-exact) and magnitudes are compared whenever the step ran the 1-bit AllReduce
+            wire = (not var) if algorithm == "alg2" else sync
+            p.compare(f"seed={seed} n={n} W={W} chunk={chunk} {algorithm} {dtype} t={t}", wire=wire)
         p.padding_is_zero()
     finally:
         p.close()      # also checks the device error flag and the guard areas

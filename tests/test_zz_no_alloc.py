@@ -4,12 +4,15 @@ loops that cannot take cudaMalloc's implicit synchronisation, pre-partitioned
 multi-tenant processes, clean-up paths that run when the device is full).  Its
 packed intermediate lives in an array built into the library, so a call makes no
 allocation.  This test calls it through the C ABI twice in a row and checks the
-results against the handle-based entry point (zoa_onebit_reduce), bit for bit.
+results against the handle-based entry point (zoa_onebit_reduce), bit for bit,
+and against the CPU oracle's Algorithm 3 within the tolerance of the parity tests.
 It is collected last on purpose, and passes alone in a fresh process as well."""
 import numpy as np
 import pytest
 import torch
 
+from helpers import assert_close
+from oracle import zoa_oracle as zo
 from paper_2202_06009_b200 import Zoa, ZoaError, binding as B
 
 pytestmark = pytest.mark.gpu
@@ -38,6 +41,7 @@ def test_static_entry_point_matches_the_handle_path_twice_in_a_row(n, W, chunk, 
     rng = np.random.default_rng(n + W)
     z_rounds = [rng.standard_normal((W, n)).astype(np.float32) * np.float32(1 + r) for r in range(2)]
     want = _existing(z_rounds, n, W, chunk)
+    cpu = zo.Oracle(n, W, chunk, dtype=np.float32)       # Algorithm 3 with errors that start at zero
 
     # `offset` shifts every buffer by one float to exercise the unaligned path
     def dev(a):
@@ -54,6 +58,12 @@ def test_static_entry_point_matches_the_handle_path_twice_in_a_row(n, W, chunk, 
         B.zoa_onebit_allreduce_static([t.data_ptr() for t in z], [t.data_ptr() for t in delta_w],
                                       delta_s.data_ptr(), z_bar.data_ptr(), n, W, chunk, stream)
         torch.cuda.synchronize()
+        z_bar_cpu = cpu.onebit_allreduce(z_rounds[r])
+        assert_close(z_bar.cpu().numpy(), z_bar_cpu, f"z_bar against the oracle, call {r}")
+        assert np.array_equal(z_bar.cpu().numpy() >= 0, z_bar_cpu >= 0), f"signs of z_bar against the oracle, call {r}"
+        assert_close(delta_s.cpu().numpy(), cpu.delta_bar, f"delta_s against the oracle, call {r}")
+        for i in range(W):
+            assert_close(delta_w[i].cpu().numpy(), cpu.delta[i], f"delta_w[{i}] against the oracle, call {r}")
         assert np.array_equal(z_bar.cpu().numpy(), want[r]["z_bar"]), f"z_bar, call {r}"
         assert np.array_equal(delta_s.cpu().numpy(), want[r]["delta_s"]), f"delta_s, call {r}"
         for i in range(W):
