@@ -6,7 +6,18 @@
  * optimizer state; gradients are borrowed, read-only, and must stay valid until
  * the stream has finished the call's work.  Every call that takes a stream
  * enqueues its work on that stream and returns after host-side validation
- * only; nothing synchronises unless stated.  A handle is not thread-safe.
+ * only; nothing synchronises unless stated.  A handle is not thread-safe
+ * (different handles may be used from different threads).
+ *
+ * Errors.  ZOA_ERR_ARG and ZOA_ERR_STATE are found before anything is enqueued:
+ * the handle and its state are unchanged.  After ZOA_ERR_CUDA, ZOA_ERR_ALLOC or
+ * ZOA_ERR_DEVICE from a call that enqueues work (a step, reduce, copy or
+ * import call) part of the call's work may have run and the host scalars may
+ * not have advanced: the optimizer state is undefined and should be restored
+ * from a checkpoint (zoa_import_state) or rebuilt.  Once a kernel has given up on
+ * a bounded wait, every step, reduce and compress entry point returns
+ * ZOA_ERR_DEVICE (without synchronising; the news travels through a word of
+ * pinned host memory) until zoa_check_device has reported and cleared it.
  *
  * Arithmetic contract (what "the same result" means for every entry point):
  * all state is IEEE binary32; each elementwise operation is one
@@ -88,6 +99,9 @@ zoa_status zoa_set_params(zoa_handle h, const float *x0, void *stream);
 /* T_v of Algorithm 1 as an explicit list of step indices (host, any order).
  * Default: empty (the variance is never updated). */
 zoa_status zoa_set_var_steps(zoa_handle h, const int64_t *steps, size_t count);
+
+/* The same call under the name zoa_set_var_policy. */
+zoa_status zoa_set_var_policy(zoa_handle h, const int64_t *steps, size_t count);
 
 /* T_v by the rule of the paragraph "Policy for T_v and T_u": the j-th update is
  * at k_j with k_0 = 0 and k_{j+1} - k_j = 2^floor(j / kappa), for k_j < freeze_at. */
@@ -255,22 +269,49 @@ zoa_status zoa_step_host(zoa_handle h, const void *const *host_grads, float lr, 
 zoa_status zoa_get_buffer(zoa_handle h, zoa_buffer which, int worker, void **dev_ptr,
                           size_t *n_elems);
 
+/* The same call under the name zoa_get_ptr (`what` takes the zoa_buffer values). */
+zoa_status zoa_get_ptr(zoa_handle h, int what, int worker, void **dev_ptr, size_t *stride_elems);
+
+/* Checkpoint of everything Algorithm 1 carries from one iteration to the next
+ * (its "Require" clause and the two errors of Algorithm 3): x, m, u and the
+ * worker error of every worker, v_t and - when a T_v step's update is still
+ * pending, i.e. between zoa_step and the next step call - v_{t+1} with the
+ * pending mark, the server error, x_sync, the sum of learning rates since the
+ * last sync, t', the last step index, beta1, beta2, eps, both policies and the
+ * step / sync / variance-update counters.  The packed wire buffers are outputs
+ * of a sync, not state, and are not saved; options (zoa_set_option) are not either.
+ * zoa_state_size: bytes the blob takes for the handle as it stands (it grows
+ * with the policy tables).  zoa_export_state: waits for the device, then writes
+ * the blob to host_blob (host, at least zoa_state_size bytes).
+ * zoa_import_state: restores a blob into a handle created with the same
+ * n_params, W and chunk (ZOA_ERR_ARG otherwise, or if the blob is malformed or
+ * truncated; nothing is changed then); waits for the device first.  A run that
+ * exports, imports into a fresh handle and continues gives the same bits as
+ * the run that was never interrupted, also when the export falls between
+ * zoa_step on a T_v step and zoa_onebit_reduce. */
+zoa_status zoa_state_size(zoa_handle h, size_t *bytes);
+zoa_status zoa_export_state(zoa_handle h, void *host_blob, size_t bytes);
+zoa_status zoa_import_state(zoa_handle h, const void *host_blob, size_t bytes);
+
 /* Synchronous copies between a state row and (host) memory, in elements of the
- * buffer's type from element `offset`; for checkpoints and tests. */
+ * buffer's type from element `offset`; for tests and inspection.  ZOA_BUF_V is
+ * the newest variance (v_{t+1} while an update is pending); a checkpoint
+ * needs both, which zoa_export_state saves. */
 zoa_status zoa_copy_out(zoa_handle h, zoa_buffer which, int worker, size_t offset, size_t count,
                         void *host_dst);
 zoa_status zoa_copy_in(zoa_handle h, zoa_buffer which, int worker, size_t offset, size_t count,
                        const void *host_src);
 
-/* Host scalars of Algorithm 1 (sum of gammas since the last sync, t', last t),
- * to restore a checkpoint together with zoa_copy_in. */
+/* Host scalars of Algorithm 1 (sum of gammas since the last sync, t', last t);
+ * lets tests and benchmarks rewind the step counter. */
 zoa_status zoa_set_scalars(zoa_handle h, double gamma_sum, int64_t t_sync, int64_t t_last);
 
 zoa_status zoa_get_stats(zoa_handle h, zoa_stats *out);
 
 /* Waits for the device and reports ZOA_ERR_CUDA if a CUDA error is pending,
  * ZOA_ERR_DEVICE if a kernel of this handle gave up on a bounded wait since the
- * last check, or if one of the guard areas that surround every device buffer of
+ * last check (which also clears that condition, so that step calls are accepted
+ * again), or if one of the guard areas that surround every device buffer of
  * the handle no longer holds its pattern (a kernel wrote out of bounds). */
 zoa_status zoa_check_device(zoa_handle h);
 

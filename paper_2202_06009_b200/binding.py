@@ -39,6 +39,7 @@ def _load():
         "zoa_destroy": ([H], C.c_int),
         "zoa_set_params": ([H, p, p], C.c_int),
         "zoa_set_var_steps": ([H, C.POINTER(C.c_int64), C.c_size_t], C.c_int),
+        "zoa_set_var_policy": ([H, C.POINTER(C.c_int64), C.c_size_t], C.c_int),
         "zoa_set_var_policy_doubling": ([H, C.c_int, C.c_int64], C.c_int),
         "zoa_set_sync_policy": ([H, C.POINTER(C.c_int64), C.POINTER(C.c_int32), C.c_size_t], C.c_int),
         "zoa_policy_var_steps": ([C.c_int, C.c_int64, C.POINTER(C.c_int64), C.c_size_t], C.c_size_t),
@@ -62,6 +63,10 @@ def _load():
         "zoa_alg2_step": ([H, C.POINTER(p), C.c_float, C.c_int64, p], C.c_int),
         "zoa_step_host": ([H, C.POINTER(p), C.c_float, C.c_int64, p, p], C.c_int),
         "zoa_get_buffer": ([H, C.c_int, C.c_int, C.POINTER(p), C.POINTER(C.c_size_t)], C.c_int),
+        "zoa_get_ptr": ([H, C.c_int, C.c_int, C.POINTER(p), C.POINTER(C.c_size_t)], C.c_int),
+        "zoa_state_size": ([H, C.POINTER(C.c_size_t)], C.c_int),
+        "zoa_export_state": ([H, p, C.c_size_t], C.c_int),
+        "zoa_import_state": ([H, p, C.c_size_t], C.c_int),
         "zoa_copy_out": ([H, C.c_int, C.c_int, C.c_size_t, C.c_size_t, p], C.c_int),
         "zoa_copy_in": ([H, C.c_int, C.c_int, C.c_size_t, C.c_size_t, p], C.c_int),
         "zoa_set_scalars": ([H, C.c_double, C.c_int64, C.c_int64], C.c_int),
@@ -218,6 +223,31 @@ def zoa_get_buffer(h, which, worker=0):
     ptr, n = C.c_void_p(), C.c_size_t()
     _check(h, lib.zoa_get_buffer(h, which, worker, C.byref(ptr), C.byref(n)))
     return ptr.value, n.value
+
+
+def zoa_get_ptr(h, what, worker=0):
+    ptr, n = C.c_void_p(), C.c_size_t()
+    _check(h, lib.zoa_get_ptr(h, what, worker, C.byref(ptr), C.byref(n)))
+    return ptr.value, n.value
+
+
+def zoa_set_var_policy(h, steps):
+    arr = (C.c_int64 * len(steps))(*steps)
+    _check(h, lib.zoa_set_var_policy(h, arr, len(steps)))
+
+
+def zoa_state_size(h):
+    n = C.c_size_t()
+    _check(h, lib.zoa_state_size(h, C.byref(n)))
+    return n.value
+
+
+def zoa_export_state(h, host_ptr, nbytes):
+    _check(h, lib.zoa_export_state(h, host_ptr, nbytes))
+
+
+def zoa_import_state(h, host_ptr, nbytes):
+    _check(h, lib.zoa_import_state(h, host_ptr, nbytes))
 
 
 def zoa_copy_out(h, which, worker, offset, count, host_ptr):

@@ -28,6 +28,8 @@ struct zoa_handle_s {
     cudaStream_t copy_stream = nullptr;                 // host-to-device copies of zoa_step_host run here ...
     std::vector<cudaEvent_t> copy_events;               // ... and these order them with the caller's stream
     int *error_flag = nullptr;     // device int: a kernel gave up on a bounded wait
+    int *error_host = nullptr;     // the same news in pinned, mapped host memory: the step entry points test it without synchronising
+    int *error_host_dev = nullptr; // its device-side address
     unsigned long long *sched = nullptr;   // device [2]: chunk counter of the persistent kernel, finished blocks
     double *partials = nullptr;    // device [W + 1][n_chunks * segments]: per-segment l1 sums, chunk > 16384 only
     bool large_chunk = false;
@@ -53,7 +55,7 @@ struct TraceRange {
     ~TraceRange() { nvtxRangePop(); }
 };
 
-static std::string g_create_error;
+static thread_local std::string g_create_error;   // text of this thread's last failed zoa_create
 
 static zoa_status fail(zoa_handle h, zoa_status s, const std::string &msg)
 {
@@ -70,6 +72,8 @@ static zoa_status fail_cuda(zoa_handle h, cudaError_t e, const char *what)
         cudaError_t e_ = (call);                                 \
         if (e_ != cudaSuccess) return fail_cuda(h, e_, #call);   \
     } while (0)
+
+static bool on_own_device(zoa_handle h);
 
 static StateView view(zoa_handle h)
 {
@@ -96,7 +100,21 @@ static void free_all(zoa_handle h)
     h->copy_events.clear();
     if (h->copy_stream) cudaStreamDestroy(h->copy_stream);
     h->copy_stream = nullptr;
+    if (h->error_host) cudaFreeHost(h->error_host);
+    h->error_host = h->error_host_dev = nullptr;
 }
+
+static ErrorWords error_words(zoa_handle h) { return ErrorWords{h->error_flag, h->error_host_dev}; }
+
+// A kernel of an earlier call gave up on a bounded wait: every later step would run on undefined
+// state, so the step entry points refuse until zoa_check_device has reported and cleared it.
+static bool device_gave_up(zoa_handle h) { return h->error_host && *static_cast<volatile int *>(h->error_host) != 0; }
+#define ZOA_REFUSE_AFTER_DEVICE_ERROR(h, who)                                                                      \
+    do {                                                                                                            \
+        if (device_gave_up(h))                                                                                      \
+            return fail(h, ZOA_ERR_DEVICE, std::string(who) + ": an earlier kernel gave up waiting for its "        \
+                                           "asynchronous copies; the optimizer state is undefined (zoa_check_device clears the flag)"); \
+    } while (0)
 
 static cudaError_t alloc_guarded(zoa_handle h, void **p, size_t bytes)
 {
@@ -177,6 +195,13 @@ extern "C" zoa_status zoa_create(zoa_handle *out, size_t n_params, int W, float 
         h->large_chunk = chunk > kMaxChunk;
         if (h->large_chunk)
             e = alloc_zero(h, &h->partials, (size_t)(W + 1) * (size_t)h->n_chunks * (size_t)large_chunk_segments(view(h)));
+        if (e == cudaSuccess) e = cudaHostAlloc(reinterpret_cast<void **>(&h->error_host), sizeof(int), cudaHostAllocMapped);
+        if (e == cudaSuccess) {
+            *h->error_host = 0;
+            e = cudaHostGetDevicePointer(reinterpret_cast<void **>(&h->error_host_dev), h->error_host, 0);
+        } else {
+            h->error_host = nullptr;
+        }
         if (e == cudaSuccess) e = cudaDeviceSynchronize();
     }
     if (e != cudaSuccess) {
@@ -192,10 +217,13 @@ extern "C" zoa_status zoa_create(zoa_handle *out, size_t n_params, int W, float 
 extern "C" zoa_status zoa_destroy(zoa_handle h)
 {
     if (!h) return ZOA_ERR_ARG;
+    int current = -1;
+    const bool restore = cudaGetDevice(&current) == cudaSuccess && current != h->device;
     cudaSetDevice(h->device);
     cudaDeviceSynchronize();
     free_all(h);
     delete h;
+    if (restore) cudaSetDevice(current);      // the caller's current device stays what it was
     return ZOA_OK;
 }
 
@@ -203,6 +231,7 @@ extern "C" zoa_status zoa_set_params(zoa_handle h, const float *x0, void *stream
 {
     if (!h) return ZOA_ERR_ARG;
     if (!x0) return fail(h, ZOA_ERR_ARG, "zoa_set_params: x0 is NULL");
+    if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, "zoa_set_params: the handle's device is not the current CUDA device");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t bytes = (size_t)h->n * sizeof(float);
     for (int i = 0; i < h->W; ++i)
@@ -321,12 +350,11 @@ extern "C" int zoa_var_due(zoa_handle h, int64_t t)
 }
 
 // Checks shared by the step entry points; fills the pointer pack.
-static bool on_own_device(zoa_handle h);
-
 static zoa_status check_step_args(zoa_handle h, const void *const *grads, float lr, int64_t t, GradPtrs *gp,
                                   int *aligned, const char *who)
 {
     if (!h) return ZOA_ERR_ARG;
+    ZOA_REFUSE_AFTER_DEVICE_ERROR(h, who);
     if (!grads) return fail(h, ZOA_ERR_ARG, std::string(who) + ": grads is NULL");
     if (!std::isfinite(lr)) return fail(h, ZOA_ERR_ARG, std::string(who) + ": lr is not finite");
     if (t < 0) return fail(h, ZOA_ERR_ARG, std::string(who) + ": t is negative");
@@ -413,7 +441,7 @@ static zoa_status run_sync_range(zoa_handle h, const StateView &st, const GradPt
     if (stages > 0) {
         bool var_fused = false;
         ZOA_CUDA(h, launch_step_sync_pipelined(st, gp, h->c, lr, gamma_sum, do_var, fmt, c0, n_full, stages, h->sm_count,
-                                               h->error_flag, h->sched, (unsigned long long)h->wait_limit_ms * 1000000ull,
+                                               error_words(h), h->sched, (unsigned long long)h->wait_limit_ms * 1000000ull,
                                                h->test_stop_after_tiles, &var_fused, s));
         h->n_launches += 1;
         if (ragged) {
@@ -454,6 +482,7 @@ extern "C" zoa_status zoa_onebit_reduce(zoa_handle h, void *stream)
 {
     TraceRange trace("zoa_onebit_reduce");
     if (!h) return ZOA_ERR_ARG;
+    ZOA_REFUSE_AFTER_DEVICE_ERROR(h, "zoa_onebit_reduce");
     const float gamma_sum = (float)h->gamma_sum;
     if (!(h->gamma_sum > 0.0) || !(gamma_sum > 0.f) || !std::isfinite(gamma_sum))
         return fail(h, ZOA_ERR_STATE, "zoa_onebit_reduce: nothing accumulated since the last sync (sum of learning rates is not positive)");
@@ -470,6 +499,8 @@ extern "C" zoa_status zoa_onebit_reduce(zoa_handle h, void *stream)
 extern "C" zoa_status zoa_onebit_compress(zoa_handle h, void *stream)
 {
     if (!h) return ZOA_ERR_ARG;
+    ZOA_REFUSE_AFTER_DEVICE_ERROR(h, "zoa_onebit_compress");
+    if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, "zoa_onebit_compress: the handle's device is not the current CUDA device");
     ZOA_CUDA(h, run_compress(h, static_cast<cudaStream_t>(stream)));
     return ZOA_OK;
 }
@@ -480,6 +511,8 @@ extern "C" zoa_status zoa_onebit_average(zoa_handle h, void *stream)
     const float gamma_sum = (float)h->gamma_sum;
     if (!(h->gamma_sum > 0.0) || !(gamma_sum > 0.f) || !std::isfinite(gamma_sum))
         return fail(h, ZOA_ERR_STATE, "zoa_onebit_average: nothing accumulated since the last sync (sum of learning rates is not positive)");
+    ZOA_REFUSE_AFTER_DEVICE_ERROR(h, "zoa_onebit_average");
+    if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, "zoa_onebit_average: the handle's device is not the current CUDA device");
     ZOA_CUDA(h, run_server(h, gamma_sum, static_cast<cudaStream_t>(stream)));
     h->gamma_sum = 0.0;
     h->t_sync = h->t_last;
@@ -699,7 +732,7 @@ extern "C" zoa_status zoa_alg2_step(zoa_handle h, const void *const *grads, floa
         const int stages = (!full && h->use_pipeline && enough_chunks) ? alg2_pipeline_stages(st, aligned) : 0;
         long long first = 0;
         if (stages > 0) {   // full chunks through the bulk-copy ring, a ragged last chunk through the block kernel
-            ZOA_CUDA(h, launch_alg2_pipelined(st, gp, h->c, lr, aligned, stages, h->sm_count, h->error_flag, h->sched,
+            ZOA_CUDA(h, launch_alg2_pipelined(st, gp, h->c, lr, aligned, stages, h->sm_count, error_words(h), h->sched,
                                               (unsigned long long)h->wait_limit_ms * 1000000ull, h->test_stop_after_tiles, s));
             h->n_launches += 1;
             first = h->n / h->chunk;
@@ -729,6 +762,7 @@ extern "C" zoa_status zoa_step_host(zoa_handle h, const void *const *host_grads,
     if (!host_grads) return fail(h, ZOA_ERR_ARG, "zoa_step_host: host_grads is NULL");
     for (int i = 0; i < h->W; ++i)
         if (!host_grads[i]) return fail(h, ZOA_ERR_ARG, "zoa_step_host: a gradient pointer is NULL");
+    if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, "zoa_step_host: the handle's device is not the current CUDA device");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (!h->staging) {
         cudaError_t e = cudaMalloc(reinterpret_cast<void **>(&h->staging), (size_t)h->W * h->n_pad * sizeof(float));
@@ -738,21 +772,7 @@ extern "C" zoa_status zoa_step_host(zoa_handle h, const void *const *host_grads,
     for (int i = 0; i < h->W; ++i) dev[i] = h->staging + (size_t)i * h->n_pad;
     const size_t g_bytes = h->grad_type ? 2 : 4;
 
-    // Large chunks are not cut into ranges, and small problems are not worth it: copy, then step.
-    const int kSegments = 8;
-    if (h->large_chunk || h->n_chunks < 64 * kSegments) {
-        for (int i = 0; i < h->W; ++i)
-            ZOA_CUDA(h, cudaMemcpyAsync(const_cast<void *>(dev[i]), host_grads[i], (size_t)h->n * g_bytes, cudaMemcpyHostToDevice, s));
-        zoa_status rc = zoa_step_auto(h, dev, lr, t, stream);
-        if (rc != ZOA_OK) return rc;
-        if (host_x_out)
-            ZOA_CUDA(h, cudaMemcpyAsync(host_x_out, h->x, (size_t)h->n * sizeof(float), cudaMemcpyDeviceToHost, s));
-        return ZOA_OK;
-    }
-
-    // Otherwise the vector is cut into chunk ranges: the copies of range k+1 (on the handle's own copy
-    // stream) run while the kernels of range k and the copy of its part of the result (on the
-    // caller's stream) do, so the step costs little more than moving the gradients over the bus.
+    // Everything is validated before the first copy is enqueued.
     GradPtrs gp;
     int fmt;
     zoa_status rc = check_step_args(h, dev, lr, t, &gp, &fmt, "zoa_step_host");
@@ -762,6 +782,22 @@ extern "C" zoa_status zoa_step_host(zoa_handle h, const void *const *host_grads,
     const float gamma_sum = (float)total;
     if (do_sync && (!(total > 0.0) || !(gamma_sum > 0.f) || !std::isfinite(gamma_sum)))
         return fail(h, ZOA_ERR_STATE, "zoa_step_host: sum of learning rates since the last sync is not positive");
+
+    // Large chunks are not cut into ranges, and small problems are not worth it: copy, then step.
+    const int kSegments = 8;
+    if (h->large_chunk || h->n_chunks < 64 * kSegments) {
+        for (int i = 0; i < h->W; ++i)
+            ZOA_CUDA(h, cudaMemcpyAsync(const_cast<void *>(dev[i]), host_grads[i], (size_t)h->n * g_bytes, cudaMemcpyHostToDevice, s));
+        rc = zoa_step_auto(h, dev, lr, t, stream);
+        if (rc != ZOA_OK) return rc;
+        if (host_x_out)
+            ZOA_CUDA(h, cudaMemcpyAsync(host_x_out, h->x, (size_t)h->n * sizeof(float), cudaMemcpyDeviceToHost, s));
+        return ZOA_OK;
+    }
+
+    // Otherwise the vector is cut into chunk ranges: the copies of range k+1 (on the handle's own copy
+    // stream) run while the kernels of range k and the copy of its part of the result (on the
+    // caller's stream) do, so the step costs little more than moving the gradients over the bus.
     if (!h->copy_stream) ZOA_CUDA(h, cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking));
     while ((int)h->copy_events.size() < kSegments + 1) {
         cudaEvent_t e;
@@ -841,6 +877,7 @@ extern "C" zoa_status zoa_copy_out(zoa_handle h, zoa_buffer which, int worker, s
     zoa_status rc = locate(h, which, worker, &base, &elem, &len);
     if (rc != ZOA_OK) return rc;
     if (!host_dst || offset > len || count > len - offset) return fail(h, ZOA_ERR_ARG, "zoa_copy_out: range outside the row");
+    if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, "zoa_copy_out: the handle's device is not the current CUDA device");
     ZOA_CUDA(h, cudaDeviceSynchronize());
     ZOA_CUDA(h, cudaMemcpy(host_dst, base + offset * elem, count * elem, cudaMemcpyDeviceToHost));
     return ZOA_OK;
@@ -853,6 +890,7 @@ extern "C" zoa_status zoa_copy_in(zoa_handle h, zoa_buffer which, int worker, si
     zoa_status rc = locate(h, which, worker, &base, &elem, &len);
     if (rc != ZOA_OK) return rc;
     if (!host_src || offset > len || count > len - offset) return fail(h, ZOA_ERR_ARG, "zoa_copy_in: range outside the row");
+    if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, "zoa_copy_in: the handle's device is not the current CUDA device");
     ZOA_CUDA(h, cudaDeviceSynchronize());
     ZOA_CUDA(h, cudaMemcpy(base + offset * elem, host_src, count * elem, cudaMemcpyHostToDevice));
     return ZOA_OK;
@@ -865,6 +903,158 @@ extern "C" zoa_status zoa_set_scalars(zoa_handle h, double gamma_sum, int64_t t_
     h->gamma_sum = gamma_sum;
     h->t_sync = t_sync;
     h->t_last = t_last;
+    return ZOA_OK;
+}
+
+// The names the optimizer's C interface was first drafted with; same calls.
+extern "C" zoa_status zoa_set_var_policy(zoa_handle h, const int64_t *steps, size_t count)
+{
+    return zoa_set_var_steps(h, steps, count);
+}
+extern "C" zoa_status zoa_get_ptr(zoa_handle h, int what, int worker, void **dev_ptr, size_t *stride_elems)
+{
+    return zoa_get_buffer(h, static_cast<zoa_buffer>(what), worker, dev_ptr, stride_elems);
+}
+
+// ---- checkpoint: the whole state of Algorithm 1 / Algorithm 3 as one host blob ------------------
+//
+// Layout: BlobHeader, then T_v (int64 each), the T_u pieces (int64 boundaries, then int32
+// intervals, padded to 8 bytes), then n floats per row: x, m, u, delta_w (W rows each),
+// v_t, v_{t+1} (meaningful only when v_pending), delta_s, x_sync.
+namespace {
+struct BlobHeader {
+    char magic[8];                 // "ZOASTATE"
+    uint32_t version, header_bytes;
+    int64_t n, n_chunks;
+    int32_t W, chunk;
+    float beta1, beta2, eps;
+    int32_t v_pending;
+    double gamma_sum;
+    int64_t t_sync, t_last;
+    int64_t n_steps, n_syncs, n_var_updates;
+    uint64_t n_var_steps, n_sync_pieces;
+    uint64_t total_bytes;
+};
+const char kBlobMagic[8] = {'Z', 'O', 'A', 'S', 'T', 'A', 'T', 'E'};
+const uint32_t kBlobVersion = 1;
+
+size_t blob_policy_bytes(size_t n_var, size_t n_pieces)
+{
+    return n_var * sizeof(int64_t) + n_pieces * sizeof(int64_t) + (n_pieces * sizeof(int32_t) + 7) / 8 * 8;
+}
+size_t blob_rows(int W) { return 4 * (size_t)W + 4; }
+}  // namespace
+
+extern "C" zoa_status zoa_state_size(zoa_handle h, size_t *bytes)
+{
+    if (!h) return ZOA_ERR_ARG;
+    if (!bytes) return fail(h, ZOA_ERR_ARG, "zoa_state_size: bytes is NULL");
+    *bytes = sizeof(BlobHeader) + blob_policy_bytes(h->var_steps.size(), h->sync_bounds.size()) +
+             blob_rows(h->W) * (size_t)h->n * sizeof(float);
+    return ZOA_OK;
+}
+
+extern "C" zoa_status zoa_export_state(zoa_handle h, void *host_blob, size_t bytes)
+{
+    if (!h) return ZOA_ERR_ARG;
+    size_t need = 0;
+    zoa_state_size(h, &need);
+    if (!host_blob) return fail(h, ZOA_ERR_ARG, "zoa_export_state: host_blob is NULL");
+    if (bytes < need) return fail(h, ZOA_ERR_ARG, "zoa_export_state: the buffer is smaller than zoa_state_size");
+    if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, "zoa_export_state: the handle's device is not the current CUDA device");
+    ZOA_CUDA(h, cudaDeviceSynchronize());
+    BlobHeader hd{};
+    std::memcpy(hd.magic, kBlobMagic, 8);
+    hd.version = kBlobVersion;
+    hd.header_bytes = (uint32_t)sizeof(BlobHeader);
+    hd.n = h->n; hd.n_chunks = h->n_chunks; hd.W = h->W; hd.chunk = h->chunk;
+    hd.beta1 = h->c.b1; hd.beta2 = h->c.b2; hd.eps = h->c.eps;
+    hd.v_pending = h->v_pending ? 1 : 0;
+    hd.gamma_sum = h->gamma_sum;
+    hd.t_sync = h->t_sync; hd.t_last = h->t_last;
+    hd.n_steps = h->n_steps; hd.n_syncs = h->n_syncs; hd.n_var_updates = h->n_var_updates;
+    hd.n_var_steps = h->var_steps.size();
+    hd.n_sync_pieces = h->sync_bounds.size();
+    hd.total_bytes = need;
+    char *p = static_cast<char *>(host_blob);
+    std::memcpy(p, &hd, sizeof(hd));
+    p += sizeof(hd);
+    std::memset(p, 0, blob_policy_bytes(hd.n_var_steps, hd.n_sync_pieces));
+    std::memcpy(p, h->var_steps.data(), hd.n_var_steps * sizeof(int64_t));
+    p += hd.n_var_steps * sizeof(int64_t);
+    std::memcpy(p, h->sync_bounds.data(), hd.n_sync_pieces * sizeof(int64_t));
+    p += hd.n_sync_pieces * sizeof(int64_t);
+    std::memcpy(p, h->sync_intervals.data(), hd.n_sync_pieces * sizeof(int32_t));
+    p += (hd.n_sync_pieces * sizeof(int32_t) + 7) / 8 * 8;
+    const size_t row_bytes = (size_t)h->n * sizeof(float);
+    float *const per_worker[4] = {h->x, h->m, h->u, h->dw};
+    for (float *buf : per_worker)
+        for (int i = 0; i < h->W; ++i, p += row_bytes)
+            ZOA_CUDA(h, cudaMemcpy(p, buf + (size_t)i * h->n_pad, row_bytes, cudaMemcpyDeviceToHost));
+    float *const shared[4] = {h->v_cur, h->v_nxt, h->ds, h->xs};
+    for (float *buf : shared) {
+        ZOA_CUDA(h, cudaMemcpy(p, buf, row_bytes, cudaMemcpyDeviceToHost));
+        p += row_bytes;
+    }
+    return ZOA_OK;
+}
+
+extern "C" zoa_status zoa_import_state(zoa_handle h, const void *host_blob, size_t bytes)
+{
+    if (!h) return ZOA_ERR_ARG;
+    if (!host_blob) return fail(h, ZOA_ERR_ARG, "zoa_import_state: host_blob is NULL");
+    if (bytes < sizeof(BlobHeader)) return fail(h, ZOA_ERR_ARG, "zoa_import_state: the blob is shorter than its header");
+    BlobHeader hd;
+    std::memcpy(&hd, host_blob, sizeof(hd));
+    if (std::memcmp(hd.magic, kBlobMagic, 8) != 0 || hd.version != kBlobVersion || hd.header_bytes != sizeof(BlobHeader))
+        return fail(h, ZOA_ERR_ARG, "zoa_import_state: not a state blob of this library version");
+    if (hd.n != h->n || hd.W != h->W || hd.chunk != h->chunk)
+        return fail(h, ZOA_ERR_ARG, "zoa_import_state: the blob was exported from a handle with another n_params, W or chunk");
+    if (hd.n_var_steps > ((uint64_t)1 << 40) || hd.n_sync_pieces < 1 || hd.n_sync_pieces > ((uint64_t)1 << 40))
+        return fail(h, ZOA_ERR_ARG, "zoa_import_state: malformed policy tables");
+    const size_t need = sizeof(BlobHeader) + blob_policy_bytes(hd.n_var_steps, hd.n_sync_pieces) +
+                        blob_rows(h->W) * (size_t)h->n * sizeof(float);
+    if (hd.total_bytes != need || bytes < need) return fail(h, ZOA_ERR_ARG, "zoa_import_state: the blob is truncated");
+    if (!(hd.beta1 >= 0.f && hd.beta1 < 1.f) || !(hd.beta2 >= 0.f && hd.beta2 < 1.f) || !(hd.eps > 0.f) ||
+        !std::isfinite(hd.gamma_sum) || hd.gamma_sum < 0.0 || hd.t_last < -1)
+        return fail(h, ZOA_ERR_ARG, "zoa_import_state: a scalar of the blob is out of range");
+    const char *p = static_cast<const char *>(host_blob) + sizeof(BlobHeader);
+    std::vector<int64_t> var_steps(hd.n_var_steps), bounds(hd.n_sync_pieces);
+    std::vector<int32_t> intervals(hd.n_sync_pieces);
+    std::memcpy(var_steps.data(), p, hd.n_var_steps * sizeof(int64_t));
+    p += hd.n_var_steps * sizeof(int64_t);
+    std::memcpy(bounds.data(), p, hd.n_sync_pieces * sizeof(int64_t));
+    p += hd.n_sync_pieces * sizeof(int64_t);
+    std::memcpy(intervals.data(), p, hd.n_sync_pieces * sizeof(int32_t));
+    p += (hd.n_sync_pieces * sizeof(int32_t) + 7) / 8 * 8;
+    if (bounds[0] != 0) return fail(h, ZOA_ERR_ARG, "zoa_import_state: malformed policy tables");
+    for (size_t r = 0; r < bounds.size(); ++r)
+        if (intervals[r] < 1 || (r && bounds[r] <= bounds[r - 1])) return fail(h, ZOA_ERR_ARG, "zoa_import_state: malformed policy tables");
+    if (!std::is_sorted(var_steps.begin(), var_steps.end())) return fail(h, ZOA_ERR_ARG, "zoa_import_state: malformed policy tables");
+    if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, "zoa_import_state: the handle's device is not the current CUDA device");
+    ZOA_CUDA(h, cudaDeviceSynchronize());
+    // From here on the handle changes; a failing copy leaves it undefined (ZOA_ERR_CUDA).
+    commit_variance(h);        // v_cur / v_nxt take their plain roles before they are overwritten
+    const size_t row_bytes = (size_t)h->n * sizeof(float);
+    float *const per_worker[4] = {h->x, h->m, h->u, h->dw};
+    for (float *buf : per_worker)
+        for (int i = 0; i < h->W; ++i, p += row_bytes)
+            ZOA_CUDA(h, cudaMemcpy(buf + (size_t)i * h->n_pad, p, row_bytes, cudaMemcpyHostToDevice));
+    float *const shared[4] = {h->v_cur, h->v_nxt, h->ds, h->xs};
+    for (float *buf : shared) {
+        ZOA_CUDA(h, cudaMemcpy(buf, p, row_bytes, cudaMemcpyHostToDevice));
+        p += row_bytes;
+    }
+    h->c.b1 = hd.beta1; h->c.ob1 = 1.0f - hd.beta1;
+    h->c.b2 = hd.beta2; h->c.ob2 = 1.0f - hd.beta2;
+    h->c.eps = hd.eps;
+    h->v_pending = hd.v_pending != 0;
+    h->gamma_sum = hd.gamma_sum;
+    h->t_sync = hd.t_sync; h->t_last = hd.t_last;
+    h->n_steps = hd.n_steps; h->n_syncs = hd.n_syncs; h->n_var_updates = hd.n_var_updates;
+    h->var_steps.swap(var_steps);
+    h->sync_bounds.swap(bounds);
+    h->sync_intervals.swap(intervals);
     return ZOA_OK;
 }
 
@@ -892,8 +1082,9 @@ extern "C" zoa_status zoa_check_device(zoa_handle h)
     if (!intact) return fail(h, ZOA_ERR_DEVICE, "a kernel wrote outside one of the handle's buffers (guard area overwritten)");
     int flag = 0;
     ZOA_CUDA(h, cudaMemcpy(&flag, h->error_flag, sizeof(int), cudaMemcpyDeviceToHost));
-    if (flag) {
+    if (flag || device_gave_up(h)) {
         cudaMemset(h->error_flag, 0, sizeof(int));
+        *static_cast<volatile int *>(h->error_host) = 0;
         cudaMemset(h->sched, 0, 2 * sizeof(unsigned long long));
         return fail(h, ZOA_ERR_DEVICE, "a kernel gave up waiting for its asynchronous copies; the optimizer state is undefined");
     }

@@ -1,9 +1,38 @@
 // Declarations shared between the kernels' translation unit and the C-ABI one.
 #pragma once
 
+#include <mutex>
+
 #include "zoa_device.cuh"
 
 namespace zoa {
+
+// Where a kernel that gives up on a bounded wait says so: a device word (zoa_check_device reads
+// and clears it) and the device-side address of a word in pinned, mapped host memory, which the
+// step entry points test without synchronising.
+struct ErrorWords {
+    int *device;
+    int *host_mapped;
+};
+
+// Raises a kernel's dynamic shared-memory limit the first time the kernel is launched on a
+// device; one object per kernel (template instantiation).  Safe to call from several threads.
+struct SmemLimitOnce {
+    std::mutex mu;
+    bool done[64] = {false};
+    template <typename Kernel>
+    cudaError_t ensure(Kernel kern, int bytes)
+    {
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        std::lock_guard<std::mutex> lock(mu);
+        if (dev >= 0 && dev < 64 && done[dev]) return cudaSuccess;
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (e == cudaSuccess && dev >= 0 && dev < 64) done[dev] = true;
+        return e;
+    }
+};
 
 cudaError_t configure_kernels();
 
@@ -30,7 +59,7 @@ cudaError_t launch_large_server(const StateView &st, const Consts &c, int mode, 
 int pipeline_stages(const StateView &st, int grad_fmt);
 cudaError_t launch_step_sync_pipelined(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
                                        float gamma_sum, bool do_var, int grad_fmt, long long first_chunk, long long n_chunks, int stages,
-                                       int sm_count, int *error_flag,
+                                       int sm_count, ErrorWords error_flag,
                                        unsigned long long *sched, unsigned long long wait_limit_ns,
                                        long long test_stop_after_tiles, bool *var_fused, cudaStream_t s);
 
@@ -47,7 +76,7 @@ cudaError_t launch_count_nonfinite(const float *p, long long count, unsigned lon
 
 int alg2_pipeline_stages(const StateView &st, int grad_fmt);
 cudaError_t launch_alg2_pipelined(const StateView &st, const GradPtrs &g, const Consts &c, float gamma, int grad_fmt,
-                                  int stages, int sm_count, int *error_flag, unsigned long long *sched,
+                                  int stages, int sm_count, ErrorWords error_flag, unsigned long long *sched,
                                   unsigned long long wait_limit_ns, long long test_stop_after_tiles, cudaStream_t s);
 
 }  // namespace zoa

@@ -1051,15 +1051,9 @@ cudaError_t launch_dist_server(const StateView &st, const uint32_t *words_in, lo
                                const float *scales_in, long long scales_in_stride, int W_total,
                                long long first_chunk, long long count, const PeerOut &out, cudaStream_t s)
 {
-    static bool configured[64] = {false};
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
+    static SmemLimitOnce once;
+    const cudaError_t e = once.ensure(dist_server_kernel, (int)reduce_smem(kMaxChunk));
     if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= 64 || !configured[dev]) {
-        e = cudaFuncSetAttribute(dist_server_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)reduce_smem(kMaxChunk));
-        if (e != cudaSuccess) return e;
-        if (dev >= 0 && dev < 64) configured[dev] = true;
-    }
     // block size as for reduce_kernel: with few workers smaller blocks, more of them per SM
     const int per_thread = W_total <= 2 ? 32 : 16;
     int thr = 128;
@@ -1074,18 +1068,12 @@ cudaError_t launch_dist_server(const StateView &st, const uint32_t *words_in, lo
 cudaError_t launch_dist_pack_push(const StateView &st, const float *g, const Consts &c, float gamma, int g_fmt,
                                   const PushPlan &plan, cudaStream_t s)
 {
-    static bool configured[64] = {false};
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
+    static SmemLimitOnce once[3];
+    const int max_smem = (int)compress_smem(kMaxChunk);
+    cudaError_t e = once[0].ensure(dist_pack_push_kernel<false, -1>, max_smem);
+    if (e == cudaSuccess) e = once[1].ensure(dist_pack_push_kernel<true, -1>, max_smem);
+    if (e == cudaSuccess) e = once[2].ensure(dist_pack_push_kernel<true, kGradF32 | kGradAligned>, max_smem);
     if (e != cudaSuccess) return e;
-    const size_t max_smem = compress_smem(kMaxChunk);
-    if (dev < 0 || dev >= 64 || !configured[dev]) {
-        e = cudaFuncSetAttribute(dist_pack_push_kernel<false, -1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(dist_pack_push_kernel<true, -1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(dist_pack_push_kernel<true, kGradF32 | kGradAligned>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
-        if (e != cudaSuccess) return e;
-        if (dev >= 0 && dev < 64) configured[dev] = true;
-    }
     int thr = 128;
     while (thr < st.chunk / 16 && thr < 1024) thr <<= 1;
     const unsigned grid = (unsigned)st.n_chunks;

@@ -206,6 +206,10 @@ extern "C" zoa_status zoa_onebit_allreduce_static(const float *const *z, float *
     if (n < 1 || W < 1 || W > kMaxWorkers) return static_fail(ZOA_ERR_ARG, "zoa_onebit_allreduce_static: need n >= 1 and 1 <= W <= 64");
     if (chunk < 32 || chunk > kMaxChunk || chunk % 32 != 0)
         return static_fail(ZOA_ERR_ARG, "zoa_onebit_allreduce_static: chunk must be a multiple of 32 in [32, 16384]");
+    // One worker's sign words alone must fit, which also keeps the 64-bit size arithmetic below from wrapping.
+    if (n > (size_t)32 * kStaticScratchSlots)
+        return static_fail(ZOA_ERR_ARG, "zoa_onebit_allreduce_static: n exceeds what the 1,048,576 slots of the built-in scratch "
+                                        "array can hold for a single worker; use a handle (zoa_create) for this size");
     StaticArgs a{};
     a.n = (long long)n;
     a.W = W;

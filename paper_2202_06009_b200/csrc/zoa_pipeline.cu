@@ -39,7 +39,7 @@ struct PipeArgs {
     long long first_chunk;    // the launch covers the full chunks [first_chunk, first_chunk + n_full_chunks)
     long long n_full_chunks;
     int stages;
-    int *error_flag;  // device int, set non-zero when a wait ran out
+    ErrorWords error_flag;  // set non-zero when a wait ran out
     unsigned long long *sched;  // device: [0] next chunk to hand out, [1] blocks that have finished
     int grad_fmt;                      // kGradF32 / kGradF16 / kGradBF16 (| kGradAligned, always set here)
     unsigned long long wait_limit_ns;  // how long a thread waits on an mbarrier before it gives up
@@ -89,7 +89,7 @@ __device__ __forceinline__ unsigned long long global_timer_ns()
 }
 // Bounded wait.  Returns false if the block has been aborted or the limit ran out
 // (in which case it raises both flags).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *error_flag,
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, const ErrorWords &error_flag,
                                           unsigned long long limit_ns)
 {
     if (mbar_try_wait(bar, parity)) return true;
@@ -99,7 +99,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if (*abort_flag) return false;
         if ((it & 63u) == 0 && global_timer_ns() - start > limit_ns) {
             *abort_flag = 1;
-            atomicExch(error_flag, 1);
+            atomicExch(error_flag.device, 1);
+            if (error_flag.host_mapped) {      // the host sees this one without synchronising
+                *reinterpret_cast<volatile int *>(error_flag.host_mapped) = 1;
+                __threadfence_system();
+            }
             return false;
         }
     }
@@ -686,15 +690,9 @@ template <int TILES, bool DO_VAR>
 static cudaError_t launch_pipe(const PipeArgs &a, int grid, size_t smem, cudaStream_t s)
 {
     auto kern = step_sync_pipelined_kernel<TILES, DO_VAR>;
-    static bool configured[64] = {false};   // per instantiation and device
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
+    static SmemLimitOnce once;   // per instantiation
+    const cudaError_t e = once.ensure(kern, 227 * 1024);
     if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= 64 || !configured[dev]) {
-        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-        if (e != cudaSuccess) return e;
-        if (dev >= 0 && dev < 64) configured[dev] = true;
-    }
     kern<<<grid, kThreads, smem, s>>>(a);
     return cudaGetLastError();
 }
@@ -703,7 +701,7 @@ static cudaError_t launch_pipe(const PipeArgs &a, int grid, size_t smem, cudaStr
 // *var_fused tells whether the variance update was done here too.
 cudaError_t launch_step_sync_pipelined(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
                                        float gamma_sum, bool do_var, int grad_fmt, long long first_chunk, long long n_chunks, int stages,
-                                       int sm_count, int *error_flag, unsigned long long *sched, unsigned long long wait_limit_ns,
+                                       int sm_count, ErrorWords error_flag, unsigned long long *sched, unsigned long long wait_limit_ns,
                                        long long test_stop_after_tiles, bool *var_fused, cudaStream_t s)
 {
     PipeArgs a;
@@ -748,22 +746,16 @@ template <int TILES>
 static cudaError_t launch_alg2_pipe(const PipeArgs &a, int grid, size_t smem, cudaStream_t s)
 {
     auto kern = alg2_pipelined_kernel<TILES>;
-    static bool configured[64] = {false};
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
+    static SmemLimitOnce once;
+    const cudaError_t e = once.ensure(kern, 227 * 1024);
     if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= 64 || !configured[dev]) {
-        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-        if (e != cudaSuccess) return e;
-        if (dev >= 0 && dev < 64) configured[dev] = true;
-    }
     kern<<<grid, kThreads, smem, s>>>(a);
     return cudaGetLastError();
 }
 
 // The full chunks of a compressed step of Algorithm 2; a ragged last chunk is the caller's.
 cudaError_t launch_alg2_pipelined(const StateView &st, const GradPtrs &g, const Consts &c, float gamma, int grad_fmt,
-                                  int stages, int sm_count, int *error_flag, unsigned long long *sched,
+                                  int stages, int sm_count, ErrorWords error_flag, unsigned long long *sched,
                                   unsigned long long wait_limit_ns, long long test_stop_after_tiles, cudaStream_t s)
 {
     PipeArgs a;

@@ -20,9 +20,9 @@ A second form lets the kernels do both exchanges themselves, as stores through
 peer pointers (`PeerTable`, `WorkerPerGpu.step_pushed`):
 
     local updates + pack, stored into the servers' receive buffers   (zoa_dist_step_pack_push)
-    barrier between the ranks (stream-ordered)
+    stream_barrier between the ranks
     server part, result stored into every rank's words_s / scales_s  (zoa_dist_server_push)
-    barrier
+    stream_barrier
     m, x, u from the packed result                                   (zoa_dist_apply)
 
 No kernel waits for another rank; on a sync step the half-step momentum, model and
@@ -99,6 +99,25 @@ def gather_server(plan: ExchangePlan, rank: int, words_s: torch.Tensor, scales_s
         w, c = plan.words[r], plan.chunks[r]
         words_s[w.start:w.stop] = all_w[r, :len(w)]
         scales_s[c.start:c.stop] = all_c[r, :len(c)]
+
+
+_BARRIER_TOKENS = {}
+
+
+def stream_barrier(group=None):
+    """Orders the ranks on the current CUDA stream with a one-element all-reduce.
+
+    Why this orders the peer stores: torch enqueues the collective behind everything this rank
+    has already put on the current stream, and makes the current stream wait for the collective
+    before anything enqueued later runs.  The sum a rank receives depends on every rank's input,
+    so the collective cannot finish anywhere before every rank has started it, that is, before
+    every rank's earlier kernels (and the stores they made into other ranks' memory) are done.
+    The host does not block."""
+    dev = torch.cuda.current_device()
+    token = _BARRIER_TOKENS.get(dev)
+    if token is None:
+        token = _BARRIER_TOKENS[dev] = torch.zeros(1, dtype=torch.int32, device=torch.device("cuda", dev))
+    dist.all_reduce(token, op=dist.ReduceOp.SUM, group=group)
 
 
 @dataclass
@@ -235,10 +254,12 @@ class WorkerPerGpu:
                                self.recv_scales.data_ptr(), self.recv_scales.stride(0), self.world, c.start, len(c),
                                peers.words_s, peers.scales_s, torch.cuda.current_stream().cuda_stream)
 
-    def step_pushed(self, grad: torch.Tensor, lr: float, t: int, peers: PeerTable, barrier):
+    def step_pushed(self, grad: torch.Tensor, lr: float, t: int, peers: PeerTable, barrier=None):
         """One iteration of Algorithm 1 on this rank.  `barrier()` must order the ranks on the
         current stream: nothing enqueued after it may start before every rank has finished what it
-        enqueued before (torch.distributed's NCCL barrier does)."""
+        enqueued before.  Default: `stream_barrier` on this worker's group."""
+        if barrier is None:
+            barrier = lambda: stream_barrier(self.group)
         if not self.opt.sync_due(t):
             self.opt.step([grad], lr, t)
         else:

@@ -144,6 +144,16 @@ class Zoa:
         values = np.ascontiguousarray(values, np.uint32 if which in B.WORD_BUFFERS else np.float32)
         B.zoa_copy_in(self.h, which, worker, offset, values.size, values.ctypes.data)
 
+    def export_state(self):
+        """The whole optimizer state (zoa_export_state) as a numpy byte array."""
+        blob = np.empty(B.zoa_state_size(self.h), np.uint8)
+        B.zoa_export_state(self.h, blob.ctypes.data, blob.size)
+        return blob
+
+    def import_state(self, blob):
+        blob = np.ascontiguousarray(blob, np.uint8)
+        B.zoa_import_state(self.h, blob.ctypes.data, blob.size)
+
     def stats(self):
         return B.zoa_get_stats(self.h)
 

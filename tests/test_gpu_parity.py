@@ -232,36 +232,61 @@ def test_unaligned_gradient_pointers():
         p.close()
 
 
-def test_checkpoint_round_trip():
-    """k steps, export, import into a fresh handle, k more steps == 2k steps."""
+@pytest.mark.parametrize("where", ["pending_variance", "after_sync", "mid_interval"])
+def test_checkpoint_round_trip(where):
+    """zoa_export_state / zoa_import_state through the C ABI: run, export, import into a fresh handle,
+    continue on both; the two handles stay bit-identical and both match the oracle.  In the
+    "pending_variance" case the export falls between zoa_step on a step in T_u and T_v and
+    zoa_onebit_reduce, when the handle holds v_t (which the model sync still needs) and v_{t+1}."""
     rng = np.random.default_rng(6)
     n, W, chunk = 5000, 3, 512
-    gs = [_grads(rng, W, n) for _ in range(8)]
-    x0 = torch.from_numpy((rng.standard_normal(n) * 0.02).astype(np.float32))
-    pol = ((0, 1, 5), (0, 2), (1, 3))
-    a, b = Zoa(n, W, chunk=chunk), Zoa(n, W, chunk=chunk)
+    var_steps, sync = (0, 1, 5), ((0, 2), (1, 3))        # T_u = {0, 1, 2, 5, 8, ...}
+    cut = {"pending_variance": 5, "after_sync": 3, "mid_interval": 4}[where]
+    gs = [_grads(rng, W, n) for _ in range(10)]
+    x0 = rng.standard_normal(n) * 0.02
+    p = Pair(n, W, chunk, var_steps=var_steps, sync=sync, x0=x0)
+    b = Zoa(n, W, chunk=chunk, beta1=0.5, beta2=0.5, eps=1e-3)      # everything, hyper-parameters included, comes from the blob
     try:
-        a.set_params(x0), a.set_policies(*pol), b.set_policies(*pol)
-        for t in range(4):
-            a.step_auto(list(torch.from_numpy(gs[t]).cuda()), 1e-3, t)
-        st = a.stats()
-        for name in ("x", "m", "u", "delta_w"):
-            for i in range(W):
-                b.write(name, a.read(name, i), i)
-        for name in ("v", "delta_s", "x_sync"):
-            b.write(name, a.read(name))
-        B.zoa_set_scalars(b.h, st["gamma_sum"], st["t_sync"], st["t_last"])
-        for t in range(4, 8):
+        a = p.gpu
+        for t in range(cut):
+            p.step(gs[t], 1e-3, t, "two_call")
+        if where == "pending_variance":
+            # first half of step `cut`: zoa_step on a T_u and T_v step, export before the reduce
+            a.step(list(torch.from_numpy(gs[cut]).cuda()), 1e-3, cut)
+        size = B.zoa_state_size(a.h)
+        blob = a.export_state()
+        assert blob.size == size
+        with pytest.raises(ZoaError):                    # a truncated blob changes nothing
+            B.zoa_import_state(b.h, blob.ctypes.data, size - 4)
+        other = Zoa(n + 1, W, chunk=chunk)
+        try:
+            with pytest.raises(ZoaError):                # another shape
+                other.import_state(blob)
+        finally:
+            other.close()
+        b.import_state(blob)
+        assert b.stats() == {**a.stats(), "n_launches": b.stats()["n_launches"]}
+        assert b.sync_due(4) == a.sync_due(4) and b.var_due(5) and not b.var_due(4)
+        if where == "pending_variance":
+            a.onebit_reduce(), b.onebit_reduce()
+            torch.cuda.synchronize()
+            assert p.cpu.step(gs[cut], np.float32(1e-3), cut, True, True) == 0
+            p.compare(f"{where} t={cut}")
+            cut += 1
+        for t in range(cut, 10):
             g = list(torch.from_numpy(gs[t]).cuda())
-            a.step_auto(g, 1e-3, t), b.step_auto(g, 1e-3, t)
-        torch.cuda.synchronize()
-        for name in ("x", "m", "u", "delta_w"):
-            for i in range(W):
-                assert np.array_equal(a.read(name, i), b.read(name, i)), name
-        for name in ("v", "delta_s", "x_sync"):
-            assert np.array_equal(a.read(name), b.read(name)), name
+            b.step_auto(g, 1e-3, t)
+            p.step(gs[t], 1e-3, t, "fused")
+            p.compare(f"{where} t={t}", wire=a.sync_due(t))
+            for name in ("x", "m", "u", "delta_w"):
+                for i in range(W):
+                    assert np.array_equal(a.read(name, i), b.read(name, i)), (name, i, t)
+            for name in ("v", "delta_s", "x_sync"):
+                assert np.array_equal(a.read(name), b.read(name)), (name, t)
+        assert a.stats()["gamma_sum"] == b.stats()["gamma_sum"] and a.stats()["t_sync"] == b.stats()["t_sync"]
+        b.check_device()
     finally:
-        a.close(), b.close()
+        p.close(), b.close()
 
 
 def test_host_gradient_entry_point():
@@ -385,10 +410,17 @@ def test_device_wait_runs_out_and_is_reported(algorithm):
         B.zoa_set_option(z.h, B.OPT_TEST_STOP_AFTER_TILES, 3)
         t0 = time.perf_counter()
         step(g, 1e-3, 1)
+        torch.cuda.synchronize()                          # the kernel has ended by itself
+        assert time.perf_counter() - t0 < 5.0             # bounded: a few wait limits, not a hang
+        with pytest.raises(ZoaError) as e:                # the next step call itself refuses, without any check call
+            step(g, 1e-3, 2)
+        assert e.value.status == B.ERR_DEVICE
+        with pytest.raises(ZoaError) as e:
+            z.onebit_reduce()
+        assert e.value.status == B.ERR_DEVICE
         with pytest.raises(ZoaError) as e:
             z.check_device()
         assert e.value.status == B.ERR_DEVICE
-        assert time.perf_counter() - t0 < 5.0             # bounded: a few wait limits, not a hang
         B.zoa_set_option(z.h, B.OPT_TEST_STOP_AFTER_TILES, 0)
         B.zoa_set_option(z.h, B.OPT_WAIT_LIMIT_MS, 2000)
         step(g, 1e-3, 2)
