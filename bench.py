@@ -124,47 +124,116 @@ class ClockSampler:
                 "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
+# ---- which steps are timed, and the config block both arms print ---------------------------
+def step_window(wl, K):
+    """The K step indices a run times.  K >= the workload's own length: its whole schedule from
+    t = 0.  Shorter runs start four steps before the schedule's first local step, so that the window
+    holds sync steps, sync + variance steps and local steps (the first steps of every schedule are
+    all sync steps)."""
+    if K >= wl.steps:
+        return list(range(K))
+    first_local = next((t for t in range(wl.steps) if not wl.in_T_u(t)), 0)
+    t0 = max(0, first_local - 4)
+    return list(range(t0, t0 + K))
+
+
+def config_block(wl, args, steps, world):
+    kinds = [("sync" if wl.in_T_u(t) else "local") + ("+var" if wl.in_T_v(t) else "") for t in steps]
+    mix = ", ".join(f"{kinds.count(k)} {k}" for k in sorted(set(kinds)))
+    return {"workload": wl.name, "n_params": wl.n, "W": wl.W, "chunk": wl.chunk,
+            "algorithm": "Algorithm 1 (0/1 Adam)" if args.algorithm == "alg1" else
+                         "Algorithm 2 (gradients through the 1-bit AllReduce, full precision on T_v steps)",
+            "schedule": f"t={steps[0]}..{steps[-1]} of the workload's T_u/T_v policies ({mix})",
+            "grad_dtype": args.grad_dtype,
+            "l2": "inputs larger than L2 (gradients and state are read once per step)",
+            "parallelism": f"{world} x independent chunk ranges, no collective"}
+
+
 # ---- the CPU oracle, timed as it stands (baseline and --impl reference) ---------------
-def time_oracle(wl, sample_elems, steps, seed=1):
-    """Runs the oracle (oracle/, single thread) on the first `sample_elems`
-    parameters of the workload for the given step indices; returns
-    (params*workers/s, description)."""
+def time_oracle(wl, steps, grads_of, x0, budget_elems, algorithm="alg1"):
+    """Times the oracle (oracle/zoa_oracle.c, float build, untouched and single-threaded) on a
+    slice of the workload: one oracle instance per chunk range on every core the process may
+    use, each called from its own thread (the C call releases the interpreter lock).
+    grads_of(t) returns the step's W gradient buffers (the ones the CUDA arm consumes for that
+    t); their first d elements are copied to the host, untimed.  Returns
+    (params*workers/s, cores, description, seconds per step scaled to the full vector)."""
     import numpy as np
+    from concurrent.futures import ThreadPoolExecutor
     from oracle import zoa_oracle as zo
 
-    d = min(sample_elems, wl.n)
-    rng = np.random.default_rng(seed)
-    o = zo.Oracle(d, wl.W, wl.chunk, wl.beta1, wl.beta2, wl.eps, dtype=np.float32)
-    o.set_params((rng.standard_normal(d) * wl.x0_std).astype(np.float32))
-    g = rng.standard_normal((wl.W, d)).astype(np.float32)
-    o.step(g, np.float32(wl.lr), 0, True, True)          # untimed: touch every page once
-    t0 = time.perf_counter()
-    for k, t in enumerate(steps):
-        o.step(g, np.float32(wl.lr), k + 1, wl.in_T_u(t), wl.in_T_v(t))
-    dt = time.perf_counter() - t0
+    cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
+    # slice: a chunk range per core (4 Mi parameters at most), about 10-30 s of oracle work in all
+    per = max(wl.chunk, min(budget_elems // cores, 1 << 22) // wl.chunk * wl.chunk)
+    if per * cores > wl.n:
+        per = max(wl.chunk, wl.n // cores // wl.chunk * wl.chunk)
+    if per * cores > wl.n:
+        cores = max(1, wl.n // per)
+    if per > wl.n:
+        per, cores = wl.n, 1
+    d = per * cores
+    x0 = np.asarray(x0[:d].cpu() if hasattr(x0, "cpu") else x0[:d], np.float32)
+    oracles = []
+    for c in range(cores):
+        o = zo.Oracle(per, wl.W, wl.chunk, wl.beta1, wl.beta2, wl.eps, dtype=np.float32)
+        for a in (o.x, o.m, o.u, o.delta, o.v, o.delta_bar, o.x_sync, o.z_hat, o.u_bar):
+            a.fill(0)                                    # touch every page before the clock starts
+        o.set_params(x0[c * per:(c + 1) * per])
+        oracles.append(o)
+    host = np.empty((wl.W, d), np.float32)
+    dt = 0.0
+    with ThreadPoolExecutor(cores) as pool:
+        for t in steps:
+            for i, g in enumerate(grads_of(t)):
+                host[i] = g[:d].float().cpu().numpy()
+            parts = [np.ascontiguousarray(host[:, c * per:(c + 1) * per]) for c in range(cores)]
+            lr = np.float32(wl.lr_at(t))
+            if algorithm == "alg2":
+                call = lambda c: oracles[c].alg2_step(parts[c], lr, wl.in_T_v(t))
+            else:
+                call = lambda c: oracles[c].step(parts[c], lr, t, wl.in_T_u(t), wl.in_T_v(t))
+            t0 = time.perf_counter()
+            list(pool.map(call, range(cores)))
+            dt += time.perf_counter() - t0
     n_sync = sum(wl.in_T_u(t) for t in steps)
-    desc = (f"first {d} parameters x {wl.W} workers of {wl.name}, {len(steps)} steps of its schedule "
-            f"(t={steps[0]}..{steps[-1]}: {n_sync} sync, {len(steps) - n_sync} local), oracle/zoa_oracle.c float build")
-    return d * wl.W * len(steps) / dt, desc, dt
+    desc = (f"first {d} parameters x {wl.W} workers of {wl.name} ({cores} chunk ranges of {per}, one oracle instance and "
+            f"one thread per core), steps t={steps[0]}..{steps[-1]} of its schedule ({n_sync} sync, {len(steps) - n_sync} local) "
+            f"on the gradient buffers the CUDA arm consumes for those steps, oracle/zoa_oracle.c float build")
+    return d * wl.W * len(steps) / dt, cores, desc, dt / len(steps) * (wl.n / d)
 
 
-def run_reference(args, wl):
+def oracle_inputs(wl, synth, seed):
+    """The gradient stream and x_0 of the CUDA arm, regenerated from the same seeds (on the GPU when
+    there is one, so that the oracle sees the very same bits; on the host otherwise)."""
+    import torch
+    if torch.cuda.is_available():
+        stream = synth.GradientStream(wl, "cuda", seed)
+        return stream.fill, synth.initial_params(wl, "cuda", seed), "generated on the GPU by the CUDA arm's seeded stream"
+    # no CUDA device: only a slice-sized layout is generated, from the host generator
+    small = synth.Workload(wl.name, [min(wl.n, 1 << 25)], wl.W, wl.chunk, wl.steps, wl.var_steps, wl.sync_boundaries,
+                           wl.sync_intervals, wl.shared, wl.noise, wl.noise_kind, False)
+    stream = synth.GradientStream(small, "cpu", seed)
+    return stream.fill, synth.initial_params(small, "cpu", seed), "generated on the host (no CUDA device)"
+
+
+def run_reference(args, wl, synth):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    steps = list(range(60, 60 + max(1, min(args.steps, 10))))
+    steps = step_window(wl, args.steps)
+    timed = steps[:max(1, min(len(steps), args.cpu_steps))]
+    grads_of, x0, how = oracle_inputs(wl, synth, synth.DEFAULT_SEED)
     for _ in range(min(args.warmup, 1)):
-        time_oracle(wl, 1 << 18, steps[:2])
-    value, desc, dt = time_oracle(wl, args.cpu_sample, steps)
-    per_step_ms = dt / len(steps) * 1e3 * (wl.n / min(args.cpu_sample, wl.n))
+        time_oracle(wl, timed[:1], grads_of, x0, 1 << 20, args.algorithm)
+    value, cores, desc, s_per_step = time_oracle(wl, timed, grads_of, x0, args.cpu_sample, args.algorithm)
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step_ms,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": s_per_step * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
-            "data": "synthetic", "config": {"workload": wl.name, "n_params": wl.n, "W": wl.W, "chunk": wl.chunk},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc},
+            "data": "synthetic", "config": config_block(wl, args, steps, int(os.environ.get("WORLD_SIZE", "1"))),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc + "; inputs " + how},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0,
-            "note": "ms_per_step is the sampled time scaled to the full parameter count"}
+            "note": f"each timed step is a bounded sample (the first {len(timed)} of the {len(steps)} step indices, a slice of "
+                    "the parameters); ms_per_step is the sampled time per step scaled to the full parameter count"}
     print(json.dumps(line))
 
 
@@ -215,11 +284,29 @@ def run_ours(args, wl):
         return g16
 
     K, Wu = args.steps, max(args.warmup, 3)
-    for t in range(Wu):                                   # warm-up: the first steps of the schedule
-        opt.step_auto(batch(t), wl.lr_at(t), t)
-    # also warm the local-step kernel, then rewind the step counter (timing does not depend on values)
-    opt.step(batch(Wu), wl.lr, Wu)
+    steps = step_window(wl, K)
+    t_first = steps[0]
+
+    def one_step(bufs, t):
+        if args.algorithm == "alg2":
+            opt.alg2_step(bufs, wl.lr_at(t), t)
+            return "alg2_full" if wl.in_T_v(t) else "alg2_compressed"
+        if args.two_call and wl.in_T_u(t):
+            opt.step(bufs, wl.lr_at(t), t)
+            opt.onebit_reduce()
+            return "two_call_sync" + ("+var" if wl.in_T_v(t) else "")
+        opt.step_auto(bufs, wl.lr_at(t), t)
+        return ("sync" if wl.in_T_u(t) else "local") + ("+var" if wl.in_T_v(t) else "")
+
+    # warm-up: the local-step kernel once, then the Wu steps of the schedule that precede the window
+    # (or its first Wu steps again when the window starts at 0), with the step counter rewound
+    # after each part (timing does not depend on the values in the state)
+    opt.step(batch(0), wl.lr, 0)
     B.zoa_set_scalars(opt.h, 0.0, 0, -1)
+    for t in (range(t_first - Wu, t_first) if t_first >= Wu else range(Wu)):
+        one_step(batch(t), t)
+    if t_first < Wu:
+        B.zoa_set_scalars(opt.h, 0.0, 0, -1)
     barrier()
 
     launches0 = opt.stats()["n_launches"]
@@ -228,20 +315,11 @@ def run_ours(args, wl):
     with ClockSampler(local_rank) as clocks:
         barrier()
         wall0 = time.perf_counter()
-        for t in range(K):
+        for k, t in enumerate(steps):
             bufs = batch(t)                               # untimed: the batch is resident before the step starts
-            ev[t][0].record()
-            if args.algorithm == "alg2":
-                opt.alg2_step(bufs, wl.lr_at(t), t)
-                kinds.append("alg2_full" if wl.in_T_v(t) else "alg2_compressed")
-            elif args.two_call and wl.in_T_u(t):
-                opt.step(bufs, wl.lr_at(t), t)
-                opt.onebit_reduce()
-                kinds.append("two_call_sync" + ("+var" if wl.in_T_v(t) else ""))
-            else:
-                opt.step_auto(bufs, wl.lr_at(t), t)
-                kinds.append(("sync" if wl.in_T_u(t) else "local") + ("+var" if wl.in_T_v(t) else ""))
-            ev[t][1].record()
+            ev[k][0].record()
+            kinds.append(one_step(bufs, t))
+            ev[k][1].record()
         barrier()
         wall = time.perf_counter() - wall0
     opt.check_device()
@@ -299,11 +377,11 @@ def run_ours(args, wl):
         host_x = torch.empty(wl.n, dtype=torch.float32, pin_memory=True)
         B.zoa_set_scalars(opt.h, 0.0, 0, -1)
         opt.step_host(host_g, wl.lr, 0, host_x)           # allocates the staging area; untimed
-        B.zoa_set_scalars(opt.h, 0.0, 0, -1)
+        B.zoa_set_scalars(opt.h, 0.0 if wl.in_T_u(steps[0]) else wl.lr, 0, -1)
         barrier()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record()
-        for t in range(ke):
+        for t in steps[:ke]:
             opt.step_host(host_g, wl.lr_at(t), t, host_x)
         b.record()
         barrier()
@@ -322,18 +400,15 @@ def run_ours(args, wl):
     if rank == 0:
         cpu = None
         if world == 1 and not args.no_cpu_baseline:
-            value, desc, _ = time_oracle(wl, args.cpu_sample, list(range(60, 70)))
-            cpu = {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc}
+            timed = steps[:max(1, min(len(steps), args.cpu_steps))]
+            value, cores, desc, _ = time_oracle(wl, timed, stream.fill, synth.initial_params(wl, "cuda", seed),
+                                                args.cpu_sample, args.algorithm)
+            cpu = {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
         line = {"metric": METRIC, "value": wl.n * wl.W * K * world / (total_ms / 1e3), "unit": UNIT,
                 "n_gpus": world, "steps": K, "warmup": Wu, "ms_per_step": total_ms / K,
                 "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
                 "data": "synthetic", "grad_dtype": args.grad_dtype,
-                "config": {"workload": wl.name, "n_params": wl.n, "W": wl.W, "chunk": wl.chunk,
-                           "algorithm": "Algorithm 1 (0/1 Adam)" if args.algorithm == "alg1" else
-                                        "Algorithm 2 (gradients through the 1-bit AllReduce, full precision on T_v steps)",
-                           "schedule": f"t=0..{K - 1} of the workload's T_u/T_v policies",
-                           "l2": "inputs larger than L2 (gradients and state are read once per step)",
-                           "parallelism": f"{world} x independent chunk ranges, no collective"},
+                "config": config_block(wl, args, steps, world),
                 "hbm_GBps": total_bytes / 1e6 / total_ms, "hbm_frac_of_measured_peak": total_bytes / 1e6 / total_ms / peak,
                 "step_types": step_types, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e,
                 "gpu_launches": launches, "clocks": clocks.summary(), "wall_s_timed_region": wall}
@@ -370,7 +445,7 @@ def run_worker_per_gpu(args, wl):
     if args.exchange == "push":          # the kernels store into the peers' buffers themselves
         from paper_2202_06009_b200.distributed import PeerTable
         peers = PeerTable.symmetric(w)
-        step = lambda g, lr, t: w.step_pushed(g, lr, t, peers, dist.barrier)
+        step = lambda g, lr, t: w.step_pushed(g, lr, t, peers)      # ranks ordered by a one-element all-reduce on the stream
     else:
         step = w.step
     for t in range(Wu):
@@ -477,7 +552,9 @@ def main():
     ap.add_argument("--workload", default="bert_large",
                     help="tiny | bert_base | bert_large (default, the headline) | gpt2_1p5b | all (one line each)")
     ap.add_argument("--e2e-steps", type=int, default=3)
-    ap.add_argument("--cpu-sample", type=int, default=1 << 22, help="parameters in the oracle's timed sample")
+    ap.add_argument("--cpu-sample", type=int, default=1 << 25,
+                    help="upper bound on the parameters in the oracle's timed sample (4 Mi per core at most)")
+    ap.add_argument("--cpu-steps", type=int, default=8, help="how many of the window's first steps the oracle is timed on")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--scale", type=int, default=1, help="shrink every tensor by this factor (profiling captures)")
     ap.add_argument("--no-pipeline", action="store_true", help="fused sync step through the chunk-per-block kernel")
@@ -512,9 +589,11 @@ def main():
         wl = synth.WORKLOADS[args.workload]()
         if args.scale > 1:
             wl = synth.scaled(wl, args.scale)
+        if args.chunk:
+            wl.chunk = args.chunk
         if args.steps is None:
             args.steps = wl.steps
-        return run_reference(args, wl)
+        return run_reference(args, wl, synth)
 
     from paper_2202_06009_b200 import synth
     if args.workload == "all":      # one JSON line per shaped workload, BERT-Large (the headline) last
