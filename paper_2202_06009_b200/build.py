@@ -5,8 +5,8 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libzoa.so")
-SOURCES = ["zoa_kernels.cu", "zoa_pipeline.cu", "zoa_api.cu", "zoa_noalloc.cu"]
-HEADERS = ["zoa_device.cuh", "zoa_internal.h", os.path.join("..", "..", "include", "zoa.h")]
+SOURCES = ["zoa_kernels.cu", "zoa_pipeline.cu", "zoa_reduce_pipeline.cu", "zoa_api.cu", "zoa_noalloc.cu"]
+HEADERS = ["zoa_device.cuh", "zoa_internal.h", "zoa_ring.cuh", os.path.join("..", "..", "include", "zoa.h")]
 
 # The arithmetic contract needs IEEE division and square root, subnormals kept,
 # and no contraction of a multiply and an add into one fused operation.

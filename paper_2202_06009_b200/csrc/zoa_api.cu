@@ -394,7 +394,7 @@ static cudaError_t run_compress(zoa_handle h, cudaStream_t s)
         GradPtrs none{};
         e = launch_large_compress(view(h), none, h->c, 0.f, 0, kGradAligned, h->partials, &launches, s);
     } else {
-        e = launch_compress(view(h), s);
+        e = launch_compress(view(h), 0, h->n_chunks, s);
         launches = 1;
     }
     h->n_launches += launches;
@@ -407,8 +407,20 @@ static cudaError_t run_server(zoa_handle h, float gamma_sum, cudaStream_t s)
     if (h->large_chunk) {
         e = launch_large_server(view(h), h->c, 1, gamma_sum, h->partials, &launches, s);
     } else {
-        e = launch_reduce(view(h), h->c, gamma_sum, s);
-        launches = 1;
+        const StateView st = view(h);
+        long long n_units = 0, first = 0;
+        const int stages = h->use_pipeline ? reduce_pipeline_stages(st, &n_units) : 0;
+        e = cudaSuccess;
+        if (stages > 0 && (h->use_pipeline == 2 || n_units >= 4ll * h->sm_count)) {
+            e = launch_reduce_pipelined(st, h->c, gamma_sum, n_units, stages, h->sm_count, error_words(h), h->sched,
+                                        (unsigned long long)h->wait_limit_ms * 1000000ull, h->test_stop_after_tiles, s);
+            ++launches;
+            first = n_units * std::max<long long>(h->chunk, 2048) / h->chunk;
+        }
+        if (e == cudaSuccess && first < h->n_chunks) {
+            e = launch_reduce(st, h->c, gamma_sum, first, h->n_chunks - first, s);
+            ++launches;
+        }
     }
     h->n_launches += launches;
     return e;

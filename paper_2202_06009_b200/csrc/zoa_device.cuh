@@ -100,6 +100,23 @@ __device__ __forceinline__ float4 ld4_stream(const float *p)
 }
 __device__ __forceinline__ void st4_stream(float *p, float4 v) { __stcs(reinterpret_cast<float4 *>(p), v); }
 
+// ---- bulk asynchronous stores (the copy engine reads shared memory and writes global memory) ----
+// A thread that wrote the shared-memory source with ordinary stores runs store_fence() before the
+// block barrier that precedes the bulk store; the issuing thread commits its stores as a group and
+// waits until the engine has read the source before the block reuses or releases it.  Both
+// addresses must be 16-byte aligned and the size a multiple of 16 bytes.
+__device__ __forceinline__ void store_fence() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void bulk_store(void *dst_global, const void *src_shared, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                 ::"l"(dst_global), "r"((uint32_t)__cvta_generic_to_shared(src_shared)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// Returns once the source of every committed group but the newest `N` has been read.
+template <int N>
+__device__ __forceinline__ void bulk_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+
 // How the W gradient buffers are to be read: bit 0 = every pointer is aligned for the
 // vector path (16 bytes for binary32, 8 for the 16-bit types), bits 1-2 = element type.
 // Gradients in binary16 / bfloat16 are converted to binary32 exactly on load; all

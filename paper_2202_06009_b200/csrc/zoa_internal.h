@@ -40,8 +40,16 @@ cudaError_t launch_local_step(const StateView &st, const GradPtrs &g, const Cons
                               bool do_var, int g_aligned, long long first, long long end, cudaStream_t s);
 cudaError_t launch_variance(const StateView &st, const GradPtrs &g, const Consts &c, int g_aligned,
                             long long first, long long end, cudaStream_t s);
-cudaError_t launch_compress(const StateView &st, cudaStream_t s);
-cudaError_t launch_reduce(const StateView &st, const Consts &c, float gamma_sum, cudaStream_t s);
+cudaError_t launch_compress(const StateView &st, long long first_chunk, long long count, cudaStream_t s);
+cudaError_t launch_reduce(const StateView &st, const Consts &c, float gamma_sum, long long first_chunk, long long count, cudaStream_t s);
+
+// Ring form of the server half of zoa_onebit_reduce, zoa_reduce_pipeline.cu.  reduce_pipeline_stages:
+// ring depth (0 = the kernel does not take this shape) and how many whole units of max(chunk, 2048)
+// coordinates the vector holds; the chunks after them go through launch_reduce.
+int reduce_pipeline_stages(const StateView &st, long long *n_units);
+cudaError_t launch_reduce_pipelined(const StateView &st, const Consts &c, float gamma_sum, long long n_units, int stages,
+                                    int sm_count, ErrorWords error_flag, unsigned long long *sched,
+                                    unsigned long long wait_limit_ns, long long test_stop_after_tiles, cudaStream_t s);
 cudaError_t launch_step_sync(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
                              float gamma_sum, int g_aligned, long long first_chunk, long long count, cudaStream_t s);
 

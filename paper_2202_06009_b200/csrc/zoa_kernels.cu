@@ -12,7 +12,11 @@
 //   alg2_compressed_kernel   Algorithm 2 on any other step (gradients through Algorithm 3)
 // Chunks larger than a block can hold, up to the whole vector (Eq. 3 as printed):
 //   lc_* kernels             per-segment partial l1 sums, fixed-order chunk sums, apply passes
+#include <cooperative_groups.h>
+
 #include "zoa_internal.h"
+
+namespace cg = cooperative_groups;
 
 namespace zoa {
 
@@ -121,41 +125,84 @@ __device__ __forceinline__ uint32_t compress_tile(float z[4], float hat[4], floa
     return pack_tile(b);
 }
 
-// Worker side of Algorithm 3 for (chunk blockIdx.x, worker blockIdx.y).
-__global__ void compress_kernel(StateView st)
+// A chunk above 4096 coordinates is shared by a thread-block cluster of CS blocks (2 or 4), each
+// taking chunk / CS consecutive coordinates, so that a block stays as small as the ones that move
+// chunk 4096 fastest.  The blocks' binary64 partial l1 sums meet through distributed shared
+// memory: every block writes its partial into slot [its rank] of every block's `slots`, and after
+// the cluster barrier every thread adds the CS slots in rank order.
+template <int CS>
+__device__ __forceinline__ double cluster_sum(double block_total, double *slots)
 {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    double *scratch = reinterpret_cast<double *>(smem_raw);        // 33 doubles
-    float *z_s = reinterpret_cast<float *>(smem_raw + 34 * sizeof(double));
-    const ChunkGeom cg = chunk_geom(st, blockIdx.x);
-    const int i = blockIdx.y;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
-    const long long row = (long long)i * st.n_pad + cg.c0;
+    if (CS == 1) return block_total;
+    cg::cluster_group cluster = cg::this_cluster();
+    const unsigned rank = cluster.block_rank();
+    if (threadIdx.x < CS) cluster.map_shared_rank(slots, threadIdx.x)[rank] = block_total;
+    cluster.sync();
+    double total = 0.0;
+#pragma unroll
+    for (int q = 0; q < CS; ++q) total += slots[q];
+    return total;
+}
 
+// The coordinates [lo, lo + mine) of the chunk that block `rank` of a CS-block cluster takes.
+struct BlockSpan {
+    int lo, mine;
+};
+template <int CS>
+__device__ __forceinline__ BlockSpan block_span(const StateView &st, const ChunkGeom &cg, int rank)
+{
+    BlockSpan b;
+    const int span = st.chunk / CS;
+    b.lo = rank * span;
+    const int hi = b.lo + span < cg.len ? b.lo + span : cg.len;
+    b.mine = hi > b.lo ? hi - b.lo : 0;
+    return b;
+}
+
+// Worker side of Algorithm 3 for (chunk first_chunk + blockIdx.x, worker blockIdx.y), the chunk
+// held in registers: thread t takes the float4 groups t, t + blockDim, ... (ITER of them), issues
+// all its loads before the first use, and keeps z = u + delta in registers across the block sum.
+// The block needs no shared memory for the chunk and has 2 ITER 128-bit loads in flight per
+// thread, which is what fills the memory pipeline (measured at n = 2^28, W = 16: chunk 4096
+// 6.94 TB/s against 6.74 with the chunk staged in shared memory by a loop of dependent
+// iterations; chunk 16384 6.54 against 5.62).
+template <int ITER>
+__global__ void __launch_bounds__(512, 2) compress_kernel(StateView st, long long first_chunk)
+{
+    __shared__ double scratch[34];
+    const long long chunk_id = first_chunk + blockIdx.x;
+    const ChunkGeom cg = chunk_geom(st, chunk_id);
+    const int i = blockIdx.y;
+    const int lane = threadIdx.x & 31;
+    const long long row = (long long)i * st.n_pad + cg.c0;
+    float4 u4[ITER], e4[ITER];
+#pragma unroll
+    for (int it = 0; it < ITER; ++it) {
+        const int idx = 4 * (it * blockDim.x + threadIdx.x);
+        const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+        u4[it] = idx < cg.len ? ld4_stream(st.u + row + idx) : zero;     // whole float4 groups: the rows' padding is zero
+        e4[it] = idx < cg.len ? ld4_stream(st.dw + row + idx) : zero;
+    }
+    float z[ITER][4];
     double l1 = 0.0;
-    for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
-        const int idx = base + 4 * lane;
-        if (idx < cg.len) {
-            const float4 u4 = ld4(st.u + row + idx), e4 = ld4(st.dw + row + idx);
-            const float4 z4 = make_float4(f_add(u4.x, e4.x), f_add(u4.y, e4.y), f_add(u4.z, e4.z), f_add(u4.w, e4.w));
-            st4(z_s + idx, z4);
-            l1 += fabs((double)z4.x) + fabs((double)z4.y) + fabs((double)z4.z) + fabs((double)z4.w);
-        }
+#pragma unroll
+    for (int it = 0; it < ITER; ++it) {
+        z[it][0] = f_add(u4[it].x, e4[it].x); z[it][1] = f_add(u4[it].y, e4[it].y);
+        z[it][2] = f_add(u4[it].z, e4[it].z); z[it][3] = f_add(u4[it].w, e4[it].w);
+        l1 += fabs((double)z[it][0]) + fabs((double)z[it][1]) + fabs((double)z[it][2]) + fabs((double)z[it][3]);
     }
     const float scale = chunk_scale(block_sum(l1, scratch), cg.len);
-    for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
-        const int idx = base + 4 * lane;
-        float z[4] = {0.f, 0.f, 0.f, 0.f}, hat[4];
-        if (idx < cg.len) {
-            const float4 z4 = ld4(z_s + idx);
-            z[0] = z4.x; z[1] = z4.y; z[2] = z4.z; z[3] = z4.w;
-        }
-        const uint32_t word = compress_tile(z, hat, scale, idx, cg.len);
-        if (idx < cg.len) st4(st.dw + row + idx, make_float4(z[0], z[1], z[2], z[3]));
+#pragma unroll
+    for (int it = 0; it < ITER; ++it) {
+        const int idx = 4 * (it * blockDim.x + threadIdx.x);
+        const int base = idx - 4 * lane;                   // first coordinate of the warp's 128
+        float hat[4];
+        const uint32_t word = compress_tile(z[it], hat, scale, idx, cg.len);
+        if (idx < cg.len) st4_stream(st.dw + row + idx, make_float4(z[it][0], z[it][1], z[it][2], z[it][3]));
         if (lane < 4 && base + 32 * lane < cg.len)
             st.words_w[(long long)i * st.words_stride + ((cg.c0 + base) >> 5) + lane] = word;
     }
-    if (threadIdx.x == 0) st.scales_w[(long long)i * st.n_chunks + blockIdx.x] = scale;
+    if (threadIdx.x == 0) st.scales_w[(long long)i * st.n_chunks + chunk_id] = scale;
 }
 
 // Server side of Algorithm 3 and the post-sync updates of Algorithm 1 for one tile whose
@@ -192,25 +239,31 @@ __device__ __forceinline__ void server_tile(const StateView &st, const Consts &c
     }
 }
 
-// Server side for chunk blockIdx.x, reading what compress_kernel sent.
-__global__ void __launch_bounds__(512, 3) reduce_kernel(StateView st, Consts c, float gamma_sum)
+// Server side for chunk first_chunk + blockIdx.x / CS, reading what compress_kernel sent: the
+// chunks the ring kernel (zoa_reduce_pipeline.cu) leaves over, and every shape it does not take.
+template <int CS>
+__global__ void __launch_bounds__(512) reduce_kernel(StateView st, Consts c, float gamma_sum, long long first_chunk)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     double *scratch = reinterpret_cast<double *>(smem_raw);
-    float *scales = reinterpret_cast<float *>(smem_raw + 34 * sizeof(double));  // kMaxWorkers floats
-    float *a_s = scales + kMaxWorkers;
-    const ChunkGeom cg = chunk_geom(st, blockIdx.x);
+    double *slots = scratch + 34;
+    float *scales = reinterpret_cast<float *>(smem_raw + 42 * sizeof(double));  // kMaxWorkers floats
+    float *a_s = scales + kMaxWorkers;                                           // [span]: the server input
+    const long long chunk_id = first_chunk + blockIdx.x / CS;
+    const ChunkGeom cg = chunk_geom(st, chunk_id);
+    const BlockSpan bs = block_span<CS>(st, cg, blockIdx.x % CS);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    const long long j0 = cg.c0 + bs.lo;          // this block's first coordinate
 
-    for (int i = threadIdx.x; i < st.W; i += blockDim.x) scales[i] = st.scales_w[(long long)i * st.n_chunks + blockIdx.x];
+    for (int i = threadIdx.x; i < st.W; i += blockDim.x) scales[i] = st.scales_w[(long long)i * st.n_chunks + chunk_id];
     __syncthreads();
 
     double l1 = 0.0;
-    for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
+    for (int base = warp * 128; base < bs.mine; base += n_warps * 128) {
         const int idx = base + 4 * lane;
-        if (idx < cg.len) {
+        if (idx < bs.mine) {
             double A[4] = {0.0, 0.0, 0.0, 0.0};
-            const long long word_idx = (cg.c0 + idx) >> 5;
+            const long long word_idx = (j0 + idx) >> 5;
             const int shift = idx & 31;
             for (int i = 0; i < st.W; ++i) {  // worker order
                 const uint32_t nib = st.words_w[(long long)i * st.words_stride + word_idx] >> shift;
@@ -218,28 +271,31 @@ __global__ void __launch_bounds__(512, 3) reduce_kernel(StateView st, Consts c, 
 #pragma unroll
                 for (int k = 0; k < 4; ++k) A[k] += ((nib >> k) & 1u) ? s : -s;
             }
-            const float4 e4 = ld4(st.ds + cg.c0 + idx);
+            const float4 e4 = ld4(st.ds + j0 + idx);
             const float ee[4] = {e4.x, e4.y, e4.z, e4.w};
             float a[4];
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                a[k] = idx + k < cg.len ? server_input(A[k], st.W, ee[k]) : 0.0f;
+                a[k] = idx + k < bs.mine ? server_input(A[k], st.W, ee[k]) : 0.0f;
                 l1 += fabs((double)a[k]);
             }
             st4(a_s + idx, make_float4(a[0], a[1], a[2], a[3]));
         }
     }
-    const float scale = chunk_scale(block_sum(l1, scratch), cg.len);
-    for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
+    const float scale = chunk_scale(cluster_sum<CS>(block_sum(l1, scratch), slots), cg.len);
+    ChunkGeom mine;             // this block's coordinates seen as a short chunk, for server_tile
+    mine.c0 = j0;
+    mine.len = bs.mine;
+    for (int base = warp * 128; base < bs.mine; base += n_warps * 128) {
         const int idx = base + 4 * lane;
         float a[4] = {0.f, 0.f, 0.f, 0.f};
-        if (idx < cg.len) {
+        if (idx < bs.mine) {
             const float4 a4 = ld4(a_s + idx);
             a[0] = a4.x; a[1] = a4.y; a[2] = a4.z; a[3] = a4.w;
         }
-        server_tile(st, c, cg, base, lane, a, scale, gamma_sum);
+        server_tile(st, c, mine, base, lane, a, scale, gamma_sum);
     }
-    if (threadIdx.x == 0) st.scales_s[blockIdx.x] = scale;
+    if (threadIdx.x == 0 && blockIdx.x % CS == 0) st.scales_s[chunk_id] = scale;
 }
 
 // A whole sync step for chunk blockIdx.x: the local updates in registers, worker
@@ -924,16 +980,25 @@ cudaError_t launch_variance(const StateView &st, const GradPtrs &g, const Consts
     return cudaGetLastError();
 }
 
-size_t compress_smem(int chunk) { return 34 * sizeof(double) + (size_t)chunk * sizeof(float); }
-size_t reduce_smem(int chunk) { return 34 * sizeof(double) + (kMaxWorkers + (size_t)chunk) * sizeof(float); }
+size_t compress_smem(int chunk) { return 34 * sizeof(double) + (size_t)chunk * sizeof(float); }                 // dist_pack_push_kernel
+size_t reduce_smem(int chunk) { return 34 * sizeof(double) + (kMaxWorkers + (size_t)chunk) * sizeof(float); }   // dist_server_kernel
+// reduce_kernel: block-sum and cluster scratch, magnitudes, the server input of `span` coordinates
+static size_t reduce_span_smem(int span) { return 42 * sizeof(double) + (kMaxWorkers + (size_t)span) * sizeof(float); }
+
+// How many blocks share a chunk in reduce_kernel (see cluster_sum): spans of 4096 coordinates for
+// the chunk sizes that divide evenly, one block otherwise.
+static int cluster_blocks(int chunk)
+{
+    if (chunk > 8192 && chunk % 512 == 0) return 4;
+    if (chunk > 4096 && chunk % 256 == 0) return 2;
+    return 1;
+}
 size_t step_sync_smem(int chunk) { return 34 * sizeof(double) + (size_t)chunk * (sizeof(double) + sizeof(float)); }
 
 cudaError_t configure_kernels()
 {
     cudaError_t e;
-    e = cudaFuncSetAttribute(compress_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)compress_smem(kMaxChunk));
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(reduce_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)reduce_smem(kMaxChunk));
+    e = cudaFuncSetAttribute(reduce_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)reduce_span_smem(kMaxChunk));
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(alg2_compressed_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)step_sync_smem(kMaxChunk));
     if (e != cudaSuccess) return e;
@@ -961,27 +1026,52 @@ cudaError_t launch_alg2(const StateView &st, const GradPtrs &g, const Consts &c,
     return cudaGetLastError();
 }
 
-cudaError_t launch_compress(const StateView &st, cudaStream_t s)
+// Launch of a kernel whose blocks form clusters of CS along x.
+template <int CS, typename... KArgs, typename... Args>
+static cudaError_t launch_clustered(void (*kern)(KArgs...), dim3 grid, int threads, size_t smem, cudaStream_t s, Args... args)
 {
-    const dim3 grid((unsigned)st.n_chunks, (unsigned)st.W);
-    // 16 coordinates per thread here (measured: 256-thread blocks move chunk 4096 at 6.7 TB/s,
-    // 512-thread ones at 6.0; at chunk 16384, 1024 threads 5.6 against 5.4 for 512)
-    int thr = 128;
-    while (thr < st.chunk / 16 && thr < 1024) thr <<= 1;
-    compress_kernel<<<grid, thr, compress_smem(st.chunk), s>>>(st);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3((unsigned)threads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = CS;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, args...);
+}
+
+// Worker side of Algorithm 3 for the chunks [first_chunk, first_chunk + count), one block per chunk and worker.
+cudaError_t launch_compress(const StateView &st, long long first_chunk, long long count, cudaStream_t s)
+{
+    // 16 coordinates per thread (32 above chunk 4096), in blocks of at most 512 threads: measured best
+    // at every chunk size from 1024 to 16384 (n = 2^28: 6.5 - 6.9 TB/s)
+    const int iter = st.chunk > 4096 ? 8 : 4;
+    const int thr = ((st.chunk + 4 * iter - 1) / (4 * iter) + 31) / 32 * 32;
+    const dim3 grid((unsigned)count, (unsigned)st.W);
+    if (iter == 8) compress_kernel<8><<<grid, thr, 0, s>>>(st, first_chunk);
+    else compress_kernel<4><<<grid, thr, 0, s>>>(st, first_chunk);
     return cudaGetLastError();
 }
 
-cudaError_t launch_reduce(const StateView &st, const Consts &c, float gamma_sum, cudaStream_t s)
+// Server side for the chunks [first_chunk, first_chunk + count), one block (or cluster) per chunk.
+cudaError_t launch_reduce(const StateView &st, const Consts &c, float gamma_sum, long long first_chunk, long long count, cudaStream_t s)
 {
+    const int cs = cluster_blocks(st.chunk), span = st.chunk / cs;
     // With few workers a block has little to move between its barriers, and smaller blocks
-    // (more of them per SM) do better: measured at chunk 4096, n = 2^28, W = 2: 4.75 TB/s with
-    // 512 threads, 5.21 with 256, 5.76 with 128; W = 4: 5.46, 6.07, 6.06; W = 16: 5.94, 5.91, 5.80.
-    // At chunk 16384, 512 threads are best at every W.
+    // (more of them per SM) do better.
     const int per_thread = st.W <= 2 ? 32 : 16;
     int thr = 128;
-    while (thr < st.chunk / per_thread && thr < 512) thr <<= 1;
-    reduce_kernel<<<(unsigned)st.n_chunks, thr, reduce_smem(st.chunk), s>>>(st, c, gamma_sum);
+    while (thr < span / per_thread && thr < 512) thr <<= 1;
+    const dim3 grid((unsigned)(count * cs));
+    const size_t smem = reduce_span_smem(span);
+    if (cs == 4) return launch_clustered<4>(reduce_kernel<4>, grid, thr, smem, s, st, c, gamma_sum, first_chunk);
+    if (cs == 2) return launch_clustered<2>(reduce_kernel<2>, grid, thr, smem, s, st, c, gamma_sum, first_chunk);
+    reduce_kernel<1><<<grid, thr, smem, s>>>(st, c, gamma_sum, first_chunk);
     return cudaGetLastError();
 }
 

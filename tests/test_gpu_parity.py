@@ -113,6 +113,42 @@ def test_pipelined_kernel_equals_chunk_per_block_kernel(W, chunk, n_chunks, tail
         a.close(), b.close()
 
 
+@pytest.mark.parametrize("W,chunk,n_units,tail", [(5, 4096, 301, 1852), (3, 2048, 700, 0), (4, 8192, 160, 704), (16, 16384, 40, 5),
+                                                  (2, 1024, 700, 1500), (7, 512, 650, 700), (3, 256, 620, 100), (64, 128, 610, 3),
+                                                  (33, 4096, 20, 0), (64, 2048, 30, 33), (1, 1024, 1300, 1024)])
+def test_two_call_ring_kernels_equal_chunk_per_block_kernels(W, chunk, n_units, tail):
+    """zoa_step + zoa_onebit_reduce with the compress / server ring kernels (chunks of 128 ... 16384,
+    several chunks per tile below 2048, several tiles per chunk above) against the same calls with
+    one block or cluster per chunk: same bits, and both within tolerance of the oracle.  The tail
+    holds whole chunks that do not fill a unit and a ragged last chunk."""
+    rng = np.random.default_rng(W + chunk)
+    n = n_units * max(chunk, 2048) + tail
+    x0 = (rng.standard_normal(n) * 0.02).astype(np.float32)
+    p = Pair(n, W, chunk, var_steps=(0, 2), x0=x0)          # ring kernels forced on
+    b = Zoa(n, W, chunk=chunk)
+    try:
+        b.set_pipeline(False)
+        b.set_params(torch.from_numpy(x0))
+        b.set_policies((0, 2), (0,), (1,))
+        for t in range(3):
+            g = (rng.standard_normal((W, n)) * 10.0 ** rng.integers(-2, 2)).astype(np.float32)
+            p.step(g, 1e-3, t, "two_call")
+            b.step(list(torch.from_numpy(g).cuda()), 1e-3, t)
+            b.onebit_reduce()
+            torch.cuda.synchronize()
+            p.gpu.check_device()
+            for name in ("x", "m", "u", "delta_w", "words_w", "scales_w"):
+                for i in (0, W // 2, W - 1):
+                    assert np.array_equal(p.gpu.read(name, i), b.read(name, i)), (name, i, t)
+            for name in ("v", "delta_s", "x_sync", "words_s", "scales_s"):
+                assert np.array_equal(p.gpu.read(name), b.read(name)), (name, t)
+            p.compare(f"t={t}")
+        p.padding_is_zero()
+        assert p.gpu.stats()["n_launches"] > b.stats()["n_launches"] or tail == 0      # ring + tail kernels
+    finally:
+        p.close(), b.close()
+
+
 @pytest.mark.parametrize("mode", ["fused", "two_call"])
 def test_special_values(mode):
     """Signed zeros, subnormals, an all-zero chunk, a chunk of one sign, a lone outlier."""
