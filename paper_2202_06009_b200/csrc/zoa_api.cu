@@ -444,23 +444,27 @@ static zoa_status run_sync_range(zoa_handle h, const StateView &st, const GradPt
 {
     const long long e0 = c0 * h->chunk, e1 = std::min<long long>(c1 * (long long)h->chunk, h->n);
     const bool ragged = c1 == h->n_chunks && h->n % h->chunk != 0;
-    const long long n_full = c1 - c0 - (ragged ? 1 : 0);
-    // The persistent kernel pays off once every SM has a few chunks to stream; below that the
+    // The ring kernel takes whole units (one chunk of 2048 coordinates or more, or the G smaller chunks of
+    // a tile) from a unit boundary; the chunks left over go to the chunk-per-block kernel.
+    const int G = pipeline_chunks_per_unit(st);
+    const long long n_units = c0 % G == 0 ? (c1 - c0 - (ragged ? 1 : 0)) / G : 0;
+    // The persistent kernel pays off once every SM has a few units to stream; below that the
     // one-block-per-chunk kernel starts faster (measured on a 512-chunk problem).
-    const bool enough_chunks = h->use_pipeline == 2 || n_full >= 4ll * h->sm_count;
-    const int stages = h->use_pipeline && enough_chunks && n_full > 0 ? pipeline_stages(st, fmt) : 0;
+    const bool enough = h->use_pipeline == 2 || n_units >= 4ll * h->sm_count;
+    const int stages = h->use_pipeline && enough && n_units > 0 ? pipeline_stages(st, fmt) : 0;
     long long var_first = e0;     // coordinates from here to e1 still need the variance update
     if (stages > 0) {
         bool var_fused = false;
-        ZOA_CUDA(h, launch_step_sync_pipelined(st, gp, h->c, lr, gamma_sum, do_var, fmt, c0, n_full, stages, h->sm_count,
+        ZOA_CUDA(h, launch_step_sync_pipelined(st, gp, h->c, lr, gamma_sum, do_var, fmt, c0 / G, n_units, stages, h->sm_count,
                                                error_words(h), h->sched, (unsigned long long)h->wait_limit_ms * 1000000ull,
                                                h->test_stop_after_tiles, &var_fused, s));
         h->n_launches += 1;
-        if (ragged) {
-            ZOA_CUDA(h, launch_step_sync(st, gp, h->c, lr, gamma_sum, fmt, c0 + n_full, 1, s));
+        const long long done = c0 + n_units * G;      // first chunk the ring kernel did not take
+        if (done < c1) {
+            ZOA_CUDA(h, launch_step_sync(st, gp, h->c, lr, gamma_sum, fmt, done, c1 - done, s));
             h->n_launches += 1;
         }
-        if (var_fused) var_first = (c0 + n_full) * h->chunk;
+        if (var_fused) var_first = done * h->chunk;
     } else {
         ZOA_CUDA(h, launch_step_sync(st, gp, h->c, lr, gamma_sum, fmt, c0, c1 - c0, s));
         h->n_launches += 1;
@@ -823,7 +827,9 @@ extern "C" zoa_status zoa_step_host(zoa_handle h, const void *const *host_grads,
     const bool do_var = zoa_var_due(h, t) == 1;
     const StateView st = view(h);
     for (int k = 0; k < kSegments; ++k) {
-        const long long c0 = h->n_chunks * k / kSegments, c1 = h->n_chunks * (k + 1) / kSegments;
+        // range boundaries on multiples of 16 chunks, so that every range starts on a unit of the ring kernels
+        const long long c0 = h->n_chunks * k / kSegments / 16 * 16;
+        const long long c1 = k + 1 == kSegments ? h->n_chunks : h->n_chunks * (k + 1) / kSegments / 16 * 16;
         const long long e0 = c0 * h->chunk, e1 = std::min<long long>(c1 * (long long)h->chunk, h->n);
         for (int i = 0; i < h->W; ++i)
             ZOA_CUDA(h, cudaMemcpyAsync(reinterpret_cast<char *>(const_cast<void *>(dev[i])) + (size_t)e0 * g_bytes,

@@ -65,8 +65,9 @@ cudaError_t launch_large_server(const StateView &st, const Consts &c, int mode, 
 
 // Pipelined (bulk-copy ring) form of the fused sync step, zoa_pipeline.cu.
 int pipeline_stages(const StateView &st, int grad_fmt);
+int pipeline_chunks_per_unit(const StateView &st);
 cudaError_t launch_step_sync_pipelined(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
-                                       float gamma_sum, bool do_var, int grad_fmt, long long first_chunk, long long n_chunks, int stages,
+                                       float gamma_sum, bool do_var, int grad_fmt, long long first_unit, long long n_units, int stages,
                                        int sm_count, ErrorWords error_flag,
                                        unsigned long long *sched, unsigned long long wait_limit_ns,
                                        long long test_stop_after_tiles, bool *var_fused, cudaStream_t s);

@@ -21,14 +21,23 @@
 
 namespace zoa {
 
-template <int TILES, bool DO_VAR>
+// A work unit is TILES tiles of 2048 coordinates: one chunk of 2048 ... 16384 coordinates (G = 1), or
+// one tile holding G = 2048 / chunk whole chunks of 128 ... 1024 coordinates (TILES = 1), in which
+// case a chunk's l1 norm is the sum over the 16 / G consumer warps that own it.
+template <int TILES, int G, bool DO_VAR>
 __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const __grid_constant__ PipeArgs a)
 {
+    constexpr int WPC = kConsumerWarps / G;          // consumer warps per chunk
+    constexpr long long kSpan = (long long)TILES * kTile;
+    // The server needs a unit's server errors before the l1 sum and its v and x_sync after it.  Up to four
+    // tiles stay in the ring over the sum; eight would fill it, so they travel twice: the errors
+    // first, each stage released as soon as it is read, then v and x_sync.
+    constexpr bool SERVER_TWO_PASS = TILES > 4;
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     PipeShared *sh = reinterpret_cast<PipeShared *>(smem_raw);
     const StateView &st = a.st;
     const int W = st.W;
-    const int words_per_chunk = st.chunk >> 5;
+    constexpr int words_per_chunk = (int)(kSpan >> 5);                                  // words of a unit
     uint32_t *bits_s = reinterpret_cast<uint32_t *>(smem_raw + 1024);                 // [W][words_per_chunk]
     float *scales_s = reinterpret_cast<float *>(bits_s + W * words_per_chunk);         // [kConsumerWarps][W]
     unsigned char *ring = smem_raw + ((1024 + (size_t)W * words_per_chunk * 4 + (size_t)kConsumerWarps * W * 4 + 1023) & ~(size_t)1023);
@@ -45,7 +54,7 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
         const uint32_t g_elem = (a.grad_fmt & kGradTypeMask) == kGradF32 ? 4u : 2u;
         long long chunk;
         for (long long k = 0; p.ok && p.next_chunk(k, &chunk); ++k) {
-            const long long c0 = chunk * st.chunk;
+            const long long c0 = chunk * kSpan;             // `chunk` numbers the units here
             for (int i = 0; p.ok && i <= W; ++i) {          // i == W: the server's tiles
                 for (int t = 0; t < TILES && p.stage_free(); ++t) {
                     const uint32_t full = p.full_barrier(), dst = p.stage_addr();
@@ -57,12 +66,25 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
                         bulk_load(dst + kTileBytes, st.m + row, kTileBytes, full);
                         bulk_load(dst + 2 * kTileBytes, st.u + row, kTileBytes, full);
                         bulk_load(dst + 3 * kTileBytes, st.dw + row, kTileBytes, full);
-                    } else {
+                    } else if (!SERVER_TWO_PASS) {
                         mbar_arrive_expect_tx(full, 3 * kTileBytes);
                         bulk_load(dst, st.ds + off, kTileBytes, full);
                         bulk_load(dst + kTileBytes, st.v + off, kTileBytes, full);
                         bulk_load(dst + 2 * kTileBytes, st.xs + off, kTileBytes, full);
+                    } else {
+                        mbar_arrive_expect_tx(full, kTileBytes);
+                        bulk_load(dst, st.ds + off, kTileBytes, full);
                     }
+                    p.advance();
+                }
+            }
+            if (SERVER_TWO_PASS) {      // v and x_sync follow once the server errors have gone through
+                for (int t = 0; t < TILES && p.stage_free(); ++t) {
+                    const uint32_t full = p.full_barrier(), dst = p.stage_addr();
+                    const long long off = c0 + (long long)t * kTile;
+                    mbar_arrive_expect_tx(full, 2 * kTileBytes);
+                    bulk_load(dst + kTileBytes, st.v + off, kTileBytes, full);
+                    bulk_load(dst + 2 * kTileBytes, st.xs + off, kTileBytes, full);
                     p.advance();
                 }
             }
@@ -84,7 +106,9 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
     // spread over the worker iterations of the next chunk (one worker's m, x, u after
     // each worker's compression) instead of leaving in one burst, so that the block's
     // stores and its ring's loads stay evenly mixed.  m is +-m_pos by the server's bit.
-    constexpr bool DEFER = !(TILES == 4 && DO_VAR);   // that variant has no registers to spare: it stores at once
+    // With eight tiles, or four tiles and the binary64 gradient sums of a T_v step, the tiles of x have no room
+    // in the registers (17 warps leave 96 per thread: one SM sub-partition hosts five of them): those store at once.
+    constexpr bool DEFER = TILES <= 2 || (TILES == 4 && !DO_VAR);
     float x_prev[DEFER ? TILES : 1][4];
     uint32_t bits_prev = 0;
     float m_pos_prev = 0.0f;
@@ -108,13 +132,15 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
         // wait that ran out is put to the vote.
         const bool gave_up = !mbar_wait(smem_addr(&sh->full[s]), phase, abort_flag, a.error_flag, a.wait_limit_ns);
         if (consumer_any(gave_up)) break;
-        const long long chunk = sh->chunk_queue[k % (kMaxStages + 2)];
+        const long long chunk = sh->chunk_queue[k % (kMaxStages + 2)];   // the unit
         if (chunk < 0) break;
-        const long long c0 = chunk * st.chunk;
-        double G[DO_VAR ? TILES : 1][4];
+        const long long c0 = chunk * kSpan;
+        const long long scale_idx = G == 1 ? chunk : chunk * G + warp / WPC;       // this thread's chunk
+        const bool scale_writer = G == 1 ? tid == 0 : (lane == 0 && warp % WPC == 0);
+        double Gs[DO_VAR ? TILES : 1][4];
         if (DO_VAR) {
 #pragma unroll
-            for (int t = 0; t < TILES; ++t) { G[t][0] = G[t][1] = G[t][2] = G[t][3] = 0.0; }
+            for (int t = 0; t < TILES; ++t) { Gs[t][0] = Gs[t][1] = Gs[t][2] = Gs[t][3] = 0.0; }
         }
         for (int i = 0; i < W; ++i) {
             float z[TILES][4];
@@ -143,10 +169,10 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
                     const float step = f_mul(a.gamma, momentum(a.c, mm[k], gg[k]));   // momentum update, buffer update
                     z[t][k] = f_add(f_add(uu[k], step), ee[k]);                       // u_{t+1/2} + delta
                     l1 += fabs((double)z[t][k]);
-                    if (DO_VAR) G[t][k] += (double)gg[k];
+                    if (DO_VAR) Gs[t][k] += (double)gg[k];
                 }
             }
-            const float scale = chunk_scale(consumer_sum(l1, sh, flip), st.chunk);
+            const float scale = chunk_scale(consumer_group_sum<WPC>(l1, sh, flip), st.chunk);
             const long long row = (long long)i * st.n_pad + c0;
 #pragma unroll
             for (int t = 0; t < TILES; ++t) {
@@ -165,7 +191,7 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
                 }
             }
             if (lane == 0) my_scales[i] = scale;
-            if (tid == 0) st.scales_w[(long long)i * st.n_chunks + chunk] = scale;
+            if (scale_writer) st.scales_w[(long long)i * st.n_chunks + scale_idx] = scale;
             if (DEFER && c0_prev >= 0) store_prev_worker(i);
         }
         __syncwarp();   // bits_s and my_scales were written by lanes of this warp
@@ -179,8 +205,12 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
             const bool ready = mbar_wait(smem_addr(&sh->full[s]), phase, abort_flag, a.error_flag, a.wait_limit_ns);
             srv_stage[t] = s;
             const float *stage = reinterpret_cast<const float *>(ring + (size_t)s * kStageBytes);
-            if (++s == R) { s = 0; phase ^= 1u; }
             const float4 d4 = ready ? ld4(stage + pos) : make_float4(0.f, 0.f, 0.f, 0.f);
+            if (SERVER_TWO_PASS) {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_addr(&sh->empty[s]));
+            }
+            if (++s == R) { s = 0; phase ^= 1u; }
             const float dd[4] = {d4.x, d4.y, d4.z, d4.w};
             double A[4] = {0.0, 0.0, 0.0, 0.0};
             const int shift = (lane & 7) * 4;
@@ -196,9 +226,14 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
                 l1 += fabs((double)av[t][k]);
             }
         }
-        const float scale = chunk_scale(consumer_sum(l1, sh, flip), st.chunk);
+        const float scale = chunk_scale(consumer_group_sum<WPC>(l1, sh, flip), st.chunk);
 #pragma unroll
         for (int t = 0; t < TILES; ++t) {
+            if (SERVER_TWO_PASS) {
+                mbar_wait(smem_addr(&sh->full[s]), phase, abort_flag, a.error_flag, a.wait_limit_ns);
+                srv_stage[t] = s;
+                if (++s == R) { s = 0; phase ^= 1u; }
+            }
             const float *stage = reinterpret_cast<const float *>(ring + (size_t)srv_stage[t] * kStageBytes);
             const float4 v4 = ld4(stage + kTile + pos), xs4 = ld4(stage + 2 * kTile + pos);
             __syncwarp();
@@ -238,7 +273,7 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
             if (DO_VAR) {
                 float vo[4];
 #pragma unroll
-                for (int k = 0; k < 4; ++k) vo[k] = variance(a.c, vv[k], mean_round(G[t][k], W));   // variance update
+                for (int k = 0; k < 4; ++k) vo[k] = variance(a.c, vv[k], mean_round(Gs[t][k], W));   // variance update
                 st4_stream(st.v_next + j, make_float4(vo[0], vo[1], vo[2], vo[3]));
             }
         }
@@ -246,7 +281,7 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
             m_pos_prev = f_div(scale, a.gamma_sum);     // momentum approximation: m = +-scale / sum(gamma); -(s/G) == (-s)/G exactly
             c0_prev = c0;
         }
-        if (tid == 0) st.scales_s[chunk] = scale;
+        if (scale_writer) st.scales_s[scale_idx] = scale;
         __syncwarp();   // the next chunk overwrites bits_s / my_scales of this warp
     }
     if (c0_prev >= 0)
@@ -448,9 +483,25 @@ __global__ void __launch_bounds__(kThreads, 1) alg2_pipelined_kernel(const __gri
 // ---------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------
+// Tiles per unit and chunks per tile for a chunk size the ring kernels take (false: they do not).
+static bool unit_shape(int chunk, int *tiles, int *chunks_per_tile)
+{
+    *tiles = 1;
+    *chunks_per_tile = 1;
+    if (chunk >= kTile) {
+        if (chunk % kTile != 0) return false;
+        *tiles = chunk / kTile;
+        return *tiles == 1 || *tiles == 2 || *tiles == 4 || *tiles == 8;
+    }
+    if (chunk < 128 || kTile % chunk != 0) return false;
+    *chunks_per_tile = kTile / chunk;      // 2, 4, 8 or 16: whole warps per chunk
+    return true;
+}
+
 static size_t pipeline_fixed_smem(int W, int chunk)
 {
-    const size_t head = 1024 + (size_t)W * (chunk / 32) * 4 + (size_t)kConsumerWarps * W * 4;
+    const int span = chunk < kTile ? kTile : chunk;
+    const size_t head = 1024 + (size_t)W * (span / 32) * 4 + (size_t)kConsumerWarps * W * 4;
     return (head + 1023) & ~(size_t)1023;
 }
 
@@ -458,21 +509,26 @@ static size_t pipeline_fixed_smem(int W, int chunk)
 int pipeline_stages(const StateView &st, int grad_fmt)
 {
     if (!(grad_fmt & kGradAligned)) return 0;
-    if (st.chunk != kTile && st.chunk != 2 * kTile && st.chunk != 4 * kTile) return 0;
-    if (st.n / st.chunk < 1) return 0;
-    const int tiles = st.chunk / kTile;
+    int tiles, g;
+    if (!unit_shape(st.chunk, &tiles, &g)) return 0;
+    if (st.n / ((long long)tiles * kTile) < 1) return 0;
     const size_t budget = 227 * 1024;
     const size_t fixed = pipeline_fixed_smem(st.W, st.chunk);
-    if (fixed + (size_t)(tiles + 1) * kStageBytes > budget) return 0;
+    // up to four server tiles of a unit stay in the ring over the l1 sum: tiles + 1 stages at least
+    const int least = tiles <= 4 ? tiles + 1 : 4;
+    if (fixed + (size_t)least * kStageBytes > budget) return 0;
     int stages = (int)((budget - fixed) / kStageBytes);
     if (stages > kSyncStages) stages = kSyncStages;
-    return stages >= tiles + 1 ? stages : 0;
+    return stages >= least ? stages : 0;
 }
 
-template <int TILES, bool DO_VAR>
+// Chunks per work unit of the ring kernels (1 for chunks of 2048 coordinates and more).
+int pipeline_chunks_per_unit(const StateView &st) { return st.chunk < kTile ? kTile / st.chunk : 1; }
+
+template <int TILES, int G, bool DO_VAR>
 static cudaError_t launch_pipe(const PipeArgs &a, int grid, size_t smem, cudaStream_t s)
 {
-    auto kern = step_sync_pipelined_kernel<TILES, DO_VAR>;
+    auto kern = step_sync_pipelined_kernel<TILES, G, DO_VAR>;
     static SmemLimitOnce once;   // per instantiation
     const cudaError_t e = once.ensure(kern, 227 * 1024);
     if (e != cudaSuccess) return e;
@@ -480,33 +536,43 @@ static cudaError_t launch_pipe(const PipeArgs &a, int grid, size_t smem, cudaStr
     return cudaGetLastError();
 }
 
-// Runs the full chunks [first_chunk, first_chunk + n_chunks) of a sync step; a ragged last chunk is the caller's.
+// Runs the units [first_unit, first_unit + n_units) of a sync step (a unit is one chunk of 2048 coordinates or
+// more, or the 2048 / chunk smaller chunks of one tile); what is left over is the caller's.
 // *var_fused tells whether the variance update was done here too.
 cudaError_t launch_step_sync_pipelined(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
-                                       float gamma_sum, bool do_var, int grad_fmt, long long first_chunk, long long n_chunks, int stages,
+                                       float gamma_sum, bool do_var, int grad_fmt, long long first_unit, long long n_units, int stages,
                                        int sm_count, ErrorWords error_flag, unsigned long long *sched, unsigned long long wait_limit_ns,
                                        long long test_stop_after_tiles, bool *var_fused, cudaStream_t s)
 {
     PipeArgs a;
     a.st = st; a.g = g; a.c = c; a.gamma = gamma; a.gamma_sum = gamma_sum;
-    a.first_chunk = first_chunk;
-    a.n_full_chunks = n_chunks;
+    a.first_chunk = first_unit;
+    a.n_full_chunks = n_units;
     a.stages = stages;
     a.error_flag = error_flag;
     a.sched = sched;
     a.grad_fmt = grad_fmt;
     a.wait_limit_ns = wait_limit_ns;
     a.test_stop_after_tiles = test_stop_after_tiles;
-    const int grid = (int)(a.n_full_chunks < sm_count ? a.n_full_chunks : sm_count);
+    const int grid = (int)(n_units < sm_count ? n_units : sm_count);
     const size_t smem = pipeline_fixed_smem(st.W, st.chunk) + (size_t)stages * kStageBytes;
-    const int tiles = st.chunk / kTile;
+    int tiles, cpt;
+    if (!unit_shape(st.chunk, &tiles, &cpt)) return cudaErrorInvalidValue;
+    if (tiles == 8) do_var = false;       // eight tiles of binary64 gradient sums have no room in the registers
     *var_fused = do_var;
-    switch (tiles) {
-    case 1: return do_var ? launch_pipe<1, true>(a, grid, smem, s) : launch_pipe<1, false>(a, grid, smem, s);
-    case 2: return do_var ? launch_pipe<2, true>(a, grid, smem, s) : launch_pipe<2, false>(a, grid, smem, s);
-    case 4: return do_var ? launch_pipe<4, true>(a, grid, smem, s) : launch_pipe<4, false>(a, grid, smem, s);
+#define ZOA_PIPE(T, GG) (do_var ? launch_pipe<T, GG, true>(a, grid, smem, s) : launch_pipe<T, GG, false>(a, grid, smem, s))
+    switch (tiles * 100 + cpt) {
+    case 101: return ZOA_PIPE(1, 1);
+    case 201: return ZOA_PIPE(2, 1);
+    case 401: return ZOA_PIPE(4, 1);
+    case 801: return launch_pipe<8, 1, false>(a, grid, smem, s);
+    case 102: return ZOA_PIPE(1, 2);
+    case 104: return ZOA_PIPE(1, 4);
+    case 108: return ZOA_PIPE(1, 8);
+    case 116: return ZOA_PIPE(1, 16);
     default: return cudaErrorInvalidValue;
     }
+#undef ZOA_PIPE
 }
 
 }  // namespace zoa

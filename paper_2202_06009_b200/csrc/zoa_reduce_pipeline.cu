@@ -24,28 +24,6 @@ namespace {
 constexpr int kStoreBufs = 3;                        // tiles of (x, m) staged for the store-issuing warp
 constexpr int kRingThreads = kConsumers + 64;        // consumers + copy-issuing warp + store-issuing warp
 
-// Sum over the consumer warps that share a chunk (WPC consecutive warps), in warp order, in
-// binary64; every thread gets its own chunk's total.  One named barrier per call.
-template <int WPC>
-__device__ __forceinline__ double consumer_group_sum(double v, PipeShared *sh, int &flip)
-{
-    if constexpr (WPC == kConsumerWarps) {
-        return consumer_sum(v, sh, flip);
-    } else {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    const int warp = threadIdx.x >> 5;
-    if ((threadIdx.x & 31) == 0) sh->sums[flip][warp] = v;
-    consumer_barrier();
-    const int first = warp / WPC * WPC;
-    double t = 0.0;
-#pragma unroll
-    for (int w = 0; w < WPC; ++w) t += sh->sums[flip][first + w];
-    flip ^= 1;
-    return t;
-    }
-}
-
 // Shared-memory header of reduce_pipelined_kernel.
 struct ReduceShared {
     PipeShared ring;

@@ -132,6 +132,28 @@ __device__ __forceinline__ double consumer_sum(double v, PipeShared *sh, int &fl
     return t;
 }
 
+// Sum over the consumer warps that share a chunk (WPC consecutive warps), in warp order, in
+// binary64; every thread gets its own chunk's total.  One named barrier per call.
+template <int WPC>
+__device__ __forceinline__ double consumer_group_sum(double v, PipeShared *sh, int &flip)
+{
+    if constexpr (WPC == kConsumerWarps) {
+        return consumer_sum(v, sh, flip);
+    } else {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    const int warp = threadIdx.x >> 5;
+    if ((threadIdx.x & 31) == 0) sh->sums[flip][warp] = v;
+    consumer_barrier();
+    const int first = warp / WPC * WPC;
+    double t = 0.0;
+#pragma unroll
+    for (int w = 0; w < WPC; ++w) t += sh->sums[flip][first + w];
+    flip ^= 1;
+    return t;
+    }
+}
+
 // Packs the sign bits of a float4-per-lane tile: lane l holds coordinates 4l..4l+3,
 // eight lanes make one word.  Returns the word in every lane of the 8-lane group.
 __device__ __forceinline__ uint32_t pack_group(const bool b[4])

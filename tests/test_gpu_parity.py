@@ -80,11 +80,15 @@ def test_fused_equals_two_call_bit_for_bit():
 
 
 @pytest.mark.parametrize("W,chunk,n_chunks,tail", [(5, 4096, 301, 1852), (3, 2048, 700, 0), (4, 8192, 160, 704),
-                                                   (16, 4096, 40, 5), (64, 2048, 20, 33), (33, 8192, 9, 0)])
+                                                   (16, 4096, 40, 5), (64, 2048, 20, 33), (33, 8192, 9, 0),
+                                                   (4, 16384, 150, 9000), (3, 1024, 1400, 1500), (5, 512, 2600, 700),
+                                                   (2, 256, 5000, 300), (7, 128, 9000, 131), (64, 1024, 41, 0)])
 def test_pipelined_kernel_equals_chunk_per_block_kernel(W, chunk, n_chunks, tail):
     """The bulk-copy ring kernel and the chunk-per-block kernel give the same bits,
     over enough chunks that every block wraps its ring many times; steps with and
-    without the fused variance update."""
+    without the fused variance update.  Chunks of 2048 ... 16384 coordinates are units of one
+    to eight tiles; chunks of 128 ... 1024 share a tile, and the whole chunks that do not fill
+    the last tile go to the chunk-per-block kernel with the ragged tail."""
     rng = np.random.default_rng(W + chunk)
     n = n_chunks * chunk + tail
     x0 = torch.from_numpy((rng.standard_normal(n) * 0.02).astype(np.float32))
@@ -107,7 +111,7 @@ def test_pipelined_kernel_equals_chunk_per_block_kernel(W, chunk, n_chunks, tail
                     assert np.array_equal(a.read(name, i), b.read(name, i)), (name, i, t)
             for name in ("v", "delta_s", "x_sync", "words_s", "scales_s"):
                 assert np.array_equal(a.read(name), b.read(name)), (name, t)
-        if chunk <= 4096 and not tail:      # the variance update rides along in the ring kernel
+        if chunk <= 8192 and not tail and n_chunks % max(1, 2048 // chunk) == 0:      # the variance update rides along in the ring kernel
             assert a.stats()["n_launches"] < b.stats()["n_launches"]
     finally:
         a.close(), b.close()
