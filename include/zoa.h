@@ -265,7 +265,12 @@ zoa_status zoa_step_host(zoa_handle h, const void *const *host_grads, float lr, 
                          float *host_x_out, void *stream);
 
 /* Borrowed (device) pointer to one row of a state buffer and its length in
- * elements (n_pad, n_pad/32 or n_chunks).  worker is ignored for shared buffers. */
+ * elements (n_pad, n_pad/32 or n_chunks).  worker is ignored for shared buffers.
+ * With chunks above 16384 the library keeps the two error buffers between syncs
+ * as "what was compressed", the magnitude still to be subtracted; asking for
+ * ZOA_BUF_DELTA_W or ZOA_BUF_DELTA_S (here, in zoa_copy_out / zoa_copy_in and in
+ * zoa_export_state) first brings them to their plain form, which waits for the
+ * device and runs one short kernel. */
 zoa_status zoa_get_buffer(zoa_handle h, zoa_buffer which, int worker, void **dev_ptr,
                           size_t *n_elems);
 

@@ -33,6 +33,9 @@ struct zoa_handle_s {
     unsigned long long *sched = nullptr;   // device [2]: chunk counter of the persistent kernel, finished blocks
     double *partials = nullptr;    // device [W + 1][n_chunks * segments]: per-segment l1 sums, chunk > 16384 only
     bool large_chunk = false;
+    // Large chunks only: the worker-error rows / the server-error row hold what was compressed at the last
+    // sync, the magnitude still to be subtracted (the large-chunk kernels read that form directly).
+    bool dw_pending = false, ds_pending = false;
     int grad_type = 0;             // 0 binary32, 1 binary16, 2 bfloat16: how `grads` buffers are read
     int use_pipeline = 1;          // ring kernels: 0 never, 1 where the shape allows and the problem is large enough, 2 wherever the shape allows
     int wait_limit_ms = 2000;      // bound on every device-side wait
@@ -385,6 +388,21 @@ static void commit_variance(zoa_handle h)
     }
 }
 
+// Brings the error rows of a large-chunk handle to their plain form before anything outside the
+// large-chunk kernels reads or writes them.  Synchronises.
+static cudaError_t plain_errors(zoa_handle h)
+{
+    if (!h->dw_pending && !h->ds_pending) return cudaSuccess;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) e = launch_plain_errors(view(h), h->dw_pending, h->ds_pending, nullptr);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) {
+        h->n_launches += (h->dw_pending ? 1 : 0) + (h->ds_pending ? 1 : 0);
+        h->dw_pending = h->ds_pending = false;
+    }
+    return e;
+}
+
 // Worker side / server side of the 1-bit AllReduce of u, by the kernels that fit the chunk size.
 static cudaError_t run_compress(zoa_handle h, cudaStream_t s)
 {
@@ -392,7 +410,8 @@ static cudaError_t run_compress(zoa_handle h, cudaStream_t s)
     cudaError_t e;
     if (h->large_chunk) {
         GradPtrs none{};
-        e = launch_large_compress(view(h), none, h->c, 0.f, 0, kGradAligned, h->partials, &launches, s);
+        e = launch_large_compress(view(h), none, h->c, 0.f, 0, kGradAligned, h->dw_pending, h->partials, &launches, s);
+        h->dw_pending = true;
     } else {
         e = launch_compress(view(h), 0, h->n_chunks, s);
         launches = 1;
@@ -405,7 +424,8 @@ static cudaError_t run_server(zoa_handle h, float gamma_sum, cudaStream_t s)
     int launches = 0;
     cudaError_t e;
     if (h->large_chunk) {
-        e = launch_large_server(view(h), h->c, 1, gamma_sum, h->partials, &launches, s);
+        e = launch_large_server(view(h), h->c, 1, gamma_sum, h->ds_pending, h->partials, &launches, s);
+        h->ds_pending = true;
     } else {
         const StateView st = view(h);
         long long n_units = 0, first = 0;
@@ -696,7 +716,8 @@ extern "C" zoa_status zoa_step_sync(zoa_handle h, const void *const *grads, floa
         // No single block can hold a chunk: the multi-pass kernels form the half-step buffer on the
         // fly (twice), so m, x, u are written once, by the server pass.
         int launches = 0;
-        ZOA_CUDA(h, launch_large_compress(st, gp, h->c, lr, 2, aligned, h->partials, &launches, s));
+        ZOA_CUDA(h, launch_large_compress(st, gp, h->c, lr, 2, aligned, h->dw_pending, h->partials, &launches, s));
+        h->dw_pending = true;
         h->n_launches += launches;
         ZOA_CUDA(h, run_server(h, gamma_sum, s));
         if (do_var) {
@@ -738,8 +759,10 @@ extern "C" zoa_status zoa_alg2_step(zoa_handle h, const void *const *grads, floa
     if (h->large_chunk && !full) {
         int launches = 0;
         cudaStream_t s = static_cast<cudaStream_t>(stream);
-        ZOA_CUDA(h, launch_large_compress(view(h), gp, h->c, lr, 1, aligned, h->partials, &launches, s));
-        ZOA_CUDA(h, launch_large_server(view(h), h->c, 2, lr, h->partials, &launches, s));
+        ZOA_CUDA(h, launch_large_compress(view(h), gp, h->c, lr, 1, aligned, h->dw_pending, h->partials, &launches, s));
+        h->dw_pending = true;
+        ZOA_CUDA(h, launch_large_server(view(h), h->c, 2, lr, h->ds_pending, h->partials, &launches, s));
+        h->ds_pending = true;
         h->n_launches += launches;
     } else {
         cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -880,6 +903,7 @@ extern "C" zoa_status zoa_get_buffer(zoa_handle h, zoa_buffer which, int worker,
 {
     if (!h) return ZOA_ERR_ARG;
     if (!dev_ptr) return fail(h, ZOA_ERR_ARG, "zoa_get_buffer: dev_ptr is NULL");
+    if (which == ZOA_BUF_DELTA_W || which == ZOA_BUF_DELTA_S) ZOA_CUDA(h, plain_errors(h));
     char *base; size_t elem, len;
     zoa_status rc = locate(h, which, worker, &base, &elem, &len);
     if (rc != ZOA_OK) return rc;
@@ -896,6 +920,7 @@ extern "C" zoa_status zoa_copy_out(zoa_handle h, zoa_buffer which, int worker, s
     if (rc != ZOA_OK) return rc;
     if (!host_dst || offset > len || count > len - offset) return fail(h, ZOA_ERR_ARG, "zoa_copy_out: range outside the row");
     if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, "zoa_copy_out: the handle's device is not the current CUDA device");
+    if (which == ZOA_BUF_DELTA_W || which == ZOA_BUF_DELTA_S) ZOA_CUDA(h, plain_errors(h));
     ZOA_CUDA(h, cudaDeviceSynchronize());
     ZOA_CUDA(h, cudaMemcpy(host_dst, base + offset * elem, count * elem, cudaMemcpyDeviceToHost));
     return ZOA_OK;
@@ -909,6 +934,7 @@ extern "C" zoa_status zoa_copy_in(zoa_handle h, zoa_buffer which, int worker, si
     if (rc != ZOA_OK) return rc;
     if (!host_src || offset > len || count > len - offset) return fail(h, ZOA_ERR_ARG, "zoa_copy_in: range outside the row");
     if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, "zoa_copy_in: the handle's device is not the current CUDA device");
+    if (which == ZOA_BUF_DELTA_W || which == ZOA_BUF_DELTA_S) ZOA_CUDA(h, plain_errors(h));
     ZOA_CUDA(h, cudaDeviceSynchronize());
     ZOA_CUDA(h, cudaMemcpy(base + offset * elem, host_src, count * elem, cudaMemcpyHostToDevice));
     return ZOA_OK;
@@ -980,6 +1006,7 @@ extern "C" zoa_status zoa_export_state(zoa_handle h, void *host_blob, size_t byt
     if (!host_blob) return fail(h, ZOA_ERR_ARG, "zoa_export_state: host_blob is NULL");
     if (bytes < need) return fail(h, ZOA_ERR_ARG, "zoa_export_state: the buffer is smaller than zoa_state_size");
     if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, "zoa_export_state: the handle's device is not the current CUDA device");
+    ZOA_CUDA(h, plain_errors(h));
     ZOA_CUDA(h, cudaDeviceSynchronize());
     BlobHeader hd{};
     std::memcpy(hd.magic, kBlobMagic, 8);
@@ -1053,6 +1080,7 @@ extern "C" zoa_status zoa_import_state(zoa_handle h, const void *host_blob, size
     ZOA_CUDA(h, cudaDeviceSynchronize());
     // From here on the handle changes; a failing copy leaves it undefined (ZOA_ERR_CUDA).
     commit_variance(h);        // v_cur / v_nxt take their plain roles before they are overwritten
+    h->dw_pending = h->ds_pending = false;      // the blob's error rows are plain
     const size_t row_bytes = (size_t)h->n * sizeof(float);
     float *const per_worker[4] = {h->x, h->m, h->u, h->dw};
     for (float *buf : per_worker)
@@ -1113,6 +1141,7 @@ extern "C" zoa_status zoa_check_finite(zoa_handle h, int64_t *n_nonfinite)
 {
     if (!h) return ZOA_ERR_ARG;
     if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, "zoa_check_finite: the handle's device is not the current CUDA device");
+    ZOA_CUDA(h, plain_errors(h));
     ZOA_CUDA(h, cudaDeviceSynchronize());
     ZOA_CUDA(h, cudaMemset(h->sched, 0, 2 * sizeof(unsigned long long)));      // borrowed as the counter; it is 0 between launches
     const long long rows = (long long)h->W * h->n_pad;

@@ -59,9 +59,10 @@ cudaError_t launch_alg2(const StateView &st, const GradPtrs &g, const Consts &c,
 // Chunks larger than kMaxChunk (up to the whole vector): multi-pass kernels, zoa_kernels.cu.
 long long large_chunk_segments(const StateView &st);
 cudaError_t launch_large_compress(const StateView &st, const GradPtrs &g, const Consts &c, float gamma, int src,
-                                  int g_aligned, double *partials, int *launches, cudaStream_t s);
-cudaError_t launch_large_server(const StateView &st, const Consts &c, int mode, float scalar, double *partials,
+                                  int g_aligned, bool pending, double *partials, int *launches, cudaStream_t s);
+cudaError_t launch_large_server(const StateView &st, const Consts &c, int mode, float scalar, bool pending, double *partials,
                                 int *launches, cudaStream_t s);
+cudaError_t launch_plain_errors(const StateView &st, bool workers, bool server, cudaStream_t s);
 
 // Pipelined (bulk-copy ring) form of the fused sync step, zoa_pipeline.cu.
 int pipeline_stages(const StateView &st, int grad_fmt);

@@ -719,10 +719,14 @@ __global__ void __launch_bounds__(512, 2) alg2_compressed_kernel(StateView st, G
 }
 
 // ---------------------------------------------------------------------------
-// Large chunks (chunk > 16384, up to the whole vector = Eq. 3 as printed): a chunk no
-// longer fits one block, so each l1 norm is taken in two steps - one binary64 partial
-// sum per segment of 4096 coordinates, then a fixed-order sum of a chunk's partials -
-// and the values being compressed are recomputed instead of kept.
+// Large chunks (chunk > 16384, up to the whole vector = Eq. 3 as printed): a chunk no longer fits
+// one block, so its l1 norm is taken in two steps - one binary64 partial sum per segment of 4096
+// coordinates, then a fixed-order sum of a chunk's partials.  Two facts keep this at one pass over
+// the data per side: the sign bits do not depend on the magnitude, so they are packed in the same
+// pass that takes the partial sums; and the new error, z - (+-magnitude), can wait - the pass writes
+// z itself into the error row, and whoever reads that row next subtracts the magnitude (still in
+// scales_w / scales_s) on the way in ("pending" form; zoa_api.cu brings a row to its plain form
+// before anything outside these kernels looks at it).
 // ---------------------------------------------------------------------------
 constexpr int kSegment = 4096;
 
@@ -748,15 +752,24 @@ __device__ __forceinline__ SegGeom seg_geom(const StateView &st, long long seg, 
     return g;
 }
 
+// An error row in pending form holds what was compressed; the error proper is that minus its
+// compressed value (Algorithm 3: delta = z - C[z]).
+__device__ __forceinline__ float pending_error(float z, float scale) { return f_sub(z, z >= 0.0f ? scale : -scale); }
+__device__ __forceinline__ float4 plain_error4(float4 e, bool pending, float scale)
+{
+    if (!pending) return e;
+    return make_float4(pending_error(e.x, scale), pending_error(e.y, scale), pending_error(e.z, scale), pending_error(e.w, scale));
+}
+
 // What a worker compresses, four coordinates from j.  SRC 0: u + delta (zoa_onebit_reduce);
 // SRC 1: g + delta (Algorithm 2); SRC 2: the half-step buffer formed on the fly,
 // (u + gamma m_{t+1/2}) + delta with m_{t+1/2} = beta1 m + (1 - beta1) g (fused sync step).
 template <int SRC>
 __device__ __forceinline__ float4 lc_worker_input(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
-                                                  int i, long long j, int g_aligned)
+                                                  int i, long long j, int g_aligned, bool pending, float old_scale)
 {
     const long long row = (long long)i * st.n_pad + j;
-    const float4 e = ld4(st.dw + row);
+    const float4 e = plain_error4(ld4(st.dw + row), pending, old_scale);
     float4 a;
     if (SRC == 0) {
         a = ld4(st.u + row);
@@ -770,22 +783,38 @@ __device__ __forceinline__ float4 lc_worker_input(const StateView &st, const Gra
     return make_float4(f_add(a.x, e.x), f_add(a.y, e.y), f_add(a.z, e.z), f_add(a.w, e.w));
 }
 
-// partials[i][seg] = sum |z| over segment `seg` of worker i = blockIdx.y.
+// Worker side of Algorithm 3, the one pass: z of segment blockIdx.x of worker blockIdx.y goes into
+// the error row (pending form), its sign bits into words_w, sum |z| into partials[i][seg].
 template <int SRC>
 __global__ void __launch_bounds__(512)
-lc_partial_l1_kernel(StateView st, GradPtrs g, Consts c, float gamma, int g_aligned, long long segs_per_chunk,
-                     long long n_segs, double *partials)
+lc_worker_pack_kernel(StateView st, GradPtrs g, Consts c, float gamma, int g_aligned, int pending, long long segs_per_chunk,
+                      long long n_segs, double *partials)
 {
     __shared__ double scratch[34];
     const SegGeom sg = seg_geom(st, blockIdx.x, segs_per_chunk);
     const int i = blockIdx.y;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    const float old_scale = pending ? st.scales_w[(long long)i * st.n_chunks + sg.c] : 0.0f;   // of the previous sync
     double l1 = 0.0;
-    for (int idx = 4 * threadIdx.x; idx < sg.len; idx += 4 * blockDim.x) {
-        const float4 z = lc_worker_input<SRC>(st, g, c, gamma, i, sg.j0 + idx, g_aligned);
-        const float zz[4] = {z.x, z.y, z.z, z.w};
+    for (int base = warp * 128; base < sg.len; base += n_warps * 128) {
+        const int idx = base + 4 * lane;
+        float z[4] = {0.f, 0.f, 0.f, 0.f};
+        if (idx < sg.len) {
+            const float4 z4 = lc_worker_input<SRC>(st, g, c, gamma, i, sg.j0 + idx, g_aligned, pending != 0, old_scale);
+            z[0] = z4.x; z[1] = z4.y; z[2] = z4.z; z[3] = z4.w;
+        }
+        bool b[4];
 #pragma unroll
-        for (int k = 0; k < 4; ++k)
-            if (idx + k < sg.len) l1 += fabs((double)zz[k]);
+        for (int k = 0; k < 4; ++k) {
+            const bool valid = idx + k < sg.len;
+            if (!valid) z[k] = 0.0f;                 // the rows' padding stays zero
+            b[k] = valid && z[k] >= 0.0f;
+            l1 += fabs((double)z[k]);
+        }
+        const uint32_t word = pack_tile(b);
+        if (idx < sg.len) st4(st.dw + (long long)i * st.n_pad + sg.j0 + idx, make_float4(z[0], z[1], z[2], z[3]));
+        if (lane < 4 && base + 32 * lane < sg.len)
+            st.words_w[(long long)i * st.words_stride + ((sg.j0 + base) >> 5) + lane] = word;
     }
     const double total = block_sum(l1, scratch);
     if (threadIdx.x == 0) partials[(long long)i * n_segs + blockIdx.x] = total;
@@ -809,111 +838,91 @@ __global__ void lc_scales_kernel(StateView st, const double *partials, long long
     }
 }
 
-// Worker side of Algorithm 3 once the magnitudes are known: bits, errors.
-template <int SRC>
+// Server side of Algorithm 3, the one pass: a = mean of the compressed buffers + server error goes
+// into the server-error row (pending form), its sign bits into words_s, sum |a| into partials[W][seg].
 __global__ void __launch_bounds__(512)
-lc_compress_apply_kernel(StateView st, GradPtrs g, Consts c, float gamma, int g_aligned, long long segs_per_chunk)
-{
-    const SegGeom sg = seg_geom(st, blockIdx.x, segs_per_chunk);
-    const int i = blockIdx.y;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
-    const float scale = st.scales_w[(long long)i * st.n_chunks + sg.c];
-    for (int base = warp * 128; base < sg.len; base += n_warps * 128) {
-        const int idx = base + 4 * lane;
-        float z[4] = {0.f, 0.f, 0.f, 0.f}, hat[4];
-        if (idx < sg.len) {
-            const float4 z4 = lc_worker_input<SRC>(st, g, c, gamma, i, sg.j0 + idx, g_aligned);
-            z[0] = z4.x; z[1] = z4.y; z[2] = z4.z; z[3] = z4.w;
-        }
-        const uint32_t word = compress_tile(z, hat, scale, idx, sg.len);
-        if (idx < sg.len) st4(st.dw + (long long)i * st.n_pad + sg.j0 + idx, make_float4(z[0], z[1], z[2], z[3]));
-        if (lane < 4 && base + 32 * lane < sg.len)
-            st.words_w[(long long)i * st.words_stride + ((sg.j0 + base) >> 5) + lane] = word;
-    }
-}
-
-// Server input of Algorithm 3 for four coordinates from j, from what the workers sent.
-__device__ __forceinline__ void lc_server_input(const StateView &st, const float *scales_sm, long long j, int valid, float a[4])
-{
-    double A[4] = {0.0, 0.0, 0.0, 0.0};
-    const long long word_idx = j >> 5;
-    const int shift = (int)(j & 31);
-    for (int i = 0; i < st.W; ++i) {   // worker order
-        const uint32_t nib = st.words_w[(long long)i * st.words_stride + word_idx] >> shift;
-        const double s = (double)scales_sm[i];
-#pragma unroll
-        for (int k = 0; k < 4; ++k) A[k] += ((nib >> k) & 1u) ? s : -s;
-    }
-    const float4 e4 = ld4(st.ds + j);
-    const float ee[4] = {e4.x, e4.y, e4.z, e4.w};
-#pragma unroll
-    for (int k = 0; k < 4; ++k) a[k] = k < valid ? server_input(A[k], st.W, ee[k]) : 0.0f;
-}
-
-// partials[W][seg] = sum |mean of the compressed buffers + server error| over the segment.
-__global__ void __launch_bounds__(512)
-lc_server_partial_kernel(StateView st, long long segs_per_chunk, long long n_segs, double *partials)
+lc_server_pack_kernel(StateView st, int pending, long long segs_per_chunk, long long n_segs, double *partials)
 {
     __shared__ double scratch[34];
     __shared__ float scales_sm[kMaxWorkers];
     const SegGeom sg = seg_geom(st, blockIdx.x, segs_per_chunk);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
     for (int i = threadIdx.x; i < st.W; i += blockDim.x) scales_sm[i] = st.scales_w[(long long)i * st.n_chunks + sg.c];
+    const float old_scale = pending ? st.scales_s[sg.c] : 0.0f;       // of the previous sync
     __syncthreads();
     double l1 = 0.0;
-    for (int idx = 4 * threadIdx.x; idx < sg.len; idx += 4 * blockDim.x) {
-        float a[4];
-        lc_server_input(st, scales_sm, sg.j0 + idx, sg.len - idx, a);
-        l1 += fabs((double)a[0]) + fabs((double)a[1]) + fabs((double)a[2]) + fabs((double)a[3]);
+    for (int base = warp * 128; base < sg.len; base += n_warps * 128) {
+        const int idx = base + 4 * lane;
+        float a[4] = {0.f, 0.f, 0.f, 0.f};
+        if (idx < sg.len) {
+            const long long j = sg.j0 + idx;
+            double A[4] = {0.0, 0.0, 0.0, 0.0};
+            const long long word_idx = j >> 5;
+            const int shift = (int)(j & 31);
+            for (int i = 0; i < st.W; ++i) {   // worker order
+                const uint32_t nib = st.words_w[(long long)i * st.words_stride + word_idx] >> shift;
+                const double sc = (double)scales_sm[i];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) A[k] += ((nib >> k) & 1u) ? sc : -sc;
+            }
+            const float4 e4 = plain_error4(ld4(st.ds + j), pending != 0, old_scale);
+            const float ee[4] = {e4.x, e4.y, e4.z, e4.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) a[k] = idx + k < sg.len ? server_input(A[k], st.W, ee[k]) : 0.0f;
+        }
+        bool b[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            b[k] = idx + k < sg.len && a[k] >= 0.0f;
+            l1 += fabs((double)a[k]);
+        }
+        const uint32_t word = pack_tile(b);
+        if (idx < sg.len) st4(st.ds + sg.j0 + idx, make_float4(a[0], a[1], a[2], a[3]));
+        if (lane < 4 && base + 32 * lane < sg.len) st.words_s[((sg.j0 + base) >> 5) + lane] = word;
     }
     const double total = block_sum(l1, scratch);
     if (threadIdx.x == 0) partials[(long long)st.W * n_segs + blockIdx.x] = total;
 }
 
-// Server compression and what follows it.  MODE 1: the post-sync updates of Algorithm 1.
-// MODE 2: momentum and model updates of Algorithm 2, driven by the received gradient.
-template <int MODE>
-__global__ void __launch_bounds__(512)
-lc_server_apply_kernel(StateView st, Consts c, float gamma_or_sum, long long segs_per_chunk)
+// Momentum and model updates of Algorithm 2 from the server's packed result: g_bar = +-scales_s by words_s.
+__global__ void __launch_bounds__(256)
+lc_alg2_apply_kernel(StateView st, Consts c, float gamma)
 {
-    __shared__ float scales_sm[kMaxWorkers];
-    const SegGeom sg = seg_geom(st, blockIdx.x, segs_per_chunk);
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
-    for (int i = threadIdx.x; i < st.W; i += blockDim.x) scales_sm[i] = st.scales_w[(long long)i * st.n_chunks + sg.c];
-    __syncthreads();
-    const float scale = st.scales_s[sg.c];
-    ChunkGeom cg;           // the segment seen as a short chunk, for server_tile
-    cg.c0 = sg.j0;
-    cg.len = sg.len;
-    for (int base = warp * 128; base < sg.len; base += n_warps * 128) {
-        const int idx = base + 4 * lane;
-        float a[4] = {0.f, 0.f, 0.f, 0.f};
-        if (idx < sg.len) lc_server_input(st, scales_sm, sg.j0 + idx, sg.len - idx, a);
-        if (MODE == 1) {
-            server_tile(st, c, cg, base, lane, a, scale, gamma_or_sum);
-        } else {
-            float gb[4];
-            const uint32_t word = compress_tile(a, gb, scale, idx, sg.len);
-            if (lane < 4 && base + 32 * lane < sg.len) st.words_s[((sg.j0 + base) >> 5) + lane] = word;
-            if (idx >= sg.len) continue;
-            const long long j = sg.j0 + idx;
-            st4(st.ds + j, make_float4(a[0], a[1], a[2], a[3]));
-            const float4 v4 = ld4(st.v + j);
-            const float d[4] = {denom(c, v4.x), denom(c, v4.y), denom(c, v4.z), denom(c, v4.w)};
-            for (int i = 0; i < st.W; ++i) {
-                const long long row = (long long)i * st.n_pad + j;
-                const float4 m4 = ld4(st.m + row), x4 = ld4(st.x + row);
-                const float mm[4] = {m4.x, m4.y, m4.z, m4.w}, xx[4] = {x4.x, x4.y, x4.z, x4.w};
-                float mo[4], xo[4];
+    const long long n4 = (st.n + 3) >> 2;
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x; q < n4; q += stride) {
+        const long long j = q << 2;
+        const uint32_t nib = st.words_s[j >> 5] >> (j & 31);
+        const float scale = st.scales_s[j / st.chunk];
+        const float4 v4 = ld4(st.v + j);
+        const float d[4] = {denom(c, v4.x), denom(c, v4.y), denom(c, v4.z), denom(c, v4.w)};
+        for (int i = 0; i < st.W; ++i) {
+            const long long row = (long long)i * st.n_pad + j;
+            const float4 m4 = ld4(st.m + row), x4 = ld4(st.x + row);
+            const float mm[4] = {m4.x, m4.y, m4.z, m4.w}, xx[4] = {x4.x, x4.y, x4.z, x4.w};
+            float mo[4], xo[4];
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    mo[k] = momentum(c, mm[k], gb[k]);
-                    xo[k] = f_sub(xx[k], f_div(f_mul(gamma_or_sum, mo[k]), d[k]));
-                }
-                st4(st.m + row, make_float4(mo[0], mo[1], mo[2], mo[3]));
-                st4(st.x + row, make_float4(xo[0], xo[1], xo[2], xo[3]));
+            for (int k = 0; k < 4; ++k) {
+                const bool valid = j + k < st.n;
+                const float g_bar = ((nib >> k) & 1u) ? scale : -scale;          // what every worker receives
+                mo[k] = valid ? momentum(c, mm[k], g_bar) : 0.0f;                               // update momentum
+                xo[k] = valid ? f_sub(xx[k], f_div(f_mul(gamma, mo[k]), d[k])) : 0.0f;          // update model
             }
+            st4(st.m + row, make_float4(mo[0], mo[1], mo[2], mo[3]));
+            st4(st.x + row, make_float4(xo[0], xo[1], xo[2], xo[3]));
         }
     }
+}
+
+// Brings an error row from pending to plain form: e = z - (+-scale of its chunk), coordinates [0, n).
+__global__ void __launch_bounds__(256)
+lc_plain_errors_kernel(float *rows, long long n, long long n_pad, int chunk, const float *scales, long long n_chunks)
+{
+    float *row = rows + (long long)blockIdx.y * n_pad;
+    const float *row_scales = scales + (long long)blockIdx.y * n_chunks;
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long j = (long long)blockIdx.x * blockDim.x + threadIdx.x; j < n; j += stride)
+        row[j] = pending_error(row[j], row_scales[j / chunk]);
 }
 
 // Debug scan: how many of p[0..count) are NaN or infinite.
@@ -1102,34 +1111,42 @@ long long large_chunk_segments(const StateView &st)
 
 // Worker side of Algorithm 3 for chunks too large for one block.  src 0: compress u + delta;
 // 1: g + delta (Algorithm 2); 2: the half-step buffer formed on the fly from g, m, u (fused sync
-// step; m, x, u are then written by the server pass only).  partials: [W + 1][n_chunks * segments].
+// step; m, x, u are then written by the server pass only).  pending: the worker-error rows are in
+// pending form on entry; they are on return in any case.  partials: [W + 1][n_chunks * segments].
 cudaError_t launch_large_compress(const StateView &st, const GradPtrs &g, const Consts &c, float gamma, int src,
-                                  int g_aligned, double *partials, int *launches, cudaStream_t s)
+                                  int g_aligned, bool pending, double *partials, int *launches, cudaStream_t s)
 {
     const long long spc = large_chunk_segments(st), n_segs = spc * st.n_chunks;
     const dim3 grid((unsigned)n_segs, (unsigned)st.W);
-    if (src == 0) lc_partial_l1_kernel<0><<<grid, 512, 0, s>>>(st, g, c, gamma, g_aligned, spc, n_segs, partials);
-    else if (src == 1) lc_partial_l1_kernel<1><<<grid, 512, 0, s>>>(st, g, c, gamma, g_aligned, spc, n_segs, partials);
-    else lc_partial_l1_kernel<2><<<grid, 512, 0, s>>>(st, g, c, gamma, g_aligned, spc, n_segs, partials);
+    if (src == 0) lc_worker_pack_kernel<0><<<grid, 512, 0, s>>>(st, g, c, gamma, g_aligned, pending, spc, n_segs, partials);
+    else if (src == 1) lc_worker_pack_kernel<1><<<grid, 512, 0, s>>>(st, g, c, gamma, g_aligned, pending, spc, n_segs, partials);
+    else lc_worker_pack_kernel<2><<<grid, 512, 0, s>>>(st, g, c, gamma, g_aligned, pending, spc, n_segs, partials);
     lc_scales_kernel<<<dim3((unsigned)st.n_chunks, (unsigned)st.W), 32, 0, s>>>(st, partials, spc, n_segs, st.scales_w);
-    if (src == 0) lc_compress_apply_kernel<0><<<grid, 512, 0, s>>>(st, g, c, gamma, g_aligned, spc);
-    else if (src == 1) lc_compress_apply_kernel<1><<<grid, 512, 0, s>>>(st, g, c, gamma, g_aligned, spc);
-    else lc_compress_apply_kernel<2><<<grid, 512, 0, s>>>(st, g, c, gamma, g_aligned, spc);
-    *launches += 3;
+    *launches += 2;
     return cudaGetLastError();
 }
 
 // Server side.  mode 1: post-sync updates of Algorithm 1 (scalar = sum of learning rates); mode 2:
-// momentum and model updates of Algorithm 2 (scalar = learning rate).
-cudaError_t launch_large_server(const StateView &st, const Consts &c, int mode, float scalar, double *partials,
+// momentum and model updates of Algorithm 2 (scalar = learning rate).  pending: as above, for the
+// server-error row.
+cudaError_t launch_large_server(const StateView &st, const Consts &c, int mode, float scalar, bool pending, double *partials,
                                 int *launches, cudaStream_t s)
 {
     const long long spc = large_chunk_segments(st), n_segs = spc * st.n_chunks;
-    lc_server_partial_kernel<<<(unsigned)n_segs, 512, 0, s>>>(st, spc, n_segs, partials);
+    lc_server_pack_kernel<<<(unsigned)n_segs, 512, 0, s>>>(st, pending, spc, n_segs, partials);
     lc_scales_kernel<<<dim3((unsigned)st.n_chunks, 1), 32, 0, s>>>(st, partials + (long long)st.W * n_segs, spc, n_segs, st.scales_s);
-    if (mode == 1) lc_server_apply_kernel<1><<<(unsigned)n_segs, 512, 0, s>>>(st, c, scalar, spc);
-    else lc_server_apply_kernel<2><<<(unsigned)n_segs, 512, 0, s>>>(st, c, scalar, spc);
+    if (mode == 1) dist_apply_kernel<<<elementwise_grid((st.n + 3) / 4), 256, 0, s>>>(st, c, scalar);
+    else lc_alg2_apply_kernel<<<elementwise_grid((st.n + 3) / 4), 256, 0, s>>>(st, c, scalar);
     *launches += 3;
+    return cudaGetLastError();
+}
+
+// Error rows from pending to plain form (both kinds, as asked).
+cudaError_t launch_plain_errors(const StateView &st, bool workers, bool server, cudaStream_t s)
+{
+    const unsigned blocks = (unsigned)elementwise_grid((st.n + 3) / 4);
+    if (workers) lc_plain_errors_kernel<<<dim3(blocks, (unsigned)st.W), 256, 0, s>>>(st.dw, st.n, st.n_pad, st.chunk, st.scales_w, st.n_chunks);
+    if (server) lc_plain_errors_kernel<<<dim3(blocks, 1), 256, 0, s>>>(st.ds, st.n, st.n_pad, st.chunk, st.scales_s, st.n_chunks);
     return cudaGetLastError();
 }
 
