@@ -481,10 +481,14 @@ def run_worker_per_gpu(args, wl):
 
 # ---- kernel sweep: worker compression and W-way decompress-average on flat vectors ---------
 def run_sweep(args):
-    """Times zoa_onebit_compress (Algorithm 3, worker side) and zoa_onebit_average (server
-    side + the post-sync updates of Algorithm 1) alone, for n = 2^20 .. 2^30 in powers of 4,
-    W in {2,4,8,16}, chunk in {1024,4096,16384}; inputs N(0,1) with 1 % of the elements
-    scaled by 100.  One JSON line per combination."""
+    """Times the two halves of Algorithm 3 alone on flat vectors, n = 2^20 .. 2^30 in powers of 4,
+    W in {2,4,8,16}, chunk in {1024,4096,16384}; inputs N(0,1) with 1 % of the elements scaled by 100.
+    `compress`: worker side (z, delta in; delta, bits, magnitudes out).  `average_alone`: server side
+    and nothing else (bits, magnitudes, server error in; server error, result, bits out), through a
+    handle that holds only Algorithm 3's state (zoa_create_allreduce), so that 2^30 x 16 fits.
+    `average_sync`: zoa_onebit_average of a full handle, i.e. the server side plus the post-sync
+    rows m, x, u of Algorithm 1 for all W workers (skipped where the full state does not fit).
+    One JSON line per combination."""
     import torch
     from paper_2202_06009_b200 import Zoa, ZoaError, binding as B
 
@@ -492,56 +496,86 @@ def run_sweep(args):
     peak, peak_kind = measured_hbm_peak()
     exps = [20, 22] if args.sweep == "quick" else [20, 22, 24, 26, 28, 30]
     gen = torch.Generator("cuda").manual_seed(5)
+
+    def fill(t):                                   # N(0,1), 1 % of the elements x100, in bounded slices
+        tmp = torch.empty(min(t.numel(), 1 << 26), device="cuda")
+        for lo in range(0, t.numel(), tmp.numel()):
+            part = t[lo:lo + tmp.numel()]
+            part.normal_(generator=gen)
+            u = tmp[:part.numel()].uniform_(generator=gen)
+            part.mul_(torch.where(u < 0.01, 100.0, 1.0))
+
+    def timed(calls, reps):
+        """calls: list of (name, fn); returns {name: [ms per rep]} with events between consecutive calls."""
+        out = {name: [] for name, _ in calls}
+        for _ in range(reps):
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(len(calls) + 1)]
+            ev[0].record()
+            for k, (_, fn) in enumerate(calls):
+                fn()
+                ev[k + 1].record()
+            torch.cuda.synchronize()
+            for k, (name, _) in enumerate(calls):
+                out[name].append(ev[k].elapsed_time(ev[k + 1]))
+        return out
+
     for e in exps:
         n = 1 << e
         for W in (2, 4, 8, 16):
             for chunk in (1024, 4096, 16384):
                 n_chunks = n // chunk
-                row = {"sweep": True, "n": n, "W": W, "chunk": chunk}
-                state_bytes = (4 * W + 4) * n * 4 + (W + 1) * n // 8
-                free, _ = torch.cuda.mem_get_info()
-                if state_bytes > 0.97 * free:
-                    row["skipped"] = f"memory: the handle's state needs {state_bytes / 1e9:.0f} GB"
-                    print(json.dumps(row), flush=True)
-                    continue
-                try:
-                    opt = Zoa(n, W, chunk=chunk)
-                except ZoaError as err:
-                    row["skipped"] = f"memory: {err}"
-                    print(json.dumps(row), flush=True)
-                    continue
-                tmp = torch.empty(min(n, 1 << 26), device="cuda")
-                for i in range(W):                        # u := N(0,1), 1 % of the elements x100
-                    u = opt.device_view("u", i)
-                    for lo in range(0, n, tmp.numel()):
-                        part = u[lo:lo + tmp.numel()]
-                        part.normal_(generator=gen)
-                        t = tmp[:part.numel()].uniform_(generator=gen)
-                        part.mul_(torch.where(t < 0.01, 100.0, 1.0))
-                del tmp
+                row = {"sweep": True, "n": n, "W": W, "chunk": chunk, "peak_kind": peak_kind}
                 bytes_c = n * W * (12 + 1 / 8) + 4 * n_chunks * W
-                bytes_a = n * W * (12 + 1 / 8) + 4 * n_chunks * W + n * (20 + 1 / 8) + 4 * n_chunks
-                times = {"compress": [], "average": []}
-                for rep in range(args.sweep_reps + 1):      # rep 0: errors start at zero; later reps: non-zero errors
-                    B.zoa_set_scalars(opt.h, 1e-3, 0, rep)
-                    e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
-                    e0.record()
-                    opt.onebit_compress()
-                    e1.record()
-                    opt.onebit_average()
-                    e2.record()
-                    torch.cuda.synchronize()
-                    times["compress"].append(e0.elapsed_time(e1))
-                    times["average"].append(e1.elapsed_time(e2))
+                bytes_alone = n * W / 8 + 4 * n_chunks * W + n * (12 + 1 / 8) + 4 * n_chunks
+                bytes_sync = n * W * (12 + 1 / 8) + 4 * n_chunks * W + n * (20 + 1 / 8) + 4 * n_chunks
+                free, _ = torch.cuda.mem_get_info()
+                light_bytes = (2 * W + 2) * n * 4 + (W + 1) * n // 8
+                if light_bytes > 0.97 * free:
+                    row["skipped"] = f"memory: inputs, errors and packed buffers need {light_bytes / 1e9:.0f} GB"
+                    print(json.dumps(row), flush=True)
+                    continue
+                # -- the two halves alone, on a handle that holds only Algorithm 3's state --
+                z = [torch.empty(n, device="cuda") for _ in range(W)]
+                for t in z:
+                    fill(t)
+                z_bar = torch.empty(n, device="cuda")
+                opt = Zoa(n, W, chunk=chunk, allreduce_only=True)
+                t = timed([("compress", lambda: opt.allreduce_compress(z)), ("average_alone", lambda: opt.allreduce_average(z_bar))],
+                          args.sweep_reps + 1)             # rep 0: errors start at zero; later reps: non-zero errors
                 opt.check_device()
                 opt.close()
-                tc0, ta0 = times["compress"][0], times["average"][0]
-                tc, ta = statistics.median(times["compress"][1:]), statistics.median(times["average"][1:])
-                row.update({"compress_ms_zero_errors": tc0, "compress_ms": tc, "compress_GBps": bytes_c / 1e6 / tc,
-                            "average_ms_zero_errors": ta0, "average_ms": ta, "average_GBps": bytes_a / 1e6 / ta,
-                            "both_GBps": (bytes_c + bytes_a) / 1e6 / (tc + ta),
-                            "both_frac_of_peak": (bytes_c + bytes_a) / 1e6 / (tc + ta) / peak, "peak_kind": peak_kind,
-                            "l2_resident": state_bytes < 126e6})
+                del z_bar
+                tc, ta = statistics.median(t["compress"][1:]), statistics.median(t["average_alone"][1:])
+                row.update({"compress_ms_zero_errors": t["compress"][0], "compress_ms": tc, "compress_GBps": bytes_c / 1e6 / tc,
+                            "compress_frac_of_peak": bytes_c / 1e6 / tc / peak,
+                            "average_alone_ms": ta, "average_alone_GBps": bytes_alone / 1e6 / ta,
+                            "average_alone_frac_of_peak": bytes_alone / 1e6 / ta / peak,
+                            "both_GBps": (bytes_c + bytes_alone) / 1e6 / (tc + ta),
+                            "l2_resident": light_bytes < 126e6})
+                # -- the server side with the post-sync rows of Algorithm 1, on a full handle --
+                del z
+                torch.cuda.empty_cache()
+                free, _ = torch.cuda.mem_get_info()
+                full_bytes = (4 * W + 4) * n * 4 + (W + 1) * n // 8
+                if full_bytes > 0.97 * free:
+                    row["average_sync_skipped"] = f"memory: a full handle needs {full_bytes / 1e9:.0f} GB"
+                else:
+                    try:
+                        opt = Zoa(n, W, chunk=chunk)
+                        for i in range(W):
+                            fill(opt.device_view("u", i)[:n])
+                        ts = []
+                        for rep in range(args.sweep_reps + 1):
+                            B.zoa_set_scalars(opt.h, 1e-3, 0, rep)
+                            t = timed([("compress", opt.onebit_compress), ("average_sync", opt.onebit_average)], 1)
+                            ts.append(t["average_sync"][0])
+                        opt.check_device()
+                        opt.close()
+                        tsync = statistics.median(ts[1:])
+                        row.update({"average_sync_ms": tsync, "average_sync_GBps": bytes_sync / 1e6 / tsync,
+                                    "average_sync_frac_of_peak": bytes_sync / 1e6 / tsync / peak})
+                    except ZoaError as err:
+                        row["average_sync_skipped"] = f"memory: {err}"
                 print(json.dumps(row), flush=True)
                 torch.cuda.empty_cache()
 

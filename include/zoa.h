@@ -162,6 +162,24 @@ zoa_status zoa_onebit_reduce(zoa_handle h, void *stream);
 zoa_status zoa_onebit_compress(zoa_handle h, void *stream);
 zoa_status zoa_onebit_average(zoa_handle h, void *stream);
 
+/* Algorithm 3 by itself, z_bar = 1bit-AllReduce(z; delta, delta_bar), on buffers the
+ * caller owns: z is a (host) array of W (device) pointers of n_params floats (read
+ * only, any alignment; 16-byte aligned ones take the vector path), z_bar (device)
+ * receives the n_params floats every worker would get back.  The worker errors, the
+ * server error and the wire buffers are the handle's (ZOA_BUF_DELTA_W, ZOA_BUF_DELTA_S,
+ * ZOA_BUF_WORDS_*, ZOA_BUF_SCALES_*); x, m, u, v are not touched.  Works on any handle
+ * with chunk <= 16384.  zoa_allreduce_compress is the worker side alone (packs z + delta
+ * into words_w / scales_w, keeps the errors), zoa_allreduce_average the server side alone
+ * (reads words_w / scales_w and the server error, writes the server error, words_s /
+ * scales_s and, if z_bar is not NULL, z_bar); compress then average == zoa_onebit_allreduce.
+ * zoa_create_allreduce makes a handle that holds only this state - W + 1 error rows
+ * and the packed buffers, about a fifth of a full handle - on which only these three
+ * calls, buffer access, the checks and zoa_destroy work (the others: ZOA_ERR_STATE). */
+zoa_status zoa_create_allreduce(zoa_handle *out, size_t n_params, int W, int chunk);
+zoa_status zoa_onebit_allreduce(zoa_handle h, const float *const *z, float *z_bar, void *stream);
+zoa_status zoa_allreduce_compress(zoa_handle h, const float *const *z, void *stream);
+zoa_status zoa_allreduce_average(zoa_handle h, float *z_bar, void *stream);
+
 /* Building blocks for the paper's own mapping, one worker per GPU (Algorithm 3:
  * every worker sends its packed buffer to the server, the server sends its
  * packed result to every worker).  Each GPU holds a handle for its own

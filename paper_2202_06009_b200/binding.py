@@ -52,6 +52,10 @@ def _load():
         "zoa_onebit_reduce": ([H, p], C.c_int),
         "zoa_onebit_compress": ([H, p], C.c_int),
         "zoa_onebit_average": ([H, p], C.c_int),
+        "zoa_create_allreduce": ([C.POINTER(H), C.c_size_t, C.c_int, C.c_int], C.c_int),
+        "zoa_onebit_allreduce": ([H, C.POINTER(p), p, p], C.c_int),
+        "zoa_allreduce_compress": ([H, C.POINTER(p), p], C.c_int),
+        "zoa_allreduce_average": ([H, p, p], C.c_int),
         "zoa_dist_server_range": ([H, p, C.c_size_t, p, C.c_size_t, C.c_int, C.c_int64, C.c_int64, p], C.c_int),
         "zoa_dist_apply": ([H, p], C.c_int),
         "zoa_dist_variance": ([H, p, p], C.c_int),
@@ -167,6 +171,24 @@ def zoa_onebit_compress(h, stream=0):
 
 def zoa_onebit_average(h, stream=0):
     _check(h, lib.zoa_onebit_average(h, stream))
+
+
+def zoa_create_allreduce(n_params, W, chunk):
+    h = C.c_void_p()
+    _check(None, lib.zoa_create_allreduce(C.byref(h), n_params, W, chunk))
+    return h
+
+
+def zoa_onebit_allreduce(h, z_ptrs, z_bar_ptr, stream=0):
+    _check(h, lib.zoa_onebit_allreduce(h, _ptr_array(z_ptrs), z_bar_ptr, stream))
+
+
+def zoa_allreduce_compress(h, z_ptrs, stream=0):
+    _check(h, lib.zoa_allreduce_compress(h, _ptr_array(z_ptrs), stream))
+
+
+def zoa_allreduce_average(h, z_bar_ptr, stream=0):
+    _check(h, lib.zoa_allreduce_average(h, z_bar_ptr, stream))
 
 
 def zoa_dist_server_range(h, words_ptr, words_stride, scales_ptr, scales_stride, W_total, first_chunk, n_chunks, stream=0):

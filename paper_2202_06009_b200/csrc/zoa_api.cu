@@ -33,6 +33,7 @@ struct zoa_handle_s {
     unsigned long long *sched = nullptr;   // device [2]: chunk counter of the persistent kernel, finished blocks
     double *partials = nullptr;    // device [W + 1][n_chunks * segments]: per-segment l1 sums, chunk > 16384 only
     bool large_chunk = false;
+    bool allreduce_only = false;   // zoa_create_allreduce: no x, m, u, v, x_sync; only Algorithm 3's own state
     // Large chunks only: the worker-error rows / the server-error row hold what was compressed at the last
     // sync, the magnitude still to be subtracted (the large-chunk kernels read that form directly).
     bool dw_pending = false, ds_pending = false;
@@ -155,8 +156,8 @@ static cudaError_t alloc_zero(zoa_handle h, T **p, size_t count)
     return alloc_guarded(h, reinterpret_cast<void **>(p), count * sizeof(T));
 }
 
-extern "C" zoa_status zoa_create(zoa_handle *out, size_t n_params, int W, float beta1, float beta2,
-                                 float eps, int chunk)
+static zoa_status create_handle(zoa_handle *out, size_t n_params, int W, float beta1, float beta2, float eps, int chunk,
+                                bool allreduce_only)
 {
     if (!out) return fail(nullptr, ZOA_ERR_ARG, "zoa_create: out is NULL");
     *out = nullptr;
@@ -186,10 +187,12 @@ extern "C" zoa_status zoa_create(zoa_handle *out, size_t n_params, int W, float 
     h->c.eps = eps;
 
     const size_t rows = (size_t)W * (size_t)h->n_pad, row = (size_t)h->n_pad;
-    if ((e = alloc_zero(h, &h->x, rows)) == cudaSuccess && (e = alloc_zero(h, &h->m, rows)) == cudaSuccess &&
-        (e = alloc_zero(h, &h->u, rows)) == cudaSuccess && (e = alloc_zero(h, &h->dw, rows)) == cudaSuccess &&
-        (e = alloc_zero(h, &h->v_cur, row)) == cudaSuccess && (e = alloc_zero(h, &h->v_nxt, row)) == cudaSuccess &&
-        (e = alloc_zero(h, &h->ds, row)) == cudaSuccess && (e = alloc_zero(h, &h->xs, row)) == cudaSuccess &&
+    h->allreduce_only = allreduce_only;
+    const size_t full_rows = allreduce_only ? 0 : rows, full_row = allreduce_only ? 0 : row;   // what Algorithm 1 adds to Algorithm 3
+    if ((e = alloc_zero(h, &h->x, full_rows)) == cudaSuccess && (e = alloc_zero(h, &h->m, full_rows)) == cudaSuccess &&
+        (e = alloc_zero(h, &h->u, full_rows)) == cudaSuccess && (e = alloc_zero(h, &h->dw, rows)) == cudaSuccess &&
+        (e = alloc_zero(h, &h->v_cur, full_row)) == cudaSuccess && (e = alloc_zero(h, &h->v_nxt, full_row)) == cudaSuccess &&
+        (e = alloc_zero(h, &h->ds, row)) == cudaSuccess && (e = alloc_zero(h, &h->xs, full_row)) == cudaSuccess &&
         (e = alloc_zero(h, &h->words_w, (size_t)W * h->words_stride)) == cudaSuccess &&
         (e = alloc_zero(h, &h->words_s, (size_t)h->words_stride)) == cudaSuccess &&
         (e = alloc_zero(h, &h->scales_w, (size_t)W * h->n_chunks)) == cudaSuccess &&
@@ -217,6 +220,26 @@ extern "C" zoa_status zoa_create(zoa_handle *out, size_t n_params, int W, float 
     return ZOA_OK;
 }
 
+extern "C" zoa_status zoa_create(zoa_handle *out, size_t n_params, int W, float beta1, float beta2,
+                                 float eps, int chunk)
+{
+    return create_handle(out, n_params, W, beta1, beta2, eps, chunk, false);
+}
+
+extern "C" zoa_status zoa_create_allreduce(zoa_handle *out, size_t n, int W, int chunk)
+{
+    if (chunk > kMaxChunk) return fail(nullptr, ZOA_ERR_ARG, "zoa_create_allreduce: chunk must be at most 16384");
+    return create_handle(out, n, W, 0.f, 0.f, 1.f, chunk, true);
+}
+
+// Entry points of Algorithm 1 / Algorithm 2 need the full state.
+#define ZOA_NEEDS_FULL_STATE(h, who)                                                                                    \
+    do {                                                                                                                \
+        if ((h)->allreduce_only)                                                                                        \
+            return fail(h, ZOA_ERR_STATE, std::string(who) + ": the handle was made by zoa_create_allreduce and holds "  \
+                                                             "only the state of Algorithm 3");                           \
+    } while (0)
+
 extern "C" zoa_status zoa_destroy(zoa_handle h)
 {
     if (!h) return ZOA_ERR_ARG;
@@ -233,6 +256,7 @@ extern "C" zoa_status zoa_destroy(zoa_handle h)
 extern "C" zoa_status zoa_set_params(zoa_handle h, const float *x0, void *stream)
 {
     if (!h) return ZOA_ERR_ARG;
+    ZOA_NEEDS_FULL_STATE(h, "zoa_set_params");
     if (!x0) return fail(h, ZOA_ERR_ARG, "zoa_set_params: x0 is NULL");
     if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, "zoa_set_params: the handle's device is not the current CUDA device");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -358,6 +382,7 @@ static zoa_status check_step_args(zoa_handle h, const void *const *grads, float 
 {
     if (!h) return ZOA_ERR_ARG;
     ZOA_REFUSE_AFTER_DEVICE_ERROR(h, who);
+    ZOA_NEEDS_FULL_STATE(h, who);
     if (!grads) return fail(h, ZOA_ERR_ARG, std::string(who) + ": grads is NULL");
     if (!std::isfinite(lr)) return fail(h, ZOA_ERR_ARG, std::string(who) + ": lr is not finite");
     if (t < 0) return fail(h, ZOA_ERR_ARG, std::string(who) + ": t is negative");
@@ -519,6 +544,7 @@ extern "C" zoa_status zoa_onebit_reduce(zoa_handle h, void *stream)
     TraceRange trace("zoa_onebit_reduce");
     if (!h) return ZOA_ERR_ARG;
     ZOA_REFUSE_AFTER_DEVICE_ERROR(h, "zoa_onebit_reduce");
+    ZOA_NEEDS_FULL_STATE(h, "zoa_onebit_reduce");
     const float gamma_sum = (float)h->gamma_sum;
     if (!(h->gamma_sum > 0.0) || !(gamma_sum > 0.f) || !std::isfinite(gamma_sum))
         return fail(h, ZOA_ERR_STATE, "zoa_onebit_reduce: nothing accumulated since the last sync (sum of learning rates is not positive)");
@@ -536,6 +562,7 @@ extern "C" zoa_status zoa_onebit_compress(zoa_handle h, void *stream)
 {
     if (!h) return ZOA_ERR_ARG;
     ZOA_REFUSE_AFTER_DEVICE_ERROR(h, "zoa_onebit_compress");
+    ZOA_NEEDS_FULL_STATE(h, "zoa_onebit_compress");
     if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, "zoa_onebit_compress: the handle's device is not the current CUDA device");
     ZOA_CUDA(h, run_compress(h, static_cast<cudaStream_t>(stream)));
     return ZOA_OK;
@@ -548,12 +575,68 @@ extern "C" zoa_status zoa_onebit_average(zoa_handle h, void *stream)
     if (!(h->gamma_sum > 0.0) || !(gamma_sum > 0.f) || !std::isfinite(gamma_sum))
         return fail(h, ZOA_ERR_STATE, "zoa_onebit_average: nothing accumulated since the last sync (sum of learning rates is not positive)");
     ZOA_REFUSE_AFTER_DEVICE_ERROR(h, "zoa_onebit_average");
+    ZOA_NEEDS_FULL_STATE(h, "zoa_onebit_average");
     if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, "zoa_onebit_average: the handle's device is not the current CUDA device");
     ZOA_CUDA(h, run_server(h, gamma_sum, static_cast<cudaStream_t>(stream)));
     h->gamma_sum = 0.0;
     h->t_sync = h->t_last;
     h->n_syncs += 1;
     return ZOA_OK;
+}
+
+// ---- Algorithm 3 on caller-owned buffers, with the handle's errors and wire buffers ---------------
+
+static zoa_status allreduce_compress(zoa_handle h, const float *const *z, cudaStream_t s, const char *who)
+{
+    ZOA_REFUSE_AFTER_DEVICE_ERROR(h, who);
+    if (h->large_chunk) return fail(h, ZOA_ERR_ARG, std::string(who) + ": chunk must be at most 16384");
+    if (!z) return fail(h, ZOA_ERR_ARG, std::string(who) + ": z is NULL");
+    if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, std::string(who) + ": the handle's device is not the current CUDA device");
+    GradPtrs zp{};
+    bool aligned = true;
+    for (int i = 0; i < h->W; ++i) {
+        if (!z[i]) return fail(h, ZOA_ERR_ARG, std::string(who) + ": a buffer pointer is NULL");
+        zp.p[i] = z[i];
+        if (reinterpret_cast<uintptr_t>(z[i]) & 15u) aligned = false;
+    }
+    ZOA_CUDA(h, launch_compress_external(view(h), zp, aligned ? kGradAligned : 0, s));
+    h->n_launches += 1;
+    return ZOA_OK;
+}
+
+static zoa_status allreduce_average(zoa_handle h, float *z_bar, cudaStream_t s, const char *who)
+{
+    ZOA_REFUSE_AFTER_DEVICE_ERROR(h, who);
+    if (h->large_chunk) return fail(h, ZOA_ERR_ARG, std::string(who) + ": chunk must be at most 16384");
+    if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, std::string(who) + ": the handle's device is not the current CUDA device");
+    PeerOut none{};
+    ZOA_CUDA(h, launch_dist_server(view(h), h->words_w, h->words_stride, h->scales_w, h->n_chunks, h->W, 0, h->n_chunks, none, z_bar, s));
+    h->n_launches += 1;
+    return ZOA_OK;
+}
+
+extern "C" zoa_status zoa_allreduce_compress(zoa_handle h, const float *const *z, void *stream)
+{
+    if (!h) return ZOA_ERR_ARG;
+    return allreduce_compress(h, z, static_cast<cudaStream_t>(stream), "zoa_allreduce_compress");
+}
+
+extern "C" zoa_status zoa_allreduce_average(zoa_handle h, float *z_bar, void *stream)
+{
+    if (!h) return ZOA_ERR_ARG;
+    return allreduce_average(h, z_bar, static_cast<cudaStream_t>(stream), "zoa_allreduce_average");
+}
+
+extern "C" zoa_status zoa_onebit_allreduce(zoa_handle h, const float *const *z, float *z_bar, void *stream)
+{
+    TraceRange trace("zoa_onebit_allreduce");
+    if (!h) return ZOA_ERR_ARG;
+    if (!z_bar) return fail(h, ZOA_ERR_ARG, "zoa_onebit_allreduce: z_bar is NULL");
+    zoa_status rc = allreduce_compress(h, z, static_cast<cudaStream_t>(stream), "zoa_onebit_allreduce");
+    if (rc != ZOA_OK) return rc;
+    rc = allreduce_average(h, z_bar, static_cast<cudaStream_t>(stream), "zoa_onebit_allreduce");
+    if (rc == ZOA_OK) h->n_syncs += 1;
+    return rc;
 }
 
 // ---- one worker per GPU: the pieces between the collectives ------------------------------------
@@ -572,7 +655,7 @@ extern "C" zoa_status zoa_dist_server_range(zoa_handle h, const uint32_t *words_
     if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, "zoa_dist_server_range: the handle's device is not the current CUDA device");
     PeerOut none{};
     ZOA_CUDA(h, launch_dist_server(view(h), words_all, (long long)words_stride, scales_all, (long long)scales_stride,
-                                   W_total, first_chunk, n_chunks, none, static_cast<cudaStream_t>(stream)));
+                                   W_total, first_chunk, n_chunks, none, nullptr, static_cast<cudaStream_t>(stream)));
     h->n_launches += 1;
     return ZOA_OK;
 }
@@ -600,7 +683,7 @@ extern "C" zoa_status zoa_dist_server_push(zoa_handle h, const uint32_t *words_a
     if (!words_all || !scales_all) return fail(h, ZOA_ERR_ARG, "zoa_dist_server_push: NULL buffer");
     if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, "zoa_dist_server_push: the handle's device is not the current CUDA device");
     ZOA_CUDA(h, launch_dist_server(view(h), words_all, (long long)words_stride, scales_all, (long long)scales_stride,
-                                   W_total, first_chunk, n_chunks, out, static_cast<cudaStream_t>(stream)));
+                                   W_total, first_chunk, n_chunks, out, nullptr, static_cast<cudaStream_t>(stream)));
     h->n_launches += 1;
     return ZOA_OK;
 }
@@ -610,6 +693,7 @@ extern "C" zoa_status zoa_dist_server_push(zoa_handle h, const uint32_t *words_a
 static zoa_status make_push_plan(zoa_handle h, int world, const int64_t *chunk_begin, void *const *peer_words,
                                  void *const *peer_scales, PushPlan *plan, const char *who)
 {
+    ZOA_NEEDS_FULL_STATE(h, who);
     if (h->W != 1) return fail(h, ZOA_ERR_ARG, std::string(who) + ": the handle must hold exactly one worker");
     if (h->large_chunk) return fail(h, ZOA_ERR_ARG, std::string(who) + ": chunk must be at most 16384");
     if (world < 1 || world > kMaxWorkers) return fail(h, ZOA_ERR_ARG, std::string(who) + ": world must be in [1, 64]");
@@ -672,6 +756,7 @@ extern "C" zoa_status zoa_dist_step_pack_push(zoa_handle h, const void *grad, fl
 extern "C" zoa_status zoa_dist_apply(zoa_handle h, void *stream)
 {
     if (!h) return ZOA_ERR_ARG;
+    ZOA_NEEDS_FULL_STATE(h, "zoa_dist_apply");
     const float gamma_sum = (float)h->gamma_sum;
     if (!(h->gamma_sum > 0.0) || !(gamma_sum > 0.f) || !std::isfinite(gamma_sum))
         return fail(h, ZOA_ERR_STATE, "zoa_dist_apply: nothing accumulated since the last sync (sum of learning rates is not positive)");
@@ -687,6 +772,7 @@ extern "C" zoa_status zoa_dist_apply(zoa_handle h, void *stream)
 extern "C" zoa_status zoa_dist_variance(zoa_handle h, const float *g_bar, void *stream)
 {
     if (!h) return ZOA_ERR_ARG;
+    ZOA_NEEDS_FULL_STATE(h, "zoa_dist_variance");
     if (!g_bar) return fail(h, ZOA_ERR_ARG, "zoa_dist_variance: g_bar is NULL");
     if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, "zoa_dist_variance: the handle's device is not the current CUDA device");
     if (h->v_pending) return fail(h, ZOA_ERR_STATE, "zoa_dist_variance: a variance update is already pending for this step");
@@ -880,6 +966,8 @@ static zoa_status locate(zoa_handle h, zoa_buffer which, int worker, char **base
     const bool per_worker = which == ZOA_BUF_X || which == ZOA_BUF_M || which == ZOA_BUF_U ||
                             which == ZOA_BUF_DELTA_W || which == ZOA_BUF_WORDS_W || which == ZOA_BUF_SCALES_W;
     if (per_worker && (worker < 0 || worker >= h->W)) return fail(h, ZOA_ERR_ARG, "worker index out of range");
+    if (h->allreduce_only && (which == ZOA_BUF_X || which == ZOA_BUF_M || which == ZOA_BUF_U || which == ZOA_BUF_V || which == ZOA_BUF_X_SYNC))
+        return fail(h, ZOA_ERR_ARG, "the handle was made by zoa_create_allreduce and has no such buffer");
     const size_t i = per_worker ? (size_t)worker : 0;
     *elem = 4;
     switch (which) {
@@ -1001,6 +1089,7 @@ extern "C" zoa_status zoa_state_size(zoa_handle h, size_t *bytes)
 extern "C" zoa_status zoa_export_state(zoa_handle h, void *host_blob, size_t bytes)
 {
     if (!h) return ZOA_ERR_ARG;
+    ZOA_NEEDS_FULL_STATE(h, "zoa_export_state");
     size_t need = 0;
     zoa_state_size(h, &need);
     if (!host_blob) return fail(h, ZOA_ERR_ARG, "zoa_export_state: host_blob is NULL");
@@ -1047,6 +1136,7 @@ extern "C" zoa_status zoa_export_state(zoa_handle h, void *host_blob, size_t byt
 extern "C" zoa_status zoa_import_state(zoa_handle h, const void *host_blob, size_t bytes)
 {
     if (!h) return ZOA_ERR_ARG;
+    ZOA_NEEDS_FULL_STATE(h, "zoa_import_state");
     if (!host_blob) return fail(h, ZOA_ERR_ARG, "zoa_import_state: host_blob is NULL");
     if (bytes < sizeof(BlobHeader)) return fail(h, ZOA_ERR_ARG, "zoa_import_state: the blob is shorter than its header");
     BlobHeader hd;
@@ -1147,7 +1237,9 @@ extern "C" zoa_status zoa_check_finite(zoa_handle h, int64_t *n_nonfinite)
     const long long rows = (long long)h->W * h->n_pad;
     const float *bufs[] = {h->x, h->m, h->u, h->dw, h->v_pending ? h->v_nxt : h->v_cur, h->ds, h->xs};
     const long long counts[] = {rows, rows, rows, rows, h->n_pad, h->n_pad, h->n_pad};
-    for (int k = 0; k < 7; ++k) ZOA_CUDA(h, launch_count_nonfinite(bufs[k], counts[k], h->sched, h->sm_count, nullptr));
+    for (int k = 0; k < 7; ++k)
+        if (!h->allreduce_only || bufs[k] == h->dw || bufs[k] == h->ds)
+            ZOA_CUDA(h, launch_count_nonfinite(bufs[k], counts[k], h->sched, h->sm_count, nullptr));
     unsigned long long bad = 0;
     ZOA_CUDA(h, cudaMemcpy(&bad, h->sched, sizeof(bad), cudaMemcpyDeviceToHost));
     ZOA_CUDA(h, cudaMemset(h->sched, 0, 2 * sizeof(unsigned long long)));

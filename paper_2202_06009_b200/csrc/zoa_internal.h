@@ -76,7 +76,8 @@ cudaError_t launch_step_sync_pipelined(const StateView &st, const GradPtrs &g, c
 // One worker per GPU: the kernels between the collectives.
 cudaError_t launch_dist_server(const StateView &st, const uint32_t *words_in, long long words_in_stride,
                                const float *scales_in, long long scales_in_stride, int W_total,
-                               long long first_chunk, long long count, const PeerOut &out, cudaStream_t s);
+                               long long first_chunk, long long count, const PeerOut &out, float *z_bar, cudaStream_t s);
+cudaError_t launch_compress_external(const StateView &st, const GradPtrs &z, int z_fmt, cudaStream_t s);
 cudaError_t launch_dist_pack_push(const StateView &st, const float *g, const Consts &c, float gamma, int g_fmt,
                                   const PushPlan &plan, cudaStream_t s);
 cudaError_t launch_dist_apply(const StateView &st, const Consts &c, float gamma_sum, cudaStream_t s);

@@ -166,8 +166,10 @@ __device__ __forceinline__ BlockSpan block_span(const StateView &st, const Chunk
 // thread, which is what fills the memory pipeline (measured at n = 2^28, W = 16: chunk 4096
 // 6.94 TB/s against 6.74 with the chunk staged in shared memory by a loop of dependent
 // iterations; chunk 16384 6.54 against 5.62).
-template <int ITER>
-__global__ void __launch_bounds__(512, 2) compress_kernel(StateView st, long long first_chunk)
+// EXTERNAL: what is compressed is z + delta with z read from caller-owned buffers (Algorithm 3 on an
+// arbitrary input, zoa_onebit_allreduce) instead of u + delta.
+template <int ITER, bool EXTERNAL>
+__global__ void __launch_bounds__(512, 2) compress_kernel(StateView st, long long first_chunk, GradPtrs z_in, int z_fmt)
 {
     __shared__ double scratch[34];
     const long long chunk_id = first_chunk + blockIdx.x;
@@ -180,7 +182,8 @@ __global__ void __launch_bounds__(512, 2) compress_kernel(StateView st, long lon
     for (int it = 0; it < ITER; ++it) {
         const int idx = 4 * (it * blockDim.x + threadIdx.x);
         const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
-        u4[it] = idx < cg.len ? ld4_stream(st.u + row + idx) : zero;     // whole float4 groups: the rows' padding is zero
+        if (EXTERNAL) u4[it] = idx < cg.len ? ld_grad4(z_in.p[i], cg.c0 + idx, st.n, z_fmt) : zero;
+        else u4[it] = idx < cg.len ? ld4_stream(st.u + row + idx) : zero;     // whole float4 groups: the rows' padding is zero
         e4[it] = idx < cg.len ? ld4_stream(st.dw + row + idx) : zero;
     }
     float z[ITER][4];
@@ -401,7 +404,7 @@ __global__ void step_sync_kernel(StateView st, GradPtrs g, Consts c, float gamma
 // words_s / scales_s, peer pointers included); out.world == 0 for none.
 __global__ void __launch_bounds__(512, 3) dist_server_kernel(StateView st, const uint32_t *words_in, long long words_in_stride,
                                    const float *scales_in, long long scales_in_stride, int W_total,
-                                   long long first_chunk, PeerOut out)
+                                   long long first_chunk, PeerOut out, float *z_bar)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     double *scratch = reinterpret_cast<double *>(smem_raw);
@@ -453,6 +456,11 @@ __global__ void __launch_bounds__(512, 3) dist_server_kernel(StateView st, const
             for (int r = 0; r < out.world; ++r) out.words_s[r][w] = word;
         }
         if (idx < cg.len) st4(st.ds + cg.c0 + idx, make_float4(a[0], a[1], a[2], a[3]));
+        if (z_bar) {             // the result of Algorithm 3 in full: caller-owned, exactly n floats, any alignment
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                if (idx + k < cg.len) z_bar[cg.c0 + idx + k] = hat[k];
+        }
     }
     if (threadIdx.x == 0) {
         st.scales_s[chunk_id] = scale;
@@ -1062,8 +1070,20 @@ cudaError_t launch_compress(const StateView &st, long long first_chunk, long lon
     const int iter = st.chunk > 4096 ? 8 : 4;
     const int thr = ((st.chunk + 4 * iter - 1) / (4 * iter) + 31) / 32 * 32;
     const dim3 grid((unsigned)count, (unsigned)st.W);
-    if (iter == 8) compress_kernel<8><<<grid, thr, 0, s>>>(st, first_chunk);
-    else compress_kernel<4><<<grid, thr, 0, s>>>(st, first_chunk);
+    const GradPtrs none{};
+    if (iter == 8) compress_kernel<8, false><<<grid, thr, 0, s>>>(st, first_chunk, none, 0);
+    else compress_kernel<4, false><<<grid, thr, 0, s>>>(st, first_chunk, none, 0);
+    return cudaGetLastError();
+}
+
+// The same for Algorithm 3 on caller-owned buffers z (W device pointers of n floats, format code as for gradients).
+cudaError_t launch_compress_external(const StateView &st, const GradPtrs &z, int z_fmt, cudaStream_t s)
+{
+    const int iter = st.chunk > 4096 ? 8 : 4;
+    const int thr = ((st.chunk + 4 * iter - 1) / (4 * iter) + 31) / 32 * 32;
+    const dim3 grid((unsigned)st.n_chunks, (unsigned)st.W);
+    if (iter == 8) compress_kernel<8, true><<<grid, thr, 0, s>>>(st, 0, z, z_fmt);
+    else compress_kernel<4, true><<<grid, thr, 0, s>>>(st, 0, z, z_fmt);
     return cudaGetLastError();
 }
 
@@ -1156,7 +1176,7 @@ namespace zoa {
 
 cudaError_t launch_dist_server(const StateView &st, const uint32_t *words_in, long long words_in_stride,
                                const float *scales_in, long long scales_in_stride, int W_total,
-                               long long first_chunk, long long count, const PeerOut &out, cudaStream_t s)
+                               long long first_chunk, long long count, const PeerOut &out, float *z_bar, cudaStream_t s)
 {
     static SmemLimitOnce once;
     const cudaError_t e = once.ensure(dist_server_kernel, (int)reduce_smem(kMaxChunk));
@@ -1166,7 +1186,7 @@ cudaError_t launch_dist_server(const StateView &st, const uint32_t *words_in, lo
     int thr = 128;
     while (thr < st.chunk / per_thread && thr < 512) thr <<= 1;
     dist_server_kernel<<<(unsigned)count, thr, reduce_smem(st.chunk), s>>>(
-        st, words_in, words_in_stride, scales_in, scales_in_stride, W_total, first_chunk, out);
+        st, words_in, words_in_stride, scales_in, scales_in_stride, W_total, first_chunk, out, z_bar);
     return cudaGetLastError();
 }
 

@@ -33,10 +33,15 @@ def _grad_ptrs(grads, n, W, dtype=torch.float32):
 
 
 class Zoa:
-    def __init__(self, n_params, W, beta1=0.9, beta2=0.999, eps=1e-8, chunk=4096):
+    def __init__(self, n_params, W, beta1=0.9, beta2=0.999, eps=1e-8, chunk=4096, allreduce_only=False):
+        """allreduce_only: a handle that holds only Algorithm 3's state (zoa_create_allreduce); only
+        onebit_allreduce / allreduce_compress / allreduce_average, reads and the checks work on it."""
         self.n, self.W, self.chunk = int(n_params), int(W), int(chunk)
         self.n_chunks = (self.n + self.chunk - 1) // self.chunk
-        self.h = B.zoa_create(self.n, self.W, beta1, beta2, eps, self.chunk)
+        if allreduce_only:
+            self.h = B.zoa_create_allreduce(self.n, self.W, self.chunk)
+        else:
+            self.h = B.zoa_create(self.n, self.W, beta1, beta2, eps, self.chunk)
         self.grad_dtype = torch.float32
 
     def close(self):
@@ -95,6 +100,17 @@ class Zoa:
 
     def onebit_average(self):
         B.zoa_onebit_average(self.h, _stream())
+
+    # -- Algorithm 3 on caller-owned buffers ------------------------------------
+    def onebit_allreduce(self, z, z_bar):
+        """z: W float32 CUDA tensors of n elements (read only), z_bar: float32 CUDA tensor of n elements."""
+        B.zoa_onebit_allreduce(self.h, [t.data_ptr() for t in z], z_bar.data_ptr(), _stream())
+
+    def allreduce_compress(self, z):
+        B.zoa_allreduce_compress(self.h, [t.data_ptr() for t in z], _stream())
+
+    def allreduce_average(self, z_bar=None):
+        B.zoa_allreduce_average(self.h, z_bar.data_ptr() if z_bar is not None else None, _stream())
 
     def device_view(self, name, worker=0):
         """The state row as a torch tensor that aliases the library's memory (no copy)."""

@@ -6,6 +6,7 @@ import pytest
 import torch
 
 from helpers import ATOL, RTOL, Pair, assert_close
+from oracle import zoa_oracle as zo
 from paper_2202_06009_b200 import Zoa, ZoaError, binding as B, synth
 
 pytestmark = pytest.mark.gpu
@@ -270,6 +271,51 @@ def test_unaligned_gradient_pointers():
             p.compare(f"t={t}", wire=False)
     finally:
         p.close()
+
+
+@pytest.mark.parametrize("light", [True, False])
+@pytest.mark.parametrize("n,W,chunk,offset", [(3 * 1024 + 77, 4, 1024, 0), (5000, 3, 256, 0), (4096 + 9, 2, 4096, 1),
+                                              (2 * 16384 + 100, 5, 16384, 0), (40, 1, 32, 3), (7 * 8192, 64, 8192, 0)])
+def test_onebit_allreduce_on_caller_buffers(n, W, chunk, offset, light):
+    """zoa_onebit_allreduce (Algorithm 3 by itself) against the oracle's zo_onebit_allreduce over three
+    rounds, so that non-zero worker and server errors enter; on a handle that holds only Algorithm 3's
+    state and on a full one; `offset` shifts the caller's buffers off 16-byte alignment."""
+    rng = np.random.default_rng(n + W)
+    cpu = zo.Oracle(n, W, chunk, dtype=np.float32)
+    gpu = Zoa(n, W, chunk=chunk, allreduce_only=light)
+    try:
+        for r in range(3):
+            z = (rng.standard_normal((W, n)) * 10.0 ** rng.integers(-2, 2)).astype(np.float32)
+            z[rng.random((W, n)) < 0.01] *= np.float32(100.0)
+            z_dev = [torch.zeros(n + offset, device="cuda")[offset:].copy_(torch.from_numpy(z[i])) for i in range(W)]
+            z_bar = torch.full((n + offset + 8,), 7.0, device="cuda")[offset:offset + n]
+            if r == 1:          # the two halves separately
+                gpu.allreduce_compress(z_dev)
+                gpu.allreduce_average(z_bar)
+            else:
+                gpu.onebit_allreduce(z_dev, z_bar)
+            torch.cuda.synchronize()
+            want = cpu.onebit_allreduce(z)
+            assert_close(z_bar.cpu().numpy(), want, f"z_bar, round {r}")
+            assert np.array_equal(gpu.read("words_s"), cpu.words_server), f"words_s, round {r}"
+            assert_close(gpu.read("scales_s"), cpu.scales_server, f"scales_s, round {r}")
+            assert_close(gpu.read("delta_s"), cpu.delta_bar, f"delta_s, round {r}")
+            for i in range(W):
+                assert np.array_equal(gpu.read("words_w", i), cpu.words_worker[i]), f"words_w[{i}], round {r}"
+                assert_close(gpu.read("scales_w", i), cpu.scales_worker[i], f"scales_w[{i}], round {r}")
+                assert_close(gpu.read("delta_w", i), cpu.delta[i], f"delta_w[{i}], round {r}")
+                assert np.array_equal(z_dev[i].cpu().numpy(), z[i]), "the input was written"
+        gpu.check_device()
+        if light:
+            g = list(torch.zeros(W, n, device="cuda"))
+            for call in (lambda: gpu.step(g, 1e-3, 0), lambda: gpu.step_sync(g, 1e-3, 0), lambda: gpu.alg2_step(g, 1e-3, 0),
+                         gpu.onebit_reduce, gpu.export_state, lambda: gpu.read("x")):
+                with pytest.raises(ZoaError) as e:
+                    call()
+                assert e.value.status in (B.ERR_STATE, B.ERR_ARG)
+            assert B.zoa_check_finite(gpu.h) == 0
+    finally:
+        gpu.close()
 
 
 @pytest.mark.parametrize("where", ["pending_variance", "after_sync", "mid_interval"])
