@@ -609,6 +609,8 @@ static zoa_status allreduce_average(zoa_handle h, float *z_bar, cudaStream_t s, 
     ZOA_REFUSE_AFTER_DEVICE_ERROR(h, who);
     if (h->large_chunk) return fail(h, ZOA_ERR_ARG, std::string(who) + ": chunk must be at most 16384");
     if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, std::string(who) + ": the handle's device is not the current CUDA device");
+    // One block per chunk: the server side alone moves so little per chunk (12 bytes and W bits per coordinate)
+    // that many resident blocks hide its latencies better than one persistent block per SM does.
     PeerOut none{};
     ZOA_CUDA(h, launch_dist_server(view(h), h->words_w, h->words_stride, h->scales_w, h->n_chunks, h->W, 0, h->n_chunks, none, z_bar, s));
     h->n_launches += 1;

@@ -74,20 +74,31 @@ __device__ __forceinline__ float variance(const Consts &c, float v, float g_bar)
 {
     return f_add(f_mul(c.b2, v), f_mul(c.ob2, f_mul(g_bar, g_bar)));
 }
+// x / count in binary64, as the IEEE division gives it.  A binary64 division is a long instruction
+// sequence and the server side runs one per coordinate; when the count is a power of two (every worker
+// count and chunk size of the benchmark configurations) the quotient is x scaled by 2^-k, which is
+// exact, so one multiplication gives the same bits (x is zero or a sum of binary32 magnitudes: the
+// scaled value cannot fall into the subnormal range of binary64).
+__device__ __forceinline__ double div_by_count(double x, int count)
+{
+    if ((count & (count - 1)) == 0)
+        return __dmul_rn(x, __longlong_as_double((long long)(1023 - (31 - __clz(count))) << 52));
+    return __ddiv_rn(x, (double)count);
+}
 // Mean over W workers of a binary64 sum, rounded once (Algorithm 4).
 __device__ __forceinline__ float mean_round(double sum, int W)
 {
-    return __double2float_rn(__ddiv_rn(sum, (double)W));
+    return __double2float_rn(div_by_count(sum, W));
 }
 // Eq. 3 magnitude of a chunk: l1 / len, rounded once.
 __device__ __forceinline__ float chunk_scale(double l1, int len)
 {
-    return __double2float_rn(__ddiv_rn(l1, (double)len));
+    return __double2float_rn(div_by_count(l1, len));
 }
 // Server input of Algorithm 3: mean of the compressed buffers plus the server error.
 __device__ __forceinline__ float server_input(double sum_hat, int W, float delta_bar)
 {
-    return __double2float_rn(__dadd_rn(__ddiv_rn(sum_hat, (double)W), (double)delta_bar));
+    return __double2float_rn(__dadd_rn(div_by_count(sum_hat, W), (double)delta_bar));
 }
 
 // ---- 128-bit accesses ----

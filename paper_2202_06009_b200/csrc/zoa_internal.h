@@ -47,8 +47,8 @@ cudaError_t launch_reduce(const StateView &st, const Consts &c, float gamma_sum,
 // ring depth (0 = the kernel does not take this shape) and how many whole units of max(chunk, 2048)
 // coordinates the vector holds; the chunks after them go through launch_reduce.
 int reduce_pipeline_stages(const StateView &st, long long *n_units);
-cudaError_t launch_reduce_pipelined(const StateView &st, const Consts &c, float gamma_sum, long long n_units, int stages,
-                                    int sm_count, ErrorWords error_flag, unsigned long long *sched,
+cudaError_t launch_reduce_pipelined(const StateView &st, const Consts &c, float gamma_sum, long long n_units,
+                                    int stages, int sm_count, ErrorWords error_flag, unsigned long long *sched,
                                     unsigned long long wait_limit_ns, long long test_stop_after_tiles, cudaStream_t s);
 cudaError_t launch_step_sync(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
                              float gamma_sum, int g_aligned, long long first_chunk, long long count, cudaStream_t s);

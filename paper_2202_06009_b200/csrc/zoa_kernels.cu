@@ -167,9 +167,11 @@ __device__ __forceinline__ BlockSpan block_span(const StateView &st, const Chunk
 // 6.94 TB/s against 6.74 with the chunk staged in shared memory by a loop of dependent
 // iterations; chunk 16384 6.54 against 5.62).
 // EXTERNAL: what is compressed is z + delta with z read from caller-owned buffers (Algorithm 3 on an
-// arbitrary input, zoa_onebit_allreduce) instead of u + delta.
-template <int ITER, bool EXTERNAL>
-__global__ void __launch_bounds__(512, 2) compress_kernel(StateView st, long long first_chunk, GradPtrs z_in, int z_fmt)
+// arbitrary input, zoa_onebit_allreduce) instead of u + delta; 1 = by guarded loads (any alignment,
+// exactly n elements), 2 = the buffers are 16-byte aligned and the chunk is full, so plain
+// 128-bit loads do (a format known at compile time keeps all the loads ahead of the first use).
+template <int ITER, int EXTERNAL>
+__global__ void __launch_bounds__(512, 2) compress_kernel(StateView st, long long first_chunk, const __grid_constant__ GradPtrs z_in, int z_fmt)
 {
     __shared__ double scratch[34];
     const long long chunk_id = first_chunk + blockIdx.x;
@@ -177,22 +179,31 @@ __global__ void __launch_bounds__(512, 2) compress_kernel(StateView st, long lon
     const int i = blockIdx.y;
     const int lane = threadIdx.x & 31;
     const long long row = (long long)i * st.n_pad + cg.c0;
-    float4 u4[ITER], e4[ITER];
-#pragma unroll
-    for (int it = 0; it < ITER; ++it) {
-        const int idx = 4 * (it * blockDim.x + threadIdx.x);
-        const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (EXTERNAL) u4[it] = idx < cg.len ? ld_grad4(z_in.p[i], cg.c0 + idx, st.n, z_fmt) : zero;
-        else u4[it] = idx < cg.len ? ld4_stream(st.u + row + idx) : zero;     // whole float4 groups: the rows' padding is zero
-        e4[it] = idx < cg.len ? ld4_stream(st.dw + row + idx) : zero;
-    }
+    const float *z_row = EXTERNAL ? z_in.p[i] : nullptr;
+    // Loads go out in batches of BATCH float4 pairs, every load of a batch before its first use (with
+    // caller-owned inputs sixteen pairs at once do not fit the registers two resident blocks leave).
+    constexpr int BATCH = (EXTERNAL && ITER > 4) ? 4 : ITER;
     float z[ITER][4];
     double l1 = 0.0;
 #pragma unroll
-    for (int it = 0; it < ITER; ++it) {
-        z[it][0] = f_add(u4[it].x, e4[it].x); z[it][1] = f_add(u4[it].y, e4[it].y);
-        z[it][2] = f_add(u4[it].z, e4[it].z); z[it][3] = f_add(u4[it].w, e4[it].w);
-        l1 += fabs((double)z[it][0]) + fabs((double)z[it][1]) + fabs((double)z[it][2]) + fabs((double)z[it][3]);
+    for (int h = 0; h < ITER; h += BATCH) {
+        float4 u4[BATCH], e4[BATCH];
+#pragma unroll
+        for (int q = 0; q < BATCH; ++q) {
+            const int idx = 4 * ((h + q) * blockDim.x + threadIdx.x);
+            const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (EXTERNAL == 2 && cg.len == st.chunk) u4[q] = idx < cg.len ? ld4_stream(z_row + cg.c0 + idx) : zero;
+            else if (EXTERNAL) u4[q] = idx < cg.len ? ld_grad4(z_row, cg.c0 + idx, st.n, z_fmt) : zero;
+            else u4[q] = idx < cg.len ? ld4_stream(st.u + row + idx) : zero;     // whole float4 groups: the rows' padding is zero
+            e4[q] = idx < cg.len ? ld4_stream(st.dw + row + idx) : zero;
+        }
+#pragma unroll
+        for (int q = 0; q < BATCH; ++q) {
+            const int it = h + q;
+            z[it][0] = f_add(u4[q].x, e4[q].x); z[it][1] = f_add(u4[q].y, e4[q].y);
+            z[it][2] = f_add(u4[q].z, e4[q].z); z[it][3] = f_add(u4[q].w, e4[q].w);
+            l1 += fabs((double)z[it][0]) + fabs((double)z[it][1]) + fabs((double)z[it][2]) + fabs((double)z[it][3]);
+        }
     }
     const float scale = chunk_scale(block_sum(l1, scratch), cg.len);
 #pragma unroll
@@ -399,67 +410,95 @@ __global__ void step_sync_kernel(StateView st, GradPtrs g, Consts c, float gamma
 
 // Server side of Algorithm 3 alone for chunk first_chunk + blockIdx.x, reading packed buffers
 // gathered from W_total workers: words_in[w][range words], scales_in[w][range chunks], both
-// starting at the range's first chunk.  Writes the server error, words_s and scales_s.
+// starting at the range's first chunk.  Writes the server error, words_s and scales_s, and the
+// result itself to z_bar if that is not NULL (caller-owned, exactly n floats, any alignment).
 // `out` lists where else the packed result of the range is to be stored (every rank's
 // words_s / scales_s, peer pointers included); out.world == 0 for none.
-__global__ void __launch_bounds__(512, 3) dist_server_kernel(StateView st, const uint32_t *words_in, long long words_in_stride,
+// All of a block's loads go out before the first barrier: the chunk's words of every worker into
+// shared memory (eight independent loads per thread at a time), the server errors into registers.
+template <int ITER>
+__global__ void __launch_bounds__(512) dist_server_kernel(StateView st, const uint32_t *words_in, long long words_in_stride,
                                    const float *scales_in, long long scales_in_stride, int W_total,
                                    long long first_chunk, PeerOut out, float *z_bar)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     double *scratch = reinterpret_cast<double *>(smem_raw);
     float *scales = reinterpret_cast<float *>(smem_raw + 34 * sizeof(double));
-    float *a_s = scales + kMaxWorkers;
+    uint32_t *words_sm = reinterpret_cast<uint32_t *>(scales + kMaxWorkers);       // [W_total][chunk / 32]
     const long long chunk_id = first_chunk + blockIdx.x;
     const ChunkGeom cg = chunk_geom(st, chunk_id);
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    const int lane = threadIdx.x & 31;
     const long long range_word0 = (first_chunk * st.chunk) >> 5;
+    const int words_per_chunk = st.chunk >> 5, n_words = (cg.len + 31) >> 5;
+    const long long chunk_word0 = (cg.c0 >> 5) - range_word0;
+    const bool z_bar_aligned = (reinterpret_cast<uintptr_t>(z_bar) & 15u) == 0;
 
     for (int i = threadIdx.x; i < W_total; i += blockDim.x) scales[i] = scales_in[(long long)i * scales_in_stride + blockIdx.x];
+    const int total = W_total * n_words;
+    for (int e0 = threadIdx.x; e0 < total; e0 += 8 * blockDim.x) {
+        uint32_t w[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int e = e0 + q * blockDim.x;
+            w[q] = e < total ? words_in[(long long)(e / n_words) * words_in_stride + chunk_word0 + e % n_words] : 0u;
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int e = e0 + q * blockDim.x;
+            if (e < total) words_sm[(e / n_words) * words_per_chunk + e % n_words] = w[q];
+        }
+    }
+    float4 e4[ITER];
+#pragma unroll
+    for (int it = 0; it < ITER; ++it) {
+        const int idx = 4 * (it * blockDim.x + threadIdx.x);
+        e4[it] = idx < cg.len ? ld4(st.ds + cg.c0 + idx) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
     __syncthreads();
+
+    float a[ITER][4];
     double l1 = 0.0;
-    for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
-        const int idx = base + 4 * lane;
+#pragma unroll
+    for (int it = 0; it < ITER; ++it) {
+        const int idx = 4 * (it * blockDim.x + threadIdx.x);
+        double A[4] = {0.0, 0.0, 0.0, 0.0};
         if (idx < cg.len) {
-            double A[4] = {0.0, 0.0, 0.0, 0.0};
-            const long long word_idx = ((cg.c0 + idx) >> 5) - range_word0;
             const int shift = idx & 31;
             for (int i = 0; i < W_total; ++i) {  // worker order
-                const uint32_t nib = words_in[(long long)i * words_in_stride + word_idx] >> shift;
+                const uint32_t nib = words_sm[i * words_per_chunk + (idx >> 5)] >> shift;
                 const double sc = (double)scales[i];
 #pragma unroll
                 for (int k = 0; k < 4; ++k) A[k] += ((nib >> k) & 1u) ? sc : -sc;
             }
-            const float4 e4 = ld4(st.ds + cg.c0 + idx);
-            const float ee[4] = {e4.x, e4.y, e4.z, e4.w};
-            float a[4];
+        }
+        const float ee[4] = {e4[it].x, e4[it].y, e4[it].z, e4[it].w};
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                a[k] = idx + k < cg.len ? server_input(A[k], W_total, ee[k]) : 0.0f;
-                l1 += fabs((double)a[k]);
-            }
-            st4(a_s + idx, make_float4(a[0], a[1], a[2], a[3]));
+        for (int k = 0; k < 4; ++k) {
+            a[it][k] = idx + k < cg.len ? server_input(A[k], W_total, ee[k]) : 0.0f;
+            l1 += fabs((double)a[it][k]);
         }
     }
     const float scale = chunk_scale(block_sum(l1, scratch), cg.len);
-    for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
-        const int idx = base + 4 * lane;
-        float a[4] = {0.f, 0.f, 0.f, 0.f}, hat[4];
-        if (idx < cg.len) {
-            const float4 a4 = ld4(a_s + idx);
-            a[0] = a4.x; a[1] = a4.y; a[2] = a4.z; a[3] = a4.w;
-        }
-        const uint32_t word = compress_tile(a, hat, scale, idx, cg.len);
+#pragma unroll
+    for (int it = 0; it < ITER; ++it) {
+        const int idx = 4 * (it * blockDim.x + threadIdx.x);
+        const int base = idx - 4 * lane;                   // first coordinate of the warp's 128
+        float hat[4];
+        const uint32_t word = compress_tile(a[it], hat, scale, idx, cg.len);
         if (lane < 4 && base + 32 * lane < cg.len) {
             const long long w = ((cg.c0 + base) >> 5) + lane;
             st.words_s[w] = word;
             for (int r = 0; r < out.world; ++r) out.words_s[r][w] = word;
         }
-        if (idx < cg.len) st4(st.ds + cg.c0 + idx, make_float4(a[0], a[1], a[2], a[3]));
-        if (z_bar) {             // the result of Algorithm 3 in full: caller-owned, exactly n floats, any alignment
+        if (idx < cg.len) st4(st.ds + cg.c0 + idx, make_float4(a[it][0], a[it][1], a[it][2], a[it][3]));
+        if (z_bar) {
+            if (z_bar_aligned && idx + 4 <= cg.len) {
+                st4_stream(z_bar + cg.c0 + idx, make_float4(hat[0], hat[1], hat[2], hat[3]));
+            } else {
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
-                if (idx + k < cg.len) z_bar[cg.c0 + idx + k] = hat[k];
+                for (int k = 0; k < 4; ++k)
+                    if (idx + k < cg.len) z_bar[cg.c0 + idx + k] = hat[k];
+            }
         }
     }
     if (threadIdx.x == 0) {
@@ -998,7 +1037,7 @@ cudaError_t launch_variance(const StateView &st, const GradPtrs &g, const Consts
 }
 
 size_t compress_smem(int chunk) { return 34 * sizeof(double) + (size_t)chunk * sizeof(float); }                 // dist_pack_push_kernel
-size_t reduce_smem(int chunk) { return 34 * sizeof(double) + (kMaxWorkers + (size_t)chunk) * sizeof(float); }   // dist_server_kernel
+
 // reduce_kernel: block-sum and cluster scratch, magnitudes, the server input of `span` coordinates
 static size_t reduce_span_smem(int span) { return 42 * sizeof(double) + (kMaxWorkers + (size_t)span) * sizeof(float); }
 
@@ -1071,8 +1110,8 @@ cudaError_t launch_compress(const StateView &st, long long first_chunk, long lon
     const int thr = ((st.chunk + 4 * iter - 1) / (4 * iter) + 31) / 32 * 32;
     const dim3 grid((unsigned)count, (unsigned)st.W);
     const GradPtrs none{};
-    if (iter == 8) compress_kernel<8, false><<<grid, thr, 0, s>>>(st, first_chunk, none, 0);
-    else compress_kernel<4, false><<<grid, thr, 0, s>>>(st, first_chunk, none, 0);
+    if (iter == 8) compress_kernel<8, 0><<<grid, thr, 0, s>>>(st, first_chunk, none, 0);
+    else compress_kernel<4, 0><<<grid, thr, 0, s>>>(st, first_chunk, none, 0);
     return cudaGetLastError();
 }
 
@@ -1082,8 +1121,13 @@ cudaError_t launch_compress_external(const StateView &st, const GradPtrs &z, int
     const int iter = st.chunk > 4096 ? 8 : 4;
     const int thr = ((st.chunk + 4 * iter - 1) / (4 * iter) + 31) / 32 * 32;
     const dim3 grid((unsigned)st.n_chunks, (unsigned)st.W);
-    if (iter == 8) compress_kernel<8, true><<<grid, thr, 0, s>>>(st, 0, z, z_fmt);
-    else compress_kernel<4, true><<<grid, thr, 0, s>>>(st, 0, z, z_fmt);
+    if (z_fmt & kGradAligned) {
+        if (iter == 8) compress_kernel<8, 2><<<grid, thr, 0, s>>>(st, 0, z, z_fmt);
+        else compress_kernel<4, 2><<<grid, thr, 0, s>>>(st, 0, z, z_fmt);
+    } else {
+        if (iter == 8) compress_kernel<8, 1><<<grid, thr, 0, s>>>(st, 0, z, z_fmt);
+        else compress_kernel<4, 1><<<grid, thr, 0, s>>>(st, 0, z, z_fmt);
+    }
     return cudaGetLastError();
 }
 
@@ -1178,15 +1222,18 @@ cudaError_t launch_dist_server(const StateView &st, const uint32_t *words_in, lo
                                const float *scales_in, long long scales_in_stride, int W_total,
                                long long first_chunk, long long count, const PeerOut &out, float *z_bar, cudaStream_t s)
 {
-    static SmemLimitOnce once;
-    const cudaError_t e = once.ensure(dist_server_kernel, (int)reduce_smem(kMaxChunk));
+    // 16 coordinates per thread (32 above chunk 4096), like compress_kernel
+    const int iter = st.chunk > 4096 ? 8 : 4;
+    const int thr = ((st.chunk + 4 * iter - 1) / (4 * iter) + 31) / 32 * 32;
+    const size_t smem = 34 * sizeof(double) + kMaxWorkers * sizeof(float) + (size_t)W_total * (st.chunk / 32) * sizeof(uint32_t);
+    static SmemLimitOnce once[2];
+    cudaError_t e = once[0].ensure(dist_server_kernel<4>, (int)(34 * sizeof(double) + kMaxWorkers * sizeof(float) + (size_t)kMaxWorkers * (4096 / 32) * 4));
+    if (e == cudaSuccess) e = once[1].ensure(dist_server_kernel<8>, (int)(34 * sizeof(double) + kMaxWorkers * sizeof(float) + (size_t)kMaxWorkers * (kMaxChunk / 32) * 4));
     if (e != cudaSuccess) return e;
-    // block size as for reduce_kernel: with few workers smaller blocks, more of them per SM
-    const int per_thread = W_total <= 2 ? 32 : 16;
-    int thr = 128;
-    while (thr < st.chunk / per_thread && thr < 512) thr <<= 1;
-    dist_server_kernel<<<(unsigned)count, thr, reduce_smem(st.chunk), s>>>(
-        st, words_in, words_in_stride, scales_in, scales_in_stride, W_total, first_chunk, out, z_bar);
+    if (iter == 8)
+        dist_server_kernel<8><<<(unsigned)count, thr, smem, s>>>(st, words_in, words_in_stride, scales_in, scales_in_stride, W_total, first_chunk, out, z_bar);
+    else
+        dist_server_kernel<4><<<(unsigned)count, thr, smem, s>>>(st, words_in, words_in_stride, scales_in, scales_in_stride, W_total, first_chunk, out, z_bar);
     return cudaGetLastError();
 }
 

@@ -369,8 +369,8 @@ static PipeArgs two_call_args(const StateView &st, const Consts &c, float gamma_
     }
 
 // Server side for the first n_units units (the caller runs the remaining chunks through reduce_kernel).
-cudaError_t launch_reduce_pipelined(const StateView &st, const Consts &c, float gamma_sum, long long n_units, int stages,
-                                    int sm_count, ErrorWords error_flag, unsigned long long *sched,
+cudaError_t launch_reduce_pipelined(const StateView &st, const Consts &c, float gamma_sum, long long n_units,
+                                    int stages, int sm_count, ErrorWords error_flag, unsigned long long *sched,
                                     unsigned long long wait_limit_ns, long long test_stop_after_tiles, cudaStream_t s)
 {
     int tiles, g;
