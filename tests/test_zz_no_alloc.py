@@ -83,3 +83,8 @@ def test_static_entry_point_rejects_what_does_not_fit():
     assert e.value.status == B.ERR_ARG and "scratch" in str(e.value)
     with pytest.raises(ZoaError):
         B.zoa_onebit_allreduce_static([p], [p], p, p, 64, 1, 48, 0)
+    # sizes whose slot count would wrap 64-bit arithmetic are refused as arguments too, not at launch
+    for n_huge, W, chunk in ((1 << 62, 64, 32), ((1 << 63) + 5, 1, 4096), (32 * slots + 1, 1, 16384)):
+        with pytest.raises(ZoaError) as e:
+            B.zoa_onebit_allreduce_static([p] * W, [p] * W, p, p, n_huge, W, chunk, 0)
+        assert e.value.status == B.ERR_ARG
