@@ -887,33 +887,62 @@ __global__ void lc_scales_kernel(StateView st, const double *partials, long long
 
 // Server side of Algorithm 3, the one pass: a = mean of the compressed buffers + server error goes
 // into the server-error row (pending form), its sign bits into words_s, sum |a| into partials[W][seg].
-__global__ void __launch_bounds__(512)
+// 256 threads x 16 coordinates per segment; every load goes out before the first barrier: the W
+// word rows of the segment into shared memory, the server errors into registers.
+constexpr int kSegIter = kSegment / (4 * 256);
+
+__global__ void __launch_bounds__(256)
 lc_server_pack_kernel(StateView st, int pending, long long segs_per_chunk, long long n_segs, double *partials)
 {
-    __shared__ double scratch[34];
-    __shared__ float scales_sm[kMaxWorkers];
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    double *scratch = reinterpret_cast<double *>(smem_raw);
+    float *scales_sm = reinterpret_cast<float *>(smem_raw + 34 * sizeof(double));
+    uint32_t *words_sm = reinterpret_cast<uint32_t *>(scales_sm + kMaxWorkers);      // [W][kSegment / 32]
     const SegGeom sg = seg_geom(st, blockIdx.x, segs_per_chunk);
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    const int lane = threadIdx.x & 31;
+    constexpr int kWordsPerSeg = kSegment / 32;
+    const int n_words = (sg.len + 31) >> 5;
+    const long long seg_word0 = sg.j0 >> 5;
     for (int i = threadIdx.x; i < st.W; i += blockDim.x) scales_sm[i] = st.scales_w[(long long)i * st.n_chunks + sg.c];
     const float old_scale = pending ? st.scales_s[sg.c] : 0.0f;       // of the previous sync
+    const int total = st.W * n_words;
+    for (int e0 = threadIdx.x; e0 < total; e0 += 8 * blockDim.x) {
+        uint32_t w[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int e = e0 + q * blockDim.x;
+            w[q] = e < total ? st.words_w[(long long)(e / n_words) * st.words_stride + seg_word0 + e % n_words] : 0u;
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int e = e0 + q * blockDim.x;
+            if (e < total) words_sm[(e / n_words) * kWordsPerSeg + e % n_words] = w[q];
+        }
+    }
+    float4 e4[kSegIter];
+#pragma unroll
+    for (int it = 0; it < kSegIter; ++it) {
+        const int idx = 4 * (it * blockDim.x + threadIdx.x);
+        e4[it] = idx < sg.len ? ld4(st.ds + sg.j0 + idx) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
     __syncthreads();
     double l1 = 0.0;
-    for (int base = warp * 128; base < sg.len; base += n_warps * 128) {
-        const int idx = base + 4 * lane;
+#pragma unroll
+    for (int it = 0; it < kSegIter; ++it) {
+        const int idx = 4 * (it * blockDim.x + threadIdx.x);
+        const int base = idx - 4 * lane;
         float a[4] = {0.f, 0.f, 0.f, 0.f};
         if (idx < sg.len) {
-            const long long j = sg.j0 + idx;
             double A[4] = {0.0, 0.0, 0.0, 0.0};
-            const long long word_idx = j >> 5;
-            const int shift = (int)(j & 31);
+            const int shift = idx & 31;
             for (int i = 0; i < st.W; ++i) {   // worker order
-                const uint32_t nib = st.words_w[(long long)i * st.words_stride + word_idx] >> shift;
+                const uint32_t nib = words_sm[i * kWordsPerSeg + (idx >> 5)] >> shift;
                 const double sc = (double)scales_sm[i];
 #pragma unroll
                 for (int k = 0; k < 4; ++k) A[k] += ((nib >> k) & 1u) ? sc : -sc;
             }
-            const float4 e4 = plain_error4(ld4(st.ds + j), pending != 0, old_scale);
-            const float ee[4] = {e4.x, e4.y, e4.z, e4.w};
+            const float4 p4 = plain_error4(e4[it], pending != 0, old_scale);
+            const float ee[4] = {p4.x, p4.y, p4.z, p4.w};
 #pragma unroll
             for (int k = 0; k < 4; ++k) a[k] = idx + k < sg.len ? server_input(A[k], st.W, ee[k]) : 0.0f;
         }
@@ -927,8 +956,8 @@ lc_server_pack_kernel(StateView st, int pending, long long segs_per_chunk, long 
         if (idx < sg.len) st4(st.ds + sg.j0 + idx, make_float4(a[0], a[1], a[2], a[3]));
         if (lane < 4 && base + 32 * lane < sg.len) st.words_s[((sg.j0 + base) >> 5) + lane] = word;
     }
-    const double total = block_sum(l1, scratch);
-    if (threadIdx.x == 0) partials[(long long)st.W * n_segs + blockIdx.x] = total;
+    const double total_l1 = block_sum(l1, scratch);
+    if (threadIdx.x == 0) partials[(long long)st.W * n_segs + blockIdx.x] = total_l1;
 }
 
 // Momentum and model updates of Algorithm 2 from the server's packed result: g_bar = +-scales_s by words_s.
@@ -1197,7 +1226,8 @@ cudaError_t launch_large_server(const StateView &st, const Consts &c, int mode, 
                                 int *launches, cudaStream_t s)
 {
     const long long spc = large_chunk_segments(st), n_segs = spc * st.n_chunks;
-    lc_server_pack_kernel<<<(unsigned)n_segs, 512, 0, s>>>(st, pending, spc, n_segs, partials);
+    const size_t pack_smem = 34 * sizeof(double) + kMaxWorkers * sizeof(float) + (size_t)st.W * (kSegment / 32) * sizeof(uint32_t);
+    lc_server_pack_kernel<<<(unsigned)n_segs, 256, pack_smem, s>>>(st, pending, spc, n_segs, partials);
     lc_scales_kernel<<<dim3((unsigned)st.n_chunks, 1), 32, 0, s>>>(st, partials + (long long)st.W * n_segs, spc, n_segs, st.scales_s);
     if (mode == 1) dist_apply_kernel<<<elementwise_grid((st.n + 3) / 4), 256, 0, s>>>(st, c, scalar);
     else lc_alg2_apply_kernel<<<elementwise_grid((st.n + 3) / 4), 256, 0, s>>>(st, c, scalar);
