@@ -40,7 +40,13 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
     constexpr int words_per_chunk = (int)(kSpan >> 5);                                  // words of a unit
     uint32_t *bits_s = reinterpret_cast<uint32_t *>(smem_raw + 1024);                 // [W][words_per_chunk]
     float *scales_s = reinterpret_cast<float *>(bits_s + W * words_per_chunk);         // [kConsumerWarps][W]
-    unsigned char *ring = smem_raw + ((1024 + (size_t)W * words_per_chunk * 4 + (size_t)kConsumerWarps * W * 4 + 1023) & ~(size_t)1023);
+    // On a T_v step with four tiles the binary64 gradient sums of the last two tiles live in shared
+    // memory ([tile][k][thread], one column per thread): sixteen of them in registers make the kernel spill.
+    constexpr int G_SHARED_TILES = (DO_VAR && TILES == 4) ? 2 : 0;
+    constexpr int G_REG_TILES = DO_VAR ? TILES - G_SHARED_TILES : 1;
+    const size_t head_bytes = (1024 + (size_t)W * words_per_chunk * 4 + (size_t)kConsumerWarps * W * 4 + 1023) & ~(size_t)1023;
+    double *gsum_s = reinterpret_cast<double *>(smem_raw + head_bytes);                 // [G_SHARED_TILES][4][kConsumers]
+    unsigned char *ring = smem_raw + head_bytes + (size_t)G_SHARED_TILES * 4 * kConsumers * sizeof(double);
     const int R = a.stages;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     volatile int *abort_flag = &sh->abort;
@@ -106,9 +112,9 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
     // spread over the worker iterations of the next chunk (one worker's m, x, u after
     // each worker's compression) instead of leaving in one burst, so that the block's
     // stores and its ring's loads stay evenly mixed.  m is +-m_pos by the server's bit.
-    // With eight tiles, or four tiles and the binary64 gradient sums of a T_v step, the tiles of x have no room
-    // in the registers (17 warps leave 96 per thread: one SM sub-partition hosts five of them): those store at once.
-    constexpr bool DEFER = TILES <= 2 || (TILES == 4 && !DO_VAR);
+    // With eight tiles the tiles of x have no room in the registers (17 warps leave 96 per thread: one SM
+    // sub-partition hosts five of them): that variant stores at once.
+    constexpr bool DEFER = TILES <= 4;
     float x_prev[DEFER ? TILES : 1][4];
     uint32_t bits_prev = 0;
     float m_pos_prev = 0.0f;
@@ -137,10 +143,12 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
         const long long c0 = chunk * kSpan;
         const long long scale_idx = G == 1 ? chunk : chunk * G + warp / WPC;       // this thread's chunk
         const bool scale_writer = G == 1 ? tid == 0 : (lane == 0 && warp % WPC == 0);
-        double Gs[DO_VAR ? TILES : 1][4];
+        double Gs[G_REG_TILES][4];
         if (DO_VAR) {
 #pragma unroll
-            for (int t = 0; t < TILES; ++t) { Gs[t][0] = Gs[t][1] = Gs[t][2] = Gs[t][3] = 0.0; }
+            for (int t = 0; t < G_REG_TILES; ++t) { Gs[t][0] = Gs[t][1] = Gs[t][2] = Gs[t][3] = 0.0; }
+#pragma unroll
+            for (int q = 0; q < G_SHARED_TILES * 4; ++q) gsum_s[q * kConsumers + tid] = 0.0;
         }
         for (int i = 0; i < W; ++i) {
             float z[TILES][4];
@@ -169,7 +177,10 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
                     const float step = f_mul(a.gamma, momentum(a.c, mm[k], gg[k]));   // momentum update, buffer update
                     z[t][k] = f_add(f_add(uu[k], step), ee[k]);                       // u_{t+1/2} + delta
                     l1 += fabs((double)z[t][k]);
-                    if (DO_VAR) Gs[t][k] += (double)gg[k];
+                    if (DO_VAR) {
+                        if (t < G_REG_TILES) Gs[t][k] += (double)gg[k];
+                        else gsum_s[((t - G_REG_TILES) * 4 + k) * kConsumers + tid] += (double)gg[k];
+                    }
                 }
             }
             const float scale = chunk_scale(consumer_group_sum<WPC>(l1, sh, flip), st.chunk);
@@ -273,7 +284,10 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
             if (DO_VAR) {
                 float vo[4];
 #pragma unroll
-                for (int k = 0; k < 4; ++k) vo[k] = variance(a.c, vv[k], mean_round(Gs[t][k], W));   // variance update
+                for (int k = 0; k < 4; ++k) {
+                    const double g_sum = t < G_REG_TILES ? Gs[t < G_REG_TILES ? t : 0][k] : gsum_s[((t - G_REG_TILES) * 4 + k) * kConsumers + tid];
+                    vo[k] = variance(a.c, vv[k], mean_round(g_sum, W));   // variance update
+                }
                 st4_stream(st.v_next + j, make_float4(vo[0], vo[1], vo[2], vo[3]));
             }
         }
@@ -555,10 +569,18 @@ cudaError_t launch_step_sync_pipelined(const StateView &st, const GradPtrs &g, c
     a.wait_limit_ns = wait_limit_ns;
     a.test_stop_after_tiles = test_stop_after_tiles;
     const int grid = (int)(n_units < sm_count ? n_units : sm_count);
-    const size_t smem = pipeline_fixed_smem(st.W, st.chunk) + (size_t)stages * kStageBytes;
     int tiles, cpt;
     if (!unit_shape(st.chunk, &tiles, &cpt)) return cudaErrorInvalidValue;
     if (tiles == 8) do_var = false;       // eight tiles of binary64 gradient sums have no room in the registers
+    size_t fixed = pipeline_fixed_smem(st.W, st.chunk);
+    if (tiles == 4 && do_var) {           // two tiles of gradient sums in shared memory; the ring gives up a stage for them
+        fixed += 2 * 4 * kConsumers * sizeof(double);
+        const int fit = (int)((227 * 1024 - fixed) / kStageBytes);
+        if (fit < tiles + 1) do_var = false;
+        else if (stages > fit) a.stages = stages = fit;
+    }
+    if (!do_var) fixed = pipeline_fixed_smem(st.W, st.chunk);
+    const size_t smem = fixed + (size_t)stages * kStageBytes;
     *var_fused = do_var;
 #define ZOA_PIPE(T, GG) (do_var ? launch_pipe<T, GG, true>(a, grid, smem, s) : launch_pipe<T, GG, false>(a, grid, smem, s))
     switch (tiles * 100 + cpt) {

@@ -112,7 +112,7 @@ def test_pipelined_kernel_equals_chunk_per_block_kernel(W, chunk, n_chunks, tail
                     assert np.array_equal(a.read(name, i), b.read(name, i)), (name, i, t)
             for name in ("v", "delta_s", "x_sync", "words_s", "scales_s"):
                 assert np.array_equal(a.read(name), b.read(name)), (name, t)
-        if chunk <= 8192 and not tail and n_chunks % max(1, 2048 // chunk) == 0:      # the variance update rides along in the ring kernel
+        if chunk <= 8192 and W <= 16 and not tail and n_chunks % max(1, 2048 // chunk) == 0:      # the variance update rides along in the ring kernel
             assert a.stats()["n_launches"] < b.stats()["n_launches"]
     finally:
         a.close(), b.close()
