@@ -477,19 +477,25 @@ def test_policies_match_the_workload_tables():
         z.close()
 
 
-@pytest.mark.parametrize("algorithm", ["alg1", "alg2"])
+@pytest.mark.parametrize("algorithm", ["alg1", "alg2", "two_call", "alg1_chunk_1024", "alg1_chunk_16384"])
 def test_device_wait_runs_out_and_is_reported(algorithm):
     """Error path of the ring kernels without any fault: the copy-issuing lane of every block
     stops after three tiles (test hook), the other threads' bounded waits run out after
     100 ms, the kernel ends by itself, zoa_check_device reports ZOA_ERR_DEVICE, and the
-    context and the handle stay usable."""
+    context and the handle stay usable.  Covers the fused kernel (one, two and eight tiles per
+    unit), Algorithm 2's, and the server kernel of the two-call path with its store-issuing warp."""
     import time
-    n, W, chunk = 300 * 4096, 4, 4096
+    chunk = 1024 if algorithm.endswith("1024") else 16384 if algorithm.endswith("16384") else 4096
+    n, W = 300 * max(chunk, 2048), 4
     z = Zoa(n, W, chunk=chunk)
     try:
         g = list(torch.randn(W, n, device="cuda"))
         z.set_pipeline("force")
-        step = z.step_sync if algorithm == "alg1" else z.alg2_step
+
+        def two_call(g, lr, t):
+            z.step(g, lr, t)
+            z.onebit_reduce()
+        step = z.alg2_step if algorithm == "alg2" else two_call if algorithm == "two_call" else z.step_sync
         step(g, 1e-3, 0)
         z.check_device()                                  # the normal path works
         B.zoa_set_option(z.h, B.OPT_WAIT_LIMIT_MS, 100)
