@@ -475,9 +475,21 @@ static cudaError_t run_server(zoa_handle h, float gamma_sum, cudaStream_t s)
 static zoa_status run_local_range(zoa_handle h, const StateView &st, const GradPtrs &gp, float lr, bool do_var, int fmt,
                                   long long c0, long long c1, cudaStream_t s)
 {
-    const long long e0 = c0 * h->chunk, e1 = std::min<long long>(c1 * (long long)h->chunk, h->n);
-    ZOA_CUDA(h, launch_local_step(st, gp, h->c, lr, do_var, fmt, e0, e1, s));
-    h->n_launches += 1;
+    long long e0 = c0 * h->chunk;
+    const long long e1 = std::min<long long>(c1 * (long long)h->chunk, h->n);
+    // whole tiles of 2048 coordinates through the ring kernel (aligned gradients, a tile-aligned start,
+    // enough tiles to feed every SM), the rest one float4 per thread
+    const long long n_units = (e0 % 2048 == 0 && (fmt & kGradAligned)) ? (e1 - e0) / 2048 : 0;
+    if (h->use_pipeline && (h->use_pipeline == 2 || n_units >= 4ll * h->sm_count) && n_units > 0) {
+        ZOA_CUDA(h, launch_local_step_pipelined(st, gp, h->c, lr, do_var, fmt, e0 / 2048, n_units, h->sm_count, error_words(h), h->sched,
+                                                (unsigned long long)h->wait_limit_ms * 1000000ull, h->test_stop_after_tiles, s));
+        h->n_launches += 1;
+        e0 += n_units * 2048;
+    }
+    if (e0 < e1) {
+        ZOA_CUDA(h, launch_local_step(st, gp, h->c, lr, do_var, fmt, e0, e1, s));
+        h->n_launches += 1;
+    }
     return ZOA_OK;
 }
 

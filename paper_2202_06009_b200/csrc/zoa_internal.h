@@ -73,6 +73,11 @@ cudaError_t launch_step_sync_pipelined(const StateView &st, const GradPtrs &g, c
                                        unsigned long long *sched, unsigned long long wait_limit_ns,
                                        long long test_stop_after_tiles, bool *var_fused, cudaStream_t s);
 
+cudaError_t launch_local_step_pipelined(const StateView &st, const GradPtrs &g, const Consts &c, float gamma, bool do_var,
+                                        int grad_fmt, long long first_unit, long long n_units, int sm_count, ErrorWords error_flag,
+                                        unsigned long long *sched, unsigned long long wait_limit_ns,
+                                        long long test_stop_after_tiles, cudaStream_t s);
+
 // One worker per GPU: the kernels between the collectives.
 cudaError_t launch_dist_server(const StateView &st, const uint32_t *words_in, long long words_in_stride,
                                const float *scales_in, long long scales_in_stride, int W_total,

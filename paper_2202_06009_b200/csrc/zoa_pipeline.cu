@@ -167,8 +167,7 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
                     u4 = ld4(stage + 2 * kTile + pos);
                     e4 = ld4(stage + 3 * kTile + pos);
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_addr(&sh->empty[s]));
+                release_stage(sh, s, dep_bits(g4, m4, u4, e4));
                 if (++s == R) { s = 0; phase ^= 1u; }
                 const float gg[4] = {g4.x, g4.y, g4.z, g4.w}, mm[4] = {m4.x, m4.y, m4.z, m4.w};
                 const float uu[4] = {u4.x, u4.y, u4.z, u4.w}, ee[4] = {e4.x, e4.y, e4.z, e4.w};
@@ -217,10 +216,7 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
             srv_stage[t] = s;
             const float *stage = reinterpret_cast<const float *>(ring + (size_t)s * kStageBytes);
             const float4 d4 = ready ? ld4(stage + pos) : make_float4(0.f, 0.f, 0.f, 0.f);
-            if (SERVER_TWO_PASS) {
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_addr(&sh->empty[s]));
-            }
+            if (SERVER_TWO_PASS) release_stage(sh, s, dep_bits(d4));
             if (++s == R) { s = 0; phase ^= 1u; }
             const float dd[4] = {d4.x, d4.y, d4.z, d4.w};
             double A[4] = {0.0, 0.0, 0.0, 0.0};
@@ -247,8 +243,7 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
             }
             const float *stage = reinterpret_cast<const float *>(ring + (size_t)srv_stage[t] * kStageBytes);
             const float4 v4 = ld4(stage + kTile + pos), xs4 = ld4(stage + 2 * kTile + pos);
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_addr(&sh->empty[srv_stage[t]]));
+            release_stage(sh, srv_stage[t], dep_bits(v4, xs4));
             const float vv[4] = {v4.x, v4.y, v4.z, v4.w}, xs[4] = {xs4.x, xs4.y, xs4.z, xs4.w};
             bool b[4];
             float e[4], xo[4];
@@ -384,8 +379,7 @@ __global__ void __launch_bounds__(kThreads, 1) alg2_pipelined_kernel(const __gri
                 slot0 = ld4(stage + pos);
             slot1 = ld4(stage + kTile + pos);
         }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_addr(&sh->empty[s]));
+        release_stage(sh, s, dep_bits(slot0, slot1));
         if (++s == R) { s = 0; phase ^= 1u; }
     };
 
@@ -495,6 +489,109 @@ __global__ void __launch_bounds__(kThreads, 1) alg2_pipelined_kernel(const __gri
 }
 
 // ---------------------------------------------------------------------------
+// The local step of Algorithm 1 (momentum, model and buffer updates; the variance update on T_v
+// steps) in the same style: a unit is one tile of 2048 coordinates of all W workers; the ring
+// carries per worker a stage of (g, m, x, u) and, with the first worker, the tile of v.  The
+// consumers need no barrier among themselves (the step is elementwise); the ring only keeps
+// more loads in flight than resident blocks of an elementwise kernel can.
+// ---------------------------------------------------------------------------
+constexpr int kLocalStageBytes = 5 * kTileBytes;      // g, m, x, u, v
+
+template <bool DO_VAR>
+__global__ void __launch_bounds__(kThreads, 1) local_step_pipelined_kernel(const __grid_constant__ PipeArgs a)
+{
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    PipeShared *sh = reinterpret_cast<PipeShared *>(smem_raw);
+    const StateView &st = a.st;
+    const int W = st.W;
+    unsigned char *ring = smem_raw + 1024;
+    const int R = a.stages;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    volatile int *abort_flag = &sh->abort;
+
+    ring_init(sh, R);
+
+    if (warp == kConsumerWarps) {
+        if (lane != 0) return;
+        RingProducer p(a, sh, ring, kLocalStageBytes);
+        const uint32_t g_elem = (a.grad_fmt & kGradTypeMask) == kGradF32 ? 4u : 2u;
+        long long unit;
+        for (long long k = 0; p.ok && p.next_chunk(k, &unit); ++k) {
+            const long long off = unit * kTile;
+            for (int i = 0; i < W && p.stage_free(); ++i) {
+                const uint32_t full = p.full_barrier(), dst = p.stage_addr();
+                const long long row = (long long)i * st.n_pad + off;
+                mbar_arrive_expect_tx(full, 3 * kTileBytes + kTile * g_elem + (i == 0 ? kTileBytes : 0));
+                bulk_load(dst, reinterpret_cast<const char *>(a.g.p[i]) + off * g_elem, kTile * g_elem, full);
+                bulk_load(dst + kTileBytes, st.m + row, kTileBytes, full);
+                bulk_load(dst + 2 * kTileBytes, st.x + row, kTileBytes, full);
+                bulk_load(dst + 3 * kTileBytes, st.u + row, kTileBytes, full);
+                if (i == 0) bulk_load(dst + 4 * kTileBytes, st.v + off, kTileBytes, full);
+                p.advance();
+            }
+        }
+        p.finish();
+        return;
+    }
+
+    int s = 0;
+    uint32_t phase = 0;
+    const int pos = 4 * tid;
+    for (long long k = 0;; ++k) {
+        const bool gave_up = !mbar_wait(smem_addr(&sh->full[s]), phase, abort_flag, a.error_flag, a.wait_limit_ns);
+        if (consumer_any(gave_up)) break;
+        const long long unit = sh->chunk_queue[k % (kMaxStages + 2)];
+        if (unit < 0) break;
+        const long long j = unit * kTile + pos;
+        float d[4] = {1.f, 1.f, 1.f, 1.f}, vv[4] = {0.f, 0.f, 0.f, 0.f};
+        double Gs[4] = {0.0, 0.0, 0.0, 0.0};
+        for (int i = 0; i < W; ++i) {
+            const bool ready = mbar_wait(smem_addr(&sh->full[s]), phase, abort_flag, a.error_flag, a.wait_limit_ns);
+            const float *stage = reinterpret_cast<const float *>(ring + (size_t)s * kLocalStageBytes);
+            float4 g4 = make_float4(0.f, 0.f, 0.f, 0.f), m4 = g4, x4 = g4, u4 = g4;
+            if (ready) {
+                if ((a.grad_fmt & kGradTypeMask) == kGradF32)
+                    g4 = ld4(stage + pos);
+                else   // 16-bit gradients fill the first half of the slot
+                    g4 = grad16x4_to_float4(*reinterpret_cast<const uint2 *>(reinterpret_cast<const unsigned short *>(stage) + pos), a.grad_fmt);
+                m4 = ld4(stage + kTile + pos);
+                x4 = ld4(stage + 2 * kTile + pos);
+                u4 = ld4(stage + 3 * kTile + pos);
+                if (i == 0) {
+                    const float4 v4 = ld4(stage + 4 * kTile + pos);
+                    vv[0] = v4.x; vv[1] = v4.y; vv[2] = v4.z; vv[3] = v4.w;
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) d[q] = denom(a.c, vv[q]);
+                }
+            }
+            release_stage(sh, s, dep_bits(g4, m4, x4, u4) ^ __float_as_uint(d[0]));
+            if (++s == R) { s = 0; phase ^= 1u; }
+            const float gg[4] = {g4.x, g4.y, g4.z, g4.w}, mm[4] = {m4.x, m4.y, m4.z, m4.w};
+            const float xx[4] = {x4.x, x4.y, x4.z, x4.w}, uu[4] = {u4.x, u4.y, u4.z, u4.w};
+            float mo[4], xo[4], uo[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                mo[q] = momentum(a.c, mm[q], gg[q]);            // momentum update
+                const float step = f_mul(a.gamma, mo[q]);
+                xo[q] = f_sub(xx[q], f_div(step, d[q]));        // model update
+                uo[q] = f_add(uu[q], step);                     // buffer update
+                if (DO_VAR) Gs[q] += (double)gg[q];
+            }
+            const long long row = (long long)i * st.n_pad + j;
+            st4_stream(st.m + row, make_float4(mo[0], mo[1], mo[2], mo[3]));
+            st4_stream(st.x + row, make_float4(xo[0], xo[1], xo[2], xo[3]));
+            st4_stream(st.u + row, make_float4(uo[0], uo[1], uo[2], uo[3]));
+        }
+        if (DO_VAR) {
+            float vo[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) vo[q] = variance(a.c, vv[q], mean_round(Gs[q], W));   // variance update
+            st4_stream(st.v_next + j, make_float4(vo[0], vo[1], vo[2], vo[3]));
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------
 // Tiles per unit and chunks per tile for a chunk size the ring kernels take (false: they do not).
@@ -595,6 +692,34 @@ cudaError_t launch_step_sync_pipelined(const StateView &st, const GradPtrs &g, c
     default: return cudaErrorInvalidValue;
     }
 #undef ZOA_PIPE
+}
+
+// The local step for the whole tiles [first_unit, first_unit + n_units) (tiles of 2048 coordinates); what is left
+// over is the caller's.  Needs 16-byte aligned gradients.
+cudaError_t launch_local_step_pipelined(const StateView &st, const GradPtrs &g, const Consts &c, float gamma, bool do_var,
+                                        int grad_fmt, long long first_unit, long long n_units, int sm_count, ErrorWords error_flag,
+                                        unsigned long long *sched, unsigned long long wait_limit_ns,
+                                        long long test_stop_after_tiles, cudaStream_t s)
+{
+    PipeArgs a;
+    a.st = st; a.g = g; a.c = c; a.gamma = gamma; a.gamma_sum = 0.f;
+    a.first_chunk = first_unit;
+    a.n_full_chunks = n_units;
+    a.stages = (227 * 1024 - 1024) / kLocalStageBytes;        // five stages of 40 KB
+    a.error_flag = error_flag;
+    a.sched = sched;
+    a.grad_fmt = grad_fmt;
+    a.wait_limit_ns = wait_limit_ns;
+    a.test_stop_after_tiles = test_stop_after_tiles;
+    const int grid = (int)(n_units < sm_count ? n_units : sm_count);
+    const size_t smem = 1024 + (size_t)a.stages * kLocalStageBytes;
+    static SmemLimitOnce once[2];
+    cudaError_t e = once[0].ensure(local_step_pipelined_kernel<false>, 227 * 1024);
+    if (e == cudaSuccess) e = once[1].ensure(local_step_pipelined_kernel<true>, 227 * 1024);
+    if (e != cudaSuccess) return e;
+    if (do_var) local_step_pipelined_kernel<true><<<grid, kThreads, smem, s>>>(a);
+    else local_step_pipelined_kernel<false><<<grid, kThreads, smem, s>>>(a);
+    return cudaGetLastError();
 }
 
 }  // namespace zoa

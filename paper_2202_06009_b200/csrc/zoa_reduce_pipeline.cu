@@ -239,8 +239,8 @@ __global__ void __launch_bounds__(kRingThreads, 1) reduce_pipelined_kernel(const
 #pragma unroll
                 for (int q = 0; q < 4; ++q) A[q] += ((nib >> q) & 1u) ? sc : -sc;
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_addr(&sh->ring.empty[s]));
+            // the sums were formed from the stage's words and magnitudes: they stand for those loads
+            release_stage(&sh->ring, s, dep_bits(d4) ^ (uint32_t)__double_as_longlong(A[0]) ^ (uint32_t)__double_as_longlong(A[3]));
             if (++s == R) { s = 0; phase ^= 1u; }
             const float dd[4] = {d4.x, d4.y, d4.z, d4.w};
 #pragma unroll
@@ -259,8 +259,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) reduce_pipelined_kernel(const
             const float *stage = reinterpret_cast<const float *>(ring + (size_t)s * lay.stage_bytes);
             const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
             const float4 v4 = ready ? ld4(stage + pos) : zero4, xs4 = ready ? ld4(stage + kTile + pos) : zero4;
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_addr(&sh->ring.empty[s]));
+            release_stage(&sh->ring, s, dep_bits(v4, xs4));
             if (++s == R) { s = 0; phase ^= 1u; }
             const float vv[4] = {v4.x, v4.y, v4.z, v4.w}, xs[4] = {xs4.x, xs4.y, xs4.z, xs4.w};
             bool b[4];

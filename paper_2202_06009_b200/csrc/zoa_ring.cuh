@@ -39,6 +39,7 @@ struct PipeShared {
     double sums[2][kConsumerWarps];
     long long chunk_queue[kMaxStages + 2];   // chunk ids in the order the producer took them; -1 = no more
     int abort;
+    uint32_t sink[32];                       // one word per warp, see release_stage
 };
 
 __device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -115,6 +116,25 @@ __device__ __forceinline__ bool consumer_any(bool flag)
         : "r"((uint32_t)flag), "n"(kConsumers)
         : "memory");
     return out != 0;
+}
+
+// Hands a ring stage back to the producer once this warp has read it.  `dep` must be computed from what
+// the warp loaded from the stage.  A shared-memory load only *issues* in program order: behind a full
+// store queue its data can return after a later mbarrier arrive has already let the producer refill
+// the stage, and the warp then reads the next tile's bytes (seen on an L2-resident problem, where the
+// refill lands within a few hundred nanoseconds).  The store of `dep` cannot issue before every
+// lane's loads have returned, and the arrive follows that store.
+__device__ __forceinline__ void release_stage(PipeShared *sh, int stage, uint32_t dep)
+{
+    *reinterpret_cast<volatile uint32_t *>(&sh->sink[(threadIdx.x >> 5) & 31]) = dep;
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) mbar_arrive(smem_addr(&sh->empty[stage]));
+}
+__device__ __forceinline__ uint32_t dep_bits(float4 a) { return __float_as_uint(a.x); }
+__device__ __forceinline__ uint32_t dep_bits(float4 a, float4 b) { return __float_as_uint(a.x) ^ __float_as_uint(b.x); }
+__device__ __forceinline__ uint32_t dep_bits(float4 a, float4 b, float4 c, float4 d)
+{
+    return __float_as_uint(a.x) ^ __float_as_uint(b.x) ^ __float_as_uint(c.x) ^ __float_as_uint(d.x);
 }
 
 // Sum over the 512 consumers in binary64; every consumer gets the same value.
