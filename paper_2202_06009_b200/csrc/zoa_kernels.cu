@@ -417,7 +417,7 @@ __global__ void step_sync_kernel(StateView st, GradPtrs g, Consts c, float gamma
 // All of a block's loads go out before the first barrier: the chunk's words of every worker into
 // shared memory (eight independent loads per thread at a time), the server errors into registers.
 template <int ITER>
-__global__ void __launch_bounds__(512) dist_server_kernel(StateView st, const uint32_t *words_in, long long words_in_stride,
+__global__ void __launch_bounds__(ITER > 4 ? 512 : 256, ITER > 4 ? 2 : 4) dist_server_kernel(StateView st, const uint32_t *words_in, long long words_in_stride,
                                    const float *scales_in, long long scales_in_stride, int W_total,
                                    long long first_chunk, PeerOut out, float *z_bar)
 {
@@ -1252,7 +1252,7 @@ cudaError_t launch_dist_server(const StateView &st, const uint32_t *words_in, lo
                                const float *scales_in, long long scales_in_stride, int W_total,
                                long long first_chunk, long long count, const PeerOut &out, float *z_bar, cudaStream_t s)
 {
-    // 16 coordinates per thread (32 above chunk 4096), like compress_kernel
+    // 16 coordinates per thread (32 above chunk 4096), like compress_kernel (32 per thread at chunk 4096 measured worse)
     const int iter = st.chunk > 4096 ? 8 : 4;
     const int thr = ((st.chunk + 4 * iter - 1) / (4 * iter) + 31) / 32 * 32;
     const size_t smem = 34 * sizeof(double) + kMaxWorkers * sizeof(float) + (size_t)W_total * (st.chunk / 32) * sizeof(uint32_t);
