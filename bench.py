@@ -359,7 +359,7 @@ def run_ours(args, wl):
                  "two_call_sync": "local_step_kernel + compress_kernel + " + ("reduce_pipelined_kernel" if uses_ring else "reduce_kernel"),
                  "alg2_compressed": "alg2_pipelined_kernel" if alg2_ring else "alg2_compressed_kernel",
                  "alg2_full": "alg2_full_kernel"}
-    roofline = {"bound": "hbm", "kernel": kernel_of.get(dominant, "local_step_kernel"),
+    roofline = {"bound": "hbm", "kernel": kernel_of.get(dominant, "local_step_pipelined_kernel" if uses_ring else "local_step_kernel"),
                 "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "peak_kind": f"of {peak_kind}", "frac_of_8TBps_nominal": achieved / 8000.0,
                 # ncu (dram__bytes_read.sum + dram__bytes_write.sum) on the layout shrunk 16x gave
