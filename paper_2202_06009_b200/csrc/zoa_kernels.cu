@@ -312,92 +312,109 @@ __global__ void __launch_bounds__(512) reduce_kernel(StateView st, Consts c, flo
     if (threadIdx.x == 0 && blockIdx.x % CS == 0) st.scales_s[chunk_id] = scale;
 }
 
-// A whole sync step for chunk blockIdx.x: the local updates in registers, worker
+// A whole sync step for chunk chunk_offset + blockIdx.x: the local updates in registers, worker
 // compression, server, the post-sync updates.  The half-step m, x, u never reach memory;
-// x is not even read (the model sync rebuilds it from x_sync).
+// x is not even read (the model sync rebuilds it from x_sync).  Takes every shape: ragged last
+// chunk, unaligned or 16-bit gradients, any chunk that is a multiple of 32 up to 16384.
+// Thread t takes the float4 groups t, t + blockDim, ... (ITER of them) of every worker in turn:
+// loads in batches of two groups (eight 128-bit loads in flight), z in registers across the block
+// sum; each worker's sign words stay in shared memory and the server part rebuilds the mean from
+// them in worker order, so nothing per coordinate is kept between workers.
 // GFMT as in local_step_kernel (aligned binary32 at compile time, or -1 for the argument).
-template <int GFMT>
-__global__ void step_sync_kernel(StateView st, GradPtrs g, Consts c, float gamma, float gamma_sum,
-                                 int g_fmt_arg, long long chunk_offset)
+template <int ITER, int GFMT>
+__global__ void __launch_bounds__(ITER > 4 ? 512 : 256, ITER > 4 ? 2 : 4)
+step_sync_kernel(StateView st, GradPtrs g, Consts c, float gamma, float gamma_sum, int g_fmt_arg, long long chunk_offset)
 {
     const int g_aligned = GFMT >= 0 ? GFMT : g_fmt_arg;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     double *scratch = reinterpret_cast<double *>(smem_raw);                      // 34 doubles
-    double *A_s = scratch + 34;                                                  // [chunk]
-    float *z_s = reinterpret_cast<float *>(A_s + st.chunk);                      // [chunk]
+    float *scales = reinterpret_cast<float *>(smem_raw + 34 * sizeof(double));   // kMaxWorkers floats
+    uint32_t *bits_sm = reinterpret_cast<uint32_t *>(scales + kMaxWorkers);      // [W][chunk / 32]
     const long long chunk_id = chunk_offset + blockIdx.x;
     const ChunkGeom cg = chunk_geom(st, chunk_id);
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int words_per_chunk = st.chunk >> 5;
+    constexpr int BATCH = ITER < 2 ? 1 : 2;
 
-    for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
-        const int idx = base + 4 * lane;
-        if (idx < cg.len) { A_s[idx] = 0.0; A_s[idx + 1] = 0.0; A_s[idx + 2] = 0.0; A_s[idx + 3] = 0.0; }
-    }
     for (int i = 0; i < st.W; ++i) {
         const long long row = (long long)i * st.n_pad + cg.c0;
         const float *gi = g.p[i];
+        float z[ITER][4];
         double l1 = 0.0;
-        for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
-            const int idx = base + 4 * lane;
-            if (idx < cg.len) {
-                const float4 g4 = ld_grad4(gi, cg.c0 + idx, st.n, g_aligned);
-                const float4 m4 = ld4_stream(st.m + row + idx), u4 = ld4_stream(st.u + row + idx);
-                const float4 e4 = ld4_stream(st.dw + row + idx);
-                const float gg[4] = {g4.x, g4.y, g4.z, g4.w}, mm[4] = {m4.x, m4.y, m4.z, m4.w};
-                const float uu[4] = {u4.x, u4.y, u4.z, u4.w}, ee[4] = {e4.x, e4.y, e4.z, e4.w};
-                float z[4];
+#pragma unroll
+        for (int h = 0; h < ITER; h += BATCH) {
+            float4 g4[BATCH], m4[BATCH], u4[BATCH], e4[BATCH];
+#pragma unroll
+            for (int q = 0; q < BATCH; ++q) {
+                const int idx = 4 * ((h + q) * blockDim.x + threadIdx.x);
+                const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+                g4[q] = idx < cg.len ? ld_grad4(gi, cg.c0 + idx, st.n, g_aligned) : zero;
+                m4[q] = idx < cg.len ? ld4_stream(st.m + row + idx) : zero;
+                u4[q] = idx < cg.len ? ld4_stream(st.u + row + idx) : zero;
+                e4[q] = idx < cg.len ? ld4_stream(st.dw + row + idx) : zero;
+            }
+#pragma unroll
+            for (int q = 0; q < BATCH; ++q) {
+                const float gg[4] = {g4[q].x, g4[q].y, g4[q].z, g4[q].w}, mm[4] = {m4[q].x, m4[q].y, m4[q].z, m4[q].w};
+                const float uu[4] = {u4[q].x, u4[q].y, u4[q].z, u4[q].w}, ee[4] = {e4[q].x, e4[q].y, e4[q].z, e4[q].w};
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
-                    const float s = f_mul(gamma, momentum(c, mm[k], gg[k]));     // momentum update, buffer update
-                    z[k] = f_add(f_add(uu[k], s), ee[k]);                        // u_{t+1/2} + delta
-                    l1 += fabs((double)z[k]);
+                    const float step = f_mul(gamma, momentum(c, mm[k], gg[k]));     // momentum update, buffer update
+                    z[h + q][k] = f_add(f_add(uu[k], step), ee[k]);                 // u_{t+1/2} + delta
+                    l1 += fabs((double)z[h + q][k]);
                 }
-                st4(z_s + idx, make_float4(z[0], z[1], z[2], z[3]));
             }
         }
         const float scale = chunk_scale(block_sum(l1, scratch), cg.len);
-        for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
-            const int idx = base + 4 * lane;
-            float z[4] = {0.f, 0.f, 0.f, 0.f}, hat[4];
-            if (idx < cg.len) {
-                const float4 z4 = ld4(z_s + idx);
-                z[0] = z4.x; z[1] = z4.y; z[2] = z4.z; z[3] = z4.w;
-            }
-            const uint32_t word = compress_tile(z, hat, scale, idx, cg.len);
-            if (idx < cg.len) {
-                st4_stream(st.dw + row + idx, make_float4(z[0], z[1], z[2], z[3]));
 #pragma unroll
-                for (int k = 0; k < 4; ++k) A_s[idx + k] += (double)hat[k];      // worker order
-            }
-            if (lane < 4 && base + 32 * lane < cg.len)
+        for (int it = 0; it < ITER; ++it) {
+            const int idx = 4 * (it * blockDim.x + threadIdx.x);
+            const int base = idx - 4 * lane;                   // first coordinate of the warp's 128
+            float hat[4];
+            const uint32_t word = compress_tile(z[it], hat, scale, idx, cg.len);
+            if (idx < cg.len) st4_stream(st.dw + row + idx, make_float4(z[it][0], z[it][1], z[it][2], z[it][3]));
+            if (lane < 4 && base + 32 * lane < cg.len) {
                 st.words_w[(long long)i * st.words_stride + ((cg.c0 + base) >> 5) + lane] = word;
-        }
-        if (threadIdx.x == 0) st.scales_w[(long long)i * st.n_chunks + chunk_id] = scale;
-    }
-    double l1 = 0.0;
-    for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
-        const int idx = base + 4 * lane;
-        if (idx < cg.len) {
-            const float4 e4 = ld4(st.ds + cg.c0 + idx);
-            const float ee[4] = {e4.x, e4.y, e4.z, e4.w};
-            float a[4];
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                a[k] = idx + k < cg.len ? server_input(A_s[idx + k], st.W, ee[k]) : 0.0f;
-                l1 += fabs((double)a[k]);
+                bits_sm[i * words_per_chunk + (base >> 5) + lane] = word;
             }
-            st4(z_s + idx, make_float4(a[0], a[1], a[2], a[3]));
+        }
+        if (threadIdx.x == 0) {
+            st.scales_w[(long long)i * st.n_chunks + chunk_id] = scale;
+            scales[i] = scale;
+        }
+    }
+    __syncthreads();      // every worker's words and magnitude are in shared memory
+
+    // ---- server: mean of the compressed buffers + server error, compress again, post-sync rows ----
+    float a[ITER][4];
+    double l1 = 0.0;
+#pragma unroll
+    for (int it = 0; it < ITER; ++it) {
+        const int idx = 4 * (it * blockDim.x + threadIdx.x);
+        double A[4] = {0.0, 0.0, 0.0, 0.0};
+        float4 e4 = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (idx < cg.len) {
+            e4 = ld4(st.ds + cg.c0 + idx);
+            const int shift = idx & 31;
+            for (int i = 0; i < st.W; ++i) {   // worker order
+                const uint32_t nib = bits_sm[i * words_per_chunk + (idx >> 5)] >> shift;
+                const double sc = (double)scales[i];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) A[k] += ((nib >> k) & 1u) ? sc : -sc;
+            }
+        }
+        const float ee[4] = {e4.x, e4.y, e4.z, e4.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            a[it][k] = idx + k < cg.len ? server_input(A[k], st.W, ee[k]) : 0.0f;
+            l1 += fabs((double)a[it][k]);
         }
     }
     const float scale = chunk_scale(block_sum(l1, scratch), cg.len);
-    for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
-        const int idx = base + 4 * lane;
-        float a[4] = {0.f, 0.f, 0.f, 0.f};
-        if (idx < cg.len) {
-            const float4 a4 = ld4(z_s + idx);
-            a[0] = a4.x; a[1] = a4.y; a[2] = a4.z; a[3] = a4.w;
-        }
-        server_tile(st, c, cg, base, lane, a, scale, gamma_sum);
+#pragma unroll
+    for (int it = 0; it < ITER; ++it) {
+        const int idx = 4 * (it * blockDim.x + threadIdx.x);
+        server_tile(st, c, cg, idx - 4 * lane, lane, a[it], scale, gamma_sum);
     }
     if (threadIdx.x == 0) st.scales_s[chunk_id] = scale;
 }
@@ -657,83 +674,102 @@ alg2_full_kernel(StateView st, GradPtrs g, Consts c, float gamma, int g_fmt_arg)
     }
 }
 
-// Any other step of Algorithm 2 for chunk blockIdx.x (Compressed-AllReduce, momentum, model): the
-// gradients go through the error-feedback 1-bit AllReduce (Algorithm 3), the
-// decompressed mean drives momentum and model on every worker.
-__global__ void __launch_bounds__(512, 2) alg2_compressed_kernel(StateView st, GradPtrs g, Consts c, float gamma, int g_aligned, long long chunk_offset)
+// Any other step of Algorithm 2 for chunk chunk_offset + blockIdx.x (Compressed-AllReduce,
+// momentum, model): the gradients go through the error-feedback 1-bit AllReduce (Algorithm 3),
+// the decompressed mean drives momentum and model on every worker.  Same shape as
+// step_sync_kernel: z in registers, the workers' sign words and magnitudes in shared memory.
+template <int ITER>
+__global__ void __launch_bounds__(ITER > 4 ? 512 : 256, ITER > 4 ? 2 : 4)
+alg2_compressed_kernel(StateView st, GradPtrs g, Consts c, float gamma, int g_aligned, long long chunk_offset)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    double *scratch = reinterpret_cast<double *>(smem_raw);
-    double *A_s = scratch + 34;
-    float *z_s = reinterpret_cast<float *>(A_s + st.chunk);
+    double *scratch = reinterpret_cast<double *>(smem_raw);                      // 34 doubles
+    float *scales = reinterpret_cast<float *>(smem_raw + 34 * sizeof(double));   // kMaxWorkers floats
+    uint32_t *bits_sm = reinterpret_cast<uint32_t *>(scales + kMaxWorkers);      // [W][chunk / 32]
     const long long chunk_id = chunk_offset + blockIdx.x;
     const ChunkGeom cg = chunk_geom(st, chunk_id);
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int words_per_chunk = st.chunk >> 5;
+    constexpr int BATCH = 4;
 
-    for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
-        const int idx = base + 4 * lane;
-        if (idx < cg.len) { A_s[idx] = 0.0; A_s[idx + 1] = 0.0; A_s[idx + 2] = 0.0; A_s[idx + 3] = 0.0; }
-    }
     for (int i = 0; i < st.W; ++i) {
         const long long row = (long long)i * st.n_pad + cg.c0;
+        const float *gi = g.p[i];
+        float z[ITER][4];
         double l1 = 0.0;
-        for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
-            const int idx = base + 4 * lane;
-            if (idx < cg.len) {
-                const float4 g4 = ld_grad4(g.p[i], cg.c0 + idx, st.n, g_aligned);
-                const float4 e4 = ld4_stream(st.dw + row + idx);
-                const float4 z4 = make_float4(f_add(g4.x, e4.x), f_add(g4.y, e4.y), f_add(g4.z, e4.z), f_add(g4.w, e4.w));
-                st4(z_s + idx, z4);
-                l1 += fabs((double)z4.x) + fabs((double)z4.y) + fabs((double)z4.z) + fabs((double)z4.w);
+#pragma unroll
+        for (int h = 0; h < ITER; h += BATCH) {
+            float4 g4[BATCH], e4[BATCH];
+#pragma unroll
+            for (int q = 0; q < BATCH; ++q) {
+                const int idx = 4 * ((h + q) * blockDim.x + threadIdx.x);
+                const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+                g4[q] = idx < cg.len ? ld_grad4(gi, cg.c0 + idx, st.n, g_aligned) : zero;
+                e4[q] = idx < cg.len ? ld4_stream(st.dw + row + idx) : zero;
+            }
+#pragma unroll
+            for (int q = 0; q < BATCH; ++q) {
+                z[h + q][0] = f_add(g4[q].x, e4[q].x); z[h + q][1] = f_add(g4[q].y, e4[q].y);
+                z[h + q][2] = f_add(g4[q].z, e4[q].z); z[h + q][3] = f_add(g4[q].w, e4[q].w);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) l1 += fabs((double)z[h + q][k]);
             }
         }
         const float scale = chunk_scale(block_sum(l1, scratch), cg.len);
-        for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
-            const int idx = base + 4 * lane;
-            float z[4] = {0.f, 0.f, 0.f, 0.f}, hat[4];
-            if (idx < cg.len) {
-                const float4 z4 = ld4(z_s + idx);
-                z[0] = z4.x; z[1] = z4.y; z[2] = z4.z; z[3] = z4.w;
-            }
-            const uint32_t word = compress_tile(z, hat, scale, idx, cg.len);
-            if (idx < cg.len) {
-                st4_stream(st.dw + row + idx, make_float4(z[0], z[1], z[2], z[3]));
 #pragma unroll
-                for (int k = 0; k < 4; ++k) A_s[idx + k] += (double)hat[k];
-            }
-            if (lane < 4 && base + 32 * lane < cg.len)
+        for (int it = 0; it < ITER; ++it) {
+            const int idx = 4 * (it * blockDim.x + threadIdx.x);
+            const int base = idx - 4 * lane;
+            float hat[4];
+            const uint32_t word = compress_tile(z[it], hat, scale, idx, cg.len);
+            if (idx < cg.len) st4_stream(st.dw + row + idx, make_float4(z[it][0], z[it][1], z[it][2], z[it][3]));
+            if (lane < 4 && base + 32 * lane < cg.len) {
                 st.words_w[(long long)i * st.words_stride + ((cg.c0 + base) >> 5) + lane] = word;
-        }
-        if (threadIdx.x == 0) st.scales_w[(long long)i * st.n_chunks + chunk_id] = scale;
-    }
-    double l1 = 0.0;
-    for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
-        const int idx = base + 4 * lane;
-        if (idx < cg.len) {
-            const float4 e4 = ld4(st.ds + cg.c0 + idx);
-            const float ee[4] = {e4.x, e4.y, e4.z, e4.w};
-            float a[4];
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                a[k] = idx + k < cg.len ? server_input(A_s[idx + k], st.W, ee[k]) : 0.0f;
-                l1 += fabs((double)a[k]);
+                bits_sm[i * words_per_chunk + (base >> 5) + lane] = word;
             }
-            st4(z_s + idx, make_float4(a[0], a[1], a[2], a[3]));
+        }
+        if (threadIdx.x == 0) {
+            st.scales_w[(long long)i * st.n_chunks + chunk_id] = scale;
+            scales[i] = scale;
+        }
+    }
+    __syncthreads();
+
+    float a[ITER][4];
+    double l1 = 0.0;
+#pragma unroll
+    for (int it = 0; it < ITER; ++it) {
+        const int idx = 4 * (it * blockDim.x + threadIdx.x);
+        double A[4] = {0.0, 0.0, 0.0, 0.0};
+        float4 e4 = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (idx < cg.len) {
+            e4 = ld4(st.ds + cg.c0 + idx);
+            const int shift = idx & 31;
+            for (int i = 0; i < st.W; ++i) {   // worker order
+                const uint32_t nib = bits_sm[i * words_per_chunk + (idx >> 5)] >> shift;
+                const double sc = (double)scales[i];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) A[k] += ((nib >> k) & 1u) ? sc : -sc;
+            }
+        }
+        const float ee[4] = {e4.x, e4.y, e4.z, e4.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            a[it][k] = idx + k < cg.len ? server_input(A[k], st.W, ee[k]) : 0.0f;
+            l1 += fabs((double)a[it][k]);
         }
     }
     const float scale = chunk_scale(block_sum(l1, scratch), cg.len);
-    for (int base = warp * 128; base < cg.len; base += n_warps * 128) {
-        const int idx = base + 4 * lane;
-        float a[4] = {0.f, 0.f, 0.f, 0.f}, gb[4];
-        if (idx < cg.len) {
-            const float4 a4 = ld4(z_s + idx);
-            a[0] = a4.x; a[1] = a4.y; a[2] = a4.z; a[3] = a4.w;
-        }
-        const uint32_t word = compress_tile(a, gb, scale, idx, cg.len);   // gb = the mean gradient the workers receive
+#pragma unroll 1
+    for (int it = 0; it < ITER; ++it) {
+        const int idx = 4 * (it * blockDim.x + threadIdx.x);
+        const int base = idx - 4 * lane;
+        float gb[4];
+        const uint32_t word = compress_tile(a[it], gb, scale, idx, cg.len);   // gb = the mean gradient the workers receive
         if (lane < 4 && base + 32 * lane < cg.len) st.words_s[((cg.c0 + base) >> 5) + lane] = word;
         if (idx >= cg.len) continue;
         const long long j = cg.c0 + idx;
-        st4(st.ds + j, make_float4(a[0], a[1], a[2], a[3]));
+        st4(st.ds + j, make_float4(a[it][0], a[it][1], a[it][2], a[it][3]));
         const float4 v4 = ld4(st.v + j);
         const float d[4] = {denom(c, v4.x), denom(c, v4.y), denom(c, v4.z), denom(c, v4.w)};
         // four workers at a time: all eight loads are issued before the first dependent store
@@ -1016,18 +1052,6 @@ __global__ void __launch_bounds__(256) count_nonfinite_kernel(const float *p, lo
 // ---------------------------------------------------------------------------
 // Launchers
 // ---------------------------------------------------------------------------
-static int block_threads_for_chunk(int chunk)
-{
-    // 8 coordinates per thread up to 512 threads: measured best on B200 for chunk 4096
-    // and 8192 (1024-thread blocks lose a third of the bandwidth to barrier stalls).
-    int t = chunk / 8;
-    if (t < 128) t = 128;
-    if (t > 512) t = 512;
-    int p = 128;
-    while (p < t) p <<= 1;
-    return p;
-}
-
 static int elementwise_grid(long long n4)
 {
     // One float4 per thread and as many blocks as that takes: SMs do not all get the same
@@ -1078,18 +1102,22 @@ static int cluster_blocks(int chunk)
     if (chunk > 4096 && chunk % 256 == 0) return 2;
     return 1;
 }
-size_t step_sync_smem(int chunk) { return 34 * sizeof(double) + (size_t)chunk * (sizeof(double) + sizeof(float)); }
+// step_sync_kernel, alg2_compressed_kernel: block-sum scratch, the workers' magnitudes and sign words
+static size_t step_sync_bits_smem(int W, int chunk) { return 34 * sizeof(double) + kMaxWorkers * sizeof(float) + (size_t)W * (chunk / 32) * sizeof(uint32_t); }
 
 cudaError_t configure_kernels()
 {
     cudaError_t e;
     e = cudaFuncSetAttribute(reduce_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)reduce_span_smem(kMaxChunk));
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(alg2_compressed_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)step_sync_smem(kMaxChunk));
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(step_sync_kernel<kGradF32 | kGradAligned>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)step_sync_smem(kMaxChunk));
-    if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(step_sync_kernel<-1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)step_sync_smem(kMaxChunk));
+    const int sync_smem = (int)step_sync_bits_smem(kMaxWorkers, kMaxChunk);
+    e = cudaFuncSetAttribute(alg2_compressed_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, sync_smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(alg2_compressed_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, sync_smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(step_sync_kernel<4, kGradF32 | kGradAligned>, cudaFuncAttributeMaxDynamicSharedMemorySize, sync_smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(step_sync_kernel<8, kGradF32 | kGradAligned>, cudaFuncAttributeMaxDynamicSharedMemorySize, sync_smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(step_sync_kernel<4, -1>, cudaFuncAttributeMaxDynamicSharedMemorySize, sync_smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(step_sync_kernel<8, -1>, cudaFuncAttributeMaxDynamicSharedMemorySize, sync_smem);
+    return e;
 }
 
 // A step of Algorithm 2: the whole vector at full precision, or the chunks
@@ -1105,9 +1133,13 @@ cudaError_t launch_alg2(const StateView &st, const GradPtrs &g, const Consts &c,
         case kGradBF16 | kGradAligned: alg2_full_kernel<kGradBF16 | kGradAligned><<<grid, 256, 0, s>>>(st, g, c, gamma, g_aligned); break;
         default: alg2_full_kernel<-1><<<grid, 256, 0, s>>>(st, g, c, gamma, g_aligned); break;
         }
-    } else
-        alg2_compressed_kernel<<<(unsigned)count, block_threads_for_chunk(st.chunk), step_sync_smem(st.chunk), s>>>(
-            st, g, c, gamma, g_aligned, first_chunk);
+    } else {
+        const int iter = st.chunk > 4096 ? 8 : 4;
+        const int threads = ((st.chunk + 4 * iter - 1) / (4 * iter) + 31) / 32 * 32;
+        const size_t smem = step_sync_bits_smem(st.W, st.chunk);
+        if (iter == 8) alg2_compressed_kernel<8><<<(unsigned)count, threads, smem, s>>>(st, g, c, gamma, g_aligned, first_chunk);
+        else alg2_compressed_kernel<4><<<(unsigned)count, threads, smem, s>>>(st, g, c, gamma, g_aligned, first_chunk);
+    }
     return cudaGetLastError();
 }
 
@@ -1181,14 +1213,15 @@ cudaError_t launch_reduce(const StateView &st, const Consts &c, float gamma_sum,
 cudaError_t launch_step_sync(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
                              float gamma_sum, int g_aligned, long long first_chunk, long long count, cudaStream_t s)
 {
-    // Above 8192 coordinates the chunk's shared memory leaves room for one block per SM only, and
-    // 1024 threads then beat 512 (chunk 16384, BERT-Large-shaped: 33.9 against 40.0 ms).
-    const int threads = st.chunk > 8192 ? 1024 : block_threads_for_chunk(st.chunk);
-    const size_t smem = step_sync_smem(st.chunk);
-    if (g_aligned == (kGradF32 | kGradAligned))
-        step_sync_kernel<kGradF32 | kGradAligned><<<(unsigned)count, threads, smem, s>>>(st, g, c, gamma, gamma_sum, g_aligned, first_chunk);
-    else
-        step_sync_kernel<-1><<<(unsigned)count, threads, smem, s>>>(st, g, c, gamma, gamma_sum, g_aligned, first_chunk);
+    // 16 coordinates per thread (32 above chunk 4096), like compress_kernel
+    const int iter = st.chunk > 4096 ? 8 : 4;
+    const int threads = ((st.chunk + 4 * iter - 1) / (4 * iter) + 31) / 32 * 32;
+    const size_t smem = step_sync_bits_smem(st.W, st.chunk);
+    const bool fast = g_aligned == (kGradF32 | kGradAligned);
+#define ZOA_SYNC(IT, FMT) step_sync_kernel<IT, FMT><<<(unsigned)count, threads, smem, s>>>(st, g, c, gamma, gamma_sum, g_aligned, first_chunk)
+    if (iter == 8) { if (fast) ZOA_SYNC(8, kGradF32 | kGradAligned); else ZOA_SYNC(8, -1); }
+    else { if (fast) ZOA_SYNC(4, kGradF32 | kGradAligned); else ZOA_SYNC(4, -1); }
+#undef ZOA_SYNC
     return cudaGetLastError();
 }
 

@@ -21,7 +21,7 @@
 
 namespace zoa {
 
-// A work unit is TILES tiles of 2048 coordinates: one chunk of 2048 ... 16384 coordinates (G = 1), or
+// A work unit is TILES tiles of 2048 coordinates: one chunk of 2048, 4096 or 8192 coordinates (G = 1), or
 // one tile holding G = 2048 / chunk whole chunks of 128 ... 1024 coordinates (TILES = 1), in which
 // case a chunk's l1 norm is the sum over the 16 / G consumer warps that own it.
 template <int TILES, int G, bool DO_VAR>
@@ -29,10 +29,8 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
 {
     constexpr int WPC = kConsumerWarps / G;          // consumer warps per chunk
     constexpr long long kSpan = (long long)TILES * kTile;
-    // The server needs a unit's server errors before the l1 sum and its v and x_sync after it.  Up to four
-    // tiles stay in the ring over the sum; eight would fill it, so they travel twice: the errors
-    // first, each stage released as soon as it is read, then v and x_sync.
-    constexpr bool SERVER_TWO_PASS = TILES > 4;
+    // The server needs a unit's server errors before the l1 sum and its v and x_sync after it: the
+    // unit's (at most four) server tiles stay in the ring over the sum.
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     PipeShared *sh = reinterpret_cast<PipeShared *>(smem_raw);
     const StateView &st = a.st;
@@ -72,25 +70,12 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
                         bulk_load(dst + kTileBytes, st.m + row, kTileBytes, full);
                         bulk_load(dst + 2 * kTileBytes, st.u + row, kTileBytes, full);
                         bulk_load(dst + 3 * kTileBytes, st.dw + row, kTileBytes, full);
-                    } else if (!SERVER_TWO_PASS) {
+                    } else {
                         mbar_arrive_expect_tx(full, 3 * kTileBytes);
                         bulk_load(dst, st.ds + off, kTileBytes, full);
                         bulk_load(dst + kTileBytes, st.v + off, kTileBytes, full);
                         bulk_load(dst + 2 * kTileBytes, st.xs + off, kTileBytes, full);
-                    } else {
-                        mbar_arrive_expect_tx(full, kTileBytes);
-                        bulk_load(dst, st.ds + off, kTileBytes, full);
                     }
-                    p.advance();
-                }
-            }
-            if (SERVER_TWO_PASS) {      // v and x_sync follow once the server errors have gone through
-                for (int t = 0; t < TILES && p.stage_free(); ++t) {
-                    const uint32_t full = p.full_barrier(), dst = p.stage_addr();
-                    const long long off = c0 + (long long)t * kTile;
-                    mbar_arrive_expect_tx(full, 2 * kTileBytes);
-                    bulk_load(dst + kTileBytes, st.v + off, kTileBytes, full);
-                    bulk_load(dst + 2 * kTileBytes, st.xs + off, kTileBytes, full);
                     p.advance();
                 }
             }
@@ -112,17 +97,16 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
     // spread over the worker iterations of the next chunk (one worker's m, x, u after
     // each worker's compression) instead of leaving in one burst, so that the block's
     // stores and its ring's loads stay evenly mixed.  m is +-m_pos by the server's bit.
-    // With eight tiles the tiles of x have no room in the registers (17 warps leave 96 per thread: one SM
-    // sub-partition hosts five of them): that variant stores at once.
-    constexpr bool DEFER = TILES <= 4;
-    float x_prev[DEFER ? TILES : 1][4];
+    // (Four tiles of x are what fits: 17 warps leave 96 registers per thread, since one SM
+    // sub-partition hosts five of them.)
+    float x_prev[TILES][4];
     uint32_t bits_prev = 0;
     float m_pos_prev = 0.0f;
     long long c0_prev = -1;
     auto store_prev_worker = [&](int i) {
         const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int t = 0; t < (DEFER ? TILES : 0); ++t) {
+        for (int t = 0; t < TILES; ++t) {
             const long long row = (long long)i * st.n_pad + c0_prev + t * kTile + pos;
             const uint32_t nib = bits_prev >> (4 * t);
             st4_stream(st.m + row, make_float4((nib & 1u) ? m_pos_prev : -m_pos_prev, (nib & 2u) ? m_pos_prev : -m_pos_prev,
@@ -202,7 +186,7 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
             }
             if (lane == 0) my_scales[i] = scale;
             if (scale_writer) st.scales_w[(long long)i * st.n_chunks + scale_idx] = scale;
-            if (DEFER && c0_prev >= 0) store_prev_worker(i);
+            if (c0_prev >= 0) store_prev_worker(i);
         }
         __syncwarp();   // bits_s and my_scales were written by lanes of this warp
 
@@ -216,7 +200,6 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
             srv_stage[t] = s;
             const float *stage = reinterpret_cast<const float *>(ring + (size_t)s * kStageBytes);
             const float4 d4 = ready ? ld4(stage + pos) : make_float4(0.f, 0.f, 0.f, 0.f);
-            if (SERVER_TWO_PASS) release_stage(sh, s, dep_bits(d4));
             if (++s == R) { s = 0; phase ^= 1u; }
             const float dd[4] = {d4.x, d4.y, d4.z, d4.w};
             double A[4] = {0.0, 0.0, 0.0, 0.0};
@@ -236,11 +219,6 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
         const float scale = chunk_scale(consumer_group_sum<WPC>(l1, sh, flip), st.chunk);
 #pragma unroll
         for (int t = 0; t < TILES; ++t) {
-            if (SERVER_TWO_PASS) {
-                mbar_wait(smem_addr(&sh->full[s]), phase, abort_flag, a.error_flag, a.wait_limit_ns);
-                srv_stage[t] = s;
-                if (++s == R) { s = 0; phase ^= 1u; }
-            }
             const float *stage = reinterpret_cast<const float *>(ring + (size_t)srv_stage[t] * kStageBytes);
             const float4 v4 = ld4(stage + kTile + pos), xs4 = ld4(stage + 2 * kTile + pos);
             release_stage(sh, srv_stage[t], dep_bits(v4, xs4));
@@ -254,28 +232,14 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
                 const float hat = b[k] ? scale : -scale;
                 e[k] = f_sub(av[t][k], hat);
                 xo[k] = f_sub(xs[k], f_div(hat, denom(a.c, vv[k])));           // model sync
-                if (DEFER) {
-                    x_prev[t][k] = xo[k];
-                    bits_prev |= (b[k] ? 1u : 0u) << (4 * t + k);
-                }
+                x_prev[t][k] = xo[k];
+                bits_prev |= (b[k] ? 1u : 0u) << (4 * t + k);
             }
             const long long j = c0 + t * kTile + pos;
             const uint32_t word = pack_group(b);
             if (group_leader) st.words_s[((c0 + t * kTile) >> 5) + word_in_tile] = word;
             st4_stream(st.ds + j, make_float4(e[0], e[1], e[2], e[3]));
             st4_stream(st.xs + j, make_float4(xo[0], xo[1], xo[2], xo[3]));
-            if (!DEFER) {
-                const float mp = f_div(scale, a.gamma_sum);                    // momentum approximation
-                const float4 m4 = make_float4(b[0] ? mp : -mp, b[1] ? mp : -mp, b[2] ? mp : -mp, b[3] ? mp : -mp);
-                const float4 x4 = make_float4(xo[0], xo[1], xo[2], xo[3]);
-                const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
-                for (int i = 0; i < W; ++i) {
-                    const long long row = (long long)i * st.n_pad + j;
-                    st4_stream(st.m + row, m4);
-                    st4_stream(st.x + row, x4);
-                    st4_stream(st.u + row, zero);                              // buffer reset
-                }
-            }
             if (DO_VAR) {
                 float vo[4];
 #pragma unroll
@@ -286,10 +250,8 @@ __global__ void __launch_bounds__(kThreads, 1) step_sync_pipelined_kernel(const 
                 st4_stream(st.v_next + j, make_float4(vo[0], vo[1], vo[2], vo[3]));
             }
         }
-        if (DEFER) {
-            m_pos_prev = f_div(scale, a.gamma_sum);     // momentum approximation: m = +-scale / sum(gamma); -(s/G) == (-s)/G exactly
-            c0_prev = c0;
-        }
+        m_pos_prev = f_div(scale, a.gamma_sum);     // momentum approximation: m = +-scale / sum(gamma); -(s/G) == (-s)/G exactly
+        c0_prev = c0;
         if (scale_writer) st.scales_s[scale_idx] = scale;
         __syncwarp();   // the next chunk overwrites bits_s / my_scales of this warp
     }
@@ -602,7 +564,9 @@ static bool unit_shape(int chunk, int *tiles, int *chunks_per_tile)
     if (chunk >= kTile) {
         if (chunk % kTile != 0) return false;
         *tiles = chunk / kTile;
-        return *tiles == 1 || *tiles == 2 || *tiles == 4 || *tiles == 8;
+        // eight tiles (chunk 16384) would fill the ring and leave no registers for the deferred
+        // stores: the chunk-per-block kernel is the faster one there
+        return *tiles == 1 || *tiles == 2 || *tiles == 4;
     }
     if (chunk < 128 || kTile % chunk != 0) return false;
     *chunks_per_tile = kTile / chunk;      // 2, 4, 8 or 16: whole warps per chunk
@@ -625,8 +589,8 @@ int pipeline_stages(const StateView &st, int grad_fmt)
     if (st.n / ((long long)tiles * kTile) < 1) return 0;
     const size_t budget = 227 * 1024;
     const size_t fixed = pipeline_fixed_smem(st.W, st.chunk);
-    // up to four server tiles of a unit stay in the ring over the l1 sum: tiles + 1 stages at least
-    const int least = tiles <= 4 ? tiles + 1 : 4;
+    // the server tiles of a unit stay in the ring over the l1 sum: tiles + 1 stages at least
+    const int least = tiles + 1;
     if (fixed + (size_t)least * kStageBytes > budget) return 0;
     int stages = (int)((budget - fixed) / kStageBytes);
     if (stages > kSyncStages) stages = kSyncStages;
@@ -668,7 +632,6 @@ cudaError_t launch_step_sync_pipelined(const StateView &st, const GradPtrs &g, c
     const int grid = (int)(n_units < sm_count ? n_units : sm_count);
     int tiles, cpt;
     if (!unit_shape(st.chunk, &tiles, &cpt)) return cudaErrorInvalidValue;
-    if (tiles == 8) do_var = false;       // eight tiles of binary64 gradient sums have no room in the registers
     size_t fixed = pipeline_fixed_smem(st.W, st.chunk);
     if (tiles == 4 && do_var) {           // two tiles of gradient sums in shared memory; the ring gives up a stage for them
         fixed += 2 * 4 * kConsumers * sizeof(double);
@@ -684,7 +647,6 @@ cudaError_t launch_step_sync_pipelined(const StateView &st, const GradPtrs &g, c
     case 101: return ZOA_PIPE(1, 1);
     case 201: return ZOA_PIPE(2, 1);
     case 401: return ZOA_PIPE(4, 1);
-    case 801: return launch_pipe<8, 1, false>(a, grid, smem, s);
     case 102: return ZOA_PIPE(1, 2);
     case 104: return ZOA_PIPE(1, 4);
     case 108: return ZOA_PIPE(1, 8);

@@ -87,9 +87,10 @@ def test_fused_equals_two_call_bit_for_bit():
 def test_pipelined_kernel_equals_chunk_per_block_kernel(W, chunk, n_chunks, tail):
     """The bulk-copy ring kernel and the chunk-per-block kernel give the same bits,
     over enough chunks that every block wraps its ring many times; steps with and
-    without the fused variance update.  Chunks of 2048 ... 16384 coordinates are units of one
-    to eight tiles; chunks of 128 ... 1024 share a tile, and the whole chunks that do not fill
-    the last tile go to the chunk-per-block kernel with the ragged tail."""
+    without the fused variance update.  Chunks of 2048, 4096 and 8192 coordinates are units of one,
+    two and four tiles; chunks of 128 ... 1024 share a tile, and the whole chunks that do not fill
+    the last tile go to the chunk-per-block kernel with the ragged tail.  (Chunk 16384 has no ring
+    variant: both handles run the chunk-per-block kernel.)"""
     rng = np.random.default_rng(W + chunk)
     n = n_chunks * chunk + tail
     x0 = torch.from_numpy((rng.standard_normal(n) * 0.02).astype(np.float32))
@@ -477,15 +478,15 @@ def test_policies_match_the_workload_tables():
         z.close()
 
 
-@pytest.mark.parametrize("algorithm", ["alg1", "alg2", "two_call", "alg1_chunk_1024", "alg1_chunk_16384"])
+@pytest.mark.parametrize("algorithm", ["alg1", "alg2", "two_call", "alg1_chunk_1024", "alg1_chunk_8192"])
 def test_device_wait_runs_out_and_is_reported(algorithm):
     """Error path of the ring kernels without any fault: the copy-issuing lane of every block
     stops after three tiles (test hook), the other threads' bounded waits run out after
     100 ms, the kernel ends by itself, zoa_check_device reports ZOA_ERR_DEVICE, and the
-    context and the handle stay usable.  Covers the fused kernel (one, two and eight tiles per
+    context and the handle stay usable.  Covers the fused kernel (one, two and four tiles per
     unit), Algorithm 2's, and the server kernel of the two-call path with its store-issuing warp."""
     import time
-    chunk = 1024 if algorithm.endswith("1024") else 16384 if algorithm.endswith("16384") else 4096
+    chunk = 1024 if algorithm.endswith("1024") else 8192 if algorithm.endswith("8192") else 4096
     n, W = 300 * max(chunk, 2048), 4
     z = Zoa(n, W, chunk=chunk)
     try:
