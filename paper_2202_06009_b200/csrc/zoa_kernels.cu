@@ -431,90 +431,120 @@ step_sync_kernel(StateView st, GradPtrs g, Consts c, float gamma, float gamma_su
 // result itself to z_bar if that is not NULL (caller-owned, exactly n floats, any alignment).
 // `out` lists where else the packed result of the range is to be stored (every rank's
 // words_s / scales_s, peer pointers included); out.world == 0 for none.
-// All of a block's loads go out before the first barrier: the chunk's words of every worker into
-// shared memory (eight independent loads per thread at a time), the server errors into registers.
-template <int ITER>
-__global__ void __launch_bounds__(ITER > 4 ? 512 : 256, ITER > 4 ? 2 : 4) dist_server_kernel(StateView st, const uint32_t *words_in, long long words_in_stride,
-                                   const float *scales_in, long long scales_in_stride, int W_total,
-                                   long long first_chunk, PeerOut out, float *z_bar)
+//
+// With 12 to 14 bytes per coordinate this step is bound by instructions, not by memory, if the sum
+// over the workers is taken bit by bit (W selects and W additions per coordinate).  So the sum is
+// looked up: the workers are taken in groups of four, a group's sixteen possible signed sums
+// sit in a table in shared memory (128 bytes: one entry per pair of banks, so a lookup never
+// conflicts), a thread owns eight consecutive coordinates = one byte of every worker's words, and
+// one mask, one multiplication and one shift turn the four workers' bits of a coordinate into the
+// table offset.  Adding the groups' entries gives the bits of the worker-by-worker binary64 sum
+// whenever every partial sum is exact: all magnitudes are multiples of the smallest one's last
+// place, so it is enough that W * 2^(e_max + 1) stays below 2^53 of those units, i.e. that the
+// exponents of the non-zero magnitudes differ by at most 29 - ceil(log2 W) (checked per chunk;
+// with up to four workers the single table holds the sequential sum itself).  A chunk that fails
+// the check takes the worker-by-worker loop.
+constexpr uint32_t kGatherMul = 0x10204080u;   // 2^28 + 2^21 + 2^14 + 2^7: bits 0, 8, 16, 24 -> bits 28 ... 31
+
+// One chunk of dist_server_kernel.  FULL: the chunk has its full length and z_bar (if any) takes
+// 128-bit stores, so that no coordinate needs a bounds check.
+template <int ITER, bool FULL>
+__device__ __forceinline__ void server_chunk(const StateView &st, const uint32_t *words_in, long long words_in_stride, int W_total,
+                                          long long chunk_word0, const PeerOut &out, float *z_bar, bool z_bar_aligned, const ChunkGeom cg, long long chunk_id,
+                                          double *scratch, const double *table, const float *scales, bool fast)
 {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    double *scratch = reinterpret_cast<double *>(smem_raw);
-    float *scales = reinterpret_cast<float *>(smem_raw + 34 * sizeof(double));
-    uint32_t *words_sm = reinterpret_cast<uint32_t *>(scales + kMaxWorkers);       // [W_total][chunk / 32]
-    const long long chunk_id = first_chunk + blockIdx.x;
-    const ChunkGeom cg = chunk_geom(st, chunk_id);
     const int lane = threadIdx.x & 31;
-    const long long range_word0 = (first_chunk * st.chunk) >> 5;
-    const int words_per_chunk = st.chunk >> 5, n_words = (cg.len + 31) >> 5;
-    const long long chunk_word0 = (cg.c0 >> 5) - range_word0;
-    const bool z_bar_aligned = (reinterpret_cast<uintptr_t>(z_bar) & 15u) == 0;
-
-    for (int i = threadIdx.x; i < W_total; i += blockDim.x) scales[i] = scales_in[(long long)i * scales_in_stride + blockIdx.x];
-    const int total = W_total * n_words;
-    for (int e0 = threadIdx.x; e0 < total; e0 += 8 * blockDim.x) {
-        uint32_t w[8];
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            const int e = e0 + q * blockDim.x;
-            w[q] = e < total ? words_in[(long long)(e / n_words) * words_in_stride + chunk_word0 + e % n_words] : 0u;
-        }
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            const int e = e0 + q * blockDim.x;
-            if (e < total) words_sm[(e / n_words) * words_per_chunk + e % n_words] = w[q];
-        }
-    }
-    float4 e4[ITER];
-#pragma unroll
-    for (int it = 0; it < ITER; ++it) {
-        const int idx = 4 * (it * blockDim.x + threadIdx.x);
-        e4[it] = idx < cg.len ? ld4(st.ds + cg.c0 + idx) : make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-    __syncthreads();
-
-    float a[ITER][4];
+    const uint32_t sel = (threadIdx.x & 3u) | ((4u + (threadIdx.x & 3u)) << 4);
+    const bool w_pow2 = (W_total & (W_total - 1)) == 0;
+    const double inv_w = __longlong_as_double((long long)(1023 - (31 - __clz(W_total))) << 52);
+    float a[ITER][8];
     double l1 = 0.0;
 #pragma unroll
     for (int it = 0; it < ITER; ++it) {
-        const int idx = 4 * (it * blockDim.x + threadIdx.x);
-        double A[4] = {0.0, 0.0, 0.0, 0.0};
-        if (idx < cg.len) {
-            const int shift = idx & 31;
-            for (int i = 0; i < W_total; ++i) {  // worker order
-                const uint32_t nib = words_sm[i * words_per_chunk + (idx >> 5)] >> shift;
-                const double sc = (double)scales[i];
+        const int idx = 8 * (it * blockDim.x + threadIdx.x);
+        const bool active = FULL || idx < cg.len;
+        float4 e0 = make_float4(0.f, 0.f, 0.f, 0.f), e1 = e0;
+        if (active) e0 = ld4(st.ds + cg.c0 + idx);
+        if (FULL || idx + 4 < cg.len) e1 = ld4(st.ds + cg.c0 + idx + 4);
+        double A[8] = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0};
+        const uint32_t *col = words_in + chunk_word0 + (idx >> 5);
+        for (int i0 = 0; i0 < W_total; i0 += 16) {
+            uint32_t w[16];
+            const int left = W_total - i0;
 #pragma unroll
-                for (int k = 0; k < 4; ++k) A[k] += ((nib >> k) & 1u) ? sc : -sc;
+            for (int gg = 0; gg < 4; ++gg) {
+                if (4 * gg < left) {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        w[4 * gg + k] = active && 4 * gg + k < left ? *col : 0u;
+                        col += words_in_stride;
+                    }
+                }
+            }
+#pragma unroll
+            for (int gg = 0; gg < 4; ++gg) {
+                if (4 * gg < left) {
+                    const uint32_t x = __byte_perm(__byte_perm(w[4 * gg], w[4 * gg + 1], sel), __byte_perm(w[4 * gg + 2], w[4 * gg + 3], sel), 0x5410u);
+                    if (fast) {
+                        const char *t = reinterpret_cast<const char *>(table + ((i0 >> 2) + gg) * 16);
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            const uint32_t off = ((x & (0x01010101u << c)) * (kGatherMul >> c)) >> 25;
+                            const double entry = *reinterpret_cast<const double *>(t + off);
+                            A[c] = (i0 == 0 && gg == 0) ? entry : __dadd_rn(A[c], entry);
+                        }
+                    } else {
+                        for (int k = 0; k < 4 && 4 * gg + k < left; ++k) {
+                            const double sc = (double)scales[i0 + 4 * gg + k];
+                            const uint32_t byte = x >> (8 * k);
+#pragma unroll
+                            for (int c = 0; c < 8; ++c) A[c] = __dadd_rn(A[c], ((byte >> c) & 1u) ? sc : -sc);
+                        }
+                    }
+                }
             }
         }
-        const float ee[4] = {e4[it].x, e4[it].y, e4[it].z, e4[it].w};
+        const float ee[8] = {e0.x, e0.y, e0.z, e0.w, e1.x, e1.y, e1.z, e1.w};
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            a[it][k] = idx + k < cg.len ? server_input(A[k], W_total, ee[k]) : 0.0f;
-            l1 += fabs((double)a[it][k]);
+        for (int c = 0; c < 8; ++c) {
+            const double q = w_pow2 ? __dmul_rn(A[c], inv_w) : __ddiv_rn(A[c], (double)W_total);
+            const float v = __double2float_rn(__dadd_rn(q, (double)ee[c]));
+            a[it][c] = FULL || idx + c < cg.len ? v : 0.0f;
+            l1 += fabs((double)a[it][c]);
         }
     }
     const float scale = chunk_scale(block_sum(l1, scratch), cg.len);
 #pragma unroll
     for (int it = 0; it < ITER; ++it) {
-        const int idx = 4 * (it * blockDim.x + threadIdx.x);
-        const int base = idx - 4 * lane;                   // first coordinate of the warp's 128
-        float hat[4];
-        const uint32_t word = compress_tile(a[it], hat, scale, idx, cg.len);
-        if (lane < 4 && base + 32 * lane < cg.len) {
-            const long long w = ((cg.c0 + base) >> 5) + lane;
-            st.words_s[w] = word;
-            for (int r = 0; r < out.world; ++r) out.words_s[r][w] = word;
+        const int idx = 8 * (it * blockDim.x + threadIdx.x);
+        float hat[8];
+        uint32_t bits = 0;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            const bool valid = FULL || idx + c < cg.len;
+            const bool b = valid && (a[it][c] >= 0.0f);
+            hat[c] = valid ? (b ? scale : -scale) : 0.0f;
+            a[it][c] = valid ? f_sub(a[it][c], hat[c]) : 0.0f;
+            bits |= (b ? 1u : 0u) << c;
         }
-        if (idx < cg.len) st4(st.ds + cg.c0 + idx, make_float4(a[it][0], a[it][1], a[it][2], a[it][3]));
+        bits <<= 8 * (lane & 3);
+        bits |= __shfl_xor_sync(0xffffffffu, bits, 1);
+        bits |= __shfl_xor_sync(0xffffffffu, bits, 2);
+        if ((lane & 3) == 0 && (FULL || idx < cg.len)) {
+            const long long w = (cg.c0 + idx) >> 5;
+            st.words_s[w] = bits;
+            for (int r = 0; r < out.world; ++r) out.words_s[r][w] = bits;
+        }
+        if (FULL || idx < cg.len) st4(st.ds + cg.c0 + idx, make_float4(a[it][0], a[it][1], a[it][2], a[it][3]));
+        if (FULL || idx + 4 < cg.len) st4(st.ds + cg.c0 + idx + 4, make_float4(a[it][4], a[it][5], a[it][6], a[it][7]));
         if (z_bar) {
-            if (z_bar_aligned && idx + 4 <= cg.len) {
+            if (z_bar_aligned && (FULL || idx + 8 <= cg.len)) {
                 st4_stream(z_bar + cg.c0 + idx, make_float4(hat[0], hat[1], hat[2], hat[3]));
+                st4_stream(z_bar + cg.c0 + idx + 4, make_float4(hat[4], hat[5], hat[6], hat[7]));
             } else {
 #pragma unroll
-                for (int k = 0; k < 4; ++k)
-                    if (idx + k < cg.len) z_bar[cg.c0 + idx + k] = hat[k];
+                for (int c = 0; c < 8; ++c)
+                    if (idx + c < cg.len) z_bar[cg.c0 + idx + c] = hat[c];
             }
         }
     }
@@ -522,6 +552,63 @@ __global__ void __launch_bounds__(ITER > 4 ? 512 : 256, ITER > 4 ? 2 : 4) dist_s
         st.scales_s[chunk_id] = scale;
         for (int r = 0; r < out.world; ++r) out.scales_s[r][chunk_id] = scale;
     }
+}
+
+template <int ITER>
+__global__ void __launch_bounds__(512, 2) dist_server_kernel(const __grid_constant__ StateView st, const uint32_t *words_in, long long words_in_stride,
+                                   const float *scales_in, long long scales_in_stride, int W_total,
+                                   long long first_chunk, const __grid_constant__ PeerOut out, float *z_bar)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    double *scratch = reinterpret_cast<double *>(smem_raw);
+    double *table = scratch + 34;
+    float *scales = reinterpret_cast<float *>(table + (kMaxWorkers / 4) * 16);
+    int *exact_flag = reinterpret_cast<int *>(scales + kMaxWorkers);
+    const long long chunk_id = first_chunk + blockIdx.x;
+    const ChunkGeom cg = chunk_geom(st, chunk_id);
+    const int lane = threadIdx.x & 31;
+    const long long range_word0 = (first_chunk * st.chunk) >> 5;
+    const long long chunk_word0 = (cg.c0 >> 5) - range_word0;
+    const bool z_bar_aligned = (reinterpret_cast<uintptr_t>(z_bar) & 15u) == 0;
+    const int groups = (W_total + 3) >> 2;
+
+    if (threadIdx.x < 32) {
+        int e_max = 0, e_min = 255;
+        bool bad = false;
+        for (int i = lane; i < W_total; i += 32) {
+            const float s = scales_in[(long long)i * scales_in_stride + blockIdx.x];
+            scales[i] = s;
+            const uint32_t u = __float_as_uint(s);
+            int e = (int)((u >> 23) & 0xFFu);
+            if (e == 255 || (u >> 31)) bad = true;
+            else if (u << 1) {
+                e = e < 1 ? 1 : e;
+                e_max = e > e_max ? e : e_max;
+                e_min = e < e_min ? e : e_min;
+            }
+        }
+        e_max = __reduce_max_sync(0xffffffffu, e_max);
+        e_min = __reduce_min_sync(0xffffffffu, e_min);
+        bad = __any_sync(0xffffffffu, bad);
+        const int log2_w = W_total > 1 ? 32 - __clz(W_total - 1) : 0;
+        if (lane == 0) *exact_flag = groups == 1 || (!bad && e_max - e_min <= 29 - log2_w);
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < 16 * groups; e += blockDim.x) {
+        const int g = e >> 4, m = e & 15;
+        double acc = 0.0;
+        for (int k = 0; k < 4; ++k) {
+            const int i = 4 * g + k;
+            if (i < W_total) acc = __dadd_rn(acc, ((m >> k) & 1) ? (double)scales[i] : -(double)scales[i]);
+        }
+        table[e] = acc;
+    }
+    __syncthreads();
+    const bool fast = *exact_flag != 0;
+    if (cg.len == st.chunk && (!z_bar || z_bar_aligned))
+        server_chunk<ITER, true>(st, words_in, words_in_stride, W_total, chunk_word0, out, z_bar, z_bar_aligned, cg, chunk_id, scratch, table, scales, fast);
+    else
+        server_chunk<ITER, false>(st, words_in, words_in_stride, W_total, chunk_word0, out, z_bar, z_bar_aligned, cg, chunk_id, scratch, table, scales, fast);
 }
 
 // Worker side of Algorithm 3 for the handle's single worker and chunk blockIdx.x, the packed
@@ -1285,18 +1372,15 @@ cudaError_t launch_dist_server(const StateView &st, const uint32_t *words_in, lo
                                const float *scales_in, long long scales_in_stride, int W_total,
                                long long first_chunk, long long count, const PeerOut &out, float *z_bar, cudaStream_t s)
 {
-    // 16 coordinates per thread (32 above chunk 4096), like compress_kernel (32 per thread at chunk 4096 measured worse)
-    const int iter = st.chunk > 4096 ? 8 : 4;
-    const int thr = ((st.chunk + 4 * iter - 1) / (4 * iter) + 31) / 32 * 32;
-    const size_t smem = 34 * sizeof(double) + kMaxWorkers * sizeof(float) + (size_t)W_total * (st.chunk / 32) * sizeof(uint32_t);
-    static SmemLimitOnce once[2];
-    cudaError_t e = once[0].ensure(dist_server_kernel<4>, (int)(34 * sizeof(double) + kMaxWorkers * sizeof(float) + (size_t)kMaxWorkers * (4096 / 32) * 4));
-    if (e == cudaSuccess) e = once[1].ensure(dist_server_kernel<8>, (int)(34 * sizeof(double) + kMaxWorkers * sizeof(float) + (size_t)kMaxWorkers * (kMaxChunk / 32) * 4));
-    if (e != cudaSuccess) return e;
-    if (iter == 8)
-        dist_server_kernel<8><<<(unsigned)count, thr, smem, s>>>(st, words_in, words_in_stride, scales_in, scales_in_stride, W_total, first_chunk, out, z_bar);
-    else
-        dist_server_kernel<4><<<(unsigned)count, thr, smem, s>>>(st, words_in, words_in_stride, scales_in, scales_in_stride, W_total, first_chunk, out, z_bar);
+    // 8, 16 or 32 coordinates per thread: blocks of 128 ... 512 threads for chunks of 1024 ... 16384
+    const int iter = st.chunk > 8192 ? 4 : st.chunk > 2048 ? 2 : 1;
+    const int thr = ((st.chunk + 8 * iter - 1) / (8 * iter) + 31) / 32 * 32;
+    const size_t smem = (34 + (kMaxWorkers / 4) * 16) * sizeof(double) + kMaxWorkers * sizeof(float) + 16;
+    switch (iter) {
+    case 4: dist_server_kernel<4><<<(unsigned)count, thr, smem, s>>>(st, words_in, words_in_stride, scales_in, scales_in_stride, W_total, first_chunk, out, z_bar); break;
+    case 2: dist_server_kernel<2><<<(unsigned)count, thr, smem, s>>>(st, words_in, words_in_stride, scales_in, scales_in_stride, W_total, first_chunk, out, z_bar); break;
+    default: dist_server_kernel<1><<<(unsigned)count, thr, smem, s>>>(st, words_in, words_in_stride, scales_in, scales_in_stride, W_total, first_chunk, out, z_bar); break;
+    }
     return cudaGetLastError();
 }
 

@@ -319,6 +319,46 @@ def test_onebit_allreduce_on_caller_buffers(n, W, chunk, offset, light):
         gpu.close()
 
 
+@pytest.mark.parametrize("W,chunk", [(6, 1024), (16, 4096), (64, 256), (3, 1024)])
+def test_onebit_allreduce_worker_magnitudes_far_apart(W, chunk):
+    """The server kernels add table entries for groups of four workers, which gives the bits of the
+    worker-by-worker binary64 sum only while every partial sum is exact; a chunk whose workers'
+    magnitudes are too far apart for that must take the worker-by-worker loop.  Here the chunks
+    alternate between magnitudes of one size, magnitudes spread over 2^100 (partial sums round), a
+    spread just inside and just outside the limit, and workers whose buffers are all zero."""
+    rng = np.random.default_rng(W * chunk)
+    n = 9 * chunk + 77
+    cpu = zo.Oracle(n, W, chunk, dtype=np.float32)
+    gpu = Zoa(n, W, chunk=chunk, allreduce_only=True)
+    limit = 29 - int(np.ceil(np.log2(W)))                  # largest exponent gap with exact partial sums
+    try:
+        for r in range(3):
+            z = rng.standard_normal((W, n)).astype(np.float32)
+            for c in range(10):
+                sl = slice(c * chunk, min((c + 1) * chunk, n))
+                for i in range(W):
+                    if c % 5 == 1:
+                        z[i, sl] *= np.float32(2.0 ** (-50 + (100 * i) // max(W - 1, 1)))
+                    elif c % 5 == 2:
+                        z[i, sl] *= np.float32(2.0 ** ((limit - 2) * (i % 2)))
+                    elif c % 5 == 3:
+                        z[i, sl] *= np.float32(2.0 ** ((limit + 3) * (i % 2)))
+                    elif c % 5 == 4 and i % 3 == 0:
+                        z[i, sl] = 0.0
+            z_dev = [torch.from_numpy(z[i]).cuda() for i in range(W)]
+            z_bar = torch.empty(n, device="cuda")
+            gpu.onebit_allreduce(z_dev, z_bar)
+            torch.cuda.synchronize()
+            want = cpu.onebit_allreduce(z)
+            assert np.array_equal(gpu.read("words_s"), cpu.words_server), f"words_s, round {r}"
+            assert_close(z_bar.cpu().numpy(), want, f"z_bar, round {r}")
+            assert_close(gpu.read("scales_s"), cpu.scales_server, f"scales_s, round {r}")
+            assert_close(gpu.read("delta_s"), cpu.delta_bar, f"delta_s, round {r}")
+        gpu.check_device()
+    finally:
+        gpu.close()
+
+
 @pytest.mark.parametrize("where", ["pending_variance", "after_sync", "mid_interval"])
 def test_checkpoint_round_trip(where):
     """zoa_export_state / zoa_import_state through the C ABI: run, export, import into a fresh handle,
