@@ -5,7 +5,7 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libzoa.so")
-SOURCES = ["zoa_kernels.cu", "zoa_pipeline.cu", "zoa_reduce_pipeline.cu", "zoa_api.cu", "zoa_noalloc.cu"]
+SOURCES = ["zoa_kernels.cu", "zoa_pipeline.cu", "zoa_reduce_pipeline.cu", "zoa_server_pipeline.cu", "zoa_api.cu", "zoa_noalloc.cu"]
 HEADERS = ["zoa_device.cuh", "zoa_internal.h", "zoa_ring.cuh", os.path.join("..", "..", "include", "zoa.h")]
 
 # The arithmetic contract needs IEEE division and square root, subnormals kept,

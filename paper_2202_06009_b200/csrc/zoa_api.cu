@@ -596,6 +596,31 @@ extern "C" zoa_status zoa_onebit_average(zoa_handle h, void *stream)
     return ZOA_OK;
 }
 
+// Server side of Algorithm 3 alone for the chunks [first, first + count) of packed buffers that start at
+// chunk `first`: the prefetching kernel for the whole chunks where the buffers allow it, the plain
+// one-block-per-chunk kernel for a ragged last chunk and every other case.
+static zoa_status run_server_alone(zoa_handle h, const uint32_t *words_in, long long words_stride, const float *scales_in,
+                                   long long scales_stride, int W_total, long long first, long long count, const PeerOut &out,
+                                   float *z_bar, cudaStream_t s)
+{
+    const StateView st = view(h);
+    const bool ragged = first + count == h->n_chunks && h->n % h->chunk != 0;
+    long long whole = 0;
+    if (h->use_pipeline && server_prefetch_applies(st, words_in, words_stride, W_total, z_bar)) whole = count - (ragged ? 1 : 0);
+    if (whole > 0) {
+        ZOA_CUDA(h, launch_server_prefetch(st, words_in, words_stride, scales_in, scales_stride, W_total, first, whole, out, z_bar,
+                                           error_words(h), (unsigned long long)h->wait_limit_ms * 1000000ull,
+                                           h->test_stop_after_tiles > 0, s));
+        h->n_launches += 1;
+    }
+    if (whole < count) {
+        ZOA_CUDA(h, launch_dist_server(st, words_in + (whole * h->chunk >> 5), words_stride, scales_in + whole, scales_stride, W_total,
+                                       first + whole, count - whole, out, z_bar, s));
+        h->n_launches += 1;
+    }
+    return ZOA_OK;
+}
+
 // ---- Algorithm 3 on caller-owned buffers, with the handle's errors and wire buffers ---------------
 
 static zoa_status allreduce_compress(zoa_handle h, const float *const *z, cudaStream_t s, const char *who)
@@ -621,12 +646,8 @@ static zoa_status allreduce_average(zoa_handle h, float *z_bar, cudaStream_t s, 
     ZOA_REFUSE_AFTER_DEVICE_ERROR(h, who);
     if (h->large_chunk) return fail(h, ZOA_ERR_ARG, std::string(who) + ": chunk must be at most 16384");
     if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, std::string(who) + ": the handle's device is not the current CUDA device");
-    // One block per chunk: the server side alone moves so little per chunk (12 bytes and W bits per coordinate)
-    // that many resident blocks hide its latencies better than one persistent block per SM does.
     PeerOut none{};
-    ZOA_CUDA(h, launch_dist_server(view(h), h->words_w, h->words_stride, h->scales_w, h->n_chunks, h->W, 0, h->n_chunks, none, z_bar, s));
-    h->n_launches += 1;
-    return ZOA_OK;
+    return run_server_alone(h, h->words_w, h->words_stride, h->scales_w, h->n_chunks, h->W, 0, h->n_chunks, none, z_bar, s);
 }
 
 extern "C" zoa_status zoa_allreduce_compress(zoa_handle h, const float *const *z, void *stream)
@@ -667,11 +688,10 @@ extern "C" zoa_status zoa_dist_server_range(zoa_handle h, const uint32_t *words_
     if (n_chunks == 0) return ZOA_OK;
     if (!words_all || !scales_all) return fail(h, ZOA_ERR_ARG, "zoa_dist_server_range: NULL buffer");
     if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, "zoa_dist_server_range: the handle's device is not the current CUDA device");
+    ZOA_REFUSE_AFTER_DEVICE_ERROR(h, "zoa_dist_server_range");
     PeerOut none{};
-    ZOA_CUDA(h, launch_dist_server(view(h), words_all, (long long)words_stride, scales_all, (long long)scales_stride,
-                                   W_total, first_chunk, n_chunks, none, nullptr, static_cast<cudaStream_t>(stream)));
-    h->n_launches += 1;
-    return ZOA_OK;
+    return run_server_alone(h, words_all, (long long)words_stride, scales_all, (long long)scales_stride, W_total, first_chunk, n_chunks,
+                            none, nullptr, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" zoa_status zoa_dist_server_push(zoa_handle h, const uint32_t *words_all, size_t words_stride,
@@ -696,10 +716,9 @@ extern "C" zoa_status zoa_dist_server_push(zoa_handle h, const uint32_t *words_a
     if (n_chunks == 0) return ZOA_OK;
     if (!words_all || !scales_all) return fail(h, ZOA_ERR_ARG, "zoa_dist_server_push: NULL buffer");
     if (!on_own_device(h)) return fail(h, ZOA_ERR_STATE, "zoa_dist_server_push: the handle's device is not the current CUDA device");
-    ZOA_CUDA(h, launch_dist_server(view(h), words_all, (long long)words_stride, scales_all, (long long)scales_stride,
-                                   W_total, first_chunk, n_chunks, out, nullptr, static_cast<cudaStream_t>(stream)));
-    h->n_launches += 1;
-    return ZOA_OK;
+    ZOA_REFUSE_AFTER_DEVICE_ERROR(h, "zoa_dist_server_push");
+    return run_server_alone(h, words_all, (long long)words_stride, scales_all, (long long)scales_stride, W_total, first_chunk, n_chunks,
+                            out, nullptr, static_cast<cudaStream_t>(stream));
 }
 
 // The table of a rank's destinations, checked: the ranges tile the chunks in rank order and

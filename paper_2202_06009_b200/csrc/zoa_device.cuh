@@ -101,6 +101,67 @@ __device__ __forceinline__ float server_input(double sum_hat, int W, float delta
     return __double2float_rn(__dadd_rn(div_by_count(sum_hat, W), (double)delta_bar));
 }
 
+// ---- the server's sum over the workers (Algorithm 3), looked up instead of added bit by bit ----
+// The workers are taken in groups of four; a group's sixteen possible signed sums of magnitudes sit
+// in a table of 128 bytes (one entry per pair of shared-memory banks, so a warp's lookups never
+// conflict).  A thread owns eight consecutive coordinates = one byte of every worker's words;
+// gather_bytes puts that byte of four workers into one register, and for coordinate c one mask, one
+// multiplication and one shift turn the four workers' bits into the byte offset of the table entry.
+// Adding the groups' entries gives the bits of the worker-by-worker binary64 sum whenever every
+// partial sum is exact: all magnitudes are multiples of the smallest one's last place, so it is
+// enough that W * 2^(e_max + 1) stays below 2^53 of those units, i.e. that the exponents of the
+// non-zero magnitudes differ by at most 29 - ceil(log2 W).  With up to four workers the single
+// table holds the sequential sum itself.  Otherwise the caller adds worker by worker.
+constexpr uint32_t kGatherMul = 0x10204080u;   // 2^28 + 2^21 + 2^14 + 2^7: bits 0, 8, 16, 24 -> bits 28 ... 31
+
+// Warp-wide.  Lane l passes the magnitudes of workers l and l + 32 (0 beyond W).
+__device__ __forceinline__ bool table_sum_is_exact(float s_lo, float s_hi, int W)
+{
+    if (W <= 4) return true;
+    int e_max = 0, e_min = 255;
+    bool bad = false;
+    const float both[2] = {s_lo, s_hi};
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+        const uint32_t u = __float_as_uint(both[q]);
+        int e = (int)((u >> 23) & 0xFFu);
+        if (e == 255 || (u >> 31)) bad = true;            // not finite
+        else if (u << 1) {                                // not zero
+            e = e < 1 ? 1 : e;                            // subnormals share the exponent of the smallest normals
+            e_max = e > e_max ? e : e_max;
+            e_min = e < e_min ? e : e_min;
+        }
+    }
+    e_max = __reduce_max_sync(0xffffffffu, e_max);
+    e_min = __reduce_min_sync(0xffffffffu, e_min);
+    bad = __any_sync(0xffffffffu, bad);
+    return !bad && e_max - e_min <= 29 - (32 - __clz(W - 1));
+}
+// Entry e = 16 * group + m of the tables: the signed sum of the group's workers in worker order, worker
+// 4 * group + k taken positive where bit k of m is set.
+__device__ __forceinline__ double table_entry(const float *scales, int W, int e)
+{
+    const int g = e >> 4, m = e & 15;
+    double acc = 0.0;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int i = 4 * g + k;
+        if (i < W) acc = __dadd_rn(acc, ((m >> k) & 1) ? (double)scales[i] : -(double)scales[i]);
+    }
+    return acc;
+}
+// Byte b of each of four words, worker k's in byte k; sel = b | ((4 + b) << 4).
+__device__ __forceinline__ uint32_t gather_bytes(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3, uint32_t sel)
+{
+    return __byte_perm(__byte_perm(w0, w1, sel), __byte_perm(w2, w3, sel), 0x5410u);
+}
+// Byte offset (8 * the four workers' bits) of coordinate c's entry; x from gather_bytes, c a constant
+// after unrolling.
+__device__ __forceinline__ uint32_t table_offset(uint32_t x, int c)
+{
+    return ((x & (0x01010101u << c)) * (kGatherMul >> c)) >> 25;
+}
+
 // ---- 128-bit accesses ----
 __device__ __forceinline__ float4 ld4(const float *p) { return *reinterpret_cast<const float4 *>(p); }
 __device__ __forceinline__ void st4(float *p, float4 v) { *reinterpret_cast<float4 *>(p) = v; }

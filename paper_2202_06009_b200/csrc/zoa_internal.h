@@ -50,6 +50,13 @@ int reduce_pipeline_stages(const StateView &st, long long *n_units);
 cudaError_t launch_reduce_pipelined(const StateView &st, const Consts &c, float gamma_sum, long long n_units,
                                     int stages, int sm_count, ErrorWords error_flag, unsigned long long *sched,
                                     unsigned long long wait_limit_ns, long long test_stop_after_tiles, cudaStream_t s);
+// Server side of Algorithm 3 alone with its inputs prefetched into shared memory (zoa_server_pipeline.cu):
+// whether the buffers allow it, and the launch for the whole chunks [first_chunk, first_chunk + count).
+bool server_prefetch_applies(const StateView &st, const uint32_t *words_in, long long words_in_stride, int W_total, const float *z_bar);
+cudaError_t launch_server_prefetch(const StateView &st, const uint32_t *words_in, long long words_in_stride,
+                                   const float *scales_in, long long scales_in_stride, int W_total, long long first_chunk,
+                                   long long count, const PeerOut &out, float *z_bar, ErrorWords error_flag,
+                                   unsigned long long wait_limit_ns, bool skip_copies, cudaStream_t s);
 cudaError_t launch_step_sync(const StateView &st, const GradPtrs &g, const Consts &c, float gamma,
                              float gamma_sum, int g_aligned, long long first_chunk, long long count, cudaStream_t s);
 

@@ -433,18 +433,9 @@ step_sync_kernel(StateView st, GradPtrs g, Consts c, float gamma, float gamma_su
 // words_s / scales_s, peer pointers included); out.world == 0 for none.
 //
 // With 12 to 14 bytes per coordinate this step is bound by instructions, not by memory, if the sum
-// over the workers is taken bit by bit (W selects and W additions per coordinate).  So the sum is
-// looked up: the workers are taken in groups of four, a group's sixteen possible signed sums
-// sit in a table in shared memory (128 bytes: one entry per pair of banks, so a lookup never
-// conflicts), a thread owns eight consecutive coordinates = one byte of every worker's words, and
-// one mask, one multiplication and one shift turn the four workers' bits of a coordinate into the
-// table offset.  Adding the groups' entries gives the bits of the worker-by-worker binary64 sum
-// whenever every partial sum is exact: all magnitudes are multiples of the smallest one's last
-// place, so it is enough that W * 2^(e_max + 1) stays below 2^53 of those units, i.e. that the
-// exponents of the non-zero magnitudes differ by at most 29 - ceil(log2 W) (checked per chunk;
-// with up to four workers the single table holds the sequential sum itself).  A chunk that fails
-// the check takes the worker-by-worker loop.
-constexpr uint32_t kGatherMul = 0x10204080u;   // 2^28 + 2^21 + 2^14 + 2^7: bits 0, 8, 16, 24 -> bits 28 ... 31
+// over the workers is taken bit by bit (W selects and W additions per coordinate), so it is looked
+// up in tables (see table_sum_is_exact in zoa_device.cuh); a chunk whose magnitudes are too far
+// apart for that takes the worker-by-worker loop.
 
 // One chunk of dist_server_kernel.  FULL: the chunk has its full length and z_bar (if any) takes
 // 128-bit stores, so that no coordinate needs a bounds check.
@@ -484,13 +475,12 @@ __device__ __forceinline__ void server_chunk(const StateView &st, const uint32_t
 #pragma unroll
             for (int gg = 0; gg < 4; ++gg) {
                 if (4 * gg < left) {
-                    const uint32_t x = __byte_perm(__byte_perm(w[4 * gg], w[4 * gg + 1], sel), __byte_perm(w[4 * gg + 2], w[4 * gg + 3], sel), 0x5410u);
+                    const uint32_t x = gather_bytes(w[4 * gg], w[4 * gg + 1], w[4 * gg + 2], w[4 * gg + 3], sel);
                     if (fast) {
                         const char *t = reinterpret_cast<const char *>(table + ((i0 >> 2) + gg) * 16);
 #pragma unroll
                         for (int c = 0; c < 8; ++c) {
-                            const uint32_t off = ((x & (0x01010101u << c)) * (kGatherMul >> c)) >> 25;
-                            const double entry = *reinterpret_cast<const double *>(t + off);
+                            const double entry = *reinterpret_cast<const double *>(t + table_offset(x, c));
                             A[c] = (i0 == 0 && gg == 0) ? entry : __dadd_rn(A[c], entry);
                         }
                     } else {
@@ -573,39 +563,18 @@ __global__ void __launch_bounds__(512, 2) dist_server_kernel(const __grid_consta
     const int groups = (W_total + 3) >> 2;
 
     if (threadIdx.x < 32) {
-        int e_max = 0, e_min = 255;
-        bool bad = false;
-        for (int i = lane; i < W_total; i += 32) {
-            const float s = scales_in[(long long)i * scales_in_stride + blockIdx.x];
-            scales[i] = s;
-            const uint32_t u = __float_as_uint(s);
-            int e = (int)((u >> 23) & 0xFFu);
-            if (e == 255 || (u >> 31)) bad = true;
-            else if (u << 1) {
-                e = e < 1 ? 1 : e;
-                e_max = e > e_max ? e : e_max;
-                e_min = e < e_min ? e : e_min;
-            }
-        }
-        e_max = __reduce_max_sync(0xffffffffu, e_max);
-        e_min = __reduce_min_sync(0xffffffffu, e_min);
-        bad = __any_sync(0xffffffffu, bad);
-        const int log2_w = W_total > 1 ? 32 - __clz(W_total - 1) : 0;
-        if (lane == 0) *exact_flag = groups == 1 || (!bad && e_max - e_min <= 29 - log2_w);
+        const float s_lo = lane < W_total ? scales_in[(long long)lane * scales_in_stride + blockIdx.x] : 0.0f;
+        const float s_hi = lane + 32 < W_total ? scales_in[(long long)(lane + 32) * scales_in_stride + blockIdx.x] : 0.0f;
+        if (lane < W_total) scales[lane] = s_lo;
+        if (lane + 32 < W_total) scales[lane + 32] = s_hi;
+        const bool exact = table_sum_is_exact(s_lo, s_hi, W_total);
+        if (lane == 0) *exact_flag = exact;
     }
     __syncthreads();
-    for (int e = threadIdx.x; e < 16 * groups; e += blockDim.x) {
-        const int g = e >> 4, m = e & 15;
-        double acc = 0.0;
-        for (int k = 0; k < 4; ++k) {
-            const int i = 4 * g + k;
-            if (i < W_total) acc = __dadd_rn(acc, ((m >> k) & 1) ? (double)scales[i] : -(double)scales[i]);
-        }
-        table[e] = acc;
-    }
+    for (int e = threadIdx.x; e < 16 * groups; e += blockDim.x) table[e] = table_entry(scales, W_total, e);
     __syncthreads();
     const bool fast = *exact_flag != 0;
-    if (cg.len == st.chunk && (!z_bar || z_bar_aligned))
+    if (cg.len == st.chunk && 8 * ITER * (int)blockDim.x == st.chunk && (!z_bar || z_bar_aligned))   // every thread has eight valid coordinates per pass
         server_chunk<ITER, true>(st, words_in, words_in_stride, W_total, chunk_word0, out, z_bar, z_bar_aligned, cg, chunk_id, scratch, table, scales, fast);
     else
         server_chunk<ITER, false>(st, words_in, words_in_stride, W_total, chunk_word0, out, z_bar, z_bar_aligned, cg, chunk_id, scratch, table, scales, fast);

@@ -319,22 +319,77 @@ def test_onebit_allreduce_on_caller_buffers(n, W, chunk, offset, light):
         gpu.close()
 
 
+@pytest.mark.parametrize("W,chunk,n_units,tail", [(5, 4096, 301, 1852), (16, 8192, 160, 704), (4, 16384, 150, 9000), (2, 2048, 600, 2048 + 33),
+                                                  (7, 1024, 650, 1500), (3, 512, 620, 0), (64, 256, 610, 3), (33, 4096, 20, 0),
+                                                  (1, 1024, 600, 1024), (16, 128, 300, 0)])
+def test_server_prefetch_kernel_equals_plain_kernel(W, chunk, n_units, tail):
+    """zoa_allreduce_average through the kernel that prefetches a chunk's inputs into shared memory
+    against the same call through the plain one-block-per-chunk kernel: same bits in everything it
+    writes, over rounds with non-zero errors, with and without a result buffer.  A ragged last chunk
+    goes to the plain kernel in both; chunk 128 has no prefetching variant.  A smaller case of the
+    same shape is also compared with the oracle."""
+    rng = np.random.default_rng(W * chunk + 1)
+    n = n_units * max(chunk, 4096) + tail
+    a, b = Zoa(n, W, chunk=chunk, allreduce_only=True), Zoa(n, W, chunk=chunk, allreduce_only=True)
+    try:
+        a.set_pipeline("force")
+        b.set_pipeline(False)
+        za, zb = torch.empty(n, device="cuda"), torch.empty(n, device="cuda")
+        for r in range(3):
+            z = [torch.randn(n, device="cuda", generator=torch.Generator("cuda").manual_seed(100 * r + i)) * 10.0 ** (r - 1) for i in range(W)]
+            for h, out in ((a, za), (b, zb)):
+                h.allreduce_compress(z)
+                h.allreduce_average(out if r != 1 else None)
+            torch.cuda.synchronize()
+            a.check_device()
+            if r != 1:
+                assert torch.equal(za, zb), f"z_bar, round {r}"
+            for name in ("delta_s", "words_s", "scales_s"):
+                assert np.array_equal(a.read(name), b.read(name)), (name, r)
+        if chunk % 256 == 0 and n % chunk != 0:
+            assert a.stats()["n_launches"] > b.stats()["n_launches"]      # prefetching kernel + the ragged chunk's
+    finally:
+        a.close(), b.close()
+    # the same shape, small, against the oracle
+    n = 3 * max(chunk, 4096) + (tail % (2 * chunk))
+    cpu = zo.Oracle(n, W, chunk, dtype=np.float32)
+    gpu = Zoa(n, W, chunk=chunk, allreduce_only=True)
+    try:
+        gpu.set_pipeline("force")
+        for r in range(2):
+            z = (rng.standard_normal((W, n)) * 10.0 ** rng.integers(-2, 2, size=(W, 1))).astype(np.float32)
+            z_bar = torch.empty(n, device="cuda")
+            gpu.onebit_allreduce([torch.from_numpy(z[i]).cuda() for i in range(W)], z_bar)
+            torch.cuda.synchronize()
+            want = cpu.onebit_allreduce(z)
+            assert np.array_equal(gpu.read("words_s"), cpu.words_server), f"words_s, round {r}"
+            assert_close(z_bar.cpu().numpy(), want, f"z_bar, round {r}")
+            assert_close(gpu.read("scales_s"), cpu.scales_server, f"scales_s, round {r}")
+            assert_close(gpu.read("delta_s"), cpu.delta_bar, f"delta_s, round {r}")
+        gpu.check_device()
+    finally:
+        gpu.close()
+
+
+@pytest.mark.parametrize("prefetch", [False, True])
 @pytest.mark.parametrize("W,chunk", [(6, 1024), (16, 4096), (64, 256), (3, 1024)])
-def test_onebit_allreduce_worker_magnitudes_far_apart(W, chunk):
+def test_onebit_allreduce_worker_magnitudes_far_apart(W, chunk, prefetch):
     """The server kernels add table entries for groups of four workers, which gives the bits of the
     worker-by-worker binary64 sum only while every partial sum is exact; a chunk whose workers'
     magnitudes are too far apart for that must take the worker-by-worker loop.  Here the chunks
     alternate between magnitudes of one size, magnitudes spread over 2^100 (partial sums round), a
-    spread just inside and just outside the limit, and workers whose buffers are all zero."""
+    spread just inside and just outside the limit, and workers whose buffers are all zero; through the
+    plain one-block-per-chunk kernel and through the prefetching kernel."""
     rng = np.random.default_rng(W * chunk)
     n = 9 * chunk + 77
     cpu = zo.Oracle(n, W, chunk, dtype=np.float32)
     gpu = Zoa(n, W, chunk=chunk, allreduce_only=True)
+    gpu.set_pipeline("force" if prefetch else False)
     limit = 29 - int(np.ceil(np.log2(W)))                  # largest exponent gap with exact partial sums
     try:
         for r in range(3):
             z = rng.standard_normal((W, n)).astype(np.float32)
-            for c in range(10):
+            for c in range((n + chunk - 1) // chunk):
                 sl = slice(c * chunk, min((c + 1) * chunk, n))
                 for i in range(W):
                     if c % 5 == 1:
@@ -518,13 +573,14 @@ def test_policies_match_the_workload_tables():
         z.close()
 
 
-@pytest.mark.parametrize("algorithm", ["alg1", "alg2", "two_call", "alg1_chunk_1024", "alg1_chunk_8192"])
+@pytest.mark.parametrize("algorithm", ["alg1", "alg2", "two_call", "allreduce", "alg1_chunk_1024", "alg1_chunk_8192"])
 def test_device_wait_runs_out_and_is_reported(algorithm):
     """Error path of the ring kernels without any fault: the copy-issuing lane of every block
     stops after three tiles (test hook), the other threads' bounded waits run out after
     100 ms, the kernel ends by itself, zoa_check_device reports ZOA_ERR_DEVICE, and the
     context and the handle stay usable.  Covers the fused kernel (one, two and four tiles per
-    unit), Algorithm 2's, and the server kernel of the two-call path with its store-issuing warp."""
+    unit), Algorithm 2's, the server kernel of the two-call path with its store-issuing warp, and the
+    prefetching server kernel of Algorithm 3 alone (whose copies are then never started)."""
     import time
     chunk = 1024 if algorithm.endswith("1024") else 8192 if algorithm.endswith("8192") else 4096
     n, W = 300 * max(chunk, 2048), 4
@@ -536,7 +592,11 @@ def test_device_wait_runs_out_and_is_reported(algorithm):
         def two_call(g, lr, t):
             z.step(g, lr, t)
             z.onebit_reduce()
-        step = z.alg2_step if algorithm == "alg2" else two_call if algorithm == "two_call" else z.step_sync
+        z_bar = torch.empty(n, device="cuda")
+
+        def allreduce(g, lr, t):
+            z.onebit_allreduce(g, z_bar)
+        step = {"alg2": z.alg2_step, "two_call": two_call, "allreduce": allreduce}.get(algorithm, z.step_sync)
         step(g, 1e-3, 0)
         z.check_device()                                  # the normal path works
         B.zoa_set_option(z.h, B.OPT_WAIT_LIMIT_MS, 100)
