@@ -499,6 +499,10 @@ def run_sweep(args):
     torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
     peak, peak_kind = measured_hbm_peak()
     exps = [20, 22] if args.sweep == "quick" else [20, 22, 24, 26, 28, 30]
+    if args.sweep_exp:
+        exps = args.sweep_exp
+    workers = args.sweep_workers or (2, 4, 8, 16)
+    chunks = args.sweep_chunks or (1024, 4096, 16384)
     gen = torch.Generator("cuda").manual_seed(5)
 
     def fill(t):                                   # N(0,1), 1 % of the elements x100, in bounded slices
@@ -525,8 +529,8 @@ def run_sweep(args):
 
     for e in exps:
         n = 1 << e
-        for W in (2, 4, 8, 16):
-            for chunk in (1024, 4096, 16384):
+        for W in workers:
+            for chunk in chunks:
                 n_chunks = n // chunk
                 row = {"sweep": True, "n": n, "W": W, "chunk": chunk, "peak_kind": peak_kind}
                 bytes_c = n * W * (12 + 1 / 8) + 4 * n_chunks * W
@@ -616,6 +620,9 @@ def main():
     ap.add_argument("--sweep", nargs="?", const="full", default=None, choices=["full", "quick"],
                     help="time the compress / decompress-average kernels over the size grid instead")
     ap.add_argument("--sweep-reps", type=int, default=3)
+    ap.add_argument("--sweep-exp", type=int, nargs="*", help="restrict the sweep to n = 2^EXP for these exponents")
+    ap.add_argument("--sweep-workers", type=int, nargs="*", help="restrict the sweep to these worker counts")
+    ap.add_argument("--sweep-chunks", type=int, nargs="*", help="restrict the sweep to these chunk sizes")
     args = ap.parse_args()
 
     if args.sweep:
