@@ -15,8 +15,8 @@
  * import call) part of the call's work may have run and the host scalars may
  * not have advanced: the optimizer state is undefined and should be restored
  * from a checkpoint (zoa_import_state) or rebuilt.  Once a kernel has given up on
- * a bounded wait, every step, reduce and compress entry point returns
- * ZOA_ERR_DEVICE (without synchronising; the news travels through a word of
+ * a bounded wait, every step, reduce, compress, allreduce and server entry point
+ * returns ZOA_ERR_DEVICE (without synchronising; the news travels through a word of
  * pinned host memory) until zoa_check_device has reported and cleared it.
  *
  * Arithmetic contract (what "the same result" means for every entry point):
@@ -353,8 +353,9 @@ zoa_status zoa_check_finite(zoa_handle h, int64_t *n_nonfinite);
  * asynchronous copy before it gives up; the kernel then ends early, the state is
  * undefined and zoa_check_device reports ZOA_ERR_DEVICE.
  * ZOA_OPT_TEST_STOP_AFTER_TILES (default 0 = off): for testing that error path
- * only - the copy-issuing lane of every block stops after this many tiles, so
- * the waits of the other threads run out after the limit.
+ * only - the copy-issuing lane of every block stops after this many tiles (in the
+ * server kernel of zoa_allreduce_average the copies are never started), so the
+ * waits of the other threads run out after the limit.
  * ZOA_OPT_GRAD_TYPE (default ZOA_GRAD_F32): element type of the buffers passed as
  * `grads` / `host_grads` from now on: binary32, binary16 (IEEE half) or bfloat16.
  * 16-bit gradients are converted to binary32 exactly when they are loaded; all
