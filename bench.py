@@ -24,7 +24,20 @@ if ROOT not in sys.path:
 METRIC = "optimizer step throughput (params*workers/s)"
 UNIT = "params*workers/s"
 FALLBACK_HBM_GBS = 6650.0
-DRAM_TRAFFIC_RATIO = 0.995   # measured DRAM bytes / algorithmic bytes, see profiles/
+# Measured DRAM bytes (ncu dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic bytes of one launch, per
+# kernel, each from a capture on the BERT-Large-shaped layout shrunk 16x (traffic is proportional to n*W, so
+# the ratio carries to a full launch), with the summary under profiles/ that holds it.  A kernel without a
+# capture reports traffic null.
+DRAM_TRAFFIC_RATIO = {
+    "step_sync_pipelined_kernel": (0.995, "step_sync_pipelined_kernel_bert_large_div16.md"),
+    "local_step_pipelined_kernel": (0.994, "step_sync_pipelined_kernel_bert_large_div16.md"),
+    "step_sync_kernel": (0.995, "step_sync_kernel_alg2_compressed_kernel_chunk_per_block_bert_large_div16.md"),
+    "step_sync_kernel@16384": (1.004, "step_sync_kernel_alg2_compressed_kernel_chunk_per_block_bert_large_div16.md"),
+    "alg2_compressed_kernel": (1.007, "step_sync_kernel_alg2_compressed_kernel_chunk_per_block_bert_large_div16.md"),
+    "alg2_pipelined_kernel": (0.996, "alg2_kernels_bert_large_div16.md"),
+    "local_step_pipelined_kernel + compress_kernel + reduce_pipelined_kernel": (0.987, "compress_kernel_reduce_pipelined_kernel_two_call_bert_large_div16.md"),
+    "lc_worker_pack_kernel + lc_server_pack_kernel + dist_apply_kernel (large-chunk kernels)": (1.004, "large_chunk_kernels_whole_vector_bert_large_div16.md"),
+}
 
 
 # ---- byte model: what the method must move, per launch -------------------------
@@ -363,14 +376,14 @@ def run_ours(args, wl):
                                   + ("reduce_pipelined_kernel" if uses_ring else "reduce_kernel"),
                  "alg2_compressed": "alg2_pipelined_kernel" if alg2_ring else "alg2_compressed_kernel",
                  "alg2_full": "alg2_full_kernel"}
-    roofline = {"bound": "hbm", "kernel": kernel_of.get(dominant, "local_step_pipelined_kernel" if local_ring else "local_step_kernel"),
+    kernel = kernel_of.get(dominant, "local_step_pipelined_kernel" if local_ring else "local_step_kernel")
+    ratio, summary = DRAM_TRAFFIC_RATIO.get(f"{kernel}@{wl.chunk}", DRAM_TRAFFIC_RATIO.get(kernel, (None, None)))
+    roofline = {"bound": "hbm", "kernel": kernel,
                 "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "peak_kind": f"of {peak_kind}", "frac_of_8TBps_nominal": achieved / 8000.0,
-                # ncu (dram__bytes_read.sum + dram__bytes_write.sum) on the layout shrunk 16x gave
-                # 0.995 x the algorithmic bytes for both sync kernels and 0.994 for the local step
-                # (profiles/); traffic is proportional to n*W, so the ratio carries to a full launch.
-                "traffic": DRAM_TRAFFIC_RATIO * bytes_of[dominant],
-                "traffic_how": "ncu capture of the same kernel on the layout shrunk 16x, scaled by n*W",
+                "traffic": ratio * bytes_of[dominant] if ratio else None,
+                "traffic_how": (f"ncu capture of the same kernel on the layout shrunk 16x (profiles/{summary}: DRAM bytes = "
+                                f"{ratio} x algorithmic), scaled by n*W") if ratio else "no ncu capture of this kernel",
                 "launch_ms": statistics.mean(by_kind[dominant]),
                 "algorithmic_bytes_per_launch": bytes_of[dominant]}
 

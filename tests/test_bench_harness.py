@@ -71,3 +71,16 @@ def test_oracle_baseline_uses_the_cores_and_the_given_gradients():
     assert asked == [3, 4, 5]
     assert cores == min(len(os.sched_getaffinity(0)), 64) and value > 0 and s_per_step > 0
     assert f"{cores} chunk ranges" in desc and "t=3..5" in desc
+
+
+def test_traffic_ratios_are_the_ones_in_the_committed_profiles():
+    """bench.py's roofline.traffic is a measured ratio times the algorithmic bytes: every ratio must be
+    printed in the ncu summary it names, so that a re-captured kernel cannot leave a stale constant."""
+    import os
+    import bench
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    for kernel, (ratio, summary) in bench.DRAM_TRAFFIC_RATIO.items():
+        path = os.path.join(root, "profiles", summary)
+        assert os.path.exists(path), (kernel, summary)
+        text = open(path).read()
+        assert f"{ratio}" in text, (kernel, ratio, summary)
