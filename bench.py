@@ -34,7 +34,8 @@ DRAM_TRAFFIC_RATIO = {
     "step_sync_kernel": (0.995, "step_sync_kernel_alg2_compressed_kernel_chunk_per_block_bert_large_div16.md"),
     "step_sync_kernel@16384": (1.004, "step_sync_kernel_alg2_compressed_kernel_chunk_per_block_bert_large_div16.md"),
     "alg2_compressed_kernel": (1.007, "step_sync_kernel_alg2_compressed_kernel_chunk_per_block_bert_large_div16.md"),
-    "alg2_pipelined_kernel": (0.996, "alg2_kernels_bert_large_div16.md"),
+    "alg2_pipelined_kernel": (0.994, "alg2_kernels_bert_large_div16.md"),
+    "alg2_full_kernel": (0.992, "alg2_kernels_bert_large_div16.md"),
     "local_step_pipelined_kernel + compress_kernel + reduce_pipelined_kernel": (0.987, "compress_kernel_reduce_pipelined_kernel_two_call_bert_large_div16.md"),
     "lc_worker_pack_kernel + lc_server_pack_kernel + dist_apply_kernel (large-chunk kernels)": (1.004, "large_chunk_kernels_whole_vector_bert_large_div16.md"),
 }
