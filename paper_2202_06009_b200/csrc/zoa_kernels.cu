@@ -988,14 +988,23 @@ lc_server_pack_kernel(StateView st, int pending, long long segs_per_chunk, long 
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     double *scratch = reinterpret_cast<double *>(smem_raw);
-    float *scales_sm = reinterpret_cast<float *>(smem_raw + 34 * sizeof(double));
-    uint32_t *words_sm = reinterpret_cast<uint32_t *>(scales_sm + kMaxWorkers);      // [W][kSegment / 32]
+    double *table = scratch + 34;                                                    // [kMaxWorkers / 4][16], see table_sum_is_exact
+    float *scales_sm = reinterpret_cast<float *>(table + (kMaxWorkers / 4) * 16);
+    int *exact_flag = reinterpret_cast<int *>(scales_sm + kMaxWorkers);
+    uint32_t *words_sm = reinterpret_cast<uint32_t *>(exact_flag + 4);               // [W][kSegment / 32]
     const SegGeom sg = seg_geom(st, blockIdx.x, segs_per_chunk);
     const int lane = threadIdx.x & 31;
     constexpr int kWordsPerSeg = kSegment / 32;
     const int n_words = (sg.len + 31) >> 5;
     const long long seg_word0 = sg.j0 >> 5;
-    for (int i = threadIdx.x; i < st.W; i += blockDim.x) scales_sm[i] = st.scales_w[(long long)i * st.n_chunks + sg.c];
+    if (threadIdx.x < 32) {
+        const float s_lo = lane < st.W ? st.scales_w[(long long)lane * st.n_chunks + sg.c] : 0.0f;
+        const float s_hi = lane + 32 < st.W ? st.scales_w[(long long)(lane + 32) * st.n_chunks + sg.c] : 0.0f;
+        if (lane < st.W) scales_sm[lane] = s_lo;
+        if (lane + 32 < st.W) scales_sm[lane + 32] = s_hi;
+        const bool exact = table_sum_is_exact(s_lo, s_hi, st.W);
+        if (lane == 0) *exact_flag = exact;
+    }
     const float old_scale = pending ? st.scales_s[sg.c] : 0.0f;       // of the previous sync
     const int total = st.W * n_words;
     for (int e0 = threadIdx.x; e0 < total; e0 += 8 * blockDim.x) {
@@ -1018,6 +1027,14 @@ lc_server_pack_kernel(StateView st, int pending, long long segs_per_chunk, long 
         e4[it] = idx < sg.len ? ld4(st.ds + sg.j0 + idx) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
     __syncthreads();
+    const int groups = (st.W + 3) >> 2;
+    for (int e = threadIdx.x; e < 16 * groups; e += blockDim.x) table[e] = table_entry(scales_sm, st.W, e);
+    __syncthreads();
+    const bool fast = *exact_flag != 0;
+    // the thread's four coordinates are one nibble of a packed word: byte (lane & 7) / 2, its upper half for odd lanes
+    const uint32_t byte_sel = ((lane & 7u) >> 1) | ((4u + ((lane & 7u) >> 1)) << 4);
+    const int half_shift = (lane & 1) * 4;
+    const int last = st.W - 1;
     double l1 = 0.0;
 #pragma unroll
     for (int it = 0; it < kSegIter; ++it) {
@@ -1026,12 +1043,24 @@ lc_server_pack_kernel(StateView st, int pending, long long segs_per_chunk, long 
         float a[4] = {0.f, 0.f, 0.f, 0.f};
         if (idx < sg.len) {
             double A[4] = {0.0, 0.0, 0.0, 0.0};
-            const int shift = idx & 31;
-            for (int i = 0; i < st.W; ++i) {   // worker order
-                const uint32_t nib = words_sm[i * kWordsPerSeg + (idx >> 5)] >> shift;
-                const double sc = (double)scales_sm[i];
+            const uint32_t *col = words_sm + (idx >> 5);
+            for (int g = 0; g < groups; ++g) {
+                // a worker index past the last one repeats the last worker's word: its bits select among equal table entries
+                const int i1 = min(4 * g + 1, last), i2 = min(4 * g + 2, last), i3 = min(4 * g + 3, last);
+                const uint32_t x = gather_bytes(col[4 * g * kWordsPerSeg], col[i1 * kWordsPerSeg], col[i2 * kWordsPerSeg],
+                                                col[i3 * kWordsPerSeg], byte_sel) >> half_shift;
+                if (fast) {
+                    const char *tb = reinterpret_cast<const char *>(table + g * 16);
 #pragma unroll
-                for (int k = 0; k < 4; ++k) A[k] += ((nib >> k) & 1u) ? sc : -sc;
+                    for (int k = 0; k < 4; ++k) A[k] = __dadd_rn(A[k], *reinterpret_cast<const double *>(tb + table_offset(x, k)));
+                } else {
+                    for (int q = 0; q < 4 && 4 * g + q < st.W; ++q) {   // worker order
+                        const double sc = (double)scales_sm[4 * g + q];
+                        const uint32_t nib = x >> (8 * q);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) A[k] += ((nib >> k) & 1u) ? sc : -sc;
+                    }
+                }
             }
             const float4 p4 = plain_error4(e4[it], pending != 0, old_scale);
             const float ee[4] = {p4.x, p4.y, p4.z, p4.w};
@@ -1315,7 +1344,8 @@ cudaError_t launch_large_server(const StateView &st, const Consts &c, int mode, 
                                 int *launches, cudaStream_t s)
 {
     const long long spc = large_chunk_segments(st), n_segs = spc * st.n_chunks;
-    const size_t pack_smem = 34 * sizeof(double) + kMaxWorkers * sizeof(float) + (size_t)st.W * (kSegment / 32) * sizeof(uint32_t);
+    const size_t pack_smem = (34 + (kMaxWorkers / 4) * 16) * sizeof(double) + kMaxWorkers * sizeof(float) + 16
+                             + (size_t)st.W * (kSegment / 32) * sizeof(uint32_t);
     lc_server_pack_kernel<<<(unsigned)n_segs, 256, pack_smem, s>>>(st, pending, spc, n_segs, partials);
     lc_scales_kernel<<<dim3((unsigned)st.n_chunks, 1), 32, 0, s>>>(st, partials + (long long)st.W * n_segs, spc, n_segs, st.scales_s);
     if (mode == 1) dist_apply_kernel<<<elementwise_grid((st.n + 3) / 4), 256, 0, s>>>(st, c, scalar);

@@ -695,6 +695,29 @@ def test_large_chunks_and_whole_vector_scale(W, chunk, n, mode):
         p.close()
 
 
+@pytest.mark.parametrize("mode", ["fused", "two_call", "alg2"])
+@pytest.mark.parametrize("W,chunk,n", [(3, 32768, 2 * 32768 + 5000), (5, 1 << 22, 70000)])
+def test_large_chunks_worker_magnitudes_far_apart(W, chunk, n, mode):
+    """The large-chunk server pass also looks the sum over the workers up in tables; with the workers'
+    gradients 2^25 apart from one another the partial sums round and it must add worker by worker."""
+    rng = np.random.default_rng(W * n)
+    p = Pair(n, W, chunk, var_steps=(0,), sync=((0,), (1,)), x0=rng.standard_normal(n) * 0.02)
+    factor = (2.0 ** (25.0 * np.arange(W) - 40.0)).astype(np.float32)[:, None]
+    try:
+        for t in range(4):
+            g = _grads(rng, W, n) * factor
+            if mode == "alg2":
+                p.gpu.alg2_step(list(torch.from_numpy(g).cuda()), 1e-3, t)
+                torch.cuda.synchronize()
+                p.cpu.alg2_step(g, np.float32(1e-3), t == 0)
+                p.compare(f"t={t}", wire=t != 0)
+            else:
+                p.step(g, 1e-3, t, mode)
+                p.compare(f"t={t}", wire=True)
+    finally:
+        p.close()
+
+
 def test_paper_schedules_on_a_handle():
     z = Zoa(64, 1, chunk=32)
     try:
