@@ -91,16 +91,40 @@ __global__ void __launch_bounds__(kRingThreads, 1) reduce_pipelined_kernel(const
     if (warp == kConsumerWarps) {
         // ------------------------- copy-issuing warp (all 32 lanes stay) -------------------------
         RingProducer p(a, &sh->ring, ring, lay.stage_bytes);
+        // The unit numbers come from a global counter and the magnitudes from global memory: two
+        // round trips that would stand between the tiles of every unit (with one tile per unit and
+        // few workers they, not the copies, set the pace).  So the warp runs ahead: it holds the
+        // numbers of the next two units, and the magnitudes of a unit's first tile are loaded one
+        // unit early into registers (two per lane; more than 64 of them are loaded in place).
+        const bool ahead = W * G <= 64;
+        long long cur = 0, nxt = 0;
+        if (lane == 0) { cur = p.take(); nxt = p.take(); }
+        float pre_c[2] = {0.f, 0.f}, pre_n[2] = {0.f, 0.f};
+        bool have_pre = false;
+        auto load_magnitudes = [&](long long unit, float (&dst)[2]) {      // of the unit's first tile
+            const long long chunk0 = G > 1 ? unit * span / st.chunk : unit;
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                const int e = lane + 32 * q;
+                dst[q] = e < W * G ? st.scales_w[(long long)(e / G) * st.n_chunks + chunk0 + (e % G)] : 0.0f;
+            }
+        };
         for (long long k = 0;; ++k) {
             long long unit = 0;
             int go = 0;
             if (lane == 0) {
-                go = (p.ok && p.next_chunk(k, &unit)) ? 1 : 0;
+                go = (p.ok && p.publish(k, cur, &unit)) ? 1 : 0;
                 if (!go && p.ok) mbar_arrive(p.full_barrier());          // the end mark needs the barrier's second arrival too
             }
             go = __shfl_sync(0xffffffffu, go, 0);
             unit = __shfl_sync(0xffffffffu, unit, 0);
             if (!go) break;
+            // next unit's magnitudes and the number of the unit after it: both in flight during this unit's tiles
+            const long long next_taken = __shfl_sync(0xffffffffu, nxt, 0);
+            const bool next_valid = next_taken < a.n_full_chunks;
+            if (ahead && next_valid) load_magnitudes(a.first_chunk + next_taken, pre_n);
+            cur = nxt;
+            if (lane == 0) nxt = p.take();
             const long long u0 = unit * span;
             int alive = 1;
             for (int t = 0; t < 2 * TILES && alive; ++t) {
@@ -125,9 +149,15 @@ __global__ void __launch_bounds__(kRingThreads, 1) reduce_pipelined_kernel(const
                     }
                     if (G > 1 || t == 0) {
                         float *dst_scales = reinterpret_cast<float *>(stage_ptr + lay.stage_scales_off);
-                        const long long chunk0 = G > 1 ? off / st.chunk : unit;
-                        for (int e = lane; e < W * G; e += 32)
-                            dst_scales[e] = st.scales_w[(long long)(e / G) * st.n_chunks + chunk0 + (e % G)];
+                        if (have_pre && t == 0) {
+#pragma unroll
+                            for (int q = 0; q < 2; ++q)
+                                if (lane + 32 * q < W * G) dst_scales[lane + 32 * q] = pre_c[q];
+                        } else {
+                            const long long chunk0 = G > 1 ? off / st.chunk : unit;
+                            for (int e = lane; e < W * G; e += 32)
+                                dst_scales[e] = st.scales_w[(long long)(e / G) * st.n_chunks + chunk0 + (e % G)];
+                        }
                     }
                 } else {                    // second pass: v and x_sync
                     const long long off = u0 + (long long)(t - TILES) * kTile;
@@ -147,6 +177,9 @@ __global__ void __launch_bounds__(kRingThreads, 1) reduce_pipelined_kernel(const
                 alive = __shfl_sync(0xffffffffu, alive, 0);
             }
             if (!alive) break;
+            pre_c[0] = pre_n[0];
+            pre_c[1] = pre_n[1];
+            have_pre = ahead && next_valid;
         }
         if (lane == 0) p.finish();
         return;

@@ -224,9 +224,12 @@ struct RingProducer {
     // travels through shared memory and the arrive on the chunk's first tile publishes it.  The queue
     // cannot wrap onto an unread entry: the producer is at most `stages` tiles, hence chunks, ahead.
     // Returns false when no chunk is left (the consumers are told) or a wait ran out.
-    __device__ __forceinline__ bool next_chunk(long long k, long long *chunk)
+    __device__ __forceinline__ bool next_chunk(long long k, long long *chunk) { return publish(k, take(), chunk); }
+    // The two halves of next_chunk, for a producer that takes its chunks ahead of time: the number of a
+    // chunk from the global counter, and (later) the announcement of it as this block's k-th chunk.
+    __device__ __forceinline__ long long take() { return (long long)atomicAdd(&a.sched[0], 1ull); }
+    __device__ __forceinline__ bool publish(long long k, long long taken, long long *chunk)
     {
-        const long long taken = (long long)atomicAdd(&a.sched[0], 1ull);
         const bool last = taken >= a.n_full_chunks;
         *chunk = a.first_chunk + taken;
         if (!stage_free()) return false;
